@@ -1,0 +1,307 @@
+/*
+ * CPU oracle for structured tensor algebra on packed layouts.  TEST INFRASTRUCTURE ONLY: it is
+ * called by the tests, by the smoke check and by the benchmark's CPU-baseline leg, never by the
+ * CUDA library, and it shares no code with it.
+ *
+ * Everything here is the plain definition written out, with no closed-form index polynomial:
+ *
+ *  - A structure is a set of integer points inside the box [0, dims) that satisfy every row of a
+ *    list of affine comparisons over the indices and the size symbols (Section 2, "Unique set";
+ *    Section 4, "Iteration space extraction").
+ *  - The packed position of a point is the number of points of the set that precede it in
+ *    lexicographic order, first index slowest, last index contiguous (Section 4, "Iteration
+ *    space extraction", "Preceding Accesses" and "Access domain linearization":
+ *    P = #{preceding accesses}).  Here that number is a counter advanced while enumerating.
+ *  - Compress / decompress copy values between the dense tensor and the packed vector while
+ *    walking the accessed indices (Section 3, "Data Layout Compression"); a redundancy map sends a
+ *    redundant index to its unique representative (Section 2, "Redundancy map").
+ *  - A contraction is the sum-of-products rule evaluated over the full dense index ranges with the
+ *    body guarded by the structure predicate, each product added to the output element
+ *    (Section 5.2, "Uncompressed Compute Code Generation"), accumulated in double.
+ *
+ * Parallelism: OpenMP static schedule over the outermost output index, which is the
+ * parallelisation the paper itself applies (Section 5.2, "Parallelization").
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_MAX_RANK 4
+
+/* rows: nrows x (rank + nparams + 1), row-major.  Row r holds
+ *   sum_k rows[r][k] * idx[k] + sum_p rows[r][rank+p] * params[p] + rows[r][rank+nparams]
+ * which must be >= 0 (is_eq[r] == 0) or == 0 (is_eq[r] != 0). */
+typedef struct {
+    int32_t rank, nparams, nrows;
+    const int64_t* dims;
+    const int64_t* rows;
+    const uint8_t* is_eq;
+    const int64_t* params;
+} orc_desc;
+
+static int in_domain(const orc_desc* d, const int64_t* idx) {
+    const int w = d->rank + d->nparams + 1;
+    for (int r = 0; r < d->nrows; ++r) {
+        const int64_t* row = d->rows + (size_t)r * w;
+        int64_t v = row[w - 1];
+        for (int k = 0; k < d->rank; ++k) v += row[k] * idx[k];
+        for (int p = 0; p < d->nparams; ++p) v += row[d->rank + p] * d->params[p];
+        if (d->is_eq[r] ? (v != 0) : (v < 0)) return 0;
+    }
+    return 1;
+}
+
+/* Advance idx to the next point of the box in lexicographic order; 0 when the box is exhausted. */
+static int box_next(const orc_desc* d, int64_t* idx) {
+    for (int k = d->rank - 1; k >= 0; --k) {
+        if (++idx[k] < d->dims[k]) return 1;
+        idx[k] = 0;
+    }
+    return 0;
+}
+
+static int box_empty(const orc_desc* d) {
+    for (int k = 0; k < d->rank; ++k)
+        if (d->dims[k] <= 0) return 1;
+    return d->rank <= 0;
+}
+
+static int64_t dense_linear(const orc_desc* d, const int64_t* idx) {
+    int64_t lin = 0;
+    for (int k = 0; k < d->rank; ++k) lin = lin * d->dims[k] + idx[k];
+    return lin;
+}
+
+/* Number of points of the set. */
+int64_t orc_count(const orc_desc* d) {
+    if (box_empty(d)) return 0;
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0}, counter = 0;
+    do {
+        if (in_domain(d, idx)) ++counter;
+    } while (box_next(d, idx));
+    return counter;
+}
+
+/* table[dense linear index] = packed position of that point, or -1 outside the set. */
+void orc_rank_table(const orc_desc* d, int64_t* table) {
+    if (box_empty(d)) return;
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0}, counter = 0;
+    do {
+        table[dense_linear(d, idx)] = in_domain(d, idx) ? counter++ : -1;
+    } while (box_next(d, idx));
+}
+
+/* idx_out[p * rank + k] = k-th index of the point stored at packed position p. */
+void orc_unrank_table(const orc_desc* d, int32_t* idx_out) {
+    if (box_empty(d)) return;
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0}, counter = 0;
+    do {
+        if (in_domain(d, idx)) {
+            for (int k = 0; k < d->rank; ++k) idx_out[counter * d->rank + k] = (int32_t)idx[k];
+            ++counter;
+        }
+    } while (box_next(d, idx));
+}
+
+/* Packed position of one point: the points preceding it are counted one by one.
+ * Returns -1 if the point is not in the set. */
+int64_t orc_rank_point(const orc_desc* d, const int64_t* point) {
+    if (box_empty(d)) return -1;
+    for (int k = 0; k < d->rank; ++k)
+        if (point[k] < 0 || point[k] >= d->dims[k]) return -1;
+    if (!in_domain(d, point)) return -1;
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0}, counter = 0;
+    do {
+        if (memcmp(idx, point, sizeof(int64_t) * (size_t)d->rank) == 0) return counter;
+        if (in_domain(d, idx)) ++counter;
+    } while (box_next(d, idx));
+    return -1;
+}
+
+/* Compress: packed[counter] = dense[idx] over the set, elements moved as raw bytes. */
+void orc_pack(const orc_desc* d, int64_t elt_size, const void* dense, void* packed) {
+    if (box_empty(d)) return;
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0}, counter = 0;
+    do {
+        if (in_domain(d, idx)) {
+            memcpy((char*)packed + counter * elt_size,
+                   (const char*)dense + dense_linear(d, idx) * elt_size, (size_t)elt_size);
+            ++counter;
+        }
+    } while (box_next(d, idx));
+}
+
+/* Decompress: dense = 0; dense[idx] = packed[counter]; with a redundancy map given as an index
+ * permutation (mirror[k] = which source index lands in position k), the permuted point receives
+ * the same value when it differs from the point itself. */
+void orc_unpack(const orc_desc* d, const int32_t* mirror, int64_t elt_size, const void* packed,
+                void* dense) {
+    if (box_empty(d)) return;
+    int64_t total = 1;
+    for (int k = 0; k < d->rank; ++k) total *= d->dims[k];
+    memset(dense, 0, (size_t)(total * elt_size));
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0}, counter = 0;
+    do {
+        if (in_domain(d, idx)) {
+            const char* src = (const char*)packed + counter * elt_size;
+            memcpy((char*)dense + dense_linear(d, idx) * elt_size, src, (size_t)elt_size);
+            if (mirror) {
+                int64_t m[ORC_MAX_RANK];
+                int ok = 1;
+                for (int k = 0; k < d->rank; ++k) {
+                    m[k] = idx[mirror[k]];
+                    if (m[k] >= d->dims[k]) ok = 0;
+                }
+                if (ok && memcmp(m, idx, sizeof(int64_t) * (size_t)d->rank) != 0)
+                    memcpy((char*)dense + dense_linear(d, m) * elt_size, src, (size_t)elt_size);
+            }
+            ++counter;
+        }
+    } while (box_next(d, idx));
+}
+
+/* ---- band stored as padded diagonals -------------------------------------------------------
+ * Layout: 2w+1 diagonals of N slots; slot (d, i), d outer, holds A[i][i + d - w] when that
+ * column exists and +0.0f otherwise.  The enumeration runs over slots. */
+void orc_band_pack(int64_t N, int64_t w, const float* dense, float* packed) {
+    int64_t counter = 0;
+    for (int64_t d = 0; d <= 2 * w; ++d)
+        for (int64_t i = 0; i < N; ++i) {
+            int64_t j = i + d - w;
+            packed[counter++] = (j >= 0 && j < N) ? dense[i * N + j] : 0.0f;
+        }
+}
+
+void orc_band_unpack(int64_t N, int64_t w, const float* packed, float* dense) {
+    memset(dense, 0, (size_t)(N * N) * sizeof(float));
+    int64_t counter = 0;
+    for (int64_t d = 0; d <= 2 * w; ++d)
+        for (int64_t i = 0; i < N; ++i) {
+            int64_t j = i + d - w;
+            if (j >= 0 && j < N) dense[i * N + j] = packed[counter];
+            ++counter;
+        }
+}
+
+/* slot_table[i * N + j] = slot of (i, j), or -1 outside the band. */
+void orc_band_slot_table(int64_t N, int64_t w, int64_t* slot_table) {
+    for (int64_t t = 0; t < N * N; ++t) slot_table[t] = -1;
+    int64_t counter = 0;
+    for (int64_t d = 0; d <= 2 * w; ++d)
+        for (int64_t i = 0; i < N; ++i) {
+            int64_t j = i + d - w;
+            if (j >= 0 && j < N) slot_table[i * N + j] = counter;
+            ++counter;
+        }
+}
+
+/* ---- contractions ---------------------------------------------------------------------------
+ * Inputs are fp32 arrays, or bf16 bit patterns (is_bf16 != 0) widened exactly to double.
+ * Outputs: `out` = the sum in double, `out_abs` = the sum of the absolute values of the same
+ * products (the denominator of the forward-error bound), both may be computed for a subset of the
+ * outermost output index: sel[s] is the logical index i of the s-th supplied slice of the
+ * structured operand. */
+static inline double widen(const void* p, int64_t at, int is_bf16) {
+    if (is_bf16) {
+        union { uint32_t u; float f; } c;
+        c.u = (uint32_t)((const uint16_t*)p)[at] << 16;
+        return (double)c.f;
+    }
+    return (double)((const float*)p)[at];
+}
+
+/* y[i] = sum_j [ (i, j) in set ] A[i][j] * x[j]           (A(i) := B(i,j) * C(j), Table 1 "SpMV")
+ * A_rows[s] is the dense row sel[s] of A (N values). */
+void orc_matvec(const orc_desc* d, int64_t nsel, const int64_t* sel, const float* A_rows,
+                const float* x, double* out, double* out_abs) {
+    const int64_t N = d->dims[1];
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        double acc = 0.0, acc_abs = 0.0;
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t idx[2] = {sel[s], j};
+            if (in_domain(d, idx)) {
+                double p = (double)A_rows[s * N + j] * (double)x[j];
+                acc += p;
+                acc_abs += fabs(p);
+            }
+        }
+        out[s] = acc;
+        out_abs[s] = acc_abs;
+    }
+}
+
+/* Symmetric product from the unique upper part:  Sfull[i][j] = U[min(i,j)][max(i,j)],
+ * y[i] = sum_j Sfull[i][j] * x[j]  (Section 2, "Redundancy map": redundant (x, y) with x > y reads
+ * the unique element (y, x)).  U is a dense N x N array; entries below the diagonal are ignored. */
+void orc_symv(int64_t N, const float* U, const float* x, double* out, double* out_abs) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < N; ++i) {
+        double acc = 0.0, acc_abs = 0.0;
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t lo = i < j ? i : j, hi = i < j ? j : i;
+            double p = (double)U[lo * N + hi] * (double)x[j];
+            acc += p;
+            acc_abs += fabs(p);
+        }
+        out[i] = acc;
+        out_abs[i] = acc_abs;
+    }
+}
+
+/* C[i][c] = sum_j [ (i, j) in set ] A[i][j] * B[j][c];  B is N x ncols row-major. */
+void orc_matmat(const orc_desc* d, int is_bf16, int64_t nsel, const int64_t* sel,
+                const void* A_rows, const void* B, int64_t ncols, double* out, double* out_abs) {
+    const int64_t N = d->dims[1];
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        for (int64_t c = 0; c < ncols; ++c) {
+            double acc = 0.0, acc_abs = 0.0;
+            for (int64_t j = 0; j < N; ++j) {
+                int64_t idx[2] = {sel[s], j};
+                if (in_domain(d, idx)) {
+                    double p = widen(A_rows, s * N + j, is_bf16) * widen(B, j * ncols + c, is_bf16);
+                    acc += p;
+                    acc_abs += fabs(p);
+                }
+            }
+            out[s * ncols + c] = acc;
+            out_abs[s * ncols + c] = acc_abs;
+        }
+    }
+}
+
+/* M[i][r] = sum_j sum_k [ (i, j, k) in set ] T[i][j][k] * B[j][r] * C[k][r]
+ * (A(i,j) := B(i,k,l) * C(k,j) * D(l,j), Table 1 "MTTKRP", with the indices renamed).
+ * T_slabs[s] is the dense n x n slab sel[s] of T. */
+void orc_mttkrp(const orc_desc* d, int64_t nsel, const int64_t* sel, const float* T_slabs,
+                const float* B, const float* C, int64_t R, double* out, double* out_abs) {
+    const int64_t nj = d->dims[1], nk = d->dims[2];
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        for (int64_t r = 0; r < R; ++r) {
+            double acc = 0.0, acc_abs = 0.0;
+            for (int64_t j = 0; j < nj; ++j)
+                for (int64_t k = 0; k < nk; ++k) {
+                    int64_t idx[3] = {sel[s], j, k};
+                    if (in_domain(d, idx)) {
+                        double p = (double)T_slabs[(s * nj + j) * nk + k] * (double)B[j * R + r] *
+                                   (double)C[k * R + r];
+                        acc += p;
+                        acc_abs += fabs(p);
+                    }
+                }
+            out[s * R + r] = acc;
+            out_abs[s * R + r] = acc_abs;
+        }
+    }
+}
+
+/* Thread count the contractions above will use. */
+#ifdef _OPENMP
+#include <omp.h>
+int orc_num_threads(void) { return omp_get_max_threads(); }
+#else
+int orc_num_threads(void) { return 1; }
+#endif
