@@ -1,0 +1,193 @@
+/*
+ * dastac.h - structured tensor algebra on densely packed layouts, CUDA (sm_100a) library, C ABI.
+ *
+ * A tensor whose nonzero, non-redundant region is a polyhedron is stored as a packed vector: the
+ * position of a logical index is the number of points of the region that precede it in
+ * lexicographic order, computed from a closed-form ranking polynomial in registers, with no index
+ * arrays in memory.  Contractions read the packed operands directly.
+ *
+ * General conventions
+ *   - Every function returns a dastac_status; nothing throws or aborts across this boundary.
+ *     Argument errors are detected before any device work is enqueued.
+ *   - Device work is only enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream); no call synchronises unless stated.  The current CUDA device must be the one that
+ *     owns the buffers.
+ *   - The caller owns every buffer.  Pointers are device pointers unless marked "host".  The
+ *     library allocates no device memory; scratch space is passed in as `workspace`.
+ *   - Indices are int32 per dimension (extents up to 2^30); packed positions are int64.
+ *   - Dense operands are described by element strides; packed operands are contiguous.
+ *   - Packed buffers must be 16-byte aligned and have a capacity of `slots` elements as reported
+ *     by dastac_structure_count (the point count rounded up to a multiple of 16 bytes); the
+ *     library never reads element values beyond `count` into a result, but it may load the
+ *     padding bytes.
+ */
+#ifndef DASTAC_H_
+#define DASTAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DASTAC_OK = 0,
+    DASTAC_ERR_INVALID_ARG = 1,           /* NULL pointer, negative size, malformed descriptor     */
+    DASTAC_ERR_UNSUPPORTED_STRUCTURE = 2, /* descriptor is valid but is not a recognised class     */
+    DASTAC_ERR_UNSUPPORTED_EXPR = 3,      /* expression x structure x dtype has no kernel          */
+    DASTAC_ERR_SHAPE = 4,                 /* operand extents disagree                              */
+    DASTAC_ERR_ALIGNMENT = 5,             /* a data pointer is not 16-byte aligned                 */
+    DASTAC_ERR_OVERFLOW = 6,              /* an extent exceeds 2^30 or a count exceeds 2^62        */
+    DASTAC_ERR_WORKSPACE = 7,             /* workspace missing, misaligned or too small            */
+    DASTAC_ERR_CUDA = 8,                  /* a CUDA runtime/driver call failed                     */
+    DASTAC_ERR_TIMEOUT = 9                /* a bounded device-side wait expired (see err_word)     */
+} dastac_status;
+
+typedef enum { DASTAC_F32 = 0, DASTAC_BF16 = 1 } dastac_dtype;
+typedef enum { DASTAC_MEM_DEVICE = 0, DASTAC_MEM_HOST = 1 } dastac_memspace;
+
+/* Recognised structure classes (result of descriptor analysis). */
+typedef enum {
+    DASTAC_KIND_EMPTY = 0,
+    DASTAC_KIND_DENSE = 1,          /* the whole box, row-major                                    */
+    DASTAC_KIND_UPPER = 2,          /* 0<=i<M, i<=j<N, optional trailing dense extent Q (rank 3)   */
+    DASTAC_KIND_LOWER = 3,          /* 0<=j<=i<N                                                   */
+    DASTAC_KIND_BAND_DIAGONALS = 4, /* |i-j|<=w stored as 2w+1 diagonals of N slots                */
+    DASTAC_KIND_TETRAHEDRON = 5     /* 0<=i<=j<=k<n                                                */
+} dastac_kind;
+
+#define DASTAC_LAYOUT_LEXICOGRAPHIC 0 /* exact pack in lexicographic order                         */
+#define DASTAC_LAYOUT_PADDED_DIAGONALS 1 /* band only: diagonal-major, N slots per diagonal        */
+
+/*
+ * Structure descriptor: the unique set of a tensor as a conjunction of affine comparisons over the
+ * indices and size symbols (paper Section 2, "Unique set"; Section 4, "Iteration space
+ * extraction"), an optional redundancy map (Section 2, "Redundancy map") and the requested layout.
+ *
+ *   rows    host, nrows x (rank + nparams + 1), row-major.  Row r states
+ *             sum_k rows[r][k]*idx[k] + sum_p rows[r][rank+p]*params[p] + rows[r][rank+nparams] >= 0
+ *           or "== 0" when is_eq[r] != 0.  The box 0 <= idx[k] < dims[k] is always implied.
+ *   mirror  host, NULL or a permutation of 0..rank-1: the redundant point (idx[mirror[0]], ...)
+ *           holds the same value as idx.  Only the swap {1,0} on a square upper triangle (a
+ *           symmetric matrix stored as its upper part) is supported.
+ *   layout  DASTAC_LAYOUT_*.
+ * All arrays are read during dastac_structure_create only.
+ */
+typedef struct {
+    int32_t rank;     /* 1..3 */
+    int32_t nparams;  /* 0..8 */
+    int32_t nrows;    /* 0..64 */
+    const int64_t* dims;
+    const int64_t* rows;
+    const uint8_t* is_eq;
+    const int64_t* params;
+    const int32_t* mirror;
+    int32_t layout;
+} dastac_structure_desc;
+
+/* Immutable host object: recognised class plus the coefficients of its ranking polynomial. */
+typedef struct dastac_structure dastac_structure;
+
+/*
+ * Analyse a descriptor (Algorithm 1, "Symbolic Indexing", restricted to classes whose counting
+ * polynomial is known in closed form).  The comparisons are normalised to difference bounds,
+ * closed under implication, and matched against the recognised classes, so redundant or
+ * re-ordered rows do not matter.  Errors: INVALID_ARG, OVERFLOW, UNSUPPORTED_STRUCTURE (a row that
+ * is not a bound or a difference of two indices, or a set that is none of the classes).
+ */
+dastac_status dastac_structure_create(const dastac_structure_desc* desc, dastac_structure** out);
+void dastac_structure_destroy(dastac_structure* s);
+
+/* slots = elements a packed buffer must hold (count, or (2w+1)*N for padded diagonals; the
+ * buffer capacity must be slots rounded up to 16 bytes); nnz = points of the set. */
+dastac_status dastac_structure_count(const dastac_structure* s, int64_t* slots, int64_t* nnz);
+/* kind = dastac_kind; symmetric = 1 if a redundancy swap is attached. */
+dastac_status dastac_structure_kind(const dastac_structure* s, int32_t* kind, int32_t* symmetric);
+
+/*
+ * Ranking polynomial P(idx) = number of preceding points (Section 4, "Access domain
+ * linearization"), evaluated in exact 64-bit integer arithmetic with a single final division
+ * (Section 3, figure of the generated loop nest).  Host versions; idx and the result are host
+ * pointers.  dastac_rank returns INVALID_ARG for a point outside the set.  dastac_unrank is the
+ * inverse; for a padding slot of the padded-diagonal layout it sets the column to -1.
+ */
+dastac_status dastac_rank(const dastac_structure* s, const int32_t* idx, int64_t* off);
+dastac_status dastac_unrank(const dastac_structure* s, int64_t off, int32_t* idx);
+
+/*
+ * Device versions over n points: idx is n x rank int32 (device), off is n int64 (device).  A point
+ * outside the set ranks to -1.  These run the same in-register maps the kernels use.
+ */
+dastac_status dastac_rank_batch(const dastac_structure* s, const int32_t* idx, int64_t n,
+                                int64_t* off, void* stream);
+dastac_status dastac_unrank_batch(const dastac_structure* s, const int64_t* off, int64_t n,
+                                  int32_t* idx, void* stream);
+
+/*
+ * Compress / decompress (Section 3, "Data Layout Compression": copy over the accessed indices).
+ *   pack    packed[P(idx)] = dense[idx] for every point of the set; padded-diagonal padding
+ *           slots receive +0.  Bit-exact copy.
+ *   unpack  dense = 0 everywhere in the box, then dense[idx] = packed[P(idx)]; with a redundancy
+ *           swap the mirrored element receives the same bits.  Padding slots are ignored.
+ * dense_strides: host array of `rank` element strides of the dense tensor.
+ */
+dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dtype, const void* dense,
+                          const int64_t* dense_strides, void* packed, void* stream);
+dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype dtype, const void* packed,
+                            void* dense, const int64_t* dense_strides, void* stream);
+
+/*
+ * Contraction operand.
+ *   structure == NULL: dense tensor, `rank` extents in dims, element strides in strides.
+ *   structure != NULL: packed tensor of that structure (dims/strides ignored except that
+ *                      batch instances are batch_stride elements apart).
+ *   space: where `data` lives.  Host operands are staged through the workspace with asynchronous
+ *          copies on `stream` (pinned memory recommended); a host output is valid after the
+ *          caller synchronises the stream.
+ *   batch: number of independent instances sharing the structure (0 or 1 = single).  Dense
+ *          operands of a batched call are batch_stride elements apart as well.
+ */
+typedef struct {
+    void* data;
+    int32_t dtype; /* dastac_dtype */
+    int32_t space; /* dastac_memspace */
+    const dastac_structure* structure;
+    int32_t rank;
+    int32_t batch;
+    int64_t batch_stride;
+    int64_t dims[4];
+    int64_t strides[4];
+} dastac_operand;
+
+/*
+ * Evaluate a sum-of-products rule (Section 3, "Input"; Table 1) whose first operand is packed.
+ * Supported (expression, structure of in[0], dtypes):
+ *   "ij,j->i"       upper triangle (square)             f32        y = A x         (batched)
+ *   "ij,j->i"       upper triangle + swap (symmetric)   f32        y = S x
+ *   "ij,jc->ic"     band, padded diagonals              f32        C = A B
+ *   "ij,jc->ic"     upper triangle (square)             bf16 -> f32 output, fp32 accumulation
+ *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)
+ * accumulate: 0 -> out = result (the library zero-fills where it needs to), 1 -> out += result.
+ * workspace: device scratch of at least dastac_contract_workspace bytes, 256-byte aligned; may be
+ *            NULL when that size is 0.  Its contents are undefined afterwards.
+ * err_word: optional device int32; a kernel whose bounded wait expires stores a non-zero code
+ *           there and drains instead of hanging.  The caller zeroes and reads it.
+ * Floating-point sums are re-associated freely (the paper generates fast-math code), so results
+ * agree with a reference to rounding, not bit for bit.
+ */
+dastac_status dastac_contract_workspace(const char* expr, const dastac_operand* in, int32_t n_in,
+                                        const dastac_operand* out, size_t* bytes);
+dastac_status dastac_contract(const char* expr, const dastac_operand* in, int32_t n_in,
+                              const dastac_operand* out, int32_t accumulate, void* workspace,
+                              size_t workspace_bytes, int32_t* err_word, void* stream);
+
+const char* dastac_status_string(dastac_status st);
+
+/* Number of kernels this library has launched in the calling process (for launch accounting). */
+int64_t dastac_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DASTAC_H_ */

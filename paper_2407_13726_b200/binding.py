@@ -1,0 +1,269 @@
+"""Thin ctypes binding over ``libdastac.so``: argument marshalling only.
+
+Function names follow ``include/dastac.h``.  torch tensors supply device memory (or pinned host
+memory) and the current CUDA stream; every step of the computation runs in the library's kernels.
+There is no fallback: if the shared library is missing or fails to load, importing this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdastac.so")
+
+F32, BF16 = 0, 1
+MEM_DEVICE, MEM_HOST = 0, 1
+KIND_EMPTY, KIND_DENSE, KIND_UPPER, KIND_LOWER, KIND_BAND_DIAGONALS, KIND_TETRAHEDRON = range(6)
+LAYOUT_LEXICOGRAPHIC, LAYOUT_PADDED_DIAGONALS = 0, 1
+
+EXPORTS = [
+    "dastac_structure_create", "dastac_structure_destroy", "dastac_structure_count",
+    "dastac_structure_kind", "dastac_rank", "dastac_unrank", "dastac_rank_batch",
+    "dastac_unrank_batch", "dastac_pack", "dastac_unpack", "dastac_contract_workspace",
+    "dastac_contract", "dastac_status_string", "dastac_launch_count",
+]
+
+
+class DastacError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class _StructureDesc(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("nparams", ctypes.c_int32), ("nrows", ctypes.c_int32),
+                ("dims", ctypes.c_void_p), ("rows", ctypes.c_void_p), ("is_eq", ctypes.c_void_p),
+                ("params", ctypes.c_void_p), ("mirror", ctypes.c_void_p), ("layout", ctypes.c_int32)]
+
+
+class _Operand(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("space", ctypes.c_int32),
+                ("structure", ctypes.c_void_p), ("rank", ctypes.c_int32), ("batch", ctypes.c_int32),
+                ("batch_stride", ctypes.c_int64), ("dims", ctypes.c_int64 * 4),
+                ("strides", ctypes.c_int64 * 4)]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2407_13726_b200.build` "
+        "(there is no non-CUDA fallback)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+_vp, _i64, _i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+_lib.dastac_structure_create.argtypes = [ctypes.POINTER(_StructureDesc), ctypes.POINTER(_vp)]
+_lib.dastac_structure_destroy.argtypes = [_vp]
+_lib.dastac_structure_destroy.restype = None
+_lib.dastac_structure_count.argtypes = [_vp, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]
+_lib.dastac_structure_kind.argtypes = [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]
+_lib.dastac_rank.argtypes = [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i64)]
+_lib.dastac_unrank.argtypes = [_vp, _i64, ctypes.POINTER(_i32)]
+_lib.dastac_rank_batch.argtypes = [_vp, _vp, _i64, _vp, _vp]
+_lib.dastac_unrank_batch.argtypes = [_vp, _vp, _i64, _vp, _vp]
+_lib.dastac_pack.argtypes = [_vp, _i32, _vp, ctypes.POINTER(_i64), _vp, _vp]
+_lib.dastac_unpack.argtypes = [_vp, _i32, _vp, _vp, ctypes.POINTER(_i64), _vp]
+_lib.dastac_contract_workspace.argtypes = [ctypes.c_char_p, ctypes.POINTER(_Operand), _i32,
+                                           ctypes.POINTER(_Operand), ctypes.POINTER(ctypes.c_size_t)]
+_lib.dastac_contract.argtypes = [ctypes.c_char_p, ctypes.POINTER(_Operand), _i32,
+                                 ctypes.POINTER(_Operand), _i32, _vp, ctypes.c_size_t, _vp, _vp]
+_lib.dastac_status_string.argtypes = [ctypes.c_int]
+_lib.dastac_status_string.restype = ctypes.c_char_p
+_lib.dastac_launch_count.argtypes = []
+_lib.dastac_launch_count.restype = _i64
+
+
+def status_string(status: int) -> str:
+    return _lib.dastac_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(_lib.dastac_launch_count())
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise DastacError(status, where)
+
+
+def _stream() -> Optional[int]:
+    return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+class Structure:
+    """Owns a ``dastac_structure`` created from a descriptor (any object with ``dims``,
+    ``params``, ``rows``, ``is_eq``, ``mirror`` and ``padded_diagonals`` attributes)."""
+
+    def __init__(self, desc):
+        import numpy as np
+
+        dims = np.ascontiguousarray(desc.dims, dtype=np.int64)
+        params = np.ascontiguousarray(desc.params, dtype=np.int64)
+        rows = np.ascontiguousarray(desc.rows, dtype=np.int64)
+        is_eq = np.ascontiguousarray(desc.is_eq, dtype=np.uint8)
+        mirror = getattr(desc, "mirror", None)
+        mirror_arr = None if mirror is None else np.ascontiguousarray(mirror, dtype=np.int32)
+        layout = LAYOUT_PADDED_DIAGONALS if getattr(desc, "padded_diagonals", False) else LAYOUT_LEXICOGRAPHIC
+        nrows = rows.shape[0] if rows.ndim == 2 else 0
+        c = _StructureDesc(len(dims), len(params), nrows, dims.ctypes.data,
+                           rows.ctypes.data if nrows else None, is_eq.ctypes.data if nrows else None,
+                           params.ctypes.data if len(params) else None,
+                           None if mirror_arr is None else mirror_arr.ctypes.data, layout)
+        handle = _vp()
+        _check(_lib.dastac_structure_create(ctypes.byref(c), ctypes.byref(handle)),
+               "dastac_structure_create")
+        self._h = handle
+        self.rank = len(dims)
+        self.dims = [int(v) for v in dims]
+        slots, nnz = _i64(), _i64()
+        _check(_lib.dastac_structure_count(self._h, ctypes.byref(slots), ctypes.byref(nnz)),
+               "dastac_structure_count")
+        self.slots, self.nnz = int(slots.value), int(nnz.value)
+        kind, sym = _i32(), _i32()
+        _check(_lib.dastac_structure_kind(self._h, ctypes.byref(kind), ctypes.byref(sym)),
+               "dastac_structure_kind")
+        self.kind, self.symmetric = int(kind.value), bool(sym.value)
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            _lib.dastac_structure_destroy(h)
+
+    def capacity(self, dtype: torch.dtype) -> int:
+        """Elements a packed buffer must hold: ``slots`` rounded up to 16 bytes."""
+        per16 = 16 // torch.empty((), dtype=dtype).element_size()
+        return (self.slots + per16 - 1) // per16 * per16
+
+    def empty_packed(self, dtype=torch.float32, device="cuda", batch: int = 1) -> torch.Tensor:
+        cap = self.capacity(dtype)
+        shape = (cap,) if batch == 1 else (batch, cap)
+        return torch.zeros(shape, dtype=dtype, device=device)
+
+
+def structure_create(desc) -> Structure:
+    return Structure(desc)
+
+
+def structure_count(s: Structure):
+    return s.slots, s.nnz
+
+
+def rank(s: Structure, idx: Sequence[int]) -> int:
+    arr = (_i32 * s.rank)(*[int(v) for v in idx])
+    off = _i64()
+    _check(_lib.dastac_rank(s._h, arr, ctypes.byref(off)), "dastac_rank")
+    return int(off.value)
+
+
+def unrank(s: Structure, off: int):
+    arr = (_i32 * 3)()
+    _check(_lib.dastac_unrank(s._h, int(off), arr), "dastac_unrank")
+    return tuple(int(arr[k]) for k in range(s.rank))
+
+
+def rank_batch(s: Structure, idx: torch.Tensor) -> torch.Tensor:
+    assert idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous() and idx.shape[-1] == s.rank
+    n = idx.numel() // s.rank
+    off = torch.empty(n, dtype=torch.int64, device=idx.device)
+    _check(_lib.dastac_rank_batch(s._h, idx.data_ptr(), n, off.data_ptr(), _stream()),
+           "dastac_rank_batch")
+    return off
+
+
+def unrank_batch(s: Structure, off: torch.Tensor) -> torch.Tensor:
+    assert off.is_cuda and off.dtype == torch.int64 and off.is_contiguous()
+    idx = torch.empty((off.numel(), s.rank), dtype=torch.int32, device=off.device)
+    _check(_lib.dastac_unrank_batch(s._h, off.data_ptr(), off.numel(), idx.data_ptr(), _stream()),
+           "dastac_unrank_batch")
+    return idx
+
+
+def pack(s: Structure, dense: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    assert dense.is_cuda and list(dense.shape) == s.dims
+    if out is None:
+        out = s.empty_packed(dense.dtype, dense.device)
+    assert out.is_cuda and out.dtype == dense.dtype and out.numel() >= s.capacity(dense.dtype)
+    strides = (_i64 * s.rank)(*dense.stride())
+    _check(_lib.dastac_pack(s._h, _dtype_code(dense), dense.data_ptr(), strides, out.data_ptr(),
+                            _stream()), "dastac_pack")
+    return out
+
+
+def unpack(s: Structure, packed: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    assert packed.is_cuda and packed.numel() >= s.capacity(packed.dtype)
+    if out is None:
+        out = torch.empty(s.dims, dtype=packed.dtype, device=packed.device)
+    assert out.is_cuda and list(out.shape) == s.dims and out.dtype == packed.dtype
+    strides = (_i64 * s.rank)(*out.stride())
+    _check(_lib.dastac_unpack(s._h, _dtype_code(packed), packed.data_ptr(), out.data_ptr(), strides,
+                              _stream()), "dastac_unpack")
+    return out
+
+
+def _operand(t: torch.Tensor, structure: Optional[Structure], batch: int) -> _Operand:
+    op = _Operand()
+    op.data = t.data_ptr()
+    op.dtype = _dtype_code(t)
+    op.space = MEM_DEVICE if t.is_cuda else MEM_HOST
+    op.structure = structure._h if structure is not None else None
+    op.batch = batch
+    if structure is not None:
+        op.rank = structure.rank
+        for k, v in enumerate(structure.dims):
+            op.dims[k] = v
+        op.batch_stride = t.stride(0) if batch > 1 else 0
+    else:
+        shape, strides = list(t.shape), list(t.stride())
+        if batch > 1:
+            op.batch_stride = strides[0]
+            shape, strides = shape[1:], strides[1:]
+        op.rank = len(shape)
+        for k in range(len(shape)):
+            op.dims[k] = shape[k]
+            op.strides[k] = strides[k]
+    return op
+
+
+def _operands(s, packed, dense_inputs, out, batch):
+    ins = (_Operand * (1 + len(dense_inputs)))()
+    ins[0] = _operand(packed, s, batch)
+    for k, t in enumerate(dense_inputs):
+        ins[1 + k] = _operand(t, None, batch)
+    o = _operand(out, None, batch)
+    return ins, o
+
+
+def contract_workspace(expr: str, s: Structure, packed: torch.Tensor,
+                       dense_inputs: Sequence[torch.Tensor], out: torch.Tensor, batch: int = 1) -> int:
+    ins, o = _operands(s, packed, dense_inputs, out, batch)
+    nbytes = ctypes.c_size_t()
+    _check(_lib.dastac_contract_workspace(expr.encode(), ins, len(ins), ctypes.byref(o),
+                                          ctypes.byref(nbytes)), "dastac_contract_workspace")
+    return int(nbytes.value)
+
+
+def contract(expr: str, s: Structure, packed: torch.Tensor, dense_inputs: Sequence[torch.Tensor],
+             out: torch.Tensor, accumulate: bool = False, workspace: Optional[torch.Tensor] = None,
+             err_word: Optional[torch.Tensor] = None, batch: int = 1) -> torch.Tensor:
+    """Evaluate ``expr`` with ``packed`` (structure ``s``) as first operand.  Tensors may live on
+    the device or in (pinned) host memory; host tensors are staged through ``workspace``."""
+    ins, o = _operands(s, packed, dense_inputs, out, batch)
+    ws_ptr, ws_bytes = None, 0
+    if workspace is not None:
+        ws_ptr, ws_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    _check(_lib.dastac_contract(expr.encode(), ins, len(ins), ctypes.byref(o), int(accumulate),
+                                ws_ptr, ws_bytes,
+                                None if err_word is None else err_word.data_ptr(), _stream()),
+           "dastac_contract")
+    return out

@@ -1,0 +1,219 @@
+// Closed-form index maps of the recognised structure classes, evaluated in registers.
+//
+// rank  = number of points of the set that precede a point in lexicographic order, i.e. the value
+//         of the counting polynomial of the preceding-access domain (Section 4, "Access domain
+//         linearization").  Every polynomial is evaluated on its integer numerator with one exact
+//         division at the end, the way the generated code of the paper's running example does
+//         (all terms doubled, one final halving).
+// unrank = the inverse map.  The paper never inverts the polynomial; it is needed here so that a
+//         thread block can start in the middle of the packed stream.  A floating-point root gives
+//         an estimate and integer comparisons against the polynomial correct it, so the result is
+//         exact.
+#pragma once
+#include <cmath>
+#include <cstdint>
+
+#ifdef __CUDACC__
+#define DASTAC_HD __host__ __device__ __forceinline__
+#else
+#define DASTAC_HD inline
+#endif
+
+namespace dastac {
+
+enum Kind : int32_t {
+    kEmpty = 0,
+    kDense = 1,
+    kUpper = 2,
+    kLower = 3,
+    kBandDiagonals = 4,
+    kTetrahedron = 5
+};
+
+// Plain data, passed to kernels by value.
+struct IndexMap {
+    int32_t kind;
+    int32_t rank;
+    int32_t symmetric;
+    int32_t reserved;
+    int64_t dims[3];  // logical extents
+    int64_t M;        // kUpper: number of non-empty rows, min(dims[0], dims[1])
+    int64_t N;        // kUpper/kLower/kBand: columns; kTetrahedron: n
+    int64_t Q;        // kUpper: trailing dense extent (1 for a matrix)
+    int64_t w;        // kBand: half width
+    int64_t count;    // points of the set
+    int64_t slots;    // elements of the packed vector (count, or (2w+1)N with padding)
+};
+
+DASTAC_HD int64_t tri(int64_t m) { return (m * (m + 1)) >> 1; }
+DASTAC_HD int64_t tet(int64_t m) { return (m * (m + 1)) / 2 * (m + 2) / 3; }  // m(m+1)(m+2)/6
+
+// Largest r >= 0 with tri(r) <= q  (q >= 0).
+DASTAC_HD int64_t tri_root(int64_t q) {
+    int64_t r = (int64_t)((sqrt(8.0 * (double)q + 1.0) - 1.0) * 0.5);
+    if (r < 0) r = 0;
+    while (tri(r) > q) --r;
+    while (tri(r + 1) <= q) ++r;
+    return r;
+}
+
+// Largest a >= 0 with tet(a) <= q  (q >= 0).
+DASTAC_HD int64_t tet_root(int64_t q) {
+    int64_t a = (int64_t)cbrt(6.0 * (double)q);
+    if (a > 0) --a;
+    while (tet(a) > q) --a;
+    while (tet(a + 1) <= q) ++a;
+    return a;
+}
+
+// Upper triangle / trapezoid: points before row i, in units of (j) positions.
+DASTAC_HD int64_t upper_row_start(int64_t N, int64_t i) { return i * N - ((i * (i - 1)) >> 1); }
+
+// rowbase(i) + j = position of (i, j): rowbase may be used with any j >= i.
+DASTAC_HD int64_t upper_row_base(int64_t N, int64_t i) { return (i * (2 * N - i - 1)) >> 1; }
+
+// Largest i with upper_row_start(N, i) <= t, for 0 <= t < tri-like count.
+DASTAC_HD int64_t upper_row_of(int64_t N, int64_t t) {
+    const double f = 2.0 * (double)N + 1.0;
+    double disc = f * f - 8.0 * (double)t;
+    if (disc < 0.0) disc = 0.0;
+    int64_t i = (int64_t)((f - sqrt(disc)) * 0.5);
+    if (i < 0) i = 0;
+    if (i > N - 1) i = N - 1;
+    while (i > 0 && upper_row_start(N, i) > t) --i;
+    while (i + 1 < N && upper_row_start(N, i + 1) <= t) ++i;
+    return i;
+}
+
+DASTAC_HD bool in_set(const IndexMap& m, const int32_t* idx) {
+    for (int k = 0; k < m.rank; ++k)
+        if (idx[k] < 0 || idx[k] >= m.dims[k]) return false;
+    switch (m.kind) {
+        case kDense: return true;
+        case kUpper: return idx[0] <= idx[1];
+        case kLower: return idx[1] <= idx[0];
+        case kBandDiagonals: {
+            int64_t d = (int64_t)idx[1] - idx[0];
+            return d <= m.w && -d <= m.w;
+        }
+        case kTetrahedron: return idx[0] <= idx[1] && idx[1] <= idx[2];
+        default: return false;
+    }
+}
+
+// Position of a point of the set (caller guarantees membership).
+DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
+    switch (m.kind) {
+        case kDense: {
+            int64_t lin = 0;
+            for (int k = 0; k < m.rank; ++k) lin = lin * m.dims[k] + idx[k];
+            return lin;
+        }
+        case kUpper: {
+            int64_t p = upper_row_base(m.N, idx[0]) + idx[1];
+            return m.rank == 3 ? p * m.Q + idx[2] : p;
+        }
+        case kLower: return tri(idx[0]) + idx[1];
+        case kBandDiagonals: return ((int64_t)idx[1] - idx[0] + m.w) * m.N + idx[0];
+        case kTetrahedron: {
+            const int64_t n = m.N;
+            return tet(n) - tet(n - idx[0]) + tri(n - idx[0]) - tri(n - idx[1]) +
+                   ((int64_t)idx[2] - idx[1]);
+        }
+        default: return -1;
+    }
+}
+
+// Point stored at position p (0 <= p < slots).  Padding slots of the diagonal layout get column -1.
+DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
+    switch (m.kind) {
+        case kDense: {
+            for (int k = m.rank - 1; k >= 0; --k) {
+                int64_t q = p / m.dims[k];
+                idx[k] = (int32_t)(p - q * m.dims[k]);
+                p = q;
+            }
+            return;
+        }
+        case kUpper: {
+            int64_t t = p;
+            if (m.rank == 3) {
+                t = p / m.Q;
+                idx[2] = (int32_t)(p - t * m.Q);
+            }
+            int64_t i = upper_row_of(m.N, t);
+            idx[0] = (int32_t)i;
+            idx[1] = (int32_t)(i + (t - upper_row_start(m.N, i)));
+            return;
+        }
+        case kLower: {
+            int64_t i = tri_root(p);
+            idx[0] = (int32_t)i;
+            idx[1] = (int32_t)(p - tri(i));
+            return;
+        }
+        case kBandDiagonals: {
+            int64_t d = p / m.N;
+            int64_t i = p - d * m.N;
+            int64_t j = i + d - m.w;
+            idx[0] = (int32_t)i;
+            idx[1] = (j < 0 || j >= m.N) ? -1 : (int32_t)j;
+            return;
+        }
+        case kTetrahedron: {
+            const int64_t n = m.N;
+            int64_t q = m.count - 1 - p;
+            int64_t a = tet_root(q);
+            q -= tet(a);
+            int64_t b = tri_root(q);
+            int64_t c = q - tri(b);
+            idx[0] = (int32_t)(n - 1 - a);
+            idx[1] = (int32_t)(n - 1 - b);
+            idx[2] = (int32_t)(n - 1 - c);
+            return;
+        }
+        default: return;
+    }
+}
+
+// Step idx to the point stored at the next position (valid while that position exists).
+// Not defined for the padded-diagonal layout, whose slots are walked by position.
+DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {
+    switch (m.kind) {
+        case kDense: {
+            for (int k = m.rank - 1; k >= 0; --k) {
+                if (++idx[k] < m.dims[k]) return;
+                idx[k] = 0;
+            }
+            return;
+        }
+        case kUpper: {
+            if (m.rank == 3) {
+                if (++idx[2] < m.Q) return;
+                idx[2] = 0;
+            }
+            if (++idx[1] < m.N) return;
+            ++idx[0];
+            idx[1] = idx[0];
+            return;
+        }
+        case kLower: {
+            if (++idx[1] <= idx[0]) return;
+            ++idx[0];
+            idx[1] = 0;
+            return;
+        }
+        case kTetrahedron: {
+            if (++idx[2] < m.N) return;
+            if (++idx[1] >= m.N) {
+                ++idx[0];
+                idx[1] = idx[0];
+            }
+            idx[2] = idx[1];
+            return;
+        }
+        default: return;
+    }
+}
+
+}  // namespace dastac

@@ -1,0 +1,338 @@
+"""GPU parity: every entry point of the C-ABI library against the CPU oracle, element by element,
+on seeded inputs at sizes spanning several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from synth import structures as st
+
+from _util import TOL_BF16, TOL_F32, dev, packed_dev, rel_err
+
+pytestmark = pytest.mark.gpu
+
+dastac = pytest.importorskip("paper_2407_13726_b200") if torch.cuda.is_available() else None
+
+
+# ---- index maps: bit exact ------------------------------------------------------------------------
+
+INDEX_CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(97), st.upper_triangle(128, True),
+               st.lower_triangle(61), st.tetrahedron(1), st.tetrahedron(2), st.tetrahedron(48),
+               st.upper_half_cube(9, 14, 5), st.upper_half_cube(14, 9, 3), st.dense_box([5, 6, 7]),
+               st.band(50, 4), st.band(7, 0), st.upper_triangle(1000)]
+
+
+@pytest.mark.parametrize("desc", INDEX_CASES, ids=lambda d: f"{d.name}{d.dims}")
+def test_rank_unrank_batch_exhaustive(desc):
+    s = dastac.Structure(desc)
+    if desc.name == "band":
+        table = oracle.band_slot_table(desc.dims[0], desc.meta["w"])
+    else:
+        table = oracle.rank_table(desc)
+    grid = np.stack(np.meshgrid(*[np.arange(d) for d in desc.dims], indexing="ij"), -1)
+    idx = torch.from_numpy(grid.reshape(-1, desc.rank).astype(np.int32)).cuda()
+    off = dastac.rank_batch(s, idx).cpu().numpy().reshape(table.shape)
+    assert np.array_equal(off, table)
+    # out-of-box points rank to -1
+    bad = torch.tensor([[-1] * desc.rank, list(desc.dims)], dtype=torch.int32).cuda()
+    assert (dastac.rank_batch(s, bad).cpu().numpy() == -1).all()
+    # unrank of every slot
+    got = dastac.unrank_batch(s, torch.arange(s.slots, dtype=torch.int64).cuda()).cpu().numpy()
+    if desc.name == "band":
+        exp = np.full((s.slots, 2), -1, np.int32)
+        ii, jj = np.nonzero(table >= 0)
+        exp[table[ii, jj], 0] = ii
+        exp[table[ii, jj], 1] = jj
+        pad = exp[:, 0] < 0
+        exp[pad, 0] = (np.arange(s.slots) % desc.dims[0])[pad]
+        assert np.array_equal(got, exp)
+    else:
+        assert np.array_equal(got, oracle.unrank_table(desc))
+    oob = dastac.unrank_batch(s, torch.tensor([-1, s.slots], dtype=torch.int64).cuda()).cpu().numpy()
+    assert (oob == -1).all()
+
+
+@pytest.mark.parametrize("desc", [st.upper_triangle(65536, True), st.upper_triangle(8192),
+                                  st.upper_triangle(1024), st.tetrahedron(512), st.upper_triangle(2 ** 30)],
+                         ids=lambda d: f"{d.name}{d.dims[0]}")
+def test_index_maps_at_config_sizes(desc):
+    """Properties that fix the map at any size: it starts at 0, ends at count-1, moves by one
+    between lexicographic neighbours, and unrank inverts it; checked around 2^31 as well."""
+    s = dastac.Structure(desc)
+    rng = np.random.default_rng(7)
+    N = desc.dims[0]
+    probes = np.concatenate([np.array([0, 1, s.nnz - 2, s.nnz - 1, 2 ** 31 - 1, 2 ** 31, 2 ** 31 + 1]) % s.nnz,
+                             rng.integers(0, s.nnz, 1_000_000)]).astype(np.int64)
+    p = torch.from_numpy(probes).cuda()
+    idx = dastac.unrank_batch(s, p)
+    back = dastac.rank_batch(s, idx)
+    assert torch.equal(back, p)
+    idn = idx.cpu().numpy().astype(np.int64)
+    if desc.rank == 2:
+        assert ((0 <= idn[:, 0]) & (idn[:, 0] <= idn[:, 1]) & (idn[:, 1] < N)).all()
+    else:
+        assert ((0 <= idn[:, 0]) & (idn[:, 0] <= idn[:, 1]) & (idn[:, 1] <= idn[:, 2]) & (idn[:, 2] < N)).all()
+    # lexicographic successor has the next position
+    nxt = idn.copy()
+    last = desc.rank - 1
+    nxt[:, last] += 1
+    for k in range(last, 0, -1):
+        wrap = nxt[:, k] >= N
+        nxt[wrap, k - 1] += 1
+        for kk in range(k, desc.rank):
+            nxt[wrap, kk] = nxt[wrap, k - 1]
+    ok = nxt[:, 0] < N
+    succ = dastac.rank_batch(s, torch.from_numpy(nxt[ok].astype(np.int32)).cuda()).cpu().numpy()
+    assert np.array_equal(succ, probes[ok] + 1)
+    ends = torch.tensor([[0] * desc.rank, [N - 1] * desc.rank], dtype=torch.int32).cuda()
+    assert dastac.rank_batch(s, ends).cpu().tolist() == [0, s.nnz - 1]
+    # host and device maps agree
+    host = [dastac.unrank(s, int(q)) for q in probes[:300]]
+    assert np.array_equal(np.array(host), idn[:300])
+
+
+# ---- compress / decompress: bit exact -----------------------------------------------------------
+
+def _bits(shape, seed, sixteen=False):
+    rng = np.random.default_rng(seed)
+    bits = rng.integers(0, 2 ** 32, size=shape, dtype=np.uint64).astype(np.uint32)
+    flat = bits.reshape(-1)
+    flat[::7] = 0x80000000
+    flat[3::11] = 0x7FC12345
+    flat[5::13] = 0xFF800000
+    return (bits >> 16).astype(np.uint16) if sixteen else bits
+
+
+PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33), st.upper_triangle(129),
+              st.upper_triangle(1000), st.upper_triangle(130, True), st.lower_triangle(77),
+              st.tetrahedron(2), st.tetrahedron(37), st.upper_half_cube(11, 17, 3),
+              st.upper_half_cube(17, 11, 6), st.dense_box([6, 10])]
+
+
+@pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
+@pytest.mark.parametrize("desc", PACK_CASES, ids=lambda d: f"{d.name}{d.dims}")
+def test_pack_unpack_bit_exact(desc, sixteen):
+    s = dastac.Structure(desc)
+    bits = _bits(tuple(desc.dims), 11, sixteen)
+    tdt = torch.bfloat16 if sixteen else torch.float32
+    idt = torch.int16 if sixteen else torch.int32
+    d_dense = torch.from_numpy(bits.view(np.int16 if sixteen else np.int32)).cuda().view(tdt)
+    packed = dastac.pack(s, d_dense)
+    got = packed.view(idt).cpu().numpy().view(bits.dtype)
+    exp = oracle.pack(desc, bits)
+    assert np.array_equal(got[: s.nnz], exp)
+    assert (got[s.nnz:] == 0).all()
+    out = torch.full(desc.dims, float("nan"), dtype=tdt, device="cuda")
+    dastac.unpack(s, packed, out)
+    back = out.view(idt).cpu().numpy().view(bits.dtype)
+    assert np.array_equal(back, oracle.unpack(desc, exp))
+    # non-contiguous dense tensors (a padded leading dimension, then a transposed view)
+    big = torch.zeros([d + 3 for d in desc.dims], dtype=tdt, device="cuda")
+    view = big[tuple(slice(1, 1 + d) for d in desc.dims)]
+    view.copy_(d_dense)
+    assert torch.equal(dastac.pack(s, view).view(idt), packed.view(idt))
+    out2 = torch.full_like(big, float("nan"))
+    v2 = out2[tuple(slice(1, 1 + d) for d in desc.dims)]
+    dastac.unpack(s, packed, v2)
+    assert np.array_equal(v2.contiguous().view(idt).cpu().numpy().view(bits.dtype), back)
+    if desc.rank == 2 and desc.dims[0] == desc.dims[1]:
+        tr = d_dense.t().contiguous().t()     # same values, column-major strides
+        assert torch.equal(dastac.pack(s, tr).view(idt), packed.view(idt))
+
+
+@pytest.mark.parametrize("N,w", [(1, 0), (9, 2), (130, 5), (1000, 32), (64, 62)])
+def test_band_pack_unpack(N, w):
+    desc = st.band(N, w)
+    s = dastac.Structure(desc)
+    dense = _bits((N, N), 5).view(np.float32)
+    packed = dastac.pack(s, torch.from_numpy(dense.view(np.int32)).cuda().view(torch.float32))
+    exp = oracle.band_pack(N, w, dense)
+    assert np.array_equal(packed.view(torch.int32).cpu().numpy()[: s.slots], exp.reshape(-1).view(np.int32))
+    # padding content must not matter to unpack
+    slots = oracle.band_slot_table(N, w)
+    poisoned = packed.clone()
+    pad = np.ones(s.slots, bool)
+    pad[slots[slots >= 0]] = False
+    poisoned[: s.slots][torch.from_numpy(pad).cuda()] = float("nan")
+    out = dastac.unpack(s, poisoned)
+    assert np.array_equal(out.view(torch.int32).cpu().numpy(), oracle.band_unpack(N, w, exp).view(np.int32))
+
+
+# ---- contractions -----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("N", [1, 2, 3, 31, 32, 33, 127, 128, 129, 1000, 1024, 2500])
+def test_trmv(N):
+    desc = st.upper_triangle(N)
+    s = dastac.Structure(desc)
+    A = synth.dense(0, 0, (N, N))
+    x = synth.dense(0, 1, (N,))
+    ref, ref_abs = oracle.matvec(desc, A, x)
+    packed = packed_dev(s, synth.upper_triangle_stream(0, 0, N))
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    # accumulate: y += A x
+    y0 = synth.dense(0, 2, (N,))
+    y2 = dev(y0)
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y2, accumulate=True)
+    assert rel_err(y2.cpu().numpy(), ref + y0, ref_abs + np.abs(y0)) <= TOL_F32
+
+
+def test_trmv_closed_forms():
+    N = 515
+    s = dastac.Structure(st.upper_triangle(N))
+    ones = packed_dev(s, np.ones(s.nnz, np.float32))
+    y = torch.empty(N, device="cuda")
+    dastac.contract("ij,j->i", s, ones, [torch.ones(N, device="cuda")], y)
+    assert np.array_equal(y.cpu().numpy(), (N - np.arange(N)).astype(np.float32))
+
+
+def test_trmv_batched():
+    N, batch = 257, 5
+    desc = st.upper_triangle(N)
+    s = dastac.Structure(desc)
+    cap = s.capacity(torch.float32)
+    packed = torch.full((batch, cap + 4), float("nan"), device="cuda")[:, :cap]   # strided instances
+    xs = torch.empty((batch, N), device="cuda")
+    refs = []
+    for b in range(batch):
+        A = synth.dense(20 + b, 0, (N, N))
+        x = synth.dense(20 + b, 1, (N,))
+        packed[b, : s.nnz] = dev(synth.upper_triangle_stream(20 + b, 0, N))
+        xs[b] = dev(x)
+        refs.append(oracle.matvec(desc, A, x))
+    y = torch.full((batch, N), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed, [xs], y, batch=batch)
+    for b in range(batch):
+        assert rel_err(y[b].cpu().numpy(), refs[b][0], refs[b][1]) <= TOL_F32
+
+
+@pytest.mark.parametrize("N", [1, 2, 63, 64, 65, 1023, 1025, 2100, 3000])
+def test_symv(N):
+    desc = st.upper_triangle(N, symmetric=True)
+    s = dastac.Structure(desc)
+    U = synth.dense(2, 0, (N, N), dist=synth.NORMAL)
+    x = synth.dense(2, 1, (N,), dist=synth.NORMAL)
+    ref, ref_abs = oracle.symv(U, x)
+    packed = packed_dev(s, synth.upper_triangle_stream(2, 0, N, dist=synth.NORMAL))
+    ws = _workspace("ij,j->i", s, packed, [dev(x)], torch.empty(N, device="cuda"))
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y, workspace=ws)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    y0 = synth.dense(2, 2, (N,))
+    y2 = dev(y0)
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y2, accumulate=True, workspace=ws)
+    assert rel_err(y2.cpu().numpy(), ref + y0, ref_abs + np.abs(y0)) <= TOL_F32
+    # repeated runs stay within tolerance of each other (atomics may reorder sums)
+    y3 = torch.empty(N, device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y3, workspace=ws)
+    assert rel_err(y3.cpu().numpy(), y.cpu().numpy().astype(np.float64), ref_abs) <= TOL_F32
+
+
+def _workspace(expr, s, packed, ins, out, batch=1):
+    n = dastac.contract_workspace(expr, s, packed, ins, out, batch=batch)
+    return torch.empty(max(n, 1), dtype=torch.uint8, device="cuda") if n else None
+
+
+@pytest.mark.parametrize("N,w,C", [(1, 0, 1), (5, 0, 3), (40, 3, 5), (300, 32, 256), (1000, 7, 130),
+                                   (2048, 32, 64), (97, 40, 33)])
+def test_band_matmat(N, w, C):
+    desc = st.band(N, w)
+    s = dastac.Structure(desc)
+    A = synth.dense(1, 0, (N, N))
+    B = synth.dense(1, 1, (N, C))
+    ref, ref_abs = oracle.matmat(desc, A, B)
+    # padding slots are poisoned: the contraction must not depend on them
+    packed = packed_dev(s, synth.band_diagonals_stream(1, 0, N, w, pad_bits=0x7FC00000))
+    out = torch.full((N, C), float("nan"), device="cuda")
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out)
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    C0 = synth.dense(1, 2, (N, C))
+    out2 = dev(C0)
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out2, accumulate=True)
+    assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_F32
+    # padded leading dimensions
+    Bp = torch.zeros((N, C + 3), device="cuda")[:, :C]
+    Bp.copy_(dev(B))
+    outp = torch.full((N, C + 5), float("nan"), device="cuda")[:, :C]
+    dastac.contract("ij,jc->ic", s, packed, [Bp], outp)
+    assert rel_err(outp.cpu().numpy(), ref, ref_abs) <= TOL_F32
+
+
+@pytest.mark.parametrize("n,R", [(1, 1), (2, 5), (7, 32), (33, 32), (70, 40), (130, 32), (96, 7)])
+def test_mttkrp(n, R):
+    desc = st.tetrahedron(n)
+    s = dastac.Structure(desc)
+    T = synth.dense(3, 0, (n, n, n))
+    B = synth.dense(3, 1, (n, R))
+    C = synth.dense(3, 2, (n, R))
+    ref, ref_abs = oracle.mttkrp(desc, T, B, C)
+    packed = packed_dev(s, synth.tetrahedron_stream(3, 0, n))
+    out = torch.full((n, R), float("nan"), device="cuda")
+    ws = _workspace("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out)
+    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out, workspace=ws)
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    M0 = synth.dense(3, 3, (n, R))
+    out2 = dev(M0)
+    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out2, accumulate=True, workspace=ws)
+    assert rel_err(out2.cpu().numpy(), ref + M0, ref_abs + np.abs(M0)) <= TOL_F32
+
+
+@pytest.mark.parametrize("N,C", [(1, 1), (17, 9), (128, 256), (129, 64), (300, 200), (1000, 264), (512, 512)])
+def test_triangular_matmat_bf16(N, C):
+    desc = st.upper_triangle(N)
+    s = dastac.Structure(desc)
+    scale = N ** -0.5
+    A = synth.dense(4, 0, (N, N), dist=synth.NORMAL, scale=scale, bf16=True)
+    B = synth.dense(4, 1, (N, C), dist=synth.NORMAL, scale=scale, bf16=True)
+    ref, ref_abs = oracle.matmat(desc, A, B)
+    packed = packed_dev(s, synth.upper_triangle_stream(4, 0, N, dist=synth.NORMAL, scale=scale, bf16=True),
+                        dtype=torch.bfloat16)
+    out = torch.full((N, C), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = _workspace("ij,jc->ic", s, packed, [dev(B, "bf16")], out)
+    dastac.contract("ij,jc->ic", s, packed, [dev(B, "bf16")], out, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_BF16
+    C0 = synth.dense(4, 2, (N, C))
+    out2 = dev(C0)
+    dastac.contract("ij,jc->ic", s, packed, [dev(B, "bf16")], out2, accumulate=True, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_BF16
+
+
+def test_host_operands_are_staged():
+    """Host (pinned) buffers through the same call: copies in, kernel, copy out."""
+    N = 700
+    desc = st.upper_triangle(N)
+    s = dastac.Structure(desc)
+    A = synth.dense(0, 0, (N, N))
+    x = synth.dense(0, 1, (N,))
+    ref, ref_abs = oracle.matvec(desc, A, x)
+    hp = torch.zeros(s.capacity(torch.float32)).pin_memory()
+    hp[: s.nnz] = torch.from_numpy(synth.upper_triangle_stream(0, 0, N))
+    hx = torch.from_numpy(x).pin_memory()
+    hy = torch.full((N,), float("nan")).pin_memory()
+    n = dastac.contract_workspace("ij,j->i", s, hp, [hx], hy)
+    assert n >= hp.numel() * 4 + 2 * N * 4
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    dastac.contract("ij,j->i", s, hp, [hx], hy, workspace=ws)
+    torch.cuda.synchronize()
+    assert rel_err(hy.numpy(), ref, ref_abs) <= TOL_F32
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.contract("ij,j->i", s, hp, [hx], hy, workspace=ws[: n // 2])
+    assert e.value.status == 7
+
+
+def test_empty_and_degenerate_inputs():
+    s0 = dastac.Structure(st.upper_triangle(0))
+    y = torch.empty(0, device="cuda")
+    dastac.contract("ij,j->i", s0, torch.empty(0, device="cuda"), [torch.empty(0, device="cuda")], y)
+    dastac.pack(s0, torch.empty((0, 0), device="cuda"))
+    assert dastac.rank_batch(s0, torch.empty((0, 2), dtype=torch.int32, device="cuda")).numel() == 0
+    # zero right-hand-side columns
+    s = dastac.Structure(st.band(16, 2))
+    out = torch.empty((16, 0), device="cuda")
+    dastac.contract("ij,jc->ic", s, s.empty_packed(), [torch.empty((16, 0), device="cuda")], out)
+    torch.cuda.synchronize()

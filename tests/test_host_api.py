@@ -1,0 +1,203 @@
+"""Host-side checks of the C-ABI library that need no GPU: exported symbols, descriptor analysis,
+host rank/unrank against the oracle's enumeration, and argument errors (none of which launch)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from synth import structures as st
+
+import paper_2407_13726_b200 as dastac
+from paper_2407_13726_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "dastac.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(dastac_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert dastac.status_string(0) == "ok" and "unsupported" in dastac.status_string(2)
+
+
+CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(37), st.upper_triangle(12, True),
+         st.lower_triangle(1), st.lower_triangle(23), st.tetrahedron(1), st.tetrahedron(2),
+         st.tetrahedron(15), st.upper_half_cube(4, 6, 3), st.upper_half_cube(6, 4, 2),
+         st.upper_half_cube(5, 5, 1), st.dense_box([3, 4]), st.dense_box([2, 3, 4]), st.dense_box([7])]
+
+
+@pytest.mark.parametrize("desc", CASES, ids=lambda d: f"{d.name}{d.dims}")
+def test_host_rank_unrank_match_enumeration(desc):
+    s = dastac.Structure(desc)
+    table = oracle.rank_table(desc)
+    points = oracle.unrank_table(desc)
+    assert s.nnz == oracle.count(desc) == s.slots
+    for idx in np.ndindex(*desc.dims):
+        if table[idx] >= 0:
+            assert dastac.rank(s, idx) == table[idx]
+        else:
+            with pytest.raises(dastac.DastacError):
+                dastac.rank(s, idx)
+    for p, pt in enumerate(points):
+        assert dastac.unrank(s, p) == tuple(int(v) for v in pt)
+    for bad in (-1, s.slots):
+        with pytest.raises(dastac.DastacError):
+            dastac.unrank(s, bad)
+
+
+@pytest.mark.parametrize("N,w", [(1, 0), (6, 0), (9, 2), (20, 3), (12, 10)])
+def test_band_padded_diagonals_host(N, w):
+    desc = st.band(N, w)
+    s = dastac.Structure(desc)
+    assert s.kind == binding.KIND_BAND_DIAGONALS
+    slots = oracle.band_slot_table(N, w)
+    assert s.slots == (2 * w + 1) * N and s.nnz == (slots >= 0).sum()
+    seen = set()
+    for i in range(N):
+        for j in range(N):
+            if slots[i, j] >= 0:
+                assert dastac.rank(s, (i, j)) == slots[i, j]
+                assert dastac.unrank(s, int(slots[i, j])) == (i, j)
+                seen.add(int(slots[i, j]))
+    for p in range(s.slots):
+        if p not in seen:
+            assert dastac.unrank(s, p)[1] == -1   # padding slot
+
+
+def test_recognition_is_independent_of_how_rows_are_written():
+    N = 9
+    base = st.upper_triangle(N)
+    # the same set with redundant, scaled and re-ordered rows:  2j - 2i >= 0,  j <= N-1 twice, i <= j + 0
+    rows = np.array([[0, -1, 1, -1], [-2, 2, 0, 0], [1, 0, 0, 0], [0, 1, 0, 0], [0, -1, 1, -1],
+                     [-1, 0, 1, -1], [-1, 1, 0, 3]], dtype=np.int64)
+    d2 = st.Descriptor([N, N], [N], rows, np.zeros(len(rows), np.uint8))
+    s1, s2 = dastac.Structure(base), dastac.Structure(d2)
+    assert (s1.kind, s1.nnz) == (s2.kind, s2.nnz) == (binding.KIND_UPPER, N * (N + 1) // 2)
+    # strict inequality written as i - j + 1 <= 0 is a different set (strictly upper): not a class
+    strict = st.Descriptor([N, N], [N], np.array([[-1, 1, 0, -1]], dtype=np.int64), np.zeros(1, np.uint8))
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(strict)
+    assert e.value.status == 2
+    # an equality row (diagonal) is a valid descriptor but not a supported class
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(st.diagonal(5))
+    assert e.value.status == 2
+    # a row coupling three indices is not a difference bound
+    three = st.Descriptor([4, 4, 4], [4], np.array([[1, 1, -1, 0, 0]], dtype=np.int64), np.zeros(1, np.uint8))
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(three)
+    # contradictory rows give the empty set
+    empty = st.Descriptor([5, 5], [5], np.array([[1, -1, 0, -1], [-1, 1, 0, -1]], dtype=np.int64),
+                          np.zeros(2, np.uint8))
+    assert dastac.Structure(empty).nnz == 0
+    assert oracle.count(empty) == 0
+    # zero extent
+    assert dastac.Structure(st.upper_triangle(0)).nnz == 0
+    # band without the padded layout, or as wide as the matrix, is refused
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(st.band(8, 2, padded_diagonals=False))
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(st.band(8, 7))
+    # symmetric swap only on a square upper triangle
+    bad = st.lower_triangle(5)
+    bad.mirror = [1, 0]
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(bad)
+    bad = st.upper_triangle(5)
+    bad.mirror = [0, 0]
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(bad)
+    assert e.value.status == 1
+
+
+def test_config_cardinalities_and_overflow():
+    assert dastac.Structure(st.upper_triangle(1024)).nnz == 524800
+    assert dastac.Structure(st.upper_triangle(65536, True)).nnz == 2147516416
+    assert dastac.Structure(st.upper_triangle(8192)).nnz == 33558528
+    assert dastac.Structure(st.tetrahedron(512)).nnz == 22500864
+    b = dastac.Structure(st.band(32768, 32))
+    assert b.slots == 65 * 32768 and b.nnz == 65 * 32768 - 32 * 33
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(st.upper_triangle(2 ** 30 + 1))
+    assert e.value.status == 6
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(st.tetrahedron(2 ** 20 + 1))
+    assert e.value.status == 6
+
+
+def test_large_offsets_round_trip_on_host():
+    """rank(unrank(p)) == p around 2^31 and at row starts of the 65536 triangle; tetra at n=512."""
+    N = 65536
+    s = dastac.Structure(st.upper_triangle(N, True))
+    rng = np.random.default_rng(0)
+    probes = [0, 1, s.nnz - 1, s.nnz - 2, 2 ** 31 - 1, 2 ** 31, 2 ** 31 + 1]
+    probes += [int(v) for v in rng.integers(0, s.nnz, 2000)]
+    start = 0
+    for i in range(0, N, 997):          # row starts by running sum, +-1
+        start = sum(N - r for r in range(i)) if i < 3000 else None
+        if start is not None:
+            probes += [start, max(start - 1, 0), start + 1]
+    for p in probes:
+        i, j = dastac.unrank(s, p)
+        assert 0 <= i <= j < N
+        assert dastac.rank(s, (i, j)) == p
+    t = dastac.Structure(st.tetrahedron(512))
+    for p in [0, 1, t.nnz - 1] + [int(v) for v in rng.integers(0, t.nnz, 2000)]:
+        i, j, k = dastac.unrank(t, p)
+        assert 0 <= i <= j <= k < 512 and dastac.rank(t, (i, j, k)) == p
+    # the largest supported triangle
+    big = dastac.Structure(st.upper_triangle(2 ** 30))
+    for p in [0, big.nnz - 1, big.nnz // 2, big.nnz // 3]:
+        assert dastac.rank(big, dastac.unrank(big, p)) == p
+
+
+def test_argument_errors_do_not_launch():
+    before = dastac.launch_count()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    lib.dastac_contract.restype = ctypes.c_int
+    assert lib.dastac_contract(b"ij,j->i", None, 2, None, 0, None, 0, None, None) == 1
+    nbytes = ctypes.c_size_t()
+    assert lib.dastac_contract_workspace(b"ij,j->i", None, 2, None, ctypes.byref(nbytes)) == 1
+    assert lib.dastac_structure_create(None, None) == 1
+    assert lib.dastac_pack(None, 0, None, None, None, None) == 1
+    assert lib.dastac_rank_batch(None, None, ctypes.c_int64(4), None, None) == 1
+    # operand-level validation: unknown expression, wrong structure, wrong shapes
+    s = dastac.Structure(st.upper_triangle(8))
+    ins = (binding._Operand * 2)()
+    ins[0].structure = s._h
+    ins[0].rank = 2
+    ins[1].rank = 1
+    ins[1].dims[0] = 8
+    ins[1].strides[0] = 1
+    out = binding._Operand()
+    out.rank = 1
+    out.dims[0] = 8
+    out.strides[0] = 1
+    args = (ins, 2, ctypes.byref(out), ctypes.byref(nbytes))
+    assert lib.dastac_contract_workspace(b"ij,jk->ik", *args) == 3
+    assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 0 and nbytes.value == 0
+    out.dims[0] = 7
+    assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 4
+    out.dims[0] = 8
+    ins[0].dtype = 1
+    assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 3
+    ins[0].dtype = 0
+    # host operands are staged: the workspace covers them
+    ins[0].space = 1
+    ins[1].space = 1
+    out.space = 1
+    assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 0
+    assert nbytes.value == 256 + 256 + 256
+    # null data with a non-empty operand is rejected before any copy or launch
+    assert lib.dastac_contract(b"ij,j->i", ins, 2, ctypes.byref(out), 0, None, 0, None, None) == 7
+    t = dastac.Structure(st.tetrahedron(4))
+    ins[0].structure = t._h
+    assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 3
+    assert dastac.launch_count() == before
