@@ -1,0 +1,492 @@
+#!/usr/bin/env python
+"""Benchmark of the packed-layout hot path on B200.
+
+One step = one pass over every kernel of the path on seeded synthetic inputs of the five
+configurations: upper-triangular matrix-vector (single and 512-instance batch), band x dense,
+symmetric matrix-vector, tetrahedral MTTKRP, bf16 triangular x dense, plus pack and unpack of the
+bf16 triangle.  Prints one JSON line (see README/DESIGN for the keys).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--small]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "useful GFLOP/s and packed-operand HBM GB/s per kernel vs B200 roofline"
+UNIT = "GFLOP/s"
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FP32 lanes x (mul+add) x max SM clock
+
+
+def tri(m):
+    return m * (m + 1) // 2
+
+
+def tet(m):
+    return m * (m + 1) * (m + 2) // 6
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---- workload definitions ---------------------------------------------------------------------------
+
+def sizes(small: bool):
+    if small:
+        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024)
+    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192)
+
+
+def accounting(z):
+    """Useful FLOPs (structure-aware iterations x (adds + muls)) and algorithmic bytes (each operand
+    read once, the output written once) of every kernel of a step."""
+    N1, b, N2, w, C2, N3, n4, R, N5 = (z[k] for k in ("N1", "batch", "N2", "w", "C2", "N3", "n4", "R", "N5"))
+    nnz2 = (2 * w + 1) * N2 - w * (w + 1)
+    acc = {
+        "trmv": dict(flops=2 * tri(N1), bytes=4 * (tri(N1) + 2 * N1), bound="hbm"),
+        "trmv_batched": dict(flops=2 * tri(N1) * b, bytes=4 * (tri(N1) + 2 * N1) * b, bound="hbm"),
+        "bandmm": dict(flops=2 * nnz2 * C2, bytes=4 * ((2 * w + 1) * N2 + 2 * N2 * C2), bound="alu"),
+        "symv": dict(flops=2 * N3 * N3, bytes=4 * (tri(N3) + 2 * N3), bound="hbm"),
+        "mttkrp": dict(flops=3 * tet(n4) * R, bytes=4 * (tet(n4) + 3 * n4 * R), bound="alu"),
+        "trimm_bf16": dict(flops=2 * tri(N5) * N5, bytes=2 * tri(N5) + 2 * N5 * N5 + 4 * N5 * N5, bound="tensor"),
+        "pack_bf16": dict(flops=0, bytes=2 * (2 * tri(N5)), bound="hbm"),          # read the set, write it
+        "unpack_bf16": dict(flops=0, bytes=2 * (tri(N5) + N5 * N5), bound="hbm"),  # read packed, write box
+    }
+    return acc
+
+
+ORDER = ["trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
+
+
+def generate_host(z, pin):
+    """All inputs of a step as host tensors (pinned when `pin`), from the seeded generator."""
+    import torch
+    import synth
+    from synth import structures as st
+
+    def host(arr, bf16=False):
+        t = torch.from_numpy(np.ascontiguousarray(arr))
+        if bf16:
+            t = t.view(torch.int16).view(torch.bfloat16)
+        return t.pin_memory() if pin else t
+
+    def cap(n, per16):
+        return (n + per16 - 1) // per16 * per16
+
+    h = {}
+    N1, b = z["N1"], z["batch"]
+    c1 = cap(tri(N1), 4)
+    a1 = np.zeros(c1, np.float32)
+    synth.upper_triangle_stream(0, 0, N1, out=a1)
+    h["trmv"] = dict(desc=st.upper_triangle(N1), A=host(a1), ins=[host(synth.dense(0, 1, (N1,)))], out=(N1,))
+    ab = np.zeros((b, c1), np.float32)
+    xb = np.empty((b, N1), np.float32)
+    for k in range(b):  # instance k of the batch: seed 0, tensor ids 2k+2 / 2k+3
+        synth.upper_triangle_stream(0, 2 * k + 2, N1, out=ab[k])
+        xb[k] = synth.dense(0, 2 * k + 3, (N1,))
+    h["trmv_batched"] = dict(desc=st.upper_triangle(N1), A=host(ab), ins=[host(xb)], out=(b, N1), batch=b)
+    N2, w, C2 = z["N2"], z["w"], z["C2"]
+    h["bandmm"] = dict(desc=st.band(N2, w), A=host(synth.band_diagonals_stream(1, 0, N2, w).reshape(-1)),
+                       ins=[host(synth.dense(1, 1, (N2, C2)))], out=(N2, C2))
+    N3 = z["N3"]
+    a3 = np.zeros(cap(tri(N3), 4), np.float32)
+    synth.upper_triangle_stream(2, 0, N3, dist=synth.NORMAL, out=a3)
+    h["symv"] = dict(desc=st.upper_triangle(N3, symmetric=True), A=host(a3),
+                     ins=[host(synth.dense(2, 1, (N3,), dist=synth.NORMAL))], out=(N3,))
+    n4, R = z["n4"], z["R"]
+    a4 = np.zeros(cap(tet(n4), 4), np.float32)
+    synth.tetrahedron_stream(3, 0, n4, out=a4)
+    h["mttkrp"] = dict(desc=st.tetrahedron(n4), A=host(a4),
+                       ins=[host(synth.dense(3, 1, (n4, R))), host(synth.dense(3, 2, (n4, R)))], out=(n4, R))
+    N5 = z["N5"]
+    sc = N5 ** -0.5
+    a5 = np.zeros(cap(tri(N5), 8), np.uint16)
+    synth.upper_triangle_stream(4, 0, N5, dist=synth.NORMAL, scale=sc, bf16=True, out=a5)
+    h["trimm_bf16"] = dict(desc=st.upper_triangle(N5), A=host(a5, True),
+                           ins=[host(synth.dense(4, 1, (N5, N5), dist=synth.NORMAL, scale=sc, bf16=True), True)],
+                           out=(N5, N5))
+    return h
+
+
+EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
+        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic"}
+
+
+# ---- clocks ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu_index), "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        os.unlink(self.tmp.name)
+        # samples taken while the GPU was working: the upper half by power draw
+        if sm:
+            order = sorted(range(len(sm)), key=lambda k: power[k])
+            busy = [sm[k] for k in order[len(order) // 2:]]
+            return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                    "samples": len(sm), "power_w_max": max(power)}
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+
+
+# ---- the GPU arm ----------------------------------------------------------------------------------
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2407_13726_b200 as dastac
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    z = sizes(args.small)
+    acct = accounting(z)
+    t0 = time.time()
+    host = generate_host(z, pin=True)
+    gen_s = time.time() - t0
+
+    # device-resident copies
+    devs, structs = {}, {}
+    for name, hw in host.items():
+        s = dastac.Structure(hw["desc"])
+        structs[name] = s
+        d = dict(A=hw["A"].cuda(), ins=[t.cuda() for t in hw["ins"]],
+                 out=torch.empty(hw["out"], dtype=torch.float32, device="cuda"), batch=hw.get("batch", 1))
+        n = dastac.contract_workspace(EXPR[name], s, d["A"], d["ins"], d["out"], batch=d["batch"])
+        d["ws"] = torch.empty(n, dtype=torch.uint8, device="cuda") if n else None
+        devs[name] = d
+    err_word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    N5 = z["N5"]
+    dense5 = torch.empty((N5, N5), dtype=torch.bfloat16, device="cuda")
+    packed5 = structs["trimm_bf16"].empty_packed(torch.bfloat16)
+
+    def run_kernel(name):
+        if name == "pack_bf16":
+            dastac.pack(structs["trimm_bf16"], dense5, packed5)
+        elif name == "unpack_bf16":
+            dastac.unpack(structs["trimm_bf16"], devs["trimm_bf16"]["A"], dense5)
+        else:
+            d = devs[name]
+            dastac.contract(EXPR[name], structs[name], d["A"], d["ins"], d["out"], workspace=d["ws"],
+                            err_word=err_word, batch=d["batch"])
+
+    order = ["unpack_bf16" if n == "pack_bf16" else "pack_bf16" if n == "unpack_bf16" else n for n in ORDER]
+    # (unpack first so that pack reads a defined dense tensor)
+
+    def step(events=None):
+        for name in order:
+            if events is not None:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                run_kernel(name)
+                b.record()
+                events.setdefault(name, []).append((a, b))
+            else:
+                run_kernel(name)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = dastac.launch_count()
+    events = {}
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_start.record()
+    for _ in range(args.steps):
+        step(events)
+    t_end.record()
+    barrier()
+    launches = dastac.launch_count() - launches0
+    total_ms = t_start.elapsed_time(t_end)
+    clocks = sampler.stop() if rank == 0 else None
+    assert int(err_word.item()) == 0, "a device-side bounded wait expired"
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    step_flops = sum(a["flops"] for a in acct.values())
+
+    pk = peaks()
+    kernels = {}
+    for name in order:
+        ms = [a.elapsed_time(b) for a, b in events[name]]
+        avg = sum(ms) / len(ms)
+        a = acct[name]
+        k = {"us": round(avg * 1e3, 2), "us_min": round(min(ms) * 1e3, 2),
+             "gbs": round(a["bytes"] / avg / 1e6, 1), "useful_gflops": round(a["flops"] / avg / 1e6, 1),
+             "bytes": a["bytes"], "flops": a["flops"], "bound": a["bound"],
+             "hbm_frac_measured": round(a["bytes"] / avg / 1e6 / pk["hbm_gbs"], 4),
+             "hbm_frac_nominal_8000": round(a["bytes"] / avg / 1e6 / 8000.0, 4)}
+        if a["bound"] == "alu":
+            k["alu_frac"] = round(a["flops"] / avg / 1e9 / FP32_ALU_PEAK_TFLOPS, 4)
+        if a["bound"] == "tensor":
+            k["tensor_frac_measured"] = round(a["flops"] / avg / 1e9 / pk["bf16_tflops"], 4)
+            k["tensor_frac_nominal_2250"] = round(a["flops"] / avg / 1e9 / 2250.0, 4)
+        kernels[name] = k
+    dominant = max(order, key=lambda n: kernels[n]["us"])
+    dk, da = kernels[dominant], acct[dominant]
+    if da["bound"] == "tensor":
+        # timed inside a long step under the power cap: the sustained figure is the denominator
+        peak = pk["bf16_tflops_sustained"]
+        roof = {"bound": "tensor", "achieved": round(dk["useful_gflops"] / 1e3, 2), "peak": peak, "unit": "TFLOP/s"}
+    elif da["bound"] == "alu":
+        roof = {"bound": "alu", "achieved": round(dk["useful_gflops"] / 1e3, 2), "peak": round(FP32_ALU_PEAK_TFLOPS, 2),
+                "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": dk["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = round(roof["achieved"] / roof["peak"], 4)
+    roof["kernel"] = dominant
+    roof["peak_source"] = pk["source"]
+    roof["traffic"] = TRAFFIC.get(dominant) if not args.small else None
+
+    # ---- end to end: host buffers through the same C-ABI call, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        hd = {}
+        h2d = d2h = 0
+        for name, hw in host.items():
+            out_h = torch.empty(hw["out"], dtype=torch.float32).pin_memory()
+            n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1))
+            hd[name] = dict(out=out_h, ws=torch.empty(n, dtype=torch.uint8, device="cuda"))
+            h2d += hw["A"].numel() * hw["A"].element_size() + sum(t.numel() * t.element_size() for t in hw["ins"])
+            d2h += out_h.numel() * 4
+
+        def e2e_step():
+            for name in ORDER:
+                if name in hd:
+                    hw = host[name]
+                    dastac.contract(EXPR[name], structs[name], hw["A"], hw["ins"], hd[name]["out"],
+                                    workspace=hd[name]["ws"], err_word=err_word, batch=hw.get("batch", 1))
+
+        e2e_flops = sum(acct[n]["flops"] for n in hd)
+        e_steps = max(1, min(args.steps, 3))
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if world > 1:
+            tt = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e_ms = float(tt.item())
+        e2e = {"value": round(world * e2e_flops * e_steps / e_ms / 1e6, 1), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e_steps,
+               "ms_per_step": round(e_ms / e_steps, 3),
+               "note": "five contractions with pinned host operands staged by dastac_contract; pack/unpack legs excluded"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(z, budget=args.cpu_rows_scale)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(world * step_flops / ms_per_step / 1e6, 1), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
+            "data": "synthetic",
+            "config": {"workload": "all five configs per step: " + json.dumps(z, separators=(",", ":")),
+                       "small": bool(args.small),
+                       "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
+                             "(the 8.6 GB symmetric stream runs once per step)",
+                       "replicas": "each rank runs the whole step on its own GPU; no collective"},
+            "roofline": roof, "kernels": kernels, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "cpu_baseline": cpu, "input_generation_s": round(gen_s, 1),
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) per launch from ncu captures, by kernel; None until captured for the
+# current kernel version.
+TRAFFIC = {}
+
+
+# ---- the CPU oracle arm -----------------------------------------------------------------------------
+
+def oracle_sample(z, scale=1.0):
+    """A bounded sample of every config, evaluated by the oracle as it stands.  Returns
+    (useful_flops, seconds, description)."""
+    import oracle
+    import synth
+    from synth import structures as st
+
+    flops, secs, parts = 0, 0.0, []
+
+    def timed(fn):
+        t = time.perf_counter()
+        fn()
+        return time.perf_counter() - t
+
+    rows = lambda n, k: np.unique(np.linspace(0, n - 1, max(1, int(k * scale))).astype(np.int64))  # noqa: E731
+    N1 = z["N1"]
+    A = synth.dense(0, 0, (N1, N1))
+    x = synth.dense(0, 1, (N1,))
+    secs += timed(lambda: oracle.matvec(st.upper_triangle(N1), A, x))
+    flops += 2 * tri(N1)
+    parts.append(f"cfg1 all {N1} rows")
+    N2, w, C2 = z["N2"], z["w"], z["C2"]
+    sel = rows(N2, 256)
+    Ar = np.stack([synth.linear_slice(1, 0, int(i) * N2, N2) for i in sel])
+    B = synth.dense(1, 1, (N2, C2))
+    secs += timed(lambda: oracle.matmat(st.band(N2, w), Ar, B, sel=sel))
+    flops += sum(2 * (min(N2 - 1, int(i) + w) - max(0, int(i) - w) + 1) * C2 for i in sel)
+    parts.append(f"cfg2 {len(sel)} rows")
+    N3 = z["N3"]
+    sel = rows(N3, 2048)
+    Sr = np.stack([synth.symmetric_row(2, 0, N3, int(i), dist=synth.NORMAL) for i in sel])
+    x3 = synth.dense(2, 1, (N3,), dist=synth.NORMAL)
+    secs += timed(lambda: oracle.matvec(st.dense_box([N3, N3]), Sr, x3, sel=sel))
+    flops += 2 * N3 * len(sel)
+    parts.append(f"cfg3 {len(sel)} rows")
+    n4, R = z["n4"], z["R"]
+    sel = rows(n4, 24)
+    Ts = np.stack([synth.linear_slice(3, 0, int(i) * n4 * n4, n4 * n4).reshape(n4, n4) for i in sel])
+    Bm, Cm = synth.dense(3, 1, (n4, R)), synth.dense(3, 2, (n4, R))
+    secs += timed(lambda: oracle.mttkrp(st.tetrahedron(n4), Ts, Bm, Cm, sel=sel))
+    flops += sum(3 * tri(n4 - int(i)) * R for i in sel)
+    parts.append(f"cfg4 {len(sel)} slabs")
+    N5 = z["N5"]
+    sc = N5 ** -0.5
+    sel = rows(N5, 16)
+    A5 = np.stack([synth.linear_slice(4, 0, int(i) * N5, N5, dist=synth.NORMAL, scale=sc, bf16=True) for i in sel])
+    B5 = synth.dense(4, 1, (N5, N5), dist=synth.NORMAL, scale=sc, bf16=True)
+    secs += timed(lambda: oracle.matmat(st.upper_triangle(N5), A5, B5, sel=sel))
+    flops += sum(2 * (N5 - int(i)) * N5 for i in sel)
+    parts.append(f"cfg5 {len(sel)} rows x {N5} cols")
+    return flops, secs, "rows spread evenly over the outer index: " + ", ".join(parts)
+
+
+def cpu_baseline(z, budget=1.0):
+    import oracle
+
+    flops, secs, desc = oracle_sample(z, budget)
+    return {"value": round(flops / secs / 1e9, 3), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": desc, "seconds": round(secs, 2)}
+
+
+def run_reference(args):
+    import oracle
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    z = sizes(args.small)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(z, 0.05)
+    tot_f, tot_s, desc = 0, 0.0, ""
+    steps = max(1, min(args.steps, 3))
+    for _ in range(steps):
+        f, s, desc = oracle_sample(z, args.cpu_rows_scale)
+        tot_f += f
+        tot_s += s
+    val = round(tot_f / tot_s / 1e9, 3)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(tot_s / steps * 1e3, 2),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "all five configs per step: " + json.dumps(z, separators=(",", ":")),
+                   "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--small", action="store_true", help="reduced sizes for a quick functional run (not a result)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-rows-scale", type=float, default=1.0)
+    args = ap.parse_args()
+    import __graft_entry__
+
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        __graft_entry__.build()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

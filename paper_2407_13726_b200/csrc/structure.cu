@@ -229,6 +229,13 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
         const bool full = hi[0] == m.dims[0] - 1 && hi[1] == m.dims[1] - 1 && hi[2] == m.dims[2] - 1;
         if (padded) return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
         if (false) {
+        } else if (full && m.dims[0] == m.dims[1] && m.dims[1] == m.dims[2] && ordered_pair(0, 1) &&
+                   ordered_pair(1, 2) && b.D[0][2] == 0 && b.D[2][0] == hi[2] - lo[0]) {
+            if (m.dims[0] > (int64_t(1) << 20)) return DASTAC_ERR_OVERFLOW;
+            m.kind = kTetrahedron;
+            m.N = m.dims[0];
+            m.count = tet(m.N);
+            matched = true;
         } else if (hi[1] == m.dims[1] - 1 && hi[2] == m.dims[2] - 1 && ordered_pair(0, 1) &&
                    free_pair(0, 2) && free_pair(1, 2) &&
                    hi[0] == (m.dims[0] < m.dims[1] ? m.dims[0] : m.dims[1]) - 1) {
@@ -237,13 +244,6 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
             m.M = hi[0] + 1;
             m.Q = m.dims[2];
             m.count = upper_row_start(m.N, m.M) * m.Q;
-            matched = true;
-        } else if (full && m.dims[0] == m.dims[1] && m.dims[1] == m.dims[2] && ordered_pair(0, 1) &&
-                   ordered_pair(1, 2) && b.D[0][2] == 0 && b.D[2][0] == hi[2] - lo[0]) {
-            if (m.dims[0] > (int64_t(1) << 20)) return DASTAC_ERR_OVERFLOW;
-            m.kind = kTetrahedron;
-            m.N = m.dims[0];
-            m.count = tet(m.N);
             matched = true;
         } else if (full && free_pair(0, 1) && free_pair(0, 2) && free_pair(1, 2)) {
             m.kind = kDense;
