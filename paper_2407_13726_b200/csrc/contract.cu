@@ -100,7 +100,7 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         if (in[1].dims[0] != p.N || out->dims[0] != m.dims[0] || out->dims[1] != p.ncols)
             return DASTAC_ERR_SHAPE;
         if (p.ncols > 1 && (in[1].strides[1] != 1 || out->strides[1] != 1)) return DASTAC_ERR_SHAPE;
-        if (tri_bf16) p.scratch = trimm_workspace_bytes(m, p.ncols);
+        if (tri_bf16) p.scratch = trimm_workspace_bytes(m, p.ncols, in[1].strides[0]);
     } else {
         if (p.batch != 1 || batch_of(in[1]) != 1 || batch_of(in[2]) != 1 || batch_of(*out) != 1)
             return DASTAC_ERR_UNSUPPORTED_EXPR;

@@ -1,5 +1,32 @@
-// C = A B for a packed upper-triangular bf16 A and a dense row-major bf16 B, fp32 accumulation and
-// fp32 output.  (First version: plain CUDA-core loops; the tensor-core pipeline replaces it.)
+// C = A B for a packed upper-triangular bf16 A (row-packed, position rowbase(i) + j) and a dense
+// row-major bf16 B, fp32 accumulation in tensor memory, fp32 output.  The paper has no tensor-core
+// kernel; this is its SpMV_UT / TTM_UT access pattern (Table 1) widened to a dense right-hand
+// side and mapped on tcgen05.
+//
+// Tiling.  An output tile is 128 rows x 256 columns.  Row block I only needs K blocks (64 columns
+// of A, 64 rows of B) from the diagonal on: kb = 2I .. ceil(N/64)-1, so the executed MMA work is
+// the triangle plus half a tile per row block.  The two K blocks that cross the diagonal are
+// zero-masked while A is staged; all others take the unmasked path.  Tiles are ordered by
+// decreasing K length and dealt round-robin to one persistent CTA per SM.
+//
+// Roles inside a CTA (14 warps):
+//   warps 0-3   epilogue: tcgen05.ld of the accumulator (warp w owns TMEM lanes 32w..32w+31),
+//               128-bit stores to C
+//   warp  4     one lane issues the TMA loads of B (four 64x64 boxes per K block, 128B swizzle)
+//   warp  5     allocates tensor memory; one lane issues tcgen05.mma (M128 N256 K16, four per
+//               K block) and the commits that release stages / publish accumulators
+//   warps 6-13  stage A: the packed row pitch changes with the row, so no tensor map can
+//               describe A and row starts are only 2-byte aligned.  Eight lanes cover one row of
+//               a K block with aligned 128-bit loads; the row's constant misalignment (0..7
+//               elements, a function of rowbase(i) only) is removed in registers with a
+//               two-level word select and a funnel shift, and the 16 bytes are stored at the
+//               swizzled position the K-major UMMA descriptor expects.
+// Accumulators are double buffered in tensor memory (2 x 256 columns) so the epilogue of a tile
+// overlaps the MMAs of the next.
+//
+// Every wait on an mbarrier is bounded by a clock budget; on expiry the thread records a code in
+// the error word and the CTA drains: nothing can spin forever.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -7,45 +34,511 @@
 namespace dastac {
 namespace {
 
-constexpr int kTile = 16;
+constexpr int kTileM = 128, kTileN = 256, kBlockK = 64;
+constexpr int kStages = 4;
+constexpr int kABytes = kTileM * kBlockK * 2;  // 16 KiB
+constexpr int kBBytes = kBlockK * kTileN * 2;  // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kEpilogueWarps = 4, kProducerWarps = 8;
+constexpr int kWarpTma = 4, kWarpMma = 5, kWarpProducer0 = 6;
+constexpr int kThreads = (kWarpProducer0 + kProducerWarps) * 32;  // 448
+constexpr int kTmemCols = 512;
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long kWaitBudget = 4000000000LL;  // clock cycles (~2 s) before a wait gives up
 
-__global__ void __launch_bounds__(kTile * kTile)
-trimm_simt_kernel(int64_t N, const __nv_bfloat16* __restrict__ A,
-                  const __nv_bfloat16* __restrict__ B, int64_t ldb, float* __restrict__ C,
-                  int64_t ldc, int64_t ncols, int accumulate) {
-    __shared__ float As[kTile][kTile + 1];
-    __shared__ float Bs[kTile][kTile + 1];
-    const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
-    const int64_t i = blockIdx.y * (int64_t)kTile + ty, c = blockIdx.x * (int64_t)kTile + tx;
-    const int64_t i_first = blockIdx.y * (int64_t)kTile;
-    const int64_t base = i < N ? upper_row_base(N, i) : 0;
-    float acc = 0.f;
-    for (int64_t j0 = i_first; j0 < N; j0 += kTile) {  // columns left of the block's first row are zero
-        const int64_t ja = j0 + tx;
-        As[ty][tx] = (i < N && ja < N && ja >= i) ? __bfloat162float(A[base + ja]) : 0.f;
-        const int64_t jb = j0 + ty;
-        Bs[ty][tx] = (jb < N && c < ncols) ? __bfloat162float(B[jb * ldb + c]) : 0.f;
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < kTile; ++k) acc = fmaf(As[ty][k], Bs[k][tx], acc);
-        __syncthreads();
+enum ErrCode : int32_t { kErrFullA = 1, kErrFullB = 2, kErrEmpty = 3, kErrTmemFull = 4, kErrTmemEmpty = 5 };
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: returns false (and records `code`) when the clock budget runs out or when another
+// thread of the CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* err_word, int32_t code) {
+    if (mbar_test(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_test(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitBudget) {
+            *abort_flag = 1;
+            if (err_word) atomicCAS(err_word, 0, code);
+            return false;
+        }
     }
-    if (i < N && c < ncols) C[i * ldc + c] = accumulate ? C[i * ldc + c] + acc : acc;
+}
+// Warp-wide form: lane 0 waits and the verdict is shared, so a warp never splits on a timeout.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* err_word, int32_t code, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, err_word, code) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
+// (all in 16-byte units), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;  // version
+    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulator, bf16 A (K-major) and bf16 B (MN-major), M128 N256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                            ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+
+struct Params {
+    const __nv_bfloat16* A;
+    float* C;
+    int64_t N, ncols, ldc;
+    int64_t cap_elems;   // capacity of the packed buffer in elements (multiple of 8)
+    int32_t row_blocks, col_blocks, k_blocks;
+    int32_t accumulate;
+    int32_t vector_store;  // C allows 128-bit stores
+    int32_t* err_word;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = (uint64_t*)(smem + (size_t)kStages * kStageBytes);
+    // barrier slots: full_a[s], full_b[s], empty[s], tmem_full[2], tmem_empty[2]
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_a = [&](int s) { return bar0 + 8u * s; };
+    auto full_b = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto empty = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
+    auto tmem_full = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
+    auto tmem_empty = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
+    auto drain_bar = [&]() { return bar0 + 8u * (3 * kStages + 4); };
+    uint32_t* tmem_slot = (uint32_t*)(bars + 3 * kStages + 5);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_a(s), kProducerWarps);
+            mbar_init(full_b(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tmem_full(a), 1);
+            mbar_init(tmem_empty(a), kEpilogueWarps);
+        }
+        mbar_init(drain_bar(), 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == kWarpMma) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int64_t tiles = (int64_t)p.row_blocks * p.col_blocks;
+
+    if (warp == kWarpTma) {
+        // ---- B producer: TMA -----------------------------------------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+                const int I = (int)(t / p.col_blocks), J = (int)(t - (int64_t)I * p.col_blocks);
+                for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (it >= kStages &&
+                        !mbar_wait(empty(s), ((it / kStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t dst = smem_base + s * kStageBytes + kABytes;
+                    mbar_arrive_expect_tx(full_b(s), kBBytes);
+#pragma unroll
+                    for (int q = 0; q < kTileN / 64; ++q)
+                        tma_load_2d(dst + q * (kBlockK * 128), &tmap_b, J * kTileN + q * 64, kb * kBlockK, full_b(s));
+                }
+            }
+            // Drain: copies already issued must land before the CTA's shared memory is released.
+            if (!ok) {
+                const long long t0 = clock64();
+                for (int s = 0; s < kStages; ++s) {
+                    const uint32_t issued = it / kStages + ((int)(it % kStages) > s ? 1 : 0);
+                    if (issued == 0) continue;
+                    while (!mbar_test(full_b(s), (issued - 1) & 1) && clock64() - t0 < kWaitBudget) {
+                    }
+                }
+            }
+        }
+    } else if (warp == kWarpMma) {
+        // ---- MMA issuer ------------------------------------------------------------------------
+        if (lane == 0) {
+            uint32_t it = 0, tile_n = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++tile_n) {
+                const int I = (int)(t / p.col_blocks);
+                const int acc = tile_n & 1;
+                if (tile_n >= 2 &&
+                    !mbar_wait(tmem_empty(acc), ((tile_n >> 1) - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kTileN;
+                for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t par = (it / kStages) & 1;
+                    if (!mbar_wait(full_a(s), par, abort_flag, p.err_word, kErrFullA) ||
+                        !mbar_wait(full_b(s), par, abort_flag, p.err_word, kErrFullB)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + s * kStageBytes;
+                    const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                    for (int k16 = 0; k16 < kBlockK / 16; ++k16) {
+                        // A: K-major, 8-row groups 1024 B apart; 16 K elements = 32 B further.
+                        const uint64_t da = smem_desc(a_addr + k16 * 32, 16, 1024);
+                        // B: MN-major, 64-column groups 8192 B apart (leading), 8-row K groups
+                        // 1024 B apart (stride); 16 K rows = 2048 B further.
+                        const uint64_t db = smem_desc(b_addr + k16 * 2048, kBlockK * 128, 1024);
+                        umma_bf16(d_tmem, da, db, kIdesc, (kb > 2 * I || k16 > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty(s));
+                }
+                if (ok) umma_commit(tmem_full(acc));
+            }
+            if (!ok) {
+                // MMAs already issued still read shared memory: wait (bounded) until they retire.
+                umma_commit(drain_bar());
+                const long long t0 = clock64();
+                while (!mbar_test(drain_bar(), 0) && clock64() - t0 < kWaitBudget) {
+                }
+            }
+        }
+    } else if (warp >= kWarpProducer0) {
+        // ---- A producers -------------------------------------------------------------------------
+        const int pw = warp - kWarpProducer0;
+        const int sub = lane >> 3, c = lane & 7;  // row within a 4-row group, 16-byte chunk in the row
+        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+            const int I = (int)(t / p.col_blocks);
+            // the four rows of the tile this lane serves, constant over the K loop
+            int64_t base[4];   // rowbase(i) + 8c, in elements
+            int row[4];
+            uint32_t soff[4];  // swizzled byte offset of the lane's 16 bytes inside a stage
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const int r = 4 * (pw + kProducerWarps * g) + sub;  // 0..127
+                const int64_t i = (int64_t)I * kTileM + r;
+                row[g] = (int)i;
+                base[g] = (i < p.N ? upper_row_base(p.N, i) : 0) + 8 * c;
+                soff[g] = (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4));
+            }
+            for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
+                const int s = it % kStages;
+                const int64_t k0 = (int64_t)kb * kBlockK;
+                // issue the global loads of this K block before waiting for the stage
+                uint4 lo[4], ninth[4];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    const int64_t e0 = base[g] + k0;       // first element of the lane's chunk
+                    const int64_t a0 = e0 & ~(int64_t)7;   // aligned down to 16 bytes
+                    const bool live = row[g] < p.N;
+                    lo[g] = (live && a0 + 8 <= p.cap_elems) ? __ldg((const uint4*)(p.A + a0)) : zero4;
+                    ninth[g] = (live && c == 7 && (e0 & 7) && a0 + 16 <= p.cap_elems)
+                                   ? __ldg((const uint4*)(p.A + a0 + 8)) : zero4;
+                }
+                if (it >= kStages &&
+                    !mbar_wait_warp(empty(s), ((it / kStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty, lane)) {
+                    ok = false;
+                    break;
+                }
+                uint8_t* stage = smem + (size_t)s * kStageBytes;
+                const bool masked = (kb < 2 * I + 2) || (k0 + kBlockK > p.N);
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    // neighbour's chunk = the 16 bytes that follow this lane's aligned chunk
+                    uint4 hi;
+                    hi.x = __shfl_down_sync(0xffffffffu, lo[g].x, 1);
+                    hi.y = __shfl_down_sync(0xffffffffu, lo[g].y, 1);
+                    hi.z = __shfl_down_sync(0xffffffffu, lo[g].z, 1);
+                    hi.w = __shfl_down_sync(0xffffffffu, lo[g].w, 1);
+                    if (c == 7) hi = ninth[g];
+                    const uint32_t se = (uint32_t)((base[g] + k0) & 7);  // misalignment in elements
+                    const bool q1 = se & 2, q2 = se & 4;
+                    const uint32_t sh = (se & 1) * 16;
+                    const uint32_t W0 = lo[g].x, W1 = lo[g].y, W2 = lo[g].z, W3 = lo[g].w;
+                    const uint32_t W4 = hi.x, W5 = hi.y, W6 = hi.z, W7 = hi.w;
+                    const uint32_t X0 = q1 ? W1 : W0, X1 = q1 ? W2 : W1, X2 = q1 ? W3 : W2, X3 = q1 ? W4 : W3,
+                                   X4 = q1 ? W5 : W4, X5 = q1 ? W6 : W5, X6 = q1 ? W7 : W6;
+                    const uint32_t T0 = q2 ? X2 : X0, T1 = q2 ? X3 : X1, T2 = q2 ? X4 : X2, T3 = q2 ? X5 : X3,
+                                   T4 = q2 ? X6 : X4;
+                    uint4 out;
+                    out.x = __funnelshift_r(T0, T1, sh);
+                    out.y = __funnelshift_r(T1, T2, sh);
+                    out.z = __funnelshift_r(T2, T3, sh);
+                    out.w = __funnelshift_r(T3, T4, sh);
+                    if (masked) {
+                        // keep column j only if row <= j < N
+                        const int64_t j0 = k0 + 8 * c;
+                        uint32_t* w = &out.x;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const int64_t j = j0 + e;
+                            if (j < row[g] || j >= p.N) w[e >> 1] &= (e & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+                        }
+                    }
+                    *(uint4*)(stage + soff[g]) = out;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_a(s));
+            }
+        }
+    } else {
+        // ---- epilogue -----------------------------------------------------------------------------
+        uint32_t tile_n = 0;
+        bool ok = true;
+        for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++tile_n) {
+            const int I = (int)(t / p.col_blocks), J = (int)(t - (int64_t)I * p.col_blocks);
+            const int acc = tile_n & 1;
+            if (!mbar_wait_warp(tmem_full(acc), (tile_n >> 1) & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const int64_t i = (int64_t)I * kTileM + warp * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + acc * kTileN;
+            float* crow = p.C + i * p.ldc + (int64_t)J * kTileN;
+#pragma unroll 1
+            for (int cc = 0; cc < kTileN / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(taddr + cc * 32, r);
+                tmem_ld_wait();
+                const int64_t col0 = (int64_t)J * kTileN + cc * 32;
+                if (i < p.N) {
+                    if (p.vector_store && col0 + 32 <= p.ncols) {
+                        float4* dst = (float4*)(crow + cc * 32);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                   __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                            if (p.accumulate) {
+                                const float4 old = dst[v];
+                                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                            }
+                            dst[v] = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 32; ++v)
+                            if (col0 + v < p.ncols) {
+                                float o = __uint_as_float(r[v]);
+                                if (p.accumulate) o += crow[cc * 32 + v];
+                                crow[cc * 32 + v] = o;
+                            }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tmem_empty(acc));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kWarpMma) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---- host ------------------------------------------------------------------------------------------
+
+__global__ void repitch_bf16_kernel(const uint16_t* __restrict__ src, int64_t lds, uint16_t* __restrict__ dst,
+                                    int64_t ldd, int64_t rows, int64_t cols) {
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < rows * ldd;
+         t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = t / ldd, c = t - r * ldd;
+        dst[t] = c < cols ? src[r * lds + c] : (uint16_t)0;
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
 }
 
 }  // namespace
 
-size_t trimm_workspace_bytes(const IndexMap&, int64_t) { return 0; }
+// B rows whose pitch is not a multiple of 16 bytes cannot be described by a tensor map: they are
+// first copied into the workspace with the pitch rounded up to 8 elements.
+size_t trimm_workspace_bytes(const IndexMap& m, int64_t ncols, int64_t ldb) {
+    if (m.N == 0 || ncols == 0 || ldb % 8 == 0) return 0;
+    return (size_t)(m.N * round_up(ncols, 8) * 2);
+}
 
-dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B, int64_t ldb,
-                                float* C, int64_t ldc, int64_t ncols, int accumulate, void*,
-                                int32_t*, cudaStream_t st) {
+dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B, int64_t ldb, float* C,
+                                int64_t ldc, int64_t ncols, int accumulate, void* workspace,
+                                int32_t* err_word, cudaStream_t st) {
     const int64_t N = m.N;
     if (N == 0 || ncols == 0) return DASTAC_OK;
-    const int64_t gx = (ncols + kTile - 1) / kTile, gy = (N + kTile - 1) / kTile;
-    if (gy > 65535 || gx > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
-    trimm_simt_kernel<<<dim3((unsigned)gx, (unsigned)gy), kTile * kTile, 0, st>>>(
-        N, (const __nv_bfloat16*)A, (const __nv_bfloat16*)B, ldb, C, ldc, ncols, accumulate);
+    // TMA needs a 16-byte aligned base and row pitch for B.
+    if (!aligned16(B)) return DASTAC_ERR_ALIGNMENT;
+    if (ldb % 8 != 0) {
+        if (!workspace) return DASTAC_ERR_WORKSPACE;
+        const int64_t ldd = round_up(ncols, 8);
+        int64_t blocks = (N * ldd + 255) / 256;
+        if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
+        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, (uint16_t*)workspace,
+                                                             ldd, N, ncols);
+        dastac_status rs = launch_status();
+        if (rs != DASTAC_OK) return rs;
+        B = workspace;
+        ldb = ldd;
+    }
+    if (ncols > 0x7fffffffLL || N > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return DASTAC_ERR_CUDA;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)ncols, (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBlockK};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DASTAC_ERR_CUDA;
+
+    Params p;
+    p.A = (const __nv_bfloat16*)A;
+    p.C = C;
+    p.N = N;
+    p.ncols = ncols;
+    p.ldc = ldc;
+    p.cap_elems = round_up(m.slots, 8);
+    p.row_blocks = (int32_t)((N + kTileM - 1) / kTileM);
+    p.col_blocks = (int32_t)((ncols + kTileN - 1) / kTileN);
+    p.k_blocks = (int32_t)((N + kBlockK - 1) / kBlockK);
+    p.accumulate = accumulate;
+    p.vector_store = ((ldc & 3) == 0) && aligned16(C);
+    p.err_word = err_word;
+
+    static bool attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(trimm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kSmemBytes) != cudaSuccess)
+            return DASTAC_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const int64_t tiles = (int64_t)p.row_blocks * p.col_blocks;
+    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    trimm_tcgen05_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmap, p);
     return launch_status();
 }
 
