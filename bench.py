@@ -78,7 +78,7 @@ def accounting(z):
 ORDER = ["trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
 
 
-def generate_host(z, pin):
+def generate_host(z, pin, only=None):
     """All inputs of a step as host tensors (pinned when `pin`), from the seeded generator."""
     import torch
     import synth
@@ -94,37 +94,44 @@ def generate_host(z, pin):
         return (n + per16 - 1) // per16 * per16
 
     h = {}
+    want = lambda name: only is None or name in only or (name == "trimm_bf16" and only & {"pack_bf16", "unpack_bf16"})  # noqa: E731
     N1, b = z["N1"], z["batch"]
     c1 = cap(tri(N1), 4)
-    a1 = np.zeros(c1, np.float32)
-    synth.upper_triangle_stream(0, 0, N1, out=a1)
-    h["trmv"] = dict(desc=st.upper_triangle(N1), A=host(a1), ins=[host(synth.dense(0, 1, (N1,)))], out=(N1,))
-    ab = np.zeros((b, c1), np.float32)
-    xb = np.empty((b, N1), np.float32)
-    for k in range(b):  # instance k of the batch: seed 0, tensor ids 2k+2 / 2k+3
-        synth.upper_triangle_stream(0, 2 * k + 2, N1, out=ab[k])
-        xb[k] = synth.dense(0, 2 * k + 3, (N1,))
-    h["trmv_batched"] = dict(desc=st.upper_triangle(N1), A=host(ab), ins=[host(xb)], out=(b, N1), batch=b)
-    N2, w, C2 = z["N2"], z["w"], z["C2"]
-    h["bandmm"] = dict(desc=st.band(N2, w), A=host(synth.band_diagonals_stream(1, 0, N2, w).reshape(-1)),
-                       ins=[host(synth.dense(1, 1, (N2, C2)))], out=(N2, C2))
-    N3 = z["N3"]
-    a3 = np.zeros(cap(tri(N3), 4), np.float32)
-    synth.upper_triangle_stream(2, 0, N3, dist=synth.NORMAL, out=a3)
-    h["symv"] = dict(desc=st.upper_triangle(N3, symmetric=True), A=host(a3),
-                     ins=[host(synth.dense(2, 1, (N3,), dist=synth.NORMAL))], out=(N3,))
-    n4, R = z["n4"], z["R"]
-    a4 = np.zeros(cap(tet(n4), 4), np.float32)
-    synth.tetrahedron_stream(3, 0, n4, out=a4)
-    h["mttkrp"] = dict(desc=st.tetrahedron(n4), A=host(a4),
-                       ins=[host(synth.dense(3, 1, (n4, R))), host(synth.dense(3, 2, (n4, R)))], out=(n4, R))
-    N5 = z["N5"]
-    sc = N5 ** -0.5
-    a5 = np.zeros(cap(tri(N5), 8), np.uint16)
-    synth.upper_triangle_stream(4, 0, N5, dist=synth.NORMAL, scale=sc, bf16=True, out=a5)
-    h["trimm_bf16"] = dict(desc=st.upper_triangle(N5), A=host(a5, True),
-                           ins=[host(synth.dense(4, 1, (N5, N5), dist=synth.NORMAL, scale=sc, bf16=True), True)],
-                           out=(N5, N5))
+    if want("trmv"):
+        a1 = np.zeros(c1, np.float32)
+        synth.upper_triangle_stream(0, 0, N1, out=a1)
+        h["trmv"] = dict(desc=st.upper_triangle(N1), A=host(a1), ins=[host(synth.dense(0, 1, (N1,)))], out=(N1,))
+    if want("trmv_batched"):
+        ab = np.zeros((b, c1), np.float32)
+        xb = np.empty((b, N1), np.float32)
+        for k in range(b):  # instance k of the batch: seed 0, tensor ids 2k+2 / 2k+3
+            synth.upper_triangle_stream(0, 2 * k + 2, N1, out=ab[k])
+            xb[k] = synth.dense(0, 2 * k + 3, (N1,))
+        h["trmv_batched"] = dict(desc=st.upper_triangle(N1), A=host(ab), ins=[host(xb)], out=(b, N1), batch=b)
+    if want("bandmm"):
+        N2, w, C2 = z["N2"], z["w"], z["C2"]
+        h["bandmm"] = dict(desc=st.band(N2, w), A=host(synth.band_diagonals_stream(1, 0, N2, w).reshape(-1)),
+                           ins=[host(synth.dense(1, 1, (N2, C2)))], out=(N2, C2))
+    if want("symv"):
+        N3 = z["N3"]
+        a3 = np.zeros(cap(tri(N3), 4), np.float32)
+        synth.upper_triangle_stream(2, 0, N3, dist=synth.NORMAL, out=a3)
+        h["symv"] = dict(desc=st.upper_triangle(N3, symmetric=True), A=host(a3),
+                         ins=[host(synth.dense(2, 1, (N3,), dist=synth.NORMAL))], out=(N3,))
+    if want("mttkrp"):
+        n4, R = z["n4"], z["R"]
+        a4 = np.zeros(cap(tet(n4), 4), np.float32)
+        synth.tetrahedron_stream(3, 0, n4, out=a4)
+        h["mttkrp"] = dict(desc=st.tetrahedron(n4), A=host(a4),
+                           ins=[host(synth.dense(3, 1, (n4, R))), host(synth.dense(3, 2, (n4, R)))], out=(n4, R))
+    if want("trimm_bf16"):
+        N5 = z["N5"]
+        sc = N5 ** -0.5
+        a5 = np.zeros(cap(tri(N5), 8), np.uint16)
+        synth.upper_triangle_stream(4, 0, N5, dist=synth.NORMAL, scale=sc, bf16=True, out=a5)
+        h["trimm_bf16"] = dict(desc=st.upper_triangle(N5), A=host(a5, True),
+                               ins=[host(synth.dense(4, 1, (N5, N5), dist=synth.NORMAL, scale=sc, bf16=True), True)],
+                               out=(N5, N5))
     return h
 
 
@@ -148,7 +155,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu_index), "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-i", str(self.gpu_index), "-lms", "20"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
@@ -201,9 +208,14 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     z = sizes(args.small)
+    for kv in args.size:
+        k, v = kv.split("=")
+        assert k in z, k
+        z[k] = int(v)
     acct = accounting(z)
     t0 = time.time()
-    host = generate_host(z, pin=True)
+    only = set(args.only.split(",")) if args.only else None
+    host = generate_host(z, pin=True, only=only)
     gen_s = time.time() - t0
 
     # device-resident copies
@@ -218,8 +230,9 @@ def run_gpu(args):
         devs[name] = d
     err_word = torch.zeros(1, dtype=torch.int32, device="cuda")
     N5 = z["N5"]
-    dense5 = torch.empty((N5, N5), dtype=torch.bfloat16, device="cuda")
-    packed5 = structs["trimm_bf16"].empty_packed(torch.bfloat16)
+    if "trimm_bf16" in structs:
+        dense5 = torch.zeros((N5, N5), dtype=torch.bfloat16, device="cuda")
+        packed5 = structs["trimm_bf16"].empty_packed(torch.bfloat16)
 
     def run_kernel(name):
         if name == "pack_bf16":
@@ -233,6 +246,8 @@ def run_gpu(args):
 
     order = ["unpack_bf16" if n == "pack_bf16" else "pack_bf16" if n == "unpack_bf16" else n for n in ORDER]
     # (unpack first so that pack reads a defined dense tensor)
+    if only is not None:
+        order = [n for n in order if n in only]
 
     def step(events=None):
         for name in order:
@@ -275,7 +290,7 @@ def run_gpu(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         total_ms = float(tt.item())
     ms_per_step = total_ms / args.steps
-    step_flops = sum(a["flops"] for a in acct.values())
+    step_flops = sum(acct[n]["flops"] for n in order)
 
     pk = peaks()
     kernels = {}
@@ -316,6 +331,8 @@ def run_gpu(args):
         hd = {}
         h2d = d2h = 0
         for name, hw in host.items():
+            if name not in order:
+                continue
             out_h = torch.empty(hw["out"], dtype=torch.float32).pin_memory()
             n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1))
             hd[name] = dict(out=out_h, ws=torch.empty(n, dtype=torch.uint8, device="cuda"))
@@ -361,7 +378,7 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
             "data": "synthetic",
             "config": {"workload": "all five configs per step: " + json.dumps(z, separators=(",", ":")),
-                       "small": bool(args.small),
+                       "small": bool(args.small), "only": args.only or None,
                        "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
                              "(the 8.6 GB symmetric stream runs once per step)",
                        "replicas": "each rank runs the whole step on its own GPU; no collective"},
@@ -470,13 +487,15 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--small", action="store_true", help="reduced sizes for a quick functional run (not a result)")
+    ap.add_argument("--only", default="", help="comma list of kernels to run (profiling aid, not a result)")
+    ap.add_argument("--size", action="append", default=[], help="override a size, e.g. N3=16384 (profiling aid)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--cpu-rows-scale", type=float, default=1.0)
+    ap.add_argument("--cpu-rows-scale", type=float, default=3.0)
     args = ap.parse_args()
     import __graft_entry__
 

@@ -5,24 +5,29 @@
 //
 // Tiling.  An output tile is 128 rows x 256 columns.  Row block I only needs K blocks (64 columns
 // of A, 64 rows of B) from the diagonal on: kb = 2I .. ceil(N/64)-1, so the executed MMA work is
-// the triangle plus half a tile per row block.  The two K blocks that cross the diagonal are
-// zero-masked while A is staged; all others take the unmasked path.  Tiles are ordered by
-// decreasing K length and dealt round-robin to one persistent CTA per SM.
+// the triangle plus half a tile per row block.  Tiles are ordered by decreasing K length and dealt
+// round-robin to one persistent CTA per SM.
 //
-// Roles inside a CTA (14 warps):
-//   warps 0-3   epilogue: tcgen05.ld of the accumulator (warp w owns TMEM lanes 32w..32w+31),
-//               128-bit stores to C
-//   warp  4     one lane issues the TMA loads of B (four 64x64 boxes per K block, 128B swizzle)
-//   warp  5     allocates tensor memory; one lane issues tcgen05.mma (M128 N256 K16, four per
-//               K block) and the commits that release stages / publish accumulators
-//   warps 6-13  stage A: the packed row pitch changes with the row, so no tensor map can
-//               describe A and row starts are only 2-byte aligned.  Eight lanes cover one row of
-//               a K block with aligned 128-bit loads; the row's constant misalignment (0..7
-//               elements, a function of rowbase(i) only) is removed in registers with a
-//               two-level word select and a funnel shift, and the 16 bytes are stored at the
-//               swizzled position the K-major UMMA descriptor expects.
-// Accumulators are double buffered in tensor memory (2 x 256 columns) so the epilogue of a tile
-// overlaps the MMAs of the next.
+// Two kernels per call:
+//  1. stage_a: the packed row pitch changes with the row and row starts are only 2-byte aligned,
+//     so no tensor map can describe A.  Every 128x64 tile of the triangle is therefore re-laid
+//     once into the workspace as the exact shared-memory image the K-major, 128-byte-swizzled
+//     UMMA descriptor expects (16 KiB per tile): eight lanes cover one row with aligned 128-bit
+//     loads, the row's constant misalignment (0..7 elements, a function of rowbase(i) only) is
+//     removed in registers with a two-level word select and a funnel shift, and entries left of
+//     the diagonal or beyond column N are zeroed.  Doing this once per call instead of once per
+//     column tile keeps the realignment off the MMA critical path (each A tile is consumed by
+//     every column tile of its row block).  The workspace stays packed: it holds the triangle's
+//     tiles only.
+//  2. trimm_tcgen05: warp-specialised pipeline,
+//       warps 0-3  epilogue: tcgen05.ld of the accumulator (warp w owns TMEM lanes 32w..32w+31),
+//                  128-bit stores to C
+//       warp  4    one lane issues, per K block, one bulk copy of the staged A tile and four TMA
+//                  boxes (64x64, 128B swizzle) of B into the stage, all on one mbarrier
+//       warp  5    allocates tensor memory; one lane issues tcgen05.mma (M128 N256 K16, four per
+//                  K block) and the commits that release stages / publish accumulators
+//     Accumulators are double buffered in tensor memory (2 x 256 columns) so the epilogue of a
+//     tile overlaps the MMAs of the next.
 //
 // Every wait on an mbarrier is bounded by a clock budget; on expiry the thread records a code in
 // the error word and the CTA drains: nothing can spin forever.
@@ -39,14 +44,14 @@ constexpr int kStages = 4;
 constexpr int kABytes = kTileM * kBlockK * 2;  // 16 KiB
 constexpr int kBBytes = kBlockK * kTileN * 2;  // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kEpilogueWarps = 4, kProducerWarps = 8;
-constexpr int kWarpTma = 4, kWarpMma = 5, kWarpProducer0 = 6;
-constexpr int kThreads = (kWarpProducer0 + kProducerWarps) * 32;  // 448
+constexpr int kEpilogueWarps = 4;
+constexpr int kWarpTma = 4, kWarpMma = 5;
+constexpr int kThreads = 6 * 32;
 constexpr int kTmemCols = 512;
 constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long kWaitBudget = 4000000000LL;  // clock cycles (~2 s) before a wait gives up
 
-enum ErrCode : int32_t { kErrFullA = 1, kErrFullB = 2, kErrEmpty = 3, kErrTmemFull = 4, kErrTmemEmpty = 5 };
+enum ErrCode : int32_t { kErrFull = 1, kErrEmpty = 3, kErrTmemFull = 4, kErrTmemEmpty = 5 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 
@@ -101,13 +106,16 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void fence_proxy_async() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
@@ -169,8 +177,17 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                             ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 
+// Staged tile (I, kb) lives at tile index tile_offset(I) + kb - 4*(I/2): row blocks are stored in
+// pairs that start at the same K block, so that two row blocks can later share one K loop; the
+// two tiles this adds in front of every odd row block are all zero.
+__host__ __device__ __forceinline__ int64_t tile_offset(int64_t I, int64_t k_blocks) {
+    const int64_t P = I >> 1;
+    return 2 * P * k_blocks - 4 * P * (P - 1) + (I & 1) * (k_blocks - 4 * P);
+}
+
 struct Params {
-    const __nv_bfloat16* A;
+    const __nv_bfloat16* A;      // packed rows (stage_a) / unused (main)
+    const uint8_t* tiles;        // staged tile images, 16 KiB each
     float* C;
     int64_t N, ncols, ldc;
     int64_t cap_elems;   // capacity of the packed buffer in elements (multiple of 8)
@@ -185,10 +202,9 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = (uint64_t*)(smem + (size_t)kStages * kStageBytes);
-    // barrier slots: full_a[s], full_b[s], empty[s], tmem_full[2], tmem_empty[2]
+    // barrier slots: full[s], (unused)[s], empty[s], tmem_full[2], tmem_empty[2], drain
     const uint32_t bar0 = smem_u32(bars);
-    auto full_a = [&](int s) { return bar0 + 8u * s; };
-    auto full_b = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
     auto tmem_full = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
     auto tmem_empty = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
@@ -201,8 +217,7 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_a(s), kProducerWarps);
-            mbar_init(full_b(s), 1);
+            mbar_init(full(s), 1);
             mbar_init(empty(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -225,7 +240,7 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
     const int64_t tiles = (int64_t)p.row_blocks * p.col_blocks;
 
     if (warp == kWarpTma) {
-        // ---- B producer: TMA -----------------------------------------------------------------
+        // ---- producer: bulk copy of the staged A tile + TMA boxes of B ------------------------------
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
@@ -238,11 +253,14 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
                         ok = false;
                         break;
                     }
-                    const uint32_t dst = smem_base + s * kStageBytes + kABytes;
-                    mbar_arrive_expect_tx(full_b(s), kBBytes);
+                    const uint32_t dst = smem_base + s * kStageBytes;
+                    mbar_arrive_expect_tx(full(s), kStageBytes);
+                    bulk_load(dst, p.tiles + (tile_offset(I, p.k_blocks) + kb - 4 * (I >> 1)) * (int64_t)kABytes,
+                              kABytes, full(s));
 #pragma unroll
                     for (int q = 0; q < kTileN / 64; ++q)
-                        tma_load_2d(dst + q * (kBlockK * 128), &tmap_b, J * kTileN + q * 64, kb * kBlockK, full_b(s));
+                        tma_load_2d(dst + kABytes + q * (kBlockK * 128), &tmap_b, J * kTileN + q * 64,
+                                    kb * kBlockK, full(s));
                 }
             }
             // Drain: copies already issued must land before the CTA's shared memory is released.
@@ -251,7 +269,7 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
                 for (int s = 0; s < kStages; ++s) {
                     const uint32_t issued = it / kStages + ((int)(it % kStages) > s ? 1 : 0);
                     if (issued == 0) continue;
-                    while (!mbar_test(full_b(s), (issued - 1) & 1) && clock64() - t0 < kWaitBudget) {
+                    while (!mbar_test(full(s), (issued - 1) & 1) && clock64() - t0 < kWaitBudget) {
                     }
                 }
             }
@@ -274,8 +292,7 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
                 for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t par = (it / kStages) & 1;
-                    if (!mbar_wait(full_a(s), par, abort_flag, p.err_word, kErrFullA) ||
-                        !mbar_wait(full_b(s), par, abort_flag, p.err_word, kErrFullB)) {
+                    if (!mbar_wait(full(s), par, abort_flag, p.err_word, kErrFull)) {
                         ok = false;
                         break;
                     }
@@ -301,88 +318,6 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
                 const long long t0 = clock64();
                 while (!mbar_test(drain_bar(), 0) && clock64() - t0 < kWaitBudget) {
                 }
-            }
-        }
-    } else if (warp >= kWarpProducer0) {
-        // ---- A producers -------------------------------------------------------------------------
-        const int pw = warp - kWarpProducer0;
-        const int sub = lane >> 3, c = lane & 7;  // row within a 4-row group, 16-byte chunk in the row
-        const uint4 zero4 = make_uint4(0, 0, 0, 0);
-        uint32_t it = 0;
-        bool ok = true;
-        for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-            const int I = (int)(t / p.col_blocks);
-            // the four rows of the tile this lane serves, constant over the K loop
-            int64_t base[4];   // rowbase(i) + 8c, in elements
-            int row[4];
-            uint32_t soff[4];  // swizzled byte offset of the lane's 16 bytes inside a stage
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                const int r = 4 * (pw + kProducerWarps * g) + sub;  // 0..127
-                const int64_t i = (int64_t)I * kTileM + r;
-                row[g] = (int)i;
-                base[g] = (i < p.N ? upper_row_base(p.N, i) : 0) + 8 * c;
-                soff[g] = (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4));
-            }
-            for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
-                const int s = it % kStages;
-                const int64_t k0 = (int64_t)kb * kBlockK;
-                // issue the global loads of this K block before waiting for the stage
-                uint4 lo[4], ninth[4];
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int64_t e0 = base[g] + k0;       // first element of the lane's chunk
-                    const int64_t a0 = e0 & ~(int64_t)7;   // aligned down to 16 bytes
-                    const bool live = row[g] < p.N;
-                    lo[g] = (live && a0 + 8 <= p.cap_elems) ? __ldg((const uint4*)(p.A + a0)) : zero4;
-                    ninth[g] = (live && c == 7 && (e0 & 7) && a0 + 16 <= p.cap_elems)
-                                   ? __ldg((const uint4*)(p.A + a0 + 8)) : zero4;
-                }
-                if (it >= kStages &&
-                    !mbar_wait_warp(empty(s), ((it / kStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty, lane)) {
-                    ok = false;
-                    break;
-                }
-                uint8_t* stage = smem + (size_t)s * kStageBytes;
-                const bool masked = (kb < 2 * I + 2) || (k0 + kBlockK > p.N);
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    // neighbour's chunk = the 16 bytes that follow this lane's aligned chunk
-                    uint4 hi;
-                    hi.x = __shfl_down_sync(0xffffffffu, lo[g].x, 1);
-                    hi.y = __shfl_down_sync(0xffffffffu, lo[g].y, 1);
-                    hi.z = __shfl_down_sync(0xffffffffu, lo[g].z, 1);
-                    hi.w = __shfl_down_sync(0xffffffffu, lo[g].w, 1);
-                    if (c == 7) hi = ninth[g];
-                    const uint32_t se = (uint32_t)((base[g] + k0) & 7);  // misalignment in elements
-                    const bool q1 = se & 2, q2 = se & 4;
-                    const uint32_t sh = (se & 1) * 16;
-                    const uint32_t W0 = lo[g].x, W1 = lo[g].y, W2 = lo[g].z, W3 = lo[g].w;
-                    const uint32_t W4 = hi.x, W5 = hi.y, W6 = hi.z, W7 = hi.w;
-                    const uint32_t X0 = q1 ? W1 : W0, X1 = q1 ? W2 : W1, X2 = q1 ? W3 : W2, X3 = q1 ? W4 : W3,
-                                   X4 = q1 ? W5 : W4, X5 = q1 ? W6 : W5, X6 = q1 ? W7 : W6;
-                    const uint32_t T0 = q2 ? X2 : X0, T1 = q2 ? X3 : X1, T2 = q2 ? X4 : X2, T3 = q2 ? X5 : X3,
-                                   T4 = q2 ? X6 : X4;
-                    uint4 out;
-                    out.x = __funnelshift_r(T0, T1, sh);
-                    out.y = __funnelshift_r(T1, T2, sh);
-                    out.z = __funnelshift_r(T2, T3, sh);
-                    out.w = __funnelshift_r(T3, T4, sh);
-                    if (masked) {
-                        // keep column j only if row <= j < N
-                        const int64_t j0 = k0 + 8 * c;
-                        uint32_t* w = &out.x;
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const int64_t j = j0 + e;
-                            if (j < row[g] || j >= p.N) w[e >> 1] &= (e & 1) ? 0x0000FFFFu : 0xFFFF0000u;
-                        }
-                    }
-                    *(uint4*)(stage + soff[g]) = out;
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full_a(s));
             }
         }
     } else {
@@ -447,6 +382,60 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
 
 // ---- host ------------------------------------------------------------------------------------------
 
+// ---- stage_a: packed rows -> swizzled tile images ----------------------------------------------------
+// One CTA builds one 128x64 tile (I, kb): 8 warps x 4 groups of 4 rows, 8 lanes per row.
+constexpr int kStageThreads = 256;
+
+__global__ void __launch_bounds__(kStageThreads)
+trimm_stage_a_kernel(const Params p, uint8_t* __restrict__ tiles) {
+    const int I = blockIdx.y;
+    const int kb = blockIdx.x + 4 * (I >> 1);
+    if (kb >= p.k_blocks) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane >> 3, c = lane & 7;  // row within a 4-row group, 16-byte chunk in the row
+    uint8_t* tile = tiles + (tile_offset(I, p.k_blocks) + blockIdx.x) * (int64_t)kABytes;
+    const int64_t k0 = (int64_t)kb * kBlockK;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    const bool masked = (kb < 2 * I + 2) || (k0 + kBlockK > p.N);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const int r = 4 * (warp + 8 * g) + sub;  // 0..127
+        const int64_t i = (int64_t)I * kTileM + r;
+        const uint32_t soff = (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4));
+        uint4 out = zero4;
+        if (i < p.N && k0 + kBlockK > i) {  // the row has entries in this K block
+            const int64_t e0 = upper_row_base(p.N, i) + k0 + 8 * c;  // first element of the lane's chunk
+            const int64_t a0 = e0 & ~(int64_t)7;                     // aligned down to 16 bytes
+            const uint32_t se = (uint32_t)(e0 & 7);                  // misalignment in elements
+            const uint4 lo = (a0 + 8 <= p.cap_elems) ? __ldg((const uint4*)(p.A + a0)) : zero4;
+            const uint4 hi = (se != 0 && a0 + 16 <= p.cap_elems) ? __ldg((const uint4*)(p.A + a0 + 8)) : zero4;
+            const bool q1 = se & 2, q2 = se & 4;
+            const uint32_t sh = (se & 1) * 16;
+            const uint32_t W0 = lo.x, W1 = lo.y, W2 = lo.z, W3 = lo.w;
+            const uint32_t W4 = hi.x, W5 = hi.y, W6 = hi.z, W7 = hi.w;
+            const uint32_t X0 = q1 ? W1 : W0, X1 = q1 ? W2 : W1, X2 = q1 ? W3 : W2, X3 = q1 ? W4 : W3,
+                           X4 = q1 ? W5 : W4, X5 = q1 ? W6 : W5, X6 = q1 ? W7 : W6;
+            const uint32_t T0 = q2 ? X2 : X0, T1 = q2 ? X3 : X1, T2 = q2 ? X4 : X2, T3 = q2 ? X5 : X3,
+                           T4 = q2 ? X6 : X4;
+            out.x = __funnelshift_r(T0, T1, sh);
+            out.y = __funnelshift_r(T1, T2, sh);
+            out.z = __funnelshift_r(T2, T3, sh);
+            out.w = __funnelshift_r(T3, T4, sh);
+            if (masked) {
+                // keep column j only if i <= j < N
+                const int64_t j0 = k0 + 8 * c;
+                uint32_t* w = &out.x;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int64_t j = j0 + e;
+                    if (j < i || j >= p.N) w[e >> 1] &= (e & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+                }
+            }
+        }
+        *(uint4*)(tile + soff) = out;
+    }
+}
+
 __global__ void repitch_bf16_kernel(const uint16_t* __restrict__ src, int64_t lds, uint16_t* __restrict__ dst,
                                     int64_t ldd, int64_t rows, int64_t cols) {
     for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < rows * ldd;
@@ -474,11 +463,17 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
-// B rows whose pitch is not a multiple of 16 bytes cannot be described by a tensor map: they are
-// first copied into the workspace with the pitch rounded up to 8 elements.
+// Workspace: the staged tile images of A, then (only when B's row pitch is not a multiple of
+// 16 bytes, which a tensor map cannot describe) a copy of B with the pitch rounded up to 8 elements.
+static int64_t staged_tile_count(int64_t N) {
+    const int64_t row_blocks = (N + kTileM - 1) / kTileM, k_blocks = (N + kBlockK - 1) / kBlockK;
+    return tile_offset(row_blocks, k_blocks);
+}
 size_t trimm_workspace_bytes(const IndexMap& m, int64_t ncols, int64_t ldb) {
-    if (m.N == 0 || ncols == 0 || ldb % 8 == 0) return 0;
-    return (size_t)(m.N * round_up(ncols, 8) * 2);
+    if (m.N == 0 || ncols == 0) return 0;
+    size_t bytes = (size_t)round_up(staged_tile_count(m.N) * kABytes, 256);
+    if (ldb % 8 != 0) bytes += (size_t)(m.N * round_up(ncols, 8) * 2);
+    return bytes;
 }
 
 dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B, int64_t ldb, float* C,
@@ -488,8 +483,10 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     if (N == 0 || ncols == 0) return DASTAC_OK;
     // TMA needs a 16-byte aligned base and row pitch for B.
     if (!aligned16(B)) return DASTAC_ERR_ALIGNMENT;
+    if (!workspace) return DASTAC_ERR_WORKSPACE;
+    uint8_t* tiles = (uint8_t*)workspace;
     if (ldb % 8 != 0) {
-        if (!workspace) return DASTAC_ERR_WORKSPACE;
+        workspace = tiles + round_up(staged_tile_count(N) * kABytes, 256);
         const int64_t ldd = round_up(ncols, 8);
         int64_t blocks = (N * ldd + 255) / 256;
         if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
@@ -515,6 +512,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
 
     Params p;
     p.A = (const __nv_bfloat16*)A;
+    p.tiles = tiles;
     p.C = C;
     p.N = N;
     p.ncols = ncols;
@@ -536,8 +534,12 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
     }
-    const int64_t tiles = (int64_t)p.row_blocks * p.col_blocks;
-    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    if (p.row_blocks > 65535) return DASTAC_ERR_OVERFLOW;  // gridDim.y of the staging kernel
+    trimm_stage_a_kernel<<<dim3((unsigned)p.k_blocks, (unsigned)p.row_blocks), kStageThreads, 0, st>>>(p, tiles);
+    dastac_status ss = launch_status();
+    if (ss != DASTAC_OK) return ss;
+    const int64_t n_tiles = (int64_t)p.row_blocks * p.col_blocks;
+    const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
     trimm_tcgen05_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmap, p);
     return launch_status();
 }
