@@ -41,7 +41,7 @@ size_t symv_workspace_bytes(const IndexMap& m);
 dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, float* y,
                           int accumulate, void* workspace, cudaStream_t st);
 dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, int64_t ldb, float* C,
-                            int64_t ldc, int64_t ncols, int accumulate, cudaStream_t st);
+                            int64_t ldc, int64_t ncols, int accumulate, int32_t* err_word, cudaStream_t st);
 dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, int64_t ldb,
                             const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
                             int accumulate, cudaStream_t st);

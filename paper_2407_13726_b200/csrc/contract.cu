@@ -200,7 +200,7 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
                          accumulate, scratch, cs);
     } else if (p.cls == kMatMat && m.kind == kBandDiagonals) {
         st = launch_bandmm(m, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0],
-                           (float*)dev_out, out->strides[0], p.ncols, accumulate, cs);
+                           (float*)dev_out, out->strides[0], p.ncols, accumulate, err_word, cs);
     } else if (p.cls == kMatMat) {
         st = launch_trimm_bf16(m, dev_in[0], dev_in[1], in[1].strides[0], (float*)dev_out,
                                out->strides[0], p.ncols, accumulate, scratch, err_word, cs);

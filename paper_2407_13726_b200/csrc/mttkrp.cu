@@ -27,6 +27,19 @@ constexpr int kTile = 32;        // fibres per unit and K elements per chunk
 constexpr int kTsPitch = 36;     // floats; 16-byte aligned rows, conflict-free 128-bit stores
 constexpr int kRTile = 32;       // rank columns per pass
 
+// Two fp32 multiply-adds per instruction (packed pair in a 64-bit register): d = a * b + d.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma2(unsigned long long& d, unsigned long long a, unsigned long long b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+
 struct WarpSmem {
     float Ts[kTile][kTsPitch];   // Ts[k][j] chunk of T, transposed
     float Cs[kTile][kRTile];     // Cs[k][r] chunk of C
@@ -62,23 +75,35 @@ mttkrp_kernel(IndexMap m, const float* __restrict__ T, const float* __restrict__
         const int64_t rowbase0 = rank_of(m, idx) - j0;
 
         for (int64_t r0 = 0; r0 < R; r0 += kRTile) {
-            float acc[4][8];
+            unsigned long long acc2[4][4];  // [fibre][pair of rank columns]
 #pragma unroll
             for (int q = 0; q < 4; ++q)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[q][e] = 0.f;
+                for (int e = 0; e < 4; ++e) acc2[q][e] = 0ull;
 
             float v[kTile];  // lane's column of the next chunk: T(i, j0+jj, kc+lane)
+            const float* Tu = T + rowbase0;  // Tu[roff(jj) + k] = T(i, j0+jj, k), roff advanced by n-j-1
+            const uint32_t n32 = (uint32_t)n, j032 = (uint32_t)j0;
             auto load_chunk = [&](int64_t kc) {
-                const int64_t k = kc + lane;
-                int64_t off = rowbase0;
+                const uint32_t k = (uint32_t)kc + lane;
+                uint32_t roff = 0;
+                if (kc > j0 && kc + kTile <= n && j0 + kTile <= n) {
+                    // interior chunk: every element is inside the tetrahedron
 #pragma unroll
-                for (int jj = 0; jj < kTile; ++jj) {
-                    const int64_t j = j0 + jj;
-                    v[jj] = (j < n && k >= j && k < n) ? __ldg(T + off + k) : 0.f;
-                    off += n - j - 1;
+                    for (int jj = 0; jj < kTile; ++jj) {
+                        v[jj] = __ldg(Tu + (roff + k));
+                        roff += n32 - (j032 + jj) - 1;
+                    }
+                } else {
+#pragma unroll
+                    for (int jj = 0; jj < kTile; ++jj) {
+                        const uint32_t j = j032 + jj;
+                        v[jj] = (j < n32 && k >= j && k < n32) ? __ldg(Tu + (roff + k)) : 0.f;
+                        roff += n32 - j - 1;
+                    }
                 }
             };
+            const bool c_fast = (r0 + kRTile <= R) && ((ldc & 3) == 0);
             load_chunk(j0);
             for (int64_t kc = j0; kc < n; kc += kTile) {
                 __syncwarp();
@@ -87,39 +112,54 @@ mttkrp_kernel(IndexMap m, const float* __restrict__ T, const float* __restrict__
                     *reinterpret_cast<float4*>(&sm.Ts[lane][4 * q]) =
                         make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
                 // rows kc..kc+31 of C, columns r0..r0+31: lane = (row within 4, 16-byte chunk)
+                if (c_fast && kc + kTile <= n) {
+                    const float4* src = reinterpret_cast<const float4*>(C + (kc + (lane >> 3)) * ldc + r0) + (lane & 7);
 #pragma unroll
-                for (int q = 0; q < kTile / 4; ++q) {
-                    const int kk = 4 * q + (lane >> 3);
-                    const int64_t k = kc + kk, r = r0 + 4 * (lane & 7);
-                    float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (k < n) {
-                        const float* src = C + k * ldc + r;
-                        if (r + 4 <= R && (ldc & 3) == 0) {
-                            c4 = __ldg(reinterpret_cast<const float4*>(src));
-                        } else {
-                            if (r < R) c4.x = __ldg(src);
-                            if (r + 1 < R) c4.y = __ldg(src + 1);
-                            if (r + 2 < R) c4.z = __ldg(src + 2);
-                            if (r + 3 < R) c4.w = __ldg(src + 3);
+                    for (int q = 0; q < kTile / 4; ++q)
+                        *reinterpret_cast<float4*>(&sm.Cs[4 * q + (lane >> 3)][4 * (lane & 7)]) = __ldg(src + q * ldc);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < kTile / 4; ++q) {
+                        const int kk = 4 * q + (lane >> 3);
+                        const int64_t k = kc + kk, r = r0 + 4 * (lane & 7);
+                        float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (k < n) {
+                            const float* src = C + k * ldc + r;
+                            if (r + 4 <= R && (ldc & 3) == 0) {
+                                c4 = __ldg(reinterpret_cast<const float4*>(src));
+                            } else {
+                                if (r < R) c4.x = __ldg(src);
+                                if (r + 1 < R) c4.y = __ldg(src + 1);
+                                if (r + 2 < R) c4.z = __ldg(src + 2);
+                                if (r + 3 < R) c4.w = __ldg(src + 3);
+                            }
                         }
+                        *reinterpret_cast<float4*>(&sm.Cs[kk][4 * (lane & 7)]) = c4;
                     }
-                    *reinterpret_cast<float4*>(&sm.Cs[kk][4 * (lane & 7)]) = c4;
                 }
                 __syncwarp();
                 if (kc + kTile < n) load_chunk(kc + kTile);  // prefetch into registers
 #pragma unroll 8
                 for (int kk = 0; kk < kTile; ++kk) {
                     const float4 t4 = *reinterpret_cast<const float4*>(&sm.Ts[kk][4 * jg]);
-                    const float4 ca = *reinterpret_cast<const float4*>(&sm.Cs[kk][8 * rg]);
-                    const float4 cb = *reinterpret_cast<const float4*>(&sm.Cs[kk][8 * rg + 4]);
-                    const float t[4] = {t4.x, t4.y, t4.z, t4.w};
-                    const float c[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+                    const ulonglong2 ca = *reinterpret_cast<const ulonglong2*>(&sm.Cs[kk][8 * rg]);
+                    const ulonglong2 cb = *reinterpret_cast<const ulonglong2*>(&sm.Cs[kk][8 * rg + 4]);
+                    const unsigned long long t2[4] = {pack2(t4.x, t4.x), pack2(t4.y, t4.y), pack2(t4.z, t4.z),
+                                                      pack2(t4.w, t4.w)};
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[q][e] = fmaf(t[q], c[e], acc[q][e]);
+                    for (int q = 0; q < 4; ++q) {
+                        fma2(acc2[q][0], t2[q], ca.x);
+                        fma2(acc2[q][1], t2[q], ca.y);
+                        fma2(acc2[q][2], t2[q], cb.x);
+                        fma2(acc2[q][3], t2[q], cb.y);
+                    }
                 }
             }
+            float acc[4][8];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) unpack2(acc2[q][e], acc[q][2 * e], acc[q][2 * e + 1]);
             // M(i, r) += sum_j B(j, r) U(j, r): the lane's 4 fibres, then the 8 fibre groups
             float s[8];
 #pragma unroll
