@@ -1,9 +1,30 @@
 """Structured tensor algebra on densely packed layouts for NVIDIA B200 (sm_100a).
 
 The product is ``libdastac.so`` (C ABI, see ``include/dastac.h``); this package is its Python
-binding.  Importing it requires the built library: ``python -m paper_2407_13726_b200.build``.
+binding.  The binding needs the built library: ``python -m paper_2407_13726_b200.build``.  It is
+loaded on first use of any public name, so that the build module itself can be imported before the
+library exists; a missing library raises ImportError at that point (there is no other code path).
 """
-from .binding import *  # noqa: F401,F403
-from .binding import (DastacError, Structure, contract, contract_workspace, launch_count, pack,
-                      rank, rank_batch, status_string, structure_count, structure_create, unpack,
-                      unrank, unrank_batch)
+import importlib
+
+_PUBLIC = ("DastacError", "Structure", "contract", "contract_workspace", "launch_count", "pack",
+           "rank", "rank_batch", "status_string", "structure_count", "structure_create", "unpack",
+           "unrank", "unrank_batch", "F32", "BF16", "MEM_DEVICE", "MEM_HOST", "KIND_EMPTY",
+           "KIND_DENSE", "KIND_UPPER", "KIND_LOWER", "KIND_BAND_DIAGONALS", "KIND_TETRAHEDRON",
+           "LAYOUT_LEXICOGRAPHIC", "LAYOUT_PADDED_DIAGONALS", "EXPORTS", "LIB_PATH")
+
+__all__ = list(_PUBLIC)
+
+
+def __getattr__(name):
+    if name.startswith("__"):
+        raise AttributeError(name)
+    if name in ("build", "binding"):
+        return importlib.import_module("." + name, __name__)
+    binding = importlib.import_module(".binding", __name__)
+    try:
+        value = getattr(binding, name)
+    except AttributeError:
+        raise AttributeError(f"module {__name__!r} has no attribute {name!r}") from None
+    globals()[name] = value
+    return value
