@@ -184,6 +184,36 @@ dastac_status dastac_contract(const char* expr, const dastac_operand* in, int32_
 
 const char* dastac_status_string(dastac_status st);
 
+/*
+ * The bf16 triangular x dense contraction ("ij,jc->ic", upper triangle, bf16 -> f32) without any
+ * workspace argument and without any memory allocation.  The paper has no counterpart: this entry
+ * point exists for callers that must not, or cannot, obtain device memory around the call - code
+ * running inside a region where allocation is forbidden (a real-time loop, a callback that holds a
+ * lock the allocator also takes, a process whose memory pool was handed out in full at start-up).
+ * dastac_contract needs about N*N bytes of caller-provided scratch for this expression; here that
+ * scratch is a fixed array inside the library image, DASTAC_NOALLOC_SCRATCH_BYTES per GPU that
+ * loads the library, held until the process exits.
+ *
+ *   s        square upper triangle, N <= DASTAC_NOALLOC_MAX_N; larger N returns DASTAC_ERR_WORKSPACE
+ *   A        device, packed bf16 rows of s (capacity as for every packed buffer), 16-byte aligned
+ *   B        device, N x ncols bf16, row pitch ldb elements; ldb must be a multiple of 8 (a pitch
+ *            that is not a multiple of 16 bytes returns DASTAC_ERR_ALIGNMENT), 16-byte aligned
+ *   C        device, N x ncols f32, row pitch ldc elements, 16-byte aligned
+ *   accumulate, err_word, stream   as for dastac_contract
+ *
+ * Results are those of dastac_contract on the same operands.  The call itself calls no cudaMalloc,
+ * cudaFree or other allocating routine.  The first call on a device looks up the array's device
+ * address (cudaGetSymbolAddress); make that first call before starting any stream capture.
+ * Every call on a device uses the same array and rewrites all of it that it needs, so nothing has
+ * to be cleared between calls, but two calls whose kernels may run at the same time (different
+ * streams, or different host threads on different streams) race on it: serialise them.
+ */
+#define DASTAC_NOALLOC_MAX_N 2048
+#define DASTAC_NOALLOC_SCRATCH_BYTES (288 * 16384)
+dastac_status dastac_trimm_bf16_noalloc(const dastac_structure* s, const void* A, const void* B,
+                                        int64_t ldb, int64_t ncols, float* C, int64_t ldc,
+                                        int32_t accumulate, int32_t* err_word, void* stream);
+
 /* Number of kernels this library has launched in the calling process (for launch accounting). */
 int64_t dastac_launch_count(void);
 

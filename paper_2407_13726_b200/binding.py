@@ -25,8 +25,9 @@ EXPORTS = [
     "dastac_structure_create", "dastac_structure_destroy", "dastac_structure_count",
     "dastac_structure_kind", "dastac_rank", "dastac_unrank", "dastac_rank_batch",
     "dastac_unrank_batch", "dastac_pack", "dastac_unpack", "dastac_contract_workspace",
-    "dastac_contract", "dastac_status_string", "dastac_launch_count",
+    "dastac_contract", "dastac_status_string", "dastac_launch_count", "dastac_trimm_bf16_noalloc",
 ]
+NOALLOC_MAX_N = 2048
 
 
 class DastacError(RuntimeError):
@@ -72,6 +73,7 @@ _lib.dastac_contract.argtypes = [ctypes.c_char_p, ctypes.POINTER(_Operand), _i32
                                  ctypes.POINTER(_Operand), _i32, _vp, ctypes.c_size_t, _vp, _vp]
 _lib.dastac_status_string.argtypes = [ctypes.c_int]
 _lib.dastac_status_string.restype = ctypes.c_char_p
+_lib.dastac_trimm_bf16_noalloc.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _i32, _vp, _vp]
 _lib.dastac_launch_count.argtypes = []
 _lib.dastac_launch_count.restype = _i64
 
@@ -266,4 +268,18 @@ def contract(expr: str, s: Structure, packed: torch.Tensor, dense_inputs: Sequen
                                 ws_ptr, ws_bytes,
                                 None if err_word is None else err_word.data_ptr(), _stream()),
            "dastac_contract")
+    return out
+
+
+def trimm_bf16_noalloc(s: Structure, packed: torch.Tensor, B: torch.Tensor, out: torch.Tensor,
+                       accumulate: bool = False, err_word: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``out = A B`` (or ``+=``) for a packed bf16 upper triangle of at most ``NOALLOC_MAX_N`` rows,
+    through the entry point that takes no workspace and allocates nothing (see ``dastac.h``)."""
+    assert packed.is_cuda and B.is_cuda and out.is_cuda and B.dim() == 2 and out.dim() == 2
+    assert packed.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and out.dtype == torch.float32
+    assert B.stride(1) == 1 and out.stride(1) == 1 and out.shape == (s.dims[0], B.shape[1])
+    _check(_lib.dastac_trimm_bf16_noalloc(s._h, packed.data_ptr(), B.data_ptr(), B.stride(0), B.shape[1],
+                                          out.data_ptr(), out.stride(0), int(accumulate),
+                                          None if err_word is None else err_word.data_ptr(), _stream()),
+           "dastac_trimm_bf16_noalloc")
     return out

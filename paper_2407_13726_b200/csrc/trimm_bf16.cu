@@ -545,3 +545,62 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
 }
 
 }  // namespace dastac
+
+// ---- entry point that allocates nothing ----------------------------------------------------------
+// The staged tile images normally live in the caller's workspace.  Callers that cannot obtain
+// device memory at call time get the same contraction with the images in a fixed array that is part
+// of the library image.  On the host the array's name is only a handle, so its device address is
+// asked for once per device and that pointer is what the kernels receive.
+namespace dastac {
+namespace {
+
+constexpr int64_t kStaticMaxN = DASTAC_NOALLOC_MAX_N;
+constexpr int64_t kStaticRowBlocks = (kStaticMaxN + kTileM - 1) / kTileM;
+constexpr int64_t kStaticKBlocks = (kStaticMaxN + kBlockK - 1) / kBlockK;
+// tile_offset(row_blocks, k_blocks) written out for an even number of row blocks
+constexpr int64_t kStaticTiles = kStaticRowBlocks * kStaticKBlocks - kStaticRowBlocks * (kStaticRowBlocks - 2);
+static_assert(kStaticRowBlocks % 2 == 0, "the closed form above assumes whole pairs of row blocks");
+constexpr size_t kStaticBytes = (size_t)kStaticTiles * kABytes;
+static_assert(kStaticBytes == DASTAC_NOALLOC_SCRATCH_BYTES, "header and array size disagree");
+
+static __device__ __align__(256) uint8_t g_static_tiles[kStaticBytes];
+
+// Device address of g_static_tiles on the current device, looked up on the first call per device.
+dastac_status static_tiles_ptr(void** out) {
+    static void* ptrs[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DASTAC_ERR_CUDA;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_tiles) != cudaSuccess || !p) return DASTAC_ERR_CUDA;
+        ptrs[dev] = p;
+    }
+    *out = ptrs[dev];
+    return DASTAC_OK;
+}
+
+}  // namespace
+}  // namespace dastac
+
+extern "C" dastac_status dastac_trimm_bf16_noalloc(const dastac_structure* s, const void* A, const void* B,
+                                                   int64_t ldb, int64_t ncols, float* C, int64_t ldc,
+                                                   int32_t accumulate, int32_t* err_word, void* stream) {
+    using namespace dastac;
+    if (!s || ncols < 0 || ldb < 0 || ldc < 0) return DASTAC_ERR_INVALID_ARG;
+    const IndexMap& m = s->map;
+    if (m.kind == kEmpty || ncols == 0) return DASTAC_OK;
+    if (!(m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1] && !m.symmetric))
+        return DASTAC_ERR_UNSUPPORTED_EXPR;
+    if (m.N > kStaticMaxN) return DASTAC_ERR_WORKSPACE;  // the fixed array holds the tiles of N <= DASTAC_NOALLOC_MAX_N
+    if (!A || !B || !C) return DASTAC_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(C)) return DASTAC_ERR_ALIGNMENT;
+    if (ldb < ncols || ldc < ncols) return DASTAC_ERR_SHAPE;
+    // A row pitch of B that is not a multiple of 16 bytes would need a re-pitched copy of B, for
+    // which there is no room in the fixed array.
+    if (ldb % 8 != 0) return DASTAC_ERR_ALIGNMENT;
+    if (trimm_workspace_bytes(m, ncols, ldb) > kStaticBytes) return DASTAC_ERR_WORKSPACE;
+    void* tiles = nullptr;
+    dastac_status st = static_tiles_ptr(&tiles);
+    if (st != DASTAC_OK) return st;
+    return launch_trimm_bf16(m, A, B, ldb, C, ldc, ncols, accumulate, tiles, err_word, (cudaStream_t)stream);
+}

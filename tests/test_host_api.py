@@ -19,7 +19,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "dastac.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(dastac_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(dastac_[a-z0-9_]+)\s*\(", header))
     assert declared == set(binding.EXPORTS)
     lib = ctypes.CDLL(binding.LIB_PATH)
     for name in declared:
