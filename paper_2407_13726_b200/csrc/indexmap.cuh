@@ -176,6 +176,46 @@ DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
     }
 }
 
+// For fixed outer indices idx[0 .. rank-2], the innermost indices of the set form one interval
+// [jlo, jhi) and the point (outer, j) is stored at pbase + j: pbase is the loop-invariant part of
+// the ranking polynomial, hoisted out of the innermost loop.  Returns false when the interval is
+// empty or the layout is not contiguous along the innermost index (padded diagonals, or the
+// trailing-extent form of the upper triangle, which is handled by position instead).
+DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int64_t& jhi, int64_t& pbase) {
+    switch (m.kind) {
+        case kDense: {
+            int64_t lin = 0;
+            for (int k = 0; k + 1 < m.rank; ++k) lin = lin * m.dims[k] + idx[k];
+            jlo = 0;
+            jhi = m.dims[m.rank - 1];
+            pbase = lin * jhi;
+            return jhi > 0;
+        }
+        case kUpper: {
+            if (m.rank != 2 || idx[0] >= m.M) return false;
+            jlo = idx[0];
+            jhi = m.N;
+            pbase = upper_row_base(m.N, idx[0]);
+            return true;
+        }
+        case kLower: {
+            jlo = 0;
+            jhi = (int64_t)idx[0] + 1;
+            pbase = tri(idx[0]);
+            return true;
+        }
+        case kTetrahedron: {
+            if (idx[1] < idx[0]) return false;
+            const int64_t n = m.N;
+            jlo = idx[1];
+            jhi = n;
+            pbase = tet(n) - tet(n - idx[0]) + tri(n - idx[0]) - tri(n - idx[1]) - idx[1];
+            return true;
+        }
+        default: return false;
+    }
+}
+
 // Step idx to the point stored at the next position (valid while that position exists).
 // Not defined for the padded-diagonal layout, whose slots are walked by position.
 DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {

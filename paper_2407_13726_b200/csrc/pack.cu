@@ -1,11 +1,20 @@
 // Index-map batch kernels and compress / decompress (Section 3, "Data Layout Compression":
 // iterate over the accessed indices and copy the data in and out of the packed buffer).
 //
-// pack walks the PACKED stream: a thread owns 16 bytes of consecutive packed positions, unranks
-// the first one and steps to the following points with index increments, so the packed side is
-// written with one aligned 128-bit store per thread and the dense side is read along rows.
-// unpack walks the DENSE box: a thread owns 16 bytes of one dense row, so the zero fill and the
-// copy are a single pass with 128-bit stores wherever the dense row allows it.
+// Row kernels (the fast path, unit inner stride): for fixed outer indices the innermost indices of
+// the set are one interval [jlo, jhi) stored contiguously at pbase + j, with pbase the hoisted part
+// of the ranking polynomial.  A group of threads walks one such row.
+//   pack    a thread owns one 16-byte aligned chunk of the PACKED stream inside the row's span.  The
+//           matching dense elements start at an arbitrary element offset, so the thread loads the
+//           two aligned 16-byte granules that cover them and shifts them into place in registers.
+//           Chunks that a row shares with its neighbour (first and last of the row) are written
+//           element by element.
+//   unpack  a thread owns one 16-byte aligned chunk of the DENSE row; the packed source is
+//           realigned the same way, elements outside [jlo, jhi) become zero, and the zero fill of
+//           the rest of the box is the same pass.
+// Generic kernels (any strides, the padded-diagonal layout, the redundancy swap): pack walks the
+// packed stream, a thread unranks the first of its positions and steps with index increments;
+// unpack walks the dense box and ranks every point.
 #include "common.cuh"
 
 namespace dastac {
@@ -131,6 +140,179 @@ __global__ void unpack_kernel(IndexMap m, const T* __restrict__ packed, T* __res
     }
 }
 
+// The 16 bytes that start `sh` bytes into the 32-byte window (lo, hi): word select on sh / 4, then
+// a funnel shift by the remaining bytes.  sh is a multiple of the element size.
+__device__ __forceinline__ uint4 realign16(const uint4 lo, const uint4 hi, const uint32_t sh) {
+    const bool q1 = sh & 4, q2 = sh & 8;
+    const uint32_t bits = (sh & 3) * 8;
+    const uint32_t X0 = q1 ? lo.y : lo.x, X1 = q1 ? lo.z : lo.y, X2 = q1 ? lo.w : lo.z, X3 = q1 ? hi.x : lo.w,
+                   X4 = q1 ? hi.y : hi.x, X5 = q1 ? hi.z : hi.y, X6 = q1 ? hi.w : hi.z;
+    const uint32_t T0 = q2 ? X2 : X0, T1 = q2 ? X3 : X1, T2 = q2 ? X4 : X2, T3 = q2 ? X5 : X3, T4 = q2 ? X6 : X4;
+    return make_uint4(__funnelshift_r(T0, T1, bits), __funnelshift_r(T1, T2, bits), __funnelshift_r(T2, T3, bits),
+                      __funnelshift_r(T3, T4, bits));
+}
+
+constexpr int kRowUnroll = 4;  // 16-byte chunks per thread and row visit
+
+struct RowGeom {
+    int64_t rows;      // product of the outer extents
+    int32_t segs;      // segments per row; a segment is tpr * kRowUnroll chunks of 16 bytes
+    int32_t tpr_log2;  // threads per row inside a block (power of two, <= 256)
+};
+
+// Outer indices of row `row` and the offset of its first dense element.
+__device__ __forceinline__ int64_t decode_row(const IndexMap& m, const Strides& st, int64_t row, int32_t* idx) {
+    if (m.rank == 2) {
+        idx[0] = (int32_t)row;
+        return row * st.s[0];
+    }
+    int64_t off = 0;
+    for (int k = m.rank - 2; k >= 0; --k) {
+        const int64_t q = row / m.dims[k];
+        idx[k] = (int32_t)(row - q * m.dims[k]);
+        off += idx[k] * st.s[k];
+        row = q;
+    }
+    return off;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+pack_rows_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed, RowGeom g) {
+    constexpr int E = 16 / sizeof(T);
+    const int tpr = 1 << g.tpr_log2, rpb = 256 >> g.tpr_log2;
+    const int t = threadIdx.x & (tpr - 1), rib = threadIdx.x >> g.tpr_log2;
+    const int64_t cap = (m.count + E - 1) / E * E;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    for (int64_t row = blockIdx.y * (int64_t)rpb + rib; row < g.rows; row += (int64_t)gridDim.y * rpb) {
+        int32_t idx[3] = {0, 0, 0};
+        const int64_t doff = decode_row(m, st, row, idx);
+        int64_t jlo, jhi, pbase;
+        if (!row_span(m, idx, jlo, jhi, pbase)) continue;
+        const int64_t ps = pbase + jlo, pe = pbase + jhi;  // the row's span in the packed stream
+        const T* drow = dense + doff - pbase;              // drow[p] = dense element stored at position p
+        const int64_t pfirst = (ps / E + (int64_t)blockIdx.x * tpr * kRowUnroll + t) * E;
+        uint4 lo[kRowUnroll], hi[kRowUnroll];
+        uint32_t sh[kRowUnroll];
+#pragma unroll
+        for (int u = 0; u < kRowUnroll; ++u) {
+            const int64_t p0 = pfirst + (int64_t)u * tpr * E;
+            sh[u] = 0;
+            if (p0 >= ps && p0 + E <= pe) {  // the chunk lies inside this row: two aligned granules cover it
+                const uintptr_t addr = reinterpret_cast<uintptr_t>(drow + p0);
+                sh[u] = (uint32_t)(addr & 15);
+                const uint4* src = reinterpret_cast<const uint4*>(addr - sh[u]);
+                lo[u] = __ldg(src);
+                hi[u] = sh[u] ? __ldg(src + 1) : zero4;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kRowUnroll; ++u) {
+            const int64_t p0 = pfirst + (int64_t)u * tpr * E;
+            if (p0 >= pe) break;
+            if (p0 >= ps && p0 + E <= pe) {
+                *reinterpret_cast<uint4*>(packed + p0) = realign16(lo[u], hi[u], sh[u]);
+            } else {  // chunk shared with the neighbouring row, or the tail of the stream
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const int64_t p = p0 + e;
+                    if (p >= ps && p < pe) packed[p] = drow[p];
+                    else if (p >= m.count && p < cap) packed[p] = T(0);
+                }
+            }
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+unpack_rows_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st, RowGeom g) {
+    constexpr int E = 16 / sizeof(T);
+    const int tpr = 1 << g.tpr_log2, rpb = 256 >> g.tpr_log2;
+    const int t = threadIdx.x & (tpr - 1), rib = threadIdx.x >> g.tpr_log2;
+    const int64_t inner = m.dims[m.rank - 1];
+    const int64_t cap = (m.count + E - 1) / E * E;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    union Chunk {
+        uint4 v;
+        T e[E];
+    };
+    for (int64_t row = blockIdx.y * (int64_t)rpb + rib; row < g.rows; row += (int64_t)gridDim.y * rpb) {
+        int32_t idx[3] = {0, 0, 0};
+        const int64_t doff = decode_row(m, st, row, idx);
+        int64_t jlo = 0, jhi = 0, pbase = 0;
+        if (!row_span(m, idx, jlo, jhi, pbase)) jlo = jhi = 0;
+        const int64_t jfirst = ((int64_t)blockIdx.x * tpr * kRowUnroll + t) * E;
+        uint4 lo[kRowUnroll], hi[kRowUnroll];
+        uint32_t sh[kRowUnroll];
+        bool fast[kRowUnroll];
+#pragma unroll
+        for (int u = 0; u < kRowUnroll; ++u) {
+            const int64_t j0 = jfirst + (int64_t)u * tpr * E;
+            const int64_t p0 = pbase + j0, a = p0 & ~(int64_t)(E - 1);
+            fast[u] = j0 < inner && j0 + E > jlo && j0 < jhi && a >= 0 && a + 2 * E <= cap;
+            sh[u] = 0;
+            if (fast[u]) {
+                sh[u] = (uint32_t)(p0 - a) * sizeof(T);
+                lo[u] = __ldg(reinterpret_cast<const uint4*>(packed + a));
+                hi[u] = sh[u] ? __ldg(reinterpret_cast<const uint4*>(packed + a + E)) : zero4;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kRowUnroll; ++u) {
+            const int64_t j0 = jfirst + (int64_t)u * tpr * E;
+            if (j0 >= inner) break;
+            Chunk out;
+            out.v = zero4;
+            if (fast[u]) {
+                out.v = realign16(lo[u], hi[u], sh[u]);
+                if (j0 < jlo || j0 + E > jhi) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e)
+                        if (j0 + e < jlo || j0 + e >= jhi) out.e[e] = T(0);
+                }
+            } else if (j0 + E > jlo && j0 < jhi) {  // the last granules of the packed buffer
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if (j0 + e >= jlo && j0 + e < jhi) out.e[e] = packed[pbase + j0 + e];
+            }
+            T* dst = dense + doff + j0;
+            if (j0 + E <= inner) {
+                *reinterpret_cast<uint4*>(dst) = out.v;
+            } else {
+                for (int e = 0; e < E && j0 + e < inner; ++e) dst[e] = out.e[e];
+            }
+        }
+    }
+}
+
+// Thread layout of the row kernels for elements of `esz` bytes.
+RowGeom row_geom(const IndexMap& m, int esz) {
+    RowGeom g;
+    g.rows = 1;
+    for (int k = 0; k + 1 < m.rank; ++k) g.rows *= m.dims[k];
+    const int64_t chunks = (m.dims[m.rank - 1] * esz + 15) / 16 + 1;  // +1: a span may straddle one more granule
+    const int64_t per_thread = (chunks + kRowUnroll - 1) / kRowUnroll;
+    int lg = 3;
+    while (lg < 8 && (int64_t(1) << lg) < per_thread) ++lg;
+    g.tpr_log2 = lg;
+    const int64_t per_seg = (int64_t(1) << lg) * kRowUnroll;
+    g.segs = (int32_t)((chunks + per_seg - 1) / per_seg);
+    return g;
+}
+
+dim3 row_grid(const RowGeom& g) {
+    const int64_t rpb = 256 >> g.tpr_log2;
+    int64_t gy = (g.rows + rpb - 1) / rpb;
+    if (gy > 32768) gy = 32768;
+    return dim3((unsigned)g.segs, (unsigned)gy);
+}
+
+bool row_path(const IndexMap& m) {
+    return (m.kind == kDense || (m.kind == kUpper && m.rank == 2) || m.kind == kLower || m.kind == kTetrahedron) &&
+           !m.symmetric;
+}
+
 int grid_for(int64_t work_items, int threads) {
     int64_t blocks = (work_items + threads - 1) / threads;
     int64_t cap = (int64_t)sm_count() * 16;
@@ -179,6 +361,17 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
     Strides st{{0, 0, 0}};
     for (int k = 0; k < m.rank; ++k) st.s[k] = dense_strides[k];
     const int E = 16 / elt_size(dtype);
+    if (row_path(m) && st.s[m.rank - 1] == 1 && (reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) {
+        const RowGeom g = row_geom(m, elt_size(dtype));
+        const dim3 grid = row_grid(g);
+        if (dtype == DASTAC_F32)
+            pack_rows_kernel<uint32_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
+                m, (const uint32_t*)dense, st, (uint32_t*)packed, g);
+        else
+            pack_rows_kernel<uint16_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
+                m, (const uint16_t*)dense, st, (uint16_t*)packed, g);
+        return launch_status();
+    }
     const int grid = grid_for((m.slots + E - 1) / E, 256);
     if (dtype == DASTAC_F32)
         pack_kernel<uint32_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
@@ -209,6 +402,17 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
     // every row start on a 16-byte boundary.
     int vector_ok = st.s[m.rank - 1] == 1 && aligned16(dense);
     for (int k = 0; k + 1 < m.rank; ++k) vector_ok = vector_ok && (st.s[k] % E == 0);
+    if (row_path(m) && vector_ok) {
+        const RowGeom g = row_geom(m, esz);
+        const dim3 grid = row_grid(g);
+        if (dtype == DASTAC_F32)
+            unpack_rows_kernel<uint32_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
+                m, (const uint32_t*)packed, (uint32_t*)dense, st, g);
+        else
+            unpack_rows_kernel<uint16_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
+                m, (const uint16_t*)packed, (uint16_t*)dense, st, g);
+        return launch_status();
+    }
     const int last = m.rank - 1;
     int64_t rows = box / m.dims[last];
     const int64_t groups = rows * ((m.dims[last] + E - 1) / E);

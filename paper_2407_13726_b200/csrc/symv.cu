@@ -2,21 +2,29 @@
 // redundancy map, Section 2, "Redundancy map"), fp32.  Every stored off-diagonal element A(i,j)
 // is loaded once and used twice: it adds A(i,j) x[j] to y[i] and A(i,j) x[i] to y[j].
 //
-// Decomposition: the triangle is cut into tiles of kRows rows by kCols columns; only tiles that
-// touch the region j >= i exist.  A thread owns kColsPerThread columns of the tile, keeps their
-// x[j] and their column sums in registers, and walks the rows; row i of the tile is the
-// contiguous packed segment rowbase(i) + j (rowbase advanced by N - i - 1 per row, never
-// re-evaluated).  Row sums are reduced with warp shuffles and shared memory, and each tile
-// issues one atomic add per row and per column it covers.
+// The packed stream is read with aligned 128-bit loads only.  Row i is the contiguous segment
+// rowbase(i) + j, and rowbase(i) mod 4 = r changes from row to row, so an aligned quad of memory
+// holds columns 4q - r .. 4q - r + 3 of the row, where q counts quads from the row's own origin.
+// A thread owns fixed values of q; over the four possible r its quad slides over the seven columns
+// 4q-3 .. 4q+3.  It keeps x and a column sum for those seven columns in registers and a uniform
+// switch on r picks the four that the current row touches, so every register index is static.
+//
+// Decomposition: tiles of kTileRows rows by kTileQuads quads (the tiles partition the memory quads
+// of each row, so every stored element belongs to exactly one tile).  Tiles entirely above the
+// diagonal run without any predicate; tiles that the diagonal or the right edge crosses mask
+// columns j < i (they are the tail of the previous row in memory) and j >= N.  rowbase advances by
+// N - i - 1 per row and is never re-evaluated.  Row sums: warp shuffle, then shared atomics; each
+// tile issues one global atomic per row and per column it covers.
 #include "common.cuh"
 
 namespace dastac {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kColsPerThread = 4;
-constexpr int kCols = kThreads * kColsPerThread;  // 1024
-constexpr int kRows = 64;
+constexpr int kQ = 4;                       // quads per thread and row
+constexpr int kTileQuads = kThreads * kQ;   // 1024 quads
+constexpr int kTileCols = 4 * kTileQuads;   // 4096 columns
+constexpr int kTileRows = 128;
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -24,46 +32,133 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-__global__ void __launch_bounds__(kThreads)
-symv_tile_kernel(int64_t N, int64_t col_tiles, const float* __restrict__ A,
+// One row's contribution for alignment class R: element e of slot k is column c0 + 1024 k - R + e,
+// register 3 - R + e of the slot's seven.
+template <int R, bool kMasked>
+__device__ __forceinline__ void row_fma(const float4 (&a)[kQ], const float (&xw)[kQ][7], float (&cacc)[kQ][7],
+                                        const float xi, float& part, const int i, const int N, const int c0) {
+#pragma unroll
+    for (int k = 0; k < kQ; ++k) {
+        const float v[4] = {a[k].x, a[k].y, a[k].z, a[k].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float vr = v[e], vc = v[e];
+            if (kMasked) {
+                const int j = c0 + k * (4 * kThreads) - R + e;
+                const bool in = j >= i && j < N;
+                vr = in ? v[e] : 0.f;
+                vc = (in && j != i) ? v[e] : 0.f;  // the diagonal element is used once
+            }
+            part = fmaf(vr, xw[k][3 - R + e], part);
+            cacc[k][3 - R + e] = fmaf(vc, xi, cacc[k][3 - R + e]);
+        }
+    }
+}
+
+template <bool kMasked>
+__device__ __forceinline__ void load_row(float4 (&a)[kQ], const float4* __restrict__ A4, const int64_t base,
+                                         const int64_t q0, const int64_t cap_quads, const int i, const int N,
+                                         const int c0) {
+    const int64_t m0 = (base >> 2) + q0;
+    const int r = (int)(base & 3);
+#pragma unroll
+    for (int k = 0; k < kQ; ++k) {
+        if (kMasked) {
+            const int jlo = c0 + k * (4 * kThreads) - r;  // first column of the quad
+            const int64_t m = m0 + k * kThreads;
+            a[k] = (jlo + 3 >= i && jlo < N && m < cap_quads) ? __ldg(A4 + m) : make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+            a[k] = __ldg(A4 + m0 + k * kThreads);
+        }
+    }
+}
+
+template <bool kMasked>
+__device__ __forceinline__ void row_step(const float4 (&a)[kQ], const float (&xw)[kQ][7], float (&cacc)[kQ][7],
+                                         const int r, const float xi, const int i, const int N, const int c0,
+                                         float* row_sum_slot, const int lane) {
+    float part = 0.f;
+    switch (r) {
+        case 0: row_fma<0, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
+        case 1: row_fma<1, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
+        case 2: row_fma<2, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
+        default: row_fma<3, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
+    }
+    part = warp_sum(part);
+    if (lane == 0) atomicAdd(row_sum_slot, part);
+}
+
+template <bool kMasked>
+__device__ __forceinline__ void tile_rows(const int N, const int64_t cap_quads, const int i0, const int i_end,
+                                          const int64_t q0, const int c0, const float4* __restrict__ A4,
+                                          const float (&xw)[kQ][7], float (&cacc)[kQ][7], const float* xs,
+                                          float* row_sum, const int lane) {
+    int64_t base = upper_row_base(N, i0);
+    int i = i0;
+    for (; i + 1 < i_end; i += 2) {
+        const int64_t base1 = base + (N - i - 1);
+        float4 a0[kQ], a1[kQ];
+        load_row<kMasked>(a0, A4, base, q0, cap_quads, i, N, c0);
+        load_row<kMasked>(a1, A4, base1, q0, cap_quads, i + 1, N, c0);
+        row_step<kMasked>(a0, xw, cacc, (int)(base & 3), xs[i - i0], i, N, c0, row_sum + (i - i0), lane);
+        row_step<kMasked>(a1, xw, cacc, (int)(base1 & 3), xs[i + 1 - i0], i + 1, N, c0, row_sum + (i + 1 - i0), lane);
+        base = base1 + (N - i - 2);
+    }
+    if (i < i_end) {
+        float4 a0[kQ];
+        load_row<kMasked>(a0, A4, base, q0, cap_quads, i, N, c0);
+        row_step<kMasked>(a0, xw, cacc, (int)(base & 3), xs[i - i0], i, N, c0, row_sum + (i - i0), lane);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, const float* __restrict__ A,
                  const float* __restrict__ x, float* __restrict__ y) {
-    __shared__ float row_sum[kRows];
-    const int64_t I = blockIdx.x / col_tiles, J = blockIdx.x - I * col_tiles;
-    const int64_t i0 = I * kRows, j0 = J * kCols;
-    if (j0 + kCols - 1 < i0) return;  // tile lies entirely below the diagonal
+    __shared__ float col_sum[kTileCols + 8];  // columns J*kTileCols - 4 ..
+    __shared__ float row_sum[kTileRows];
+    __shared__ float xs[kTileRows];
+    const int I = blockIdx.x / col_tiles, J = blockIdx.x - I * col_tiles;
+    const int i0 = I * kTileRows;
+    const int64_t col_lo = (int64_t)J * kTileCols;  // column of the tile's first quad when r = 0
+    if (col_lo + kTileCols - 1 < i0) return;          // every column of the tile lies left of the diagonal
+    const int i_end = (i0 + kTileRows < N) ? i0 + kTileRows : N;
     const int tid = threadIdx.x, lane = tid & 31;
-    if (tid < kRows) row_sum[tid] = 0.f;
+    for (int t = tid; t < kTileCols + 8; t += kThreads) col_sum[t] = 0.f;
+    if (tid < kTileRows) {
+        row_sum[tid] = 0.f;
+        xs[tid] = (i0 + tid < N) ? x[i0 + tid] : 0.f;
+    }
+    const int c0 = (int)col_lo + 4 * tid;  // column 4q of the thread's slot 0
+    float xw[kQ][7], cacc[kQ][7];
+#pragma unroll
+    for (int k = 0; k < kQ; ++k)
+#pragma unroll
+        for (int d = 0; d < 7; ++d) {
+            const int j = c0 + k * (4 * kThreads) - 3 + d;
+            xw[k][d] = (j >= 0 && j < N) ? __ldg(x + j) : 0.f;
+            cacc[k][d] = 0.f;
+        }
     __syncthreads();
 
-    int64_t j[kColsPerThread];
-    float xj[kColsPerThread], col_acc[kColsPerThread];
+    const float4* A4 = reinterpret_cast<const float4*>(A);
+    const int64_t q0 = (int64_t)J * kTileQuads + tid;
+    // strictly above the diagonal for every row and alignment, and inside the matrix
+    const bool interior = (col_lo - 3 > (int64_t)i_end - 1) && (col_lo + kTileCols - 1 < N);
+    if (interior)
+        tile_rows<false>(N, cap_quads, i0, i_end, q0, c0, A4, xw, cacc, xs, row_sum, lane);
+    else
+        tile_rows<true>(N, cap_quads, i0, i_end, q0, c0, A4, xw, cacc, xs, row_sum, lane);
+
 #pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c) {
-        j[c] = j0 + tid + c * kThreads;
-        xj[c] = j[c] < N ? x[j[c]] : 0.f;
-        col_acc[c] = 0.f;
-    }
-    const int64_t i_end = (i0 + kRows < N) ? i0 + kRows : N;
-    int64_t base = upper_row_base(N, i0);
-#pragma unroll 4
-    for (int64_t i = i0; i < i_end; ++i) {
-        const float xi = x[i];
-        float part = 0.f;
+    for (int k = 0; k < kQ; ++k)
 #pragma unroll
-        for (int c = 0; c < kColsPerThread; ++c) {
-            float a = (j[c] >= i && j[c] < N) ? A[base + j[c]] : 0.f;
-            part = fmaf(a, xj[c], part);
-            if (j[c] != i) col_acc[c] = fmaf(a, xi, col_acc[c]);
-        }
-        part = warp_sum(part);
-        if (lane == 0) atomicAdd(&row_sum[i - i0], part);
-        base += N - i - 1;
-    }
+        for (int d = 0; d < 7; ++d) atomicAdd(&col_sum[4 * (k * kThreads + tid) + 1 + d], cacc[k][d]);
     __syncthreads();
-    if (tid < kRows && i0 + tid < N) atomicAdd(&y[i0 + tid], row_sum[tid]);
-#pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c)
-        if (j[c] < N && j[c] > i0) atomicAdd(&y[j[c]], col_acc[c]);
+    if (tid < kTileRows && i0 + tid < N) atomicAdd(&y[i0 + tid], row_sum[tid]);
+    for (int t = tid; t < kTileCols + 8; t += kThreads) {
+        const int64_t j = col_lo - 4 + t;
+        if (j > i0 && j < N) atomicAdd(&y[j], col_sum[t]);  // column j only receives from rows i < j
+    }
 }
 
 }  // namespace
@@ -76,9 +171,11 @@ dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, flo
     if (N == 0) return DASTAC_OK;
     if (!accumulate && cudaMemsetAsync(y, 0, (size_t)N * sizeof(float), st) != cudaSuccess)
         return DASTAC_ERR_CUDA;
-    const int64_t row_tiles = (N + kRows - 1) / kRows, col_tiles = (N + kCols - 1) / kCols;
+    const int64_t quads_per_row = (N + 2) / 4 + 1;  // quads that can hold a column < N for some alignment
+    const int64_t row_tiles = (N + kTileRows - 1) / kTileRows, col_tiles = (quads_per_row + kTileQuads - 1) / kTileQuads;
     if (row_tiles * col_tiles > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
-    symv_tile_kernel<<<(unsigned)(row_tiles * col_tiles), kThreads, 0, st>>>(N, col_tiles, A, x, y);
+    const int64_t cap_quads = (m.count + 3) / 4;
+    symv_quad_kernel<<<(unsigned)(row_tiles * col_tiles), kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
     return launch_status();
 }
 
