@@ -1,17 +1,18 @@
 // Index-map batch kernels and compress / decompress (Section 3, "Data Layout Compression":
 // iterate over the accessed indices and copy the data in and out of the packed buffer).
 //
-// Row kernels (the fast path, unit inner stride): for fixed outer indices the innermost indices of
-// the set are one interval [jlo, jhi) stored contiguously at pbase + j, with pbase the hoisted part
-// of the ranking polynomial.  A group of threads walks one such row.
-//   pack    a thread owns one 16-byte aligned chunk of the PACKED stream inside the row's span.  The
-//           matching dense elements start at an arbitrary element offset, so the thread loads the
-//           two aligned 16-byte granules that cover them and shifts them into place in registers.
-//           Chunks that a row shares with its neighbour (first and last of the row) are written
-//           element by element.
-//   unpack  a thread owns one 16-byte aligned chunk of the DENSE row; the packed source is
-//           realigned the same way, elements outside [jlo, jhi) become zero, and the zero fill of
-//           the rest of the box is the same pass.
+// Stream kernels (the fast path, unit inner stride): for fixed outer indices the innermost indices
+// of the set are one interval [jlo, jhi) stored contiguously at pbase + j, with pbase the hoisted
+// part of the ranking polynomial.
+//   pack    a lane owns 16-byte aligned chunks of the PACKED stream.  The matching dense elements
+//           start at an arbitrary element offset, so the lane loads the two aligned 16-byte granules
+//           that cover them and shifts them into place in registers.  Chunks that a row shares with
+//           its neighbour (first and last of the row) are written element by element.  Warps own
+//           equal ranges of the stream, found by one unrank each: the uneven row lengths do not
+//           unbalance the work.
+//   unpack  a lane owns 16-byte aligned chunks of a DENSE row; the packed source is realigned the
+//           same way, elements outside [jlo, jhi) become zero, and the zero fill of the rest of the
+//           box is the same pass.
 // Generic kernels (any strides, the padded-diagonal layout, the redundancy swap): pack walks the
 // packed stream, a thread unranks the first of its positions and steps with index increments;
 // unpack walks the dense box and ranks every point.
@@ -152,84 +153,116 @@ __device__ __forceinline__ uint4 realign16(const uint4 lo, const uint4 hi, const
                       __funnelshift_r(T3, T4, bits));
 }
 
-constexpr int kRowUnroll = 4;  // 16-byte chunks per thread and row visit
+constexpr int kUnroll = 4;         // 16-byte chunks per lane and pass
+constexpr int kWarpsPerBlock = 8;
 
-struct RowGeom {
-    int64_t rows;      // product of the outer extents
-    int32_t segs;      // segments per row; a segment is tpr * kRowUnroll chunks of 16 bytes
-    int32_t tpr_log2;  // threads per row inside a block (power of two, <= 256)
-};
-
-// Outer indices of row `row` and the offset of its first dense element.
-__device__ __forceinline__ int64_t decode_row(const IndexMap& m, const Strides& st, int64_t row, int32_t* idx) {
-    if (m.rank == 2) {
-        idx[0] = (int32_t)row;
-        return row * st.s[0];
-    }
+// Offset of the first dense element of the row that holds idx (outer indices only).
+__device__ __forceinline__ int64_t dense_row_offset(const IndexMap& m, const Strides& st, const int32_t* idx) {
     int64_t off = 0;
-    for (int k = m.rank - 2; k >= 0; --k) {
-        const int64_t q = row / m.dims[k];
-        idx[k] = (int32_t)(row - q * m.dims[k]);
-        off += idx[k] * st.s[k];
-        row = q;
-    }
+    for (int k = 0; k + 1 < m.rank; ++k) off += idx[k] * st.s[k];
     return off;
 }
 
+// One 16-byte chunk of the packed stream by the generic walk: unrank its first position, then step.
 template <typename T>
-__global__ void __launch_bounds__(256)
-pack_rows_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed, RowGeom g) {
+__device__ __forceinline__ void pack_chunk_by_points(const IndexMap& m, const T* __restrict__ dense, const Strides& st,
+                                                     T* __restrict__ packed, const int64_t p0) {
     constexpr int E = 16 / sizeof(T);
-    const int tpr = 1 << g.tpr_log2, rpb = 256 >> g.tpr_log2;
-    const int t = threadIdx.x & (tpr - 1), rib = threadIdx.x >> g.tpr_log2;
-    const int64_t cap = (m.count + E - 1) / E * E;
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    for (int64_t row = blockIdx.y * (int64_t)rpb + rib; row < g.rows; row += (int64_t)gridDim.y * rpb) {
-        int32_t idx[3] = {0, 0, 0};
-        const int64_t doff = decode_row(m, st, row, idx);
-        int64_t jlo, jhi, pbase;
-        if (!row_span(m, idx, jlo, jhi, pbase)) continue;
-        const int64_t ps = pbase + jlo, pe = pbase + jhi;  // the row's span in the packed stream
-        const T* drow = dense + doff - pbase;              // drow[p] = dense element stored at position p
-        const int64_t pfirst = (ps / E + (int64_t)blockIdx.x * tpr * kRowUnroll + t) * E;
-        uint4 lo[kRowUnroll], hi[kRowUnroll];
-        uint32_t sh[kRowUnroll];
+    Vec16<T> out;
+    int32_t idx[3] = {0, 0, 0};
+    unrank_of(m, p0, idx);
 #pragma unroll
-        for (int u = 0; u < kRowUnroll; ++u) {
-            const int64_t p0 = pfirst + (int64_t)u * tpr * E;
-            sh[u] = 0;
-            if (p0 >= ps && p0 + E <= pe) {  // the chunk lies inside this row: two aligned granules cover it
-                const uintptr_t addr = reinterpret_cast<uintptr_t>(drow + p0);
-                sh[u] = (uint32_t)(addr & 15);
-                const uint4* src = reinterpret_cast<const uint4*>(addr - sh[u]);
-                lo[u] = __ldg(src);
-                hi[u] = sh[u] ? __ldg(src + 1) : zero4;
-            }
+    for (int e = 0; e < E; ++e) {
+        T val = T(0);
+        if (p0 + e < m.count) {
+            val = dense[idx[0] * st.s[0] + idx[1] * st.s[1] + idx[2] * st.s[2]];
+            advance(m, idx);
         }
+        out.v[e] = val;
+    }
+    *reinterpret_cast<uint4*>(packed + p0) = *reinterpret_cast<const uint4*>(out.v);
+}
+
+// pack: every warp owns an equal, contiguous range of 16-byte chunks of the packed stream, whatever
+// the row lengths are.  It unranks the first position of its range once and then walks from row to
+// row with index increments.  Where rows are shorter than one pass of the warp (the tip of a
+// triangle) the lanes stop cooperating and each takes whole chunks by the generic walk.
+template <typename T>
+__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
+pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed,
+                   int64_t chunks_per_warp) {
+    constexpr int E = 16 / sizeof(T);
+    const int lane = threadIdx.x & 31;
+    const int64_t total = (m.count + E - 1) / E;
+    const int64_t cA = (blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5)) * chunks_per_warp;
+    if (cA >= total) return;
+    const int64_t cB = (cA + chunks_per_warp < total) ? cA + chunks_per_warp : total;
+    const int last = m.rank - 1;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    int32_t idx[3] = {0, 0, 0};
+    unrank_of(m, cA * E, idx);
+    int64_t c_cur = cA;
+    while (c_cur < cB) {
+        int64_t jlo = 0, jhi = 0, pbase = 0;
+        row_span(m, idx, jlo, jhi, pbase);
+        if ((jhi - jlo) < 32 * E) {
+            const int64_t batch_end = (c_cur + 32 * kUnroll < cB) ? c_cur + 32 * kUnroll : cB;
+            for (int64_t c = c_cur + lane; c < batch_end; c += 32) pack_chunk_by_points<T>(m, dense, st, packed, c * E);
+            c_cur = batch_end;
+            if (c_cur < cB) unrank_of(m, c_cur * E, idx);
+            continue;
+        }
+        const int64_t ps = pbase + jlo, pe = pbase + jhi;  // the row's span in the packed stream
+        const T* drow = dense + dense_row_offset(m, st, idx) - pbase;  // drow[p]: element stored at position p
+        const int64_t c_lo = (ps / E > c_cur) ? ps / E : c_cur;
+        const int64_t c_end = (pe + E - 1) / E;
+        const int64_t c_hi = (c_end < cB) ? c_end : cB;
+        for (int64_t c0 = c_lo + lane; c0 < c_hi; c0 += 32 * kUnroll) {
+            uint4 lo[kUnroll], hi[kUnroll];
+            uint32_t sh[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kRowUnroll; ++u) {
-            const int64_t p0 = pfirst + (int64_t)u * tpr * E;
-            if (p0 >= pe) break;
-            if (p0 >= ps && p0 + E <= pe) {
-                *reinterpret_cast<uint4*>(packed + p0) = realign16(lo[u], hi[u], sh[u]);
-            } else {  // chunk shared with the neighbouring row, or the tail of the stream
+            for (int u = 0; u < kUnroll; ++u) {
+                const int64_t p0 = (c0 + 32 * u) * E;
+                sh[u] = 0;
+                if (c0 + 32 * u < c_hi && p0 >= ps && p0 + E <= pe) {  // whole chunk inside this row
+                    const uintptr_t addr = reinterpret_cast<uintptr_t>(drow + p0);
+                    sh[u] = (uint32_t)(addr & 15);
+                    const uint4* src = reinterpret_cast<const uint4*>(addr - sh[u]);
+                    lo[u] = __ldg(src);
+                    hi[u] = sh[u] ? __ldg(src + 1) : zero4;
+                }
+            }
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const int64_t p = p0 + e;
-                    if (p >= ps && p < pe) packed[p] = drow[p];
-                    else if (p >= m.count && p < cap) packed[p] = T(0);
+            for (int u = 0; u < kUnroll; ++u) {
+                const int64_t p0 = (c0 + 32 * u) * E;
+                if (c0 + 32 * u >= c_hi) break;
+                if (p0 >= ps && p0 + E <= pe) {
+                    *reinterpret_cast<uint4*>(packed + p0) = realign16(lo[u], hi[u], sh[u]);
+                } else {  // chunk shared with the neighbouring row, or the tail of the stream
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const int64_t p = p0 + e;
+                        if (p >= ps && p < pe) packed[p] = drow[p];
+                        else if (p >= m.count) packed[p] = T(0);
+                    }
                 }
             }
         }
+        if (pe >= m.count) break;
+        c_cur = pe / E;  // a chunk shared with the next row is visited again for that row's part
+        idx[last] = (int32_t)(jhi - 1);
+        advance(m, idx);  // first point of the next row
     }
 }
 
+// unpack: a warp item is a window of 32 * kUnroll chunks of one dense row; the zero fill outside
+// the set and the copy are the same pass.
 template <typename T>
-__global__ void __launch_bounds__(256)
-unpack_rows_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st, RowGeom g) {
+__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
+unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st,
+                     int64_t rows, int64_t windows_per_row) {
     constexpr int E = 16 / sizeof(T);
-    const int tpr = 1 << g.tpr_log2, rpb = 256 >> g.tpr_log2;
-    const int t = threadIdx.x & (tpr - 1), rib = threadIdx.x >> g.tpr_log2;
+    const int lane = threadIdx.x & 31;
     const int64_t inner = m.dims[m.rank - 1];
     const int64_t cap = (m.count + E - 1) / E * E;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
@@ -237,34 +270,41 @@ unpack_rows_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
         uint4 v;
         T e[E];
     };
-    for (int64_t row = blockIdx.y * (int64_t)rpb + rib; row < g.rows; row += (int64_t)gridDim.y * rpb) {
+    const int64_t warps = (int64_t)gridDim.x * kWarpsPerBlock;
+    for (int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5); item < rows * windows_per_row;
+         item += warps) {
+        int64_t row = item / windows_per_row;
+        const int64_t win = item - row * windows_per_row;
         int32_t idx[3] = {0, 0, 0};
-        const int64_t doff = decode_row(m, st, row, idx);
+        for (int k = m.rank - 2; k >= 0; --k) {
+            const int64_t q = row / m.dims[k];
+            idx[k] = (int32_t)(row - q * m.dims[k]);
+            row = q;
+        }
         int64_t jlo = 0, jhi = 0, pbase = 0;
         if (!row_span(m, idx, jlo, jhi, pbase)) jlo = jhi = 0;
-        const int64_t jfirst = ((int64_t)blockIdx.x * tpr * kRowUnroll + t) * E;
-        uint4 lo[kRowUnroll], hi[kRowUnroll];
-        uint32_t sh[kRowUnroll];
-        bool fast[kRowUnroll];
+        T* drow = dense + dense_row_offset(m, st, idx);
+        const int64_t jfirst = (win * (32 * kUnroll) + lane) * E;
+        uint4 lo[kUnroll], hi[kUnroll];
+        uint32_t sh[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kRowUnroll; ++u) {
-            const int64_t j0 = jfirst + (int64_t)u * tpr * E;
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t j0 = jfirst + 32 * u * E;
             const int64_t p0 = pbase + j0, a = p0 & ~(int64_t)(E - 1);
-            fast[u] = j0 < inner && j0 + E > jlo && j0 < jhi && a >= 0 && a + 2 * E <= cap;
-            sh[u] = 0;
-            if (fast[u]) {
+            sh[u] = 0xffffffffu;  // no vector load for this chunk
+            if (j0 < inner && j0 + E > jlo && j0 < jhi && a >= 0 && a + 2 * E <= cap) {
                 sh[u] = (uint32_t)(p0 - a) * sizeof(T);
                 lo[u] = __ldg(reinterpret_cast<const uint4*>(packed + a));
                 hi[u] = sh[u] ? __ldg(reinterpret_cast<const uint4*>(packed + a + E)) : zero4;
             }
         }
 #pragma unroll
-        for (int u = 0; u < kRowUnroll; ++u) {
-            const int64_t j0 = jfirst + (int64_t)u * tpr * E;
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t j0 = jfirst + 32 * u * E;
             if (j0 >= inner) break;
             Chunk out;
             out.v = zero4;
-            if (fast[u]) {
+            if (sh[u] != 0xffffffffu) {
                 out.v = realign16(lo[u], hi[u], sh[u]);
                 if (j0 < jlo || j0 + E > jhi) {
 #pragma unroll
@@ -276,36 +316,13 @@ unpack_rows_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
                 for (int e = 0; e < E; ++e)
                     if (j0 + e >= jlo && j0 + e < jhi) out.e[e] = packed[pbase + j0 + e];
             }
-            T* dst = dense + doff + j0;
             if (j0 + E <= inner) {
-                *reinterpret_cast<uint4*>(dst) = out.v;
+                *reinterpret_cast<uint4*>(drow + j0) = out.v;
             } else {
-                for (int e = 0; e < E && j0 + e < inner; ++e) dst[e] = out.e[e];
+                for (int e = 0; e < E && j0 + e < inner; ++e) drow[j0 + e] = out.e[e];
             }
         }
     }
-}
-
-// Thread layout of the row kernels for elements of `esz` bytes.
-RowGeom row_geom(const IndexMap& m, int esz) {
-    RowGeom g;
-    g.rows = 1;
-    for (int k = 0; k + 1 < m.rank; ++k) g.rows *= m.dims[k];
-    const int64_t chunks = (m.dims[m.rank - 1] * esz + 15) / 16 + 1;  // +1: a span may straddle one more granule
-    const int64_t per_thread = (chunks + kRowUnroll - 1) / kRowUnroll;
-    int lg = 3;
-    while (lg < 8 && (int64_t(1) << lg) < per_thread) ++lg;
-    g.tpr_log2 = lg;
-    const int64_t per_seg = (int64_t(1) << lg) * kRowUnroll;
-    g.segs = (int32_t)((chunks + per_seg - 1) / per_seg);
-    return g;
-}
-
-dim3 row_grid(const RowGeom& g) {
-    const int64_t rpb = 256 >> g.tpr_log2;
-    int64_t gy = (g.rows + rpb - 1) / rpb;
-    if (gy > 32768) gy = 32768;
-    return dim3((unsigned)g.segs, (unsigned)gy);
 }
 
 bool row_path(const IndexMap& m) {
@@ -362,14 +379,15 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
     for (int k = 0; k < m.rank; ++k) st.s[k] = dense_strides[k];
     const int E = 16 / elt_size(dtype);
     if (row_path(m) && st.s[m.rank - 1] == 1 && (reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) {
-        const RowGeom g = row_geom(m, elt_size(dtype));
-        const dim3 grid = row_grid(g);
+        const int64_t total = (m.count + E - 1) / E;
+        const int64_t cpw = 2 * 32 * kUnroll;  // two passes of a warp: short enough to balance the tip of a triangle
+        const int64_t blocks = ((total + cpw - 1) / cpw + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (dtype == DASTAC_F32)
-            pack_rows_kernel<uint32_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
-                m, (const uint32_t*)dense, st, (uint32_t*)packed, g);
+            pack_stream_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
+                m, (const uint32_t*)dense, st, (uint32_t*)packed, cpw);
         else
-            pack_rows_kernel<uint16_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
-                m, (const uint16_t*)dense, st, (uint16_t*)packed, g);
+            pack_stream_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
+                m, (const uint16_t*)dense, st, (uint16_t*)packed, cpw);
         return launch_status();
     }
     const int grid = grid_for((m.slots + E - 1) / E, 256);
@@ -403,14 +421,16 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
     int vector_ok = st.s[m.rank - 1] == 1 && aligned16(dense);
     for (int k = 0; k + 1 < m.rank; ++k) vector_ok = vector_ok && (st.s[k] % E == 0);
     if (row_path(m) && vector_ok) {
-        const RowGeom g = row_geom(m, esz);
-        const dim3 grid = row_grid(g);
+        const int64_t rows = box / m.dims[m.rank - 1];
+        const int64_t chunks_per_row = (m.dims[m.rank - 1] + E - 1) / E;
+        const int64_t wpr = (chunks_per_row + 32 * kUnroll - 1) / (32 * kUnroll);
+        const int grid = grid_for(rows * wpr * 32, 32 * kWarpsPerBlock);
         if (dtype == DASTAC_F32)
-            unpack_rows_kernel<uint32_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
-                m, (const uint32_t*)packed, (uint32_t*)dense, st, g);
+            unpack_stream_kernel<uint32_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
+                m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, wpr);
         else
-            unpack_rows_kernel<uint16_t><<<grid, 256, 0, (cudaStream_t)stream>>>(
-                m, (const uint16_t*)packed, (uint16_t*)dense, st, g);
+            unpack_stream_kernel<uint16_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
+                m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, wpr);
         return launch_status();
     }
     const int last = m.rank - 1;

@@ -21,9 +21,9 @@ namespace dastac {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kQ = 4;                       // quads per thread and row
-constexpr int kTileQuads = kThreads * kQ;   // 1024 quads
-constexpr int kTileCols = 4 * kTileQuads;   // 4096 columns
+constexpr int kQ = 2;                       // quads per thread and row
+constexpr int kTileQuads = kThreads * kQ;   // 512 quads
+constexpr int kTileCols = 4 * kTileQuads;   // 2048 columns
 constexpr int kTileRows = 128;
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -32,7 +32,7 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// One row's contribution for alignment class R: element e of slot k is column c0 + 1024 k - R + e,
+// One row's contribution for alignment class R: element e of slot k is column c0 + 4 kThreads k - R + e,
 // register 3 - R + e of the slot's seven.
 template <int R, bool kMasked>
 __device__ __forceinline__ void row_fma(const float4 (&a)[kQ], const float (&xw)[kQ][7], float (&cacc)[kQ][7],
@@ -111,7 +111,7 @@ __device__ __forceinline__ void tile_rows(const int N, const int64_t cap_quads, 
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 4)
 symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, const float* __restrict__ A,
                  const float* __restrict__ x, float* __restrict__ y) {
     __shared__ float col_sum[kTileCols + 8];  // columns J*kTileCols - 4 ..
