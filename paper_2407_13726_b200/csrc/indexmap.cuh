@@ -86,8 +86,10 @@ DASTAC_HD int64_t upper_row_of(int64_t N, int64_t t) {
 }
 
 DASTAC_HD bool in_set(const IndexMap& m, const int32_t* idx) {
-    for (int k = 0; k < m.rank; ++k)
-        if (idx[k] < 0 || idx[k] >= m.dims[k]) return false;
+    // fixed trip counts with a guard keep idx and m in registers (no dynamically indexed arrays)
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+        if (k < m.rank && (idx[k] < 0 || idx[k] >= m.dims[k])) return false;
     switch (m.kind) {
         case kDense: return true;
         case kUpper: return idx[0] <= idx[1];
@@ -106,7 +108,9 @@ DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
     switch (m.kind) {
         case kDense: {
             int64_t lin = 0;
-            for (int k = 0; k < m.rank; ++k) lin = lin * m.dims[k] + idx[k];
+#pragma unroll
+            for (int k = 0; k < 3; ++k)
+                if (k < m.rank) lin = lin * m.dims[k] + idx[k];
             return lin;
         }
         case kUpper: {
@@ -128,11 +132,13 @@ DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
 DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
     switch (m.kind) {
         case kDense: {
-            for (int k = m.rank - 1; k >= 0; --k) {
-                int64_t q = p / m.dims[k];
-                idx[k] = (int32_t)(p - q * m.dims[k]);
-                p = q;
-            }
+#pragma unroll
+            for (int k = 2; k >= 0; --k)
+                if (k < m.rank) {
+                    int64_t q = p / m.dims[k];
+                    idx[k] = (int32_t)(p - q * m.dims[k]);
+                    p = q;
+                }
             return;
         }
         case kUpper: {
@@ -185,9 +191,11 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
     switch (m.kind) {
         case kDense: {
             int64_t lin = 0;
-            for (int k = 0; k + 1 < m.rank; ++k) lin = lin * m.dims[k] + idx[k];
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+                if (k + 1 < m.rank) lin = lin * m.dims[k] + idx[k];
             jlo = 0;
-            jhi = m.dims[m.rank - 1];
+            jhi = m.rank == 3 ? m.dims[2] : m.rank == 2 ? m.dims[1] : m.dims[0];
             pbase = lin * jhi;
             return jhi > 0;
         }
@@ -221,10 +229,12 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
 DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {
     switch (m.kind) {
         case kDense: {
-            for (int k = m.rank - 1; k >= 0; --k) {
-                if (++idx[k] < m.dims[k]) return;
-                idx[k] = 0;
-            }
+#pragma unroll
+            for (int k = 2; k >= 0; --k)
+                if (k < m.rank) {
+                    if (++idx[k] < m.dims[k]) return;
+                    idx[k] = 0;
+                }
             return;
         }
         case kUpper: {

@@ -30,7 +30,9 @@ __global__ void rank_batch_kernel(IndexMap m, const int32_t* __restrict__ idx, i
     for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < n;
          t += (int64_t)gridDim.x * blockDim.x) {
         int32_t p[3] = {0, 0, 0};
-        for (int k = 0; k < m.rank; ++k) p[k] = idx[t * m.rank + k];
+#pragma unroll
+        for (int k = 0; k < 3; ++k)
+            if (k < m.rank) p[k] = idx[t * m.rank + k];
         off[t] = in_set(m, p) ? rank_of(m, p) : -1;
     }
 }
@@ -42,7 +44,9 @@ __global__ void unrank_batch_kernel(IndexMap m, const int64_t* __restrict__ off,
         int32_t p[3] = {-1, -1, -1};
         int64_t o = off[t];
         if (o >= 0 && o < m.slots) unrank_of(m, o, p);
-        for (int k = 0; k < m.rank; ++k) idx[t * m.rank + k] = p[k];
+#pragma unroll
+        for (int k = 0; k < 3; ++k)
+            if (k < m.rank) idx[t * m.rank + k] = p[k];
     }
 }
 
@@ -159,7 +163,9 @@ constexpr int kWarpsPerBlock = 8;
 // Offset of the first dense element of the row that holds idx (outer indices only).
 __device__ __forceinline__ int64_t dense_row_offset(const IndexMap& m, const Strides& st, const int32_t* idx) {
     int64_t off = 0;
-    for (int k = 0; k + 1 < m.rank; ++k) off += idx[k] * st.s[k];
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+        if (k + 1 < m.rank) off += idx[k] * st.s[k];
     return off;
 }
 
@@ -197,7 +203,6 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
     const int64_t cA = (blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5)) * chunks_per_warp;
     if (cA >= total) return;
     const int64_t cB = (cA + chunks_per_warp < total) ? cA + chunks_per_warp : total;
-    const int last = m.rank - 1;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     int32_t idx[3] = {0, 0, 0};
     unrank_of(m, cA * E, idx);
@@ -250,7 +255,9 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
         }
         if (pe >= m.count) break;
         c_cur = pe / E;  // a chunk shared with the next row is visited again for that row's part
-        idx[last] = (int32_t)(jhi - 1);
+        if (m.rank == 3) idx[2] = (int32_t)(jhi - 1);
+        else if (m.rank == 2) idx[1] = (int32_t)(jhi - 1);
+        else idx[0] = (int32_t)(jhi - 1);
         advance(m, idx);  // first point of the next row
     }
 }
@@ -263,7 +270,7 @@ unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ d
                      int64_t rows, int64_t windows_per_row) {
     constexpr int E = 16 / sizeof(T);
     const int lane = threadIdx.x & 31;
-    const int64_t inner = m.dims[m.rank - 1];
+    const int64_t inner = m.rank == 3 ? m.dims[2] : m.rank == 2 ? m.dims[1] : m.dims[0];
     const int64_t cap = (m.count + E - 1) / E * E;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     union Chunk {
@@ -276,11 +283,13 @@ unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ d
         int64_t row = item / windows_per_row;
         const int64_t win = item - row * windows_per_row;
         int32_t idx[3] = {0, 0, 0};
-        for (int k = m.rank - 2; k >= 0; --k) {
-            const int64_t q = row / m.dims[k];
-            idx[k] = (int32_t)(row - q * m.dims[k]);
-            row = q;
-        }
+#pragma unroll
+        for (int k = 1; k >= 0; --k)
+            if (k + 1 < m.rank) {
+                const int64_t q = row / m.dims[k];
+                idx[k] = (int32_t)(row - q * m.dims[k]);
+                row = q;
+            }
         int64_t jlo = 0, jhi = 0, pbase = 0;
         if (!row_span(m, idx, jlo, jhi, pbase)) jlo = jhi = 0;
         T* drow = dense + dense_row_offset(m, st, idx);
