@@ -3,10 +3,14 @@
 // kernel; this is its SpMV_UT / TTM_UT access pattern (Table 1) widened to a dense right-hand
 // side and mapped on tcgen05.
 //
-// Tiling.  An output tile is 128 rows x 256 columns.  Row block I only needs K blocks (64 columns
-// of A, 64 rows of B) from the diagonal on: kb = 2I .. ceil(N/64)-1, so the executed MMA work is
-// the triangle plus half a tile per row block.  Tiles are ordered by decreasing K length and dealt
-// round-robin to one persistent CTA per SM.
+// Tiling.  An output tile is 256 rows x 256 columns: two 128-row blocks (2P, 2P+1), each with its
+// own accumulator, that share every staged 64 x 256 block of B.  Per 64-deep K block a CTA then
+// moves 64 KiB through shared memory for two M128 N256 MMAs, instead of 48 KiB for one: with the
+// few hundred KB a CTA can keep in flight, the bytes per MMA cycle, not the tensor pipe, set the
+// pace of this kernel.  A pair only needs K blocks from its diagonal on: kb = 4P .. ceil(N/64)-1,
+// so the executed MMA work is the triangle plus one tile per pair.  Tiles are ordered by
+// decreasing K length and dealt to one persistent CTA per SM in boustrophedon order, which gives
+// every CTA the same mix of long and short tiles.
 //
 // Two kernels per call:
 //  1. stage_a: the packed row pitch changes with the row and row starts are only 2-byte aligned,
@@ -20,14 +24,14 @@
 //     every column tile of its row block).  The workspace stays packed: it holds the triangle's
 //     tiles only.
 //  2. trimm_tcgen05: warp-specialised pipeline,
-//       warps 0-3  epilogue: tcgen05.ld of the accumulator (warp w owns TMEM lanes 32w..32w+31),
-//                  128-bit stores to C
-//       warp  4    one lane issues, per K block, one bulk copy of the staged A tile and four TMA
+//       warps 0-7  epilogue: tcgen05.ld of the accumulators (warps 0-3 the upper row block, 4-7
+//                  the lower; warp w owns TMEM lanes 32(w%4)..32(w%4)+31), 128-bit stores to C
+//       warp  8    one lane issues, per K block, two bulk copies of staged A tiles and four TMA
 //                  boxes (64x64, 128B swizzle) of B into the stage, all on one mbarrier
-//       warp  5    allocates tensor memory; one lane issues tcgen05.mma (M128 N256 K16, four per
+//       warp  9    allocates tensor memory; one lane issues tcgen05.mma (M128 N256 K16, eight per
 //                  K block) and the commits that release stages / publish accumulators
-//     Accumulators are double buffered in tensor memory (2 x 256 columns) so the epilogue of a
-//     tile overlaps the MMAs of the next.
+//     The two accumulators fill tensor memory (2 x 256 columns), so a tile's epilogue does not
+//     overlap the next tile's MMAs; the producer keeps filling the stages meanwhile.
 //
 // Every wait on an mbarrier is bounded by a clock budget; on expiry the thread records a code in
 // the error word and the CTA drains: nothing can spin forever.
@@ -40,13 +44,13 @@ namespace dastac {
 namespace {
 
 constexpr int kTileM = 128, kTileN = 256, kBlockK = 64;
-constexpr int kStages = 4;
+constexpr int kStages = 3;
 constexpr int kABytes = kTileM * kBlockK * 2;  // 16 KiB
 constexpr int kBBytes = kBlockK * kTileN * 2;  // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kEpilogueWarps = 4;
-constexpr int kWarpTma = 4, kWarpMma = 5;
-constexpr int kThreads = 6 * 32;
+constexpr int kStageBytes = 2 * kABytes + kBBytes;  // two row blocks of A, one block of B
+constexpr int kEpilogueWarps = 8;
+constexpr int kWarpTma = 8, kWarpMma = 9;
+constexpr int kThreads = 10 * 32;
 constexpr int kTmemCols = 512;
 constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long kWaitBudget = 4000000000LL;  // clock cycles (~2 s) before a wait gives up
@@ -237,16 +241,30 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int64_t tiles = (int64_t)p.row_blocks * p.col_blocks;
+    // Tile t = (pair P, column block J), P ascending = K length descending.  The CTA's n-th tile is
+    // taken from round n of the list, forwards in even rounds and backwards in odd ones.
+    const int pair_blocks = (p.row_blocks + 1) >> 1;
+    const int64_t tiles = (int64_t)pair_blocks * p.col_blocks;
+    auto tile_of = [&](uint32_t n) -> int64_t {
+        const int64_t G = gridDim.x;
+        return (int64_t)n * G + ((n & 1) ? (G - 1 - (int64_t)blockIdx.x) : (int64_t)blockIdx.x);
+    };
+    // rounds in which this CTA's slot is past the end of the list are skipped, not final
+    const uint32_t rounds = (uint32_t)((tiles + gridDim.x - 1) / gridDim.x);
 
     if (warp == kWarpTma) {
-        // ---- producer: bulk copy of the staged A tile + TMA boxes of B ------------------------------
+        // ---- producer: bulk copies of the staged A tiles + TMA boxes of B ---------------------------
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-                const int I = (int)(t / p.col_blocks), J = (int)(t - (int64_t)I * p.col_blocks);
-                for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
+            for (uint32_t n = 0; n < rounds && ok; ++n) {
+                const int64_t t = tile_of(n);
+                if (t >= tiles) continue;
+                const int P = (int)(t / p.col_blocks), J = (int)(t - (int64_t)P * p.col_blocks);
+                const bool two = 2 * P + 1 < p.row_blocks;
+                const int64_t tile0 = tile_offset(2 * P, p.k_blocks) - 4 * P;  // + kb: staged tile (2P, kb)
+                const int64_t tile1 = tile_offset(2 * P + 1, p.k_blocks) - 4 * P;
+                for (int kb = 4 * P; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     if (it >= kStages &&
                         !mbar_wait(empty(s), ((it / kStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty)) {
@@ -254,12 +272,12 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
                         break;
                     }
                     const uint32_t dst = smem_base + s * kStageBytes;
-                    mbar_arrive_expect_tx(full(s), kStageBytes);
-                    bulk_load(dst, p.tiles + (tile_offset(I, p.k_blocks) + kb - 4 * (I >> 1)) * (int64_t)kABytes,
-                              kABytes, full(s));
+                    mbar_arrive_expect_tx(full(s), (two ? 2 : 1) * kABytes + kBBytes);
+                    bulk_load(dst, p.tiles + (tile0 + kb) * (int64_t)kABytes, kABytes, full(s));
+                    if (two) bulk_load(dst + kABytes, p.tiles + (tile1 + kb) * (int64_t)kABytes, kABytes, full(s));
 #pragma unroll
                     for (int q = 0; q < kTileN / 64; ++q)
-                        tma_load_2d(dst + kABytes + q * (kBlockK * 128), &tmap_b, J * kTileN + q * 64,
+                        tma_load_2d(dst + 2 * kABytes + q * (kBlockK * 128), &tmap_b, J * kTileN + q * 64,
                                     kb * kBlockK, full(s));
                 }
             }
@@ -279,17 +297,19 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
         if (lane == 0) {
             uint32_t it = 0, tile_n = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++tile_n) {
-                const int I = (int)(t / p.col_blocks);
-                const int acc = tile_n & 1;
-                if (tile_n >= 2 &&
-                    !mbar_wait(tmem_empty(acc), ((tile_n >> 1) - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
+            for (uint32_t n = 0; n < rounds && ok; ++n) {
+                const int64_t t = tile_of(n);
+                if (t >= tiles) continue;
+                const int P = (int)(t / p.col_blocks);
+                const bool two = 2 * P + 1 < p.row_blocks;
+                // the epilogue of the previous tile must have drained both accumulators
+                if (tile_n >= 1 &&
+                    !mbar_wait(tmem_empty(0), (tile_n - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * kTileN;
-                for (int kb = 2 * I; kb < p.k_blocks; ++kb, ++it) {
+                for (int kb = 4 * P; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t par = (it / kStages) & 1;
                     if (!mbar_wait(full(s), par, abort_flag, p.err_word, kErrFull)) {
@@ -298,19 +318,23 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
                     }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * kStageBytes;
-                    const uint32_t b_addr = a_addr + kABytes;
+                    const uint32_t b_addr = a_addr + 2 * kABytes;
+                    const uint32_t acc_flag = kb > 4 * P ? 1u : 0u;
 #pragma unroll
                     for (int k16 = 0; k16 < kBlockK / 16; ++k16) {
                         // A: K-major, 8-row groups 1024 B apart; 16 K elements = 32 B further.
-                        const uint64_t da = smem_desc(a_addr + k16 * 32, 16, 1024);
+                        const uint64_t da0 = smem_desc(a_addr + k16 * 32, 16, 1024);
+                        const uint64_t da1 = smem_desc(a_addr + kABytes + k16 * 32, 16, 1024);
                         // B: MN-major, 64-column groups 8192 B apart (leading), 8-row K groups
                         // 1024 B apart (stride); 16 K rows = 2048 B further.
                         const uint64_t db = smem_desc(b_addr + k16 * 2048, kBlockK * 128, 1024);
-                        umma_bf16(d_tmem, da, db, kIdesc, (kb > 2 * I || k16 > 0) ? 1u : 0u);
+                        umma_bf16(tmem_base, da0, db, kIdesc, (acc_flag || k16 > 0) ? 1u : 0u);
+                        if (two) umma_bf16(tmem_base + kTileN, da1, db, kIdesc, (acc_flag || k16 > 0) ? 1u : 0u);
                     }
                     umma_commit(empty(s));
                 }
-                if (ok) umma_commit(tmem_full(acc));
+                if (ok) umma_commit(tmem_full(0));
+                ++tile_n;
             }
             if (!ok) {
                 // MMAs already issued still read shared memory: wait (bounded) until they retire.
@@ -322,52 +346,58 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
         }
     } else {
         // ---- epilogue -----------------------------------------------------------------------------
+        const int half = warp >> 2, quarter = warp & 3;  // which accumulator / which 32 TMEM lanes
         uint32_t tile_n = 0;
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++tile_n) {
-            const int I = (int)(t / p.col_blocks), J = (int)(t - (int64_t)I * p.col_blocks);
-            const int acc = tile_n & 1;
-            if (!mbar_wait_warp(tmem_full(acc), (tile_n >> 1) & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
+        for (uint32_t n = 0; n < rounds && ok; ++n) {
+            const int64_t t = tile_of(n);
+            if (t >= tiles) continue;
+            const int P = (int)(t / p.col_blocks), J = (int)(t - (int64_t)P * p.col_blocks);
+            const int I = 2 * P + half;
+            if (!mbar_wait_warp(tmem_full(0), tile_n & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            const int64_t i = (int64_t)I * kTileM + warp * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + acc * kTileN;
+            const int64_t i = (int64_t)I * kTileM + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * kTileN;
             float* crow = p.C + i * p.ldc + (int64_t)J * kTileN;
+            if (I < p.row_blocks) {
 #pragma unroll 1
-            for (int cc = 0; cc < kTileN / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(taddr + cc * 32, r);
-                tmem_ld_wait();
-                const int64_t col0 = (int64_t)J * kTileN + cc * 32;
-                if (i < p.N) {
-                    if (p.vector_store && col0 + 32 <= p.ncols) {
-                        float4* dst = (float4*)(crow + cc * 32);
+                for (int cc = 0; cc < kTileN / 32; ++cc) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + cc * 32, r);
+                    tmem_ld_wait();
+                    const int64_t col0 = (int64_t)J * kTileN + cc * 32;
+                    if (i < p.N) {
+                        if (p.vector_store && col0 + 32 <= p.ncols) {
+                            float4* dst = (float4*)(crow + cc * 32);
 #pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                                   __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
-                            if (p.accumulate) {
-                                const float4 old = dst[v];
-                                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                            for (int v = 0; v < 8; ++v) {
+                                float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                       __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                                if (p.accumulate) {
+                                    const float4 old = dst[v];
+                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                }
+                                dst[v] = o;
                             }
-                            dst[v] = o;
+                        } else {
+#pragma unroll
+                            for (int v = 0; v < 32; ++v)
+                                if (col0 + v < p.ncols) {
+                                    float o = __uint_as_float(r[v]);
+                                    if (p.accumulate) o += crow[cc * 32 + v];
+                                    crow[cc * 32 + v] = o;
+                                }
                         }
-                    } else {
-#pragma unroll
-                        for (int v = 0; v < 32; ++v)
-                            if (col0 + v < p.ncols) {
-                                float o = __uint_as_float(r[v]);
-                                if (p.accumulate) o += crow[cc * 32 + v];
-                                crow[cc * 32 + v] = o;
-                            }
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tmem_empty(acc));
+            if (lane == 0) mbar_arrive(tmem_empty(0));
+            ++tile_n;
         }
     }
 
@@ -538,7 +568,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     trimm_stage_a_kernel<<<dim3((unsigned)p.k_blocks, (unsigned)p.row_blocks), kStageThreads, 0, st>>>(p, tiles);
     dastac_status ss = launch_status();
     if (ss != DASTAC_OK) return ss;
-    const int64_t n_tiles = (int64_t)p.row_blocks * p.col_blocks;
+    const int64_t n_tiles = (int64_t)((p.row_blocks + 1) / 2) * p.col_blocks;  // pairs of row blocks x column blocks
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
     trimm_tcgen05_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmap, p);
     return launch_status();
