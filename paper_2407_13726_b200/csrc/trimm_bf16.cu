@@ -3,14 +3,12 @@
 // kernel; this is its SpMV_UT / TTM_UT access pattern (Table 1) widened to a dense right-hand
 // side and mapped on tcgen05.
 //
-// Tiling.  An output tile is 256 rows x 256 columns: two 128-row blocks (2P, 2P+1), each with its
-// own accumulator, that share every staged 64 x 256 block of B.  Per 64-deep K block a CTA then
-// moves 64 KiB through shared memory for two M128 N256 MMAs, instead of 48 KiB for one: with the
-// few hundred KB a CTA can keep in flight, the bytes per MMA cycle, not the tensor pipe, set the
-// pace of this kernel.  A pair only needs K blocks from its diagonal on: kb = 4P .. ceil(N/64)-1,
-// so the executed MMA work is the triangle plus one tile per pair.  Tiles are ordered by
-// decreasing K length and dealt to one persistent CTA per SM in boustrophedon order, which gives
-// every CTA the same mix of long and short tiles.
+// Tiling.  An output tile is 256 rows x 256 columns, computed by a cluster of two CTAs (one SM
+// each) with tcgen05.mma.cta_group::2: CTA r holds row block 2P + r (128 rows).  A pair only needs
+// K blocks (64 columns of A, 64 rows of B) from its diagonal on: kb = 4P .. ceil(N/64)-1, so the
+// executed MMA work is the triangle plus one tile per pair.  Tiles are ordered by decreasing K
+// length and dealt to the persistent clusters in boustrophedon order, which gives every cluster
+// the same mix of long and short tiles.
 //
 // Two kernels per call:
 //  1. stage_a: the packed row pitch changes with the row and row starts are only 2-byte aligned,
@@ -22,16 +20,9 @@
 //     the diagonal or beyond column N are zeroed.  Doing this once per call instead of once per
 //     column tile keeps the realignment off the MMA critical path (each A tile is consumed by
 //     every column tile of its row block).  The workspace stays packed: it holds the triangle's
-//     tiles only.
-//  2. trimm_tcgen05: warp-specialised pipeline,
-//       warps 0-7  epilogue: tcgen05.ld of the accumulators (warps 0-3 the upper row block, 4-7
-//                  the lower; warp w owns TMEM lanes 32(w%4)..32(w%4)+31), 128-bit stores to C
-//       warp  8    one lane issues, per K block, two bulk copies of staged A tiles and four TMA
-//                  boxes (64x64, 128B swizzle) of B into the stage, all on one mbarrier
-//       warp  9    allocates tensor memory; one lane issues tcgen05.mma (M128 N256 K16, eight per
-//                  K block) and the commits that release stages / publish accumulators
-//     The two accumulators fill tensor memory (2 x 256 columns), so a tile's epilogue does not
-//     overlap the next tile's MMAs; the producer keeps filling the stages meanwhile.
+//     tiles only.  The images form a plain [tiles x 128][64] array, which a tensor map without
+//     swizzle copies verbatim.
+//  2. trimm_pair: warp-specialised pipeline (details at the kernel).
 //
 // Every wait on an mbarrier is bounded by a clock budget; on expiry the thread records a code in
 // the error word and the CTA drains: nothing can spin forever.
@@ -44,15 +35,8 @@ namespace dastac {
 namespace {
 
 constexpr int kTileM = 128, kTileN = 256, kBlockK = 64;
-constexpr int kStages = 3;
 constexpr int kABytes = kTileM * kBlockK * 2;  // 16 KiB
-constexpr int kBBytes = kBlockK * kTileN * 2;  // 32 KiB
-constexpr int kStageBytes = 2 * kABytes + kBBytes;  // two row blocks of A, one block of B
-constexpr int kEpilogueWarps = 8;
-constexpr int kWarpTma = 8, kWarpMma = 9;
-constexpr int kThreads = 10 * 32;
 constexpr int kTmemCols = 512;
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long kWaitBudget = 4000000000LL;  // clock cycles (~2 s) before a wait gives up
 
 enum ErrCode : int32_t { kErrFull = 1, kErrEmpty = 3, kErrTmemFull = 4, kErrTmemEmpty = 5 };
@@ -110,44 +94,11 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_after() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -177,10 +128,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return d;
 }
 
-// Instruction descriptor: fp32 accumulator, bf16 A (K-major) and bf16 B (MN-major), M128 N256.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                            ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-
 // Staged tile (I, kb) lives at tile index tile_offset(I) + kb - 4*(I/2): row blocks are stored in
 // pairs that start at the same K block, so that two row blocks can later share one K loop; the
 // two tiles this adds in front of every odd row block are all zero.
@@ -201,166 +148,255 @@ struct Params {
     int32_t* err_word;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
-trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+// ---- CTA-pair kernel ------------------------------------------------------------------------------
+// A 256 x 256 output tile is computed by a cluster of two CTAs with tcgen05.mma.cta_group::2
+// (M256 N256 K16).  CTA r of the pair stages the A tile of row block 2P + r and the 128-column half
+// r of the B block, so each SM moves 32 KiB per K block and the tensor core of each SM reads half
+// of B from its own shared memory and half from its peer's.  Each CTA holds the 128 x 256
+// accumulator of its own row block, double buffered in its tensor memory, and its four epilogue
+// warps drain one buffer while the MMAs of the next tile fill the other.
+//   - Both CTAs' loads of a stage complete on the full barrier of CTA 0 (the MMA issuer); a
+//     cta_group::2 tensor copy may name a barrier of the peer CTA.
+//   - One commit with a two-CTA mask releases a stage (or publishes an accumulator) in both CTAs.
+//   - CTA 1's epilogue warps release an accumulator with an arrive on CTA 0's barrier.
+constexpr int kPStages = 6;
+constexpr int kPBBytes = kBlockK * (kTileN / 2) * 2;   // 16 KiB: this CTA's half of the B block
+constexpr int kPStageBytes = kABytes + kPBBytes;       // 32 KiB
+constexpr int kPThreads = 6 * 32;                      // warps 0-3 epilogue, 4 producer, 5 MMA
+constexpr int kPWarpTma = 4, kPWarpMma = 5;
+constexpr size_t kPSmemBytes = (size_t)kPStages * kPStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// fp32 accumulator, bf16 A (K-major) and bf16 B (MN-major), M256 N256 across the pair
+constexpr uint32_t kPIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                             ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)((2 * kTileM) >> 4) << 24);
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_test_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  int32_t* err_word, int32_t code) {
+    if (mbar_test_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_test_cluster(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitBudget) {
+            *abort_flag = 1;
+            if (err_word) atomicCAS(err_word, 0, code);
+            return false;
+        }
+    }
+}
+// Tensor copy whose completion bytes go to `bar`, a shared::cluster address that may lie in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far retire.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3)
+        : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = (uint64_t*)(smem + (size_t)kStages * kStageBytes);
-    // barrier slots: full[s], (unused)[s], empty[s], tmem_full[2], tmem_empty[2], drain
+    uint64_t* bars = (uint64_t*)(smem + (size_t)kPStages * kPStageBytes);
+    // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2], drain
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * s; };
-    auto empty = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
-    auto tmem_full = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
-    auto tmem_empty = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
-    auto drain_bar = [&]() { return bar0 + 8u * (3 * kStages + 4); };
-    uint32_t* tmem_slot = (uint32_t*)(bars + 3 * kStages + 5);
+    auto empty = [&](int s) { return bar0 + 8u * (kPStages + s); };
+    auto tmem_full = [&](int a) { return bar0 + 8u * (2 * kPStages + a); };
+    auto tmem_empty = [&](int a) { return bar0 + 8u * (2 * kPStages + 2 + a); };
+    auto drain_bar = [&]() { return bar0 + 8u * (2 * kPStages + 4); };
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * kPStages + 5);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = smem_u32(smem);
+    const uint32_t rank = cluster_ctarank();  // 0: issues the MMAs, owns the full / tmem_empty barriers
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kPStages; ++s) {
             mbar_init(full(s), 1);
             mbar_init(empty(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
-            mbar_init(tmem_empty(a), kEpilogueWarps);
+            mbar_init(tmem_empty(a), 2 * 4);  // four epilogue warps in each CTA
         }
         mbar_init(drain_bar(), 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == kWarpMma) {
-        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-        tmem_relinquish();
+    if (warp == kPWarpMma) {
+        tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // Tile t = (pair P, column block J), P ascending = K length descending.  The CTA's n-th tile is
-    // taken from round n of the list, forwards in even rounds and backwards in odd ones.
+    // Tile t = (pair P, column block J), P ascending = K length descending, dealt to the clusters in
+    // boustrophedon order.
     const int pair_blocks = (p.row_blocks + 1) >> 1;
     const int64_t tiles = (int64_t)pair_blocks * p.col_blocks;
-    auto tile_of = [&](uint32_t n) -> int64_t {
-        const int64_t G = gridDim.x;
-        return (int64_t)n * G + ((n & 1) ? (G - 1 - (int64_t)blockIdx.x) : (int64_t)blockIdx.x);
-    };
-    // rounds in which this CTA's slot is past the end of the list are skipped, not final
-    const uint32_t rounds = (uint32_t)((tiles + gridDim.x - 1) / gridDim.x);
+    const int64_t G = gridDim.x >> 1, cid = blockIdx.x >> 1;
+    auto tile_of = [&](uint32_t n) -> int64_t { return (int64_t)n * G + ((n & 1) ? (G - 1 - cid) : cid); };
+    const uint32_t rounds = (uint32_t)((tiles + G - 1) / G);
 
-    if (warp == kWarpTma) {
-        // ---- producer: bulk copies of the staged A tiles + TMA boxes of B ---------------------------
+    if (warp == kPWarpTma) {
+        // ---- producer (both CTAs): this CTA's A tile and its half of the B block ---------------------
         if (lane == 0) {
+            const uint32_t full0 = map_to_cta(full(0), 0);  // CTA 0's full barriers, 8 bytes apart
             uint32_t it = 0;
             bool ok = true;
             for (uint32_t n = 0; n < rounds && ok; ++n) {
                 const int64_t t = tile_of(n);
                 if (t >= tiles) continue;
                 const int P = (int)(t / p.col_blocks), J = (int)(t - (int64_t)P * p.col_blocks);
-                const bool two = 2 * P + 1 < p.row_blocks;
-                const int64_t tile0 = tile_offset(2 * P, p.k_blocks) - 4 * P;  // + kb: staged tile (2P, kb)
-                const int64_t tile1 = tile_offset(2 * P + 1, p.k_blocks) - 4 * P;
+                const int I = 2 * P + (int)rank;
+                // staged tile (I, kb) sits at tile index tile_base + kb; a row block past the end of
+                // the matrix has no tiles and its loads are out of range of the map: zero fill
+                const int64_t tile_base = (I < p.row_blocks) ? tile_offset(I, p.k_blocks) - 4 * P : (int64_t)1 << 22;
                 for (int kb = 4 * P; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    if (it >= kStages &&
-                        !mbar_wait(empty(s), ((it / kStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty)) {
+                    const int s = it % kPStages;
+                    if (it >= kPStages &&
+                        !mbar_wait(empty(s), ((it / kPStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty)) {
                         ok = false;
                         break;
                     }
-                    const uint32_t dst = smem_base + s * kStageBytes;
-                    mbar_arrive_expect_tx(full(s), (two ? 2 : 1) * kABytes + kBBytes);
-                    bulk_load(dst, p.tiles + (tile0 + kb) * (int64_t)kABytes, kABytes, full(s));
-                    if (two) bulk_load(dst + kABytes, p.tiles + (tile1 + kb) * (int64_t)kABytes, kABytes, full(s));
+                    const uint32_t dst = smem_base + s * kPStageBytes;
+                    if (leader) mbar_arrive_expect_tx(full(s), 2 * kPStageBytes);  // both CTAs' bytes
+                    const uint32_t bar = full0 + 8u * s;
+                    tma_load_2d_pair(dst, &tmap_a, 0, (int)((tile_base + kb) * kTileM), bar);
 #pragma unroll
-                    for (int q = 0; q < kTileN / 64; ++q)
-                        tma_load_2d(dst + 2 * kABytes + q * (kBlockK * 128), &tmap_b, J * kTileN + q * 64,
-                                    kb * kBlockK, full(s));
+                    for (int q = 0; q < kTileN / 128; ++q)
+                        tma_load_2d_pair(dst + kABytes + q * (kBlockK * 128), &tmap_b,
+                                         J * kTileN + (int)rank * (kTileN / 2) + q * 64, kb * kBlockK, bar);
                 }
             }
-            // Drain: copies already issued must land before the CTA's shared memory is released.
             if (!ok) {
+                // give copies that are still in flight time to land before shared memory is released
                 const long long t0 = clock64();
-                for (int s = 0; s < kStages; ++s) {
-                    const uint32_t issued = it / kStages + ((int)(it % kStages) > s ? 1 : 0);
-                    if (issued == 0) continue;
-                    while (!mbar_test(full(s), (issued - 1) & 1) && clock64() - t0 < kWaitBudget) {
-                    }
+                while (clock64() - t0 < 2000000) {
                 }
             }
         }
-    } else if (warp == kWarpMma) {
-        // ---- MMA issuer ------------------------------------------------------------------------
-        if (lane == 0) {
+    } else if (warp == kPWarpMma) {
+        // ---- MMA issuer (CTA 0 only) -----------------------------------------------------------------
+        if (leader && lane == 0) {
             uint32_t it = 0, tile_n = 0;
             bool ok = true;
             for (uint32_t n = 0; n < rounds && ok; ++n) {
                 const int64_t t = tile_of(n);
                 if (t >= tiles) continue;
                 const int P = (int)(t / p.col_blocks);
-                const bool two = 2 * P + 1 < p.row_blocks;
-                // the epilogue of the previous tile must have drained both accumulators
-                if (tile_n >= 1 &&
-                    !mbar_wait(tmem_empty(0), (tile_n - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
+                const int acc = tile_n & 1;
+                if (tile_n >= 2 &&
+                    !mbar_wait_cluster(tmem_empty(acc), ((tile_n >> 1) - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kTileN;
                 for (int kb = 4 * P; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t par = (it / kStages) & 1;
-                    if (!mbar_wait(full(s), par, abort_flag, p.err_word, kErrFull)) {
+                    const int s = it % kPStages;
+                    if (!mbar_wait_cluster(full(s), (it / kPStages) & 1, abort_flag, p.err_word, kErrFull)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + s * kStageBytes;
-                    const uint32_t b_addr = a_addr + 2 * kABytes;
-                    const uint32_t acc_flag = kb > 4 * P ? 1u : 0u;
+                    const uint32_t a_addr = smem_base + s * kPStageBytes;
+                    const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
                     for (int k16 = 0; k16 < kBlockK / 16; ++k16) {
-                        // A: K-major, 8-row groups 1024 B apart; 16 K elements = 32 B further.
-                        const uint64_t da0 = smem_desc(a_addr + k16 * 32, 16, 1024);
-                        const uint64_t da1 = smem_desc(a_addr + kABytes + k16 * 32, 16, 1024);
-                        // B: MN-major, 64-column groups 8192 B apart (leading), 8-row K groups
-                        // 1024 B apart (stride); 16 K rows = 2048 B further.
+                        const uint64_t da = smem_desc(a_addr + k16 * 32, 16, 1024);
                         const uint64_t db = smem_desc(b_addr + k16 * 2048, kBlockK * 128, 1024);
-                        umma_bf16(tmem_base, da0, db, kIdesc, (acc_flag || k16 > 0) ? 1u : 0u);
-                        if (two) umma_bf16(tmem_base + kTileN, da1, db, kIdesc, (acc_flag || k16 > 0) ? 1u : 0u);
+                        umma_bf16_pair(d_tmem, da, db, kPIdesc, (kb > 4 * P || k16 > 0) ? 1u : 0u);
                     }
-                    umma_commit(empty(s));
+                    umma_commit_pair(empty(s));
                 }
-                if (ok) umma_commit(tmem_full(0));
+                if (ok) umma_commit_pair(tmem_full(acc));
                 ++tile_n;
             }
             if (!ok) {
-                // MMAs already issued still read shared memory: wait (bounded) until they retire.
-                umma_commit(drain_bar());
+                umma_commit_pair(drain_bar());
                 const long long t0 = clock64();
                 while (!mbar_test(drain_bar(), 0) && clock64() - t0 < kWaitBudget) {
                 }
             }
         }
     } else {
-        // ---- epilogue -----------------------------------------------------------------------------
-        const int half = warp >> 2, quarter = warp & 3;  // which accumulator / which 32 TMEM lanes
+        // ---- epilogue (both CTAs): this CTA's 128 rows of the tile ------------------------------------
+        const uint32_t empty0 = map_to_cta(tmem_empty(0), 0);
         uint32_t tile_n = 0;
         bool ok = true;
         for (uint32_t n = 0; n < rounds && ok; ++n) {
             const int64_t t = tile_of(n);
             if (t >= tiles) continue;
             const int P = (int)(t / p.col_blocks), J = (int)(t - (int64_t)P * p.col_blocks);
-            const int I = 2 * P + half;
-            if (!mbar_wait_warp(tmem_full(0), tile_n & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
+            const int I = 2 * P + (int)rank;
+            const int acc = tile_n & 1;
+            if (!mbar_wait_warp(tmem_full(acc), (tile_n >> 1) & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            const int64_t i = (int64_t)I * kTileM + quarter * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * kTileN;
+            const int64_t i = (int64_t)I * kTileM + warp * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + acc * kTileN;
             float* crow = p.C + i * p.ldc + (int64_t)J * kTileN;
             if (I < p.row_blocks) {
 #pragma unroll 1
@@ -396,17 +432,19 @@ trimm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_b, const Params p)
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tmem_empty(0));
+            if (lane == 0) mbar_arrive_cluster(empty0 + 8u * acc);
             ++tile_n;
         }
     }
 
+    // Neither CTA may leave, or give back tensor memory, while its peer can still touch it.
     tc_fence_before();
     __syncthreads();
-    if (warp == kWarpMma) {
+    cluster_sync_all();
+    if (warp == kPWarpMma) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 
@@ -555,12 +593,24 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     p.vector_store = ((ldc & 3) == 0) && aligned16(C);
     p.err_word = err_word;
 
+    // The staged tile images as a tensor: one 128-byte row per tile row, already in shared-memory order.
+    const int64_t staged_tiles = staged_tile_count(N);
+    if (staged_tiles * kTileM > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
+    CUtensorMap tmap_a;
+    const cuuint64_t adims[2] = {(cuuint64_t)kBlockK, (cuuint64_t)(staged_tiles * kTileM)};
+    const cuuint64_t astrides[1] = {(cuuint64_t)kBlockK * 2};
+    const cuuint32_t abox[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM};
+    if (enc(&tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, tiles, adims, astrides, abox, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DASTAC_ERR_CUDA;
+
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(trimm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(trimm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kPSmemBytes) != cudaSuccess)
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
     }
@@ -569,8 +619,9 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     dastac_status ss = launch_status();
     if (ss != DASTAC_OK) return ss;
     const int64_t n_tiles = (int64_t)((p.row_blocks + 1) / 2) * p.col_blocks;  // pairs of row blocks x column blocks
-    const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
-    trimm_tcgen05_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmap, p);
+    const int64_t max_clusters = sm_count() / 2;
+    const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
+    trimm_pair_kernel<<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, p);
     return launch_status();
 }
 
