@@ -194,6 +194,26 @@ class ClockSampler:
         return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
 
 
+# ---- multi-rank plumbing: replicas only, the one collective is the MAX of the timings ----------------
+
+def max_over_ranks(ms: float, device="cuda") -> float:
+    """The slowest rank's time: every rank runs the whole step on its own GPU, so the job's step
+    time is the maximum.  A no-op for a single process."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gflops(world: int, flops_per_rank_step: float, ms_per_step: float) -> float:
+    """Aggregate useful GFLOP/s of `world` replicas that each do `flops_per_rank_step` per step."""
+    return world * flops_per_rank_step / ms_per_step / 1e6
+
+
 # ---- the GPU arm ----------------------------------------------------------------------------------
 
 def run_gpu(args):
@@ -290,10 +310,7 @@ def run_gpu(args):
     total_ms = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
     assert int(err_word.item()) == 0, "a device-side bounded wait expired"
-    if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
     step_flops = sum(acct[n]["flops"] for n in order)
 
@@ -382,11 +399,8 @@ def run_gpu(args):
         b.record()
         barrier()
         e_ms = a.elapsed_time(b)
-        if world > 1:
-            tt = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e_ms = float(tt.item())
-        e2e = {"value": round(world * e2e_flops * e_steps / e_ms / 1e6, 1), "unit": UNIT,
+        e_ms = max_over_ranks(e_ms)
+        e2e = {"value": round(whole_job_gflops(world, e2e_flops, e_ms / e_steps), 1), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e_steps,
                "ms_per_step": round(e_ms / e_steps, 3),
                "note": "five contractions with pinned host operands staged by dastac_contract; pack/unpack legs excluded"}
@@ -397,7 +411,7 @@ def run_gpu(args):
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": round(world * step_flops / ms_per_step / 1e6, 1), "unit": UNIT,
+            "metric": METRIC, "value": round(whole_job_gflops(world, step_flops, ms_per_step), 1), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",

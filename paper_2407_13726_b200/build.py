@@ -45,7 +45,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in sources():
         obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", src, "-o", obj]
+        # DASTAC_NVCC_EXTRA: extra nvcc flags (e.g. -DNAME=value) for experiments
+        cmd = [_nvcc(), *NVCC_FLAGS, *os.environ.get("DASTAC_NVCC_EXTRA", "").split(), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
