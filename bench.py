@@ -330,6 +330,7 @@ def run_gpu(args):
         if a["bound"] == "tensor":
             k["tensor_frac_measured"] = round(a["flops"] / avg / 1e9 / pk["bf16_tflops"], 4)
             k["tensor_frac_nominal_2250"] = round(a["flops"] / avg / 1e9 / 2250.0, 4)
+        k["traffic"] = TRAFFIC.get(name) if not (args.small or args.size) else None
         kernels[name] = k
     # ---- each kernel alone, steady state: back-to-back launches over rotating copies of its buffers
     # (footprint >= 3x L2, so every launch starts cold and pays for its own write-backs), replayed
@@ -467,9 +468,18 @@ def isolated_times(order, devs, structs, run_kernel_on, z, acct, launches):
     return out
 
 
-# DRAM bytes (read + write) per launch from ncu captures, by kernel; None until captured for the
-# current kernel version.
-TRAFFIC = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per bench launch from the ncu captures
+# summarised under profiles/, by bench kernel; a kernel changed since its capture has no entry.
+# symv and trmv_batched were captured on smaller cases (N=16384; 128 instances) and scaled by the
+# number of stored elements, which their traffic is proportional to.
+TRAFFIC = {
+    "symv": int((537.292800e6 + 4.572672e6) * (65536 * 65537 // 2) / (16384 * 16385 // 2)),
+    "trmv_batched": int((269.286144e6 + 4.292096e6) * 4),
+    "mttkrp": int(91.026944e6 + 6.966272e6),
+    "trimm_bf16": int(855.178240e6 + 215.225600e6 + 67.129856e6 + 28.432640e6),  # main kernel + tile staging
+    "pack_bf16": int(67.703552e6 + 26.094336e6),
+    "unpack_bf16": int(67.148800e6 + 78.674432e6),
+}
 
 
 # ---- the CPU oracle arm -----------------------------------------------------------------------------

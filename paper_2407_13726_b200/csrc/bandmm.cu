@@ -17,8 +17,8 @@
 // window that slides down by one row per diagonal: each step loads the eight A values (two
 // broadcast 128-bit shared loads) and one new B row segment (one 128-bit shared load) and issues 32
 // multiply-adds as 16 packed fp32x2 instructions.  The window lives in registers and rotates with
-// period 8; the loop is unrolled by 8 so every register index is static.  Only the band is visited:
-// the executed work is the diagonal count rounded up to a multiple of 8.
+// period 8; the loop is unrolled by 8 so every register index is static, with a guarded copy of the body for
+// the last 1..7 diagonals.  Only the band is visited.
 #include <cuda.h>
 
 #include <cstring>
@@ -178,22 +178,29 @@ bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant_
 #pragma unroll
         for (int q = 0; q < 7; ++q)
             load_row<TMA_B>(win[q], Bs, br0 + q, B, ldb, i_f + dc - w + q, N, c0, cl, ncols);
-        const int64_t d_end = (diagonals - dc < kChunk) ? diagonals - dc : kChunk;
-        for (int db = 0; db < d_end; db += 8) {
+        const int d_end = (int)((diagonals - dc < kChunk) ? diagonals - dc : kChunk);
+        // one diagonal: slide the window down by one row of B, then 8 rows x 4 columns of multiply-adds
+        auto step = [&](const int db, const int u) {
+            load_row<TMA_B>(win[(u + 7) & 7], Bs, br0 + db + u + 7, B, ldb, i_f + dc + db + u - w + 7, N, c0, cl, ncols);
+            const float4 a_lo = *reinterpret_cast<const float4*>(&Ad[(db + u) * kRows + il]);
+            const float4 a_hi = *reinterpret_cast<const float4*>(&Ad[(db + u) * kRows + il + 4]);
+            const pair_t a2[8] = {pack2(a_lo.x, a_lo.x), pack2(a_lo.y, a_lo.y), pack2(a_lo.z, a_lo.z),
+                                  pack2(a_lo.w, a_lo.w), pack2(a_hi.x, a_hi.x), pack2(a_hi.y, a_hi.y),
+                                  pack2(a_hi.z, a_hi.z), pack2(a_hi.w, a_hi.w)};
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                load_row<TMA_B>(win[(u + 7) & 7], Bs, br0 + db + u + 7, B, ldb, i_f + dc + db + u - w + 7, N, c0, cl,
-                                ncols);
-                const float4 a_lo = *reinterpret_cast<const float4*>(&Ad[(db + u) * kRows + il]);
-                const float4 a_hi = *reinterpret_cast<const float4*>(&Ad[(db + u) * kRows + il + 4]);
-                const pair_t a2[8] = {pack2(a_lo.x, a_lo.x), pack2(a_lo.y, a_lo.y), pack2(a_lo.z, a_lo.z),
-                                      pack2(a_lo.w, a_lo.w), pack2(a_hi.x, a_hi.x), pack2(a_hi.y, a_hi.y),
-                                      pack2(a_hi.z, a_hi.z), pack2(a_hi.w, a_hi.w)};
+            for (int q = 0; q < 8; ++q)
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
+                for (int e = 0; e < kPairs; ++e) fma2(acc2[q][e], a2[q], win[(u + q) & 7][e]);
+        };
+        int db = 0;
+        for (; db + 8 <= d_end; db += 8) {
 #pragma unroll
-                    for (int e = 0; e < kPairs; ++e) fma2(acc2[q][e], a2[q], win[(u + q) & 7][e]);
-            }
+            for (int u = 0; u < 8; ++u) step(db, u);
+        }
+        if (db < d_end) {  // the last 1..7 diagonals: same rotation, no work on diagonals that do not exist
+#pragma unroll
+            for (int u = 0; u < 7; ++u)
+                if (db + u < d_end) step(db, u);
         }
     }
     if (c0 >= ncols || i_f >= N) return;
