@@ -200,7 +200,9 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
     constexpr int E = 16 / sizeof(T);
     const int lane = threadIdx.x & 31;
     const int64_t total = (m.count + E - 1) / E;
-    const int64_t cA = (blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5)) * chunks_per_warp;
+    // blocks are issued in index order: give the first ones the end of the stream, where a triangle's
+    // rows are shortest and the walk is slowest, so that they do not form the tail of the launch
+    const int64_t cA = ((gridDim.x - 1 - blockIdx.x) * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5)) * chunks_per_warp;
     if (cA >= total) return;
     const int64_t cB = (cA + chunks_per_warp < total) ? cA + chunks_per_warp : total;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
@@ -262,15 +264,16 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
     }
 }
 
-// unpack: a warp item is a window of 32 * kUnroll chunks of one dense row; the zero fill outside
-// the set and the copy are the same pass.
+// unpack: a warp item is a run of windows (32 * kUnroll chunks each) of one dense row, so the row's
+// span and base are worked out once per item; the zero fill outside the set and the copy are the
+// same pass.
 template <typename T>
 __global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
 unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st,
-                     int64_t rows, int64_t windows_per_row) {
+                     int64_t rows, int groups_per_row, int windows_per_group) {
     constexpr int E = 16 / sizeof(T);
     const int lane = threadIdx.x & 31;
-    const int64_t inner = m.rank == 3 ? m.dims[2] : m.rank == 2 ? m.dims[1] : m.dims[0];
+    const int inner = (int)(m.rank == 3 ? m.dims[2] : m.rank == 2 ? m.dims[1] : m.dims[0]);
     const int64_t cap = (m.count + E - 1) / E * E;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     union Chunk {
@@ -278,57 +281,69 @@ unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ d
         T e[E];
     };
     const int64_t warps = (int64_t)gridDim.x * kWarpsPerBlock;
-    for (int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5); item < rows * windows_per_row;
+    for (int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5); item < rows * groups_per_row;
          item += warps) {
-        int64_t row = item / windows_per_row;
-        const int64_t win = item - row * windows_per_row;
-        int32_t idx[3] = {0, 0, 0};
-#pragma unroll
-        for (int k = 1; k >= 0; --k)
-            if (k + 1 < m.rank) {
-                const int64_t q = row / m.dims[k];
-                idx[k] = (int32_t)(row - q * m.dims[k]);
-                row = q;
-            }
-        int64_t jlo = 0, jhi = 0, pbase = 0;
-        if (!row_span(m, idx, jlo, jhi, pbase)) jlo = jhi = 0;
-        T* drow = dense + dense_row_offset(m, st, idx);
-        const int64_t jfirst = (win * (32 * kUnroll) + lane) * E;
-        uint4 lo[kUnroll], hi[kUnroll];
-        uint32_t sh[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int64_t j0 = jfirst + 32 * u * E;
-            const int64_t p0 = pbase + j0, a = p0 & ~(int64_t)(E - 1);
-            sh[u] = 0xffffffffu;  // no vector load for this chunk
-            if (j0 < inner && j0 + E > jlo && j0 < jhi && a >= 0 && a + 2 * E <= cap) {
-                sh[u] = (uint32_t)(p0 - a) * sizeof(T);
-                lo[u] = __ldg(reinterpret_cast<const uint4*>(packed + a));
-                hi[u] = sh[u] ? __ldg(reinterpret_cast<const uint4*>(packed + a + E)) : zero4;
-            }
+        int64_t row = item;
+        int grp = 0;
+        if (groups_per_row > 1) {
+            row = item / groups_per_row;
+            grp = (int)(item - row * groups_per_row);
         }
+        int32_t idx[3] = {0, 0, 0};
+        if (m.rank == 2) {
+            idx[0] = (int32_t)row;
+        } else if (m.rank == 3) {
+            const int64_t q = row / m.dims[1];
+            idx[1] = (int32_t)(row - q * m.dims[1]);
+            idx[0] = (int32_t)q;
+        }
+        int64_t jlo64 = 0, jhi64 = 0, pbase = 0;
+        if (!row_span(m, idx, jlo64, jhi64, pbase)) jlo64 = jhi64 = 0;
+        const int jlo = (int)jlo64, jhi = (int)jhi64;
+        T* drow = dense + dense_row_offset(m, st, idx);
+        const T* prow = packed + pbase;  // prow[j] = stored element (row, j)
+        // the vector path reads the two aligned granules around a chunk: both must lie inside the buffer
+        const int jsafe = (int)((cap - pbase - 2 * E < (int64_t)inner) ? cap - pbase - 2 * E : (int64_t)inner);
+        for (int win = grp * windows_per_group; win < (grp + 1) * windows_per_group; ++win) {
+            const int jfirst = (win * (32 * kUnroll) + lane) * E;
+            if (win * (32 * kUnroll) * E >= inner) break;
+            uint4 lo[kUnroll], hi[kUnroll];
+            uint32_t sh[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int64_t j0 = jfirst + 32 * u * E;
-            if (j0 >= inner) break;
-            Chunk out;
-            out.v = zero4;
-            if (sh[u] != 0xffffffffu) {
-                out.v = realign16(lo[u], hi[u], sh[u]);
-                if (j0 < jlo || j0 + E > jhi) {
+            for (int u = 0; u < kUnroll; ++u) {
+                const int j0 = jfirst + 32 * u * E;
+                sh[u] = 0xffffffffu;  // no vector load for this chunk
+                if (j0 < inner && j0 + E > jlo && j0 < jhi && j0 <= jsafe) {
+                    const uintptr_t addr = reinterpret_cast<uintptr_t>(prow + j0);
+                    sh[u] = (uint32_t)(addr & 15);
+                    const uint4* src = reinterpret_cast<const uint4*>(addr - sh[u]);
+                    lo[u] = __ldg(src);
+                    hi[u] = sh[u] ? __ldg(src + 1) : zero4;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int j0 = jfirst + 32 * u * E;
+                if (j0 >= inner) break;
+                Chunk out;
+                out.v = zero4;
+                if (sh[u] != 0xffffffffu) {
+                    out.v = realign16(lo[u], hi[u], sh[u]);
+                    if (j0 < jlo || j0 + E > jhi) {
+#pragma unroll
+                        for (int e = 0; e < E; ++e)
+                            if (j0 + e < jlo || j0 + e >= jhi) out.e[e] = T(0);
+                    }
+                } else if (j0 + E > jlo && j0 < jhi) {  // the last granules of the packed buffer
 #pragma unroll
                     for (int e = 0; e < E; ++e)
-                        if (j0 + e < jlo || j0 + e >= jhi) out.e[e] = T(0);
+                        if (j0 + e >= jlo && j0 + e < jhi) out.e[e] = prow[j0 + e];
                 }
-            } else if (j0 + E > jlo && j0 < jhi) {  // the last granules of the packed buffer
-#pragma unroll
-                for (int e = 0; e < E; ++e)
-                    if (j0 + e >= jlo && j0 + e < jhi) out.e[e] = packed[pbase + j0 + e];
-            }
-            if (j0 + E <= inner) {
-                *reinterpret_cast<uint4*>(drow + j0) = out.v;
-            } else {
-                for (int e = 0; e < E && j0 + e < inner; ++e) drow[j0 + e] = out.e[e];
+                if (j0 + E <= inner) {
+                    *reinterpret_cast<uint4*>(drow + j0) = out.v;
+                } else {
+                    for (int e = 0; e < E && j0 + e < inner; ++e) drow[j0 + e] = out.e[e];
+                }
             }
         }
     }
@@ -389,7 +404,7 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
     const int E = 16 / elt_size(dtype);
     if (row_path(m) && st.s[m.rank - 1] == 1 && (reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) {
         const int64_t total = (m.count + E - 1) / E;
-        const int64_t cpw = 2 * 32 * kUnroll;  // two passes of a warp: short enough to balance the tip of a triangle
+        const int64_t cpw = 4 * 32 * kUnroll;  // four passes of a warp: short enough to balance the tip of a triangle
         const int64_t blocks = ((total + cpw - 1) / cpw + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (dtype == DASTAC_F32)
             pack_stream_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
@@ -433,13 +448,19 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
         const int64_t rows = box / m.dims[m.rank - 1];
         const int64_t chunks_per_row = (m.dims[m.rank - 1] + E - 1) / E;
         const int64_t wpr = (chunks_per_row + 32 * kUnroll - 1) / (32 * kUnroll);
-        const int grid = grid_for(rows * wpr * 32, 32 * kWarpsPerBlock);
+        // a warp takes a whole row unless there are too few rows to fill the GPU
+        const int64_t want_items = (int64_t)sm_count() * 3 * kWarpsPerBlock * 4;
+        int64_t gpr = rows >= want_items ? 1 : (want_items + rows - 1) / rows;
+        if (gpr > wpr) gpr = wpr;
+        const int64_t wpg = (wpr + gpr - 1) / gpr;
+        gpr = (wpr + wpg - 1) / wpg;
+        const int grid = grid_for(rows * gpr * 32, 32 * kWarpsPerBlock);
         if (dtype == DASTAC_F32)
             unpack_stream_kernel<uint32_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
-                m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, wpr);
+                m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)gpr, (int)wpg);
         else
             unpack_stream_kernel<uint16_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
-                m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, wpr);
+                m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)gpr, (int)wpg);
         return launch_status();
     }
     const int last = m.rank - 1;
