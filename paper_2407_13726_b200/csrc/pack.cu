@@ -4,12 +4,11 @@
 // Stream kernels (the fast path, unit inner stride): for fixed outer indices the innermost indices
 // of the set are one interval [jlo, jhi) stored contiguously at pbase + j, with pbase the hoisted
 // part of the ranking polynomial.
-//   pack    a lane owns 16-byte aligned chunks of the PACKED stream.  The matching dense elements
-//           start at an arbitrary element offset, so the lane loads the two aligned 16-byte granules
-//           that cover them and shifts them into place in registers.  Chunks that a row shares with
-//           its neighbour (first and last of the row) are written element by element.  Warps own
-//           equal ranges of the stream, found by one unrank each: the uneven row lengths do not
-//           unbalance the work.
+//   pack    a lane owns 16-byte aligned chunks of the PACKED span of a row.  The matching dense
+//           elements start at an arbitrary element offset, so the lane loads the two aligned
+//           16-byte granules that cover them and shifts them into place in registers.  Chunks that
+//           a row shares with its neighbour (first and last of the row) are written element by
+//           element by both rows.
 //   unpack  a lane owns 16-byte aligned chunks of a DENSE row; the packed source is realigned the
 //           same way, elements outside [jlo, jhi) become zero, and the zero fill of the rest of the
 //           box is the same pass.
@@ -169,69 +168,48 @@ __device__ __forceinline__ int64_t dense_row_offset(const IndexMap& m, const Str
     return off;
 }
 
-// One 16-byte chunk of the packed stream by the generic walk: unrank its first position, then step.
-template <typename T>
-__device__ __forceinline__ void pack_chunk_by_points(const IndexMap& m, const T* __restrict__ dense, const Strides& st,
-                                                     T* __restrict__ packed, const int64_t p0) {
-    constexpr int E = 16 / sizeof(T);
-    Vec16<T> out;
-    int32_t idx[3] = {0, 0, 0};
-    unrank_of(m, p0, idx);
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-        T val = T(0);
-        if (p0 + e < m.count) {
-            val = dense[idx[0] * st.s[0] + idx[1] * st.s[1] + idx[2] * st.s[2]];
-            advance(m, idx);
-        }
-        out.v[e] = val;
-    }
-    *reinterpret_cast<uint4*>(packed + p0) = *reinterpret_cast<const uint4*>(out.v);
-}
-
-// pack: every warp owns an equal, contiguous range of 16-byte chunks of the packed stream, whatever
-// the row lengths are.  It unranks the first position of its range once and then walks from row to
-// row with index increments.  Where rows are shorter than one pass of the warp (the tip of a
-// triangle) the lanes stop cooperating and each takes whole chunks by the generic walk.
+// pack: a warp item is a run of windows (32 * kUnroll chunks each) of the packed span of one row.
+// Items are independent, so short rows (the tip of a triangle) cost one pass each instead of
+// serialising a walk, and rows that are shorter than the longest simply have fewer live windows.
 template <typename T>
 __global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
 pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed,
-                   int64_t chunks_per_warp) {
+                   int64_t rows, int groups_per_row, int windows_per_group) {
     constexpr int E = 16 / sizeof(T);
     const int lane = threadIdx.x & 31;
-    const int64_t total = (m.count + E - 1) / E;
-    // blocks are issued in index order: give the first ones the end of the stream, where a triangle's
-    // rows are shortest and the walk is slowest, so that they do not form the tail of the launch
-    const int64_t cA = ((gridDim.x - 1 - blockIdx.x) * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5)) * chunks_per_warp;
-    if (cA >= total) return;
-    const int64_t cB = (cA + chunks_per_warp < total) ? cA + chunks_per_warp : total;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    int32_t idx[3] = {0, 0, 0};
-    unrank_of(m, cA * E, idx);
-    int64_t c_cur = cA;
-    while (c_cur < cB) {
-        int64_t jlo = 0, jhi = 0, pbase = 0;
-        row_span(m, idx, jlo, jhi, pbase);
-        if ((jhi - jlo) < 32 * E) {
-            const int64_t batch_end = (c_cur + 32 * kUnroll < cB) ? c_cur + 32 * kUnroll : cB;
-            for (int64_t c = c_cur + lane; c < batch_end; c += 32) pack_chunk_by_points<T>(m, dense, st, packed, c * E);
-            c_cur = batch_end;
-            if (c_cur < cB) unrank_of(m, c_cur * E, idx);
-            continue;
+    const int64_t warps = (int64_t)gridDim.x * kWarpsPerBlock;
+    for (int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5); item < rows * groups_per_row;
+         item += warps) {
+        int64_t row = item;
+        int grp = 0;
+        if (groups_per_row > 1) {
+            row = item / groups_per_row;
+            grp = (int)(item - row * groups_per_row);
         }
-        const int64_t ps = pbase + jlo, pe = pbase + jhi;  // the row's span in the packed stream
+        int32_t idx[3] = {0, 0, 0};
+        if (m.rank == 2) {
+            idx[0] = (int32_t)row;
+        } else if (m.rank == 3) {
+            const int64_t q = row / m.dims[1];
+            idx[1] = (int32_t)(row - q * m.dims[1]);
+            idx[0] = (int32_t)q;
+        }
+        int64_t jlo = 0, jhi = 0, pbase = 0;
+        if (!row_span(m, idx, jlo, jhi, pbase)) continue;
+        const int64_t ps = pbase + jlo, pe = pbase + jhi;              // the row's span in the packed stream
         const T* drow = dense + dense_row_offset(m, st, idx) - pbase;  // drow[p]: element stored at position p
-        const int64_t c_lo = (ps / E > c_cur) ? ps / E : c_cur;
-        const int64_t c_end = (pe + E - 1) / E;
-        const int64_t c_hi = (c_end < cB) ? c_end : cB;
-        for (int64_t c0 = c_lo + lane; c0 < c_hi; c0 += 32 * kUnroll) {
+        const int64_t c_first = ps / E;
+        for (int win = grp * windows_per_group; win < (grp + 1) * windows_per_group; ++win) {
+            const int64_t c0 = c_first + (int64_t)win * (32 * kUnroll) + lane;
+            if ((c0 - lane) * E >= pe) break;
             uint4 lo[kUnroll], hi[kUnroll];
             uint32_t sh[kUnroll];
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const int64_t p0 = (c0 + 32 * u) * E;
                 sh[u] = 0;
-                if (c0 + 32 * u < c_hi && p0 >= ps && p0 + E <= pe) {  // whole chunk inside this row
+                if (p0 >= ps && p0 + E <= pe) {  // whole chunk inside this row: two aligned granules cover it
                     const uintptr_t addr = reinterpret_cast<uintptr_t>(drow + p0);
                     sh[u] = (uint32_t)(addr & 15);
                     const uint4* src = reinterpret_cast<const uint4*>(addr - sh[u]);
@@ -242,7 +220,7 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const int64_t p0 = (c0 + 32 * u) * E;
-                if (c0 + 32 * u >= c_hi) break;
+                if (p0 >= pe) break;
                 if (p0 >= ps && p0 + E <= pe) {
                     *reinterpret_cast<uint4*>(packed + p0) = realign16(lo[u], hi[u], sh[u]);
                 } else {  // chunk shared with the neighbouring row, or the tail of the stream
@@ -255,12 +233,6 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
                 }
             }
         }
-        if (pe >= m.count) break;
-        c_cur = pe / E;  // a chunk shared with the next row is visited again for that row's part
-        if (m.rank == 3) idx[2] = (int32_t)(jhi - 1);
-        else if (m.rank == 2) idx[1] = (int32_t)(jhi - 1);
-        else idx[0] = (int32_t)(jhi - 1);
-        advance(m, idx);  // first point of the next row
     }
 }
 
@@ -403,15 +375,22 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
     for (int k = 0; k < m.rank; ++k) st.s[k] = dense_strides[k];
     const int E = 16 / elt_size(dtype);
     if (row_path(m) && st.s[m.rank - 1] == 1 && (reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) {
-        const int64_t total = (m.count + E - 1) / E;
-        const int64_t cpw = 4 * 32 * kUnroll;  // four passes of a warp: short enough to balance the tip of a triangle
-        const int64_t blocks = ((total + cpw - 1) / cpw + kWarpsPerBlock - 1) / kWarpsPerBlock;
+        int64_t rows = 1;
+        for (int k = 0; k + 1 < m.rank; ++k) rows *= m.dims[k];
+        const int64_t chunks_per_row = (m.dims[m.rank - 1] + E - 1) / E + 1;  // a span may straddle one more chunk
+        const int64_t wpr = (chunks_per_row + 32 * kUnroll - 1) / (32 * kUnroll);
+        const int64_t want_items = (int64_t)sm_count() * 3 * kWarpsPerBlock * 4;
+        int64_t gpr = rows >= want_items ? 1 : (want_items + rows - 1) / rows;
+        if (gpr > wpr) gpr = wpr;
+        const int64_t wpg = (wpr + gpr - 1) / gpr;
+        gpr = (wpr + wpg - 1) / wpg;
+        const int grid = grid_for(rows * gpr * 32, 32 * kWarpsPerBlock);
         if (dtype == DASTAC_F32)
-            pack_stream_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
-                m, (const uint32_t*)dense, st, (uint32_t*)packed, cpw);
+            pack_stream_kernel<uint32_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
+                m, (const uint32_t*)dense, st, (uint32_t*)packed, rows, (int)gpr, (int)wpg);
         else
-            pack_stream_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
-                m, (const uint16_t*)dense, st, (uint16_t*)packed, cpw);
+            pack_stream_kernel<uint16_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
+                m, (const uint16_t*)dense, st, (uint16_t*)packed, rows, (int)gpr, (int)wpg);
         return launch_status();
     }
     const int grid = grid_for((m.slots + E - 1) / E, 256);
