@@ -172,7 +172,7 @@ __device__ __forceinline__ int64_t dense_row_offset(const IndexMap& m, const Str
 // Items are independent, so short rows (the tip of a triangle) cost one pass each instead of
 // serialising a walk, and rows that are shorter than the longest simply have fewer live windows.
 template <typename T>
-__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
+__global__ void __launch_bounds__(32 * kWarpsPerBlock, 4)
 pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed,
                    int64_t rows, int groups_per_row, int windows_per_group) {
     constexpr int E = 16 / sizeof(T);
