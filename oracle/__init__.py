@@ -64,10 +64,11 @@ def _load():
         lib.orc_symv.argtypes = [i64, vp, vp, vp, vp]
         lib.orc_matmat.argtypes = [P, ctypes.c_int, i64, vp, vp, vp, i64, vp, vp]
         lib.orc_mttkrp.argtypes = [P, i64, vp, vp, vp, vp, i64, vp, vp]
+        lib.orc_ttm.argtypes = [P, i64, vp, vp, vp, i64, vp, vp]
         lib.orc_num_threads.restype = ctypes.c_int
         for name in ("orc_rank_table", "orc_unrank_table", "orc_pack", "orc_unpack", "orc_band_pack",
                      "orc_band_unpack", "orc_band_slot_table", "orc_matvec", "orc_symv",
-                     "orc_matmat", "orc_mttkrp"):
+                     "orc_matmat", "orc_mttkrp", "orc_ttm"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -238,4 +239,19 @@ def mttkrp(desc, T_slabs, B, C, sel=None):
     out, out_abs = np.empty((len(sel), R)), np.empty((len(sel), R))
     _load().orc_mttkrp(h.ref, len(sel), sel.ctypes.data, T_slabs.ctypes.data, B.ctypes.data,
                        C.ctypes.data, R, out.ctypes.data, out_abs.ctypes.data)
+    return out, out_abs
+
+
+def ttm(desc, B_slabs, C, sel=None):
+    """``A[i][j][k] = sum_l [(i,j,l) in set] B[i][j][l] C[k][l]``; ``B_slabs[s]`` is the dense
+    ``N x Q`` slab ``sel[s]`` of B, C is ``K x Q``.  Returns ``[len(sel), N, K]`` arrays."""
+    h = _Held(desc)
+    sel = _sel(sel, int(h.dims[0]))
+    B_slabs, C = _f32(B_slabs), _f32(C)
+    N, Q = int(h.dims[1]), int(h.dims[2])
+    assert B_slabs.shape == (len(sel), N, Q) and C.shape[1] == Q
+    K = C.shape[0]
+    out, out_abs = np.empty((len(sel), N, K)), np.empty((len(sel), N, K))
+    _load().orc_ttm(h.ref, len(sel), sel.ctypes.data, B_slabs.ctypes.data, C.ctypes.data, K,
+                    out.ctypes.data, out_abs.ctypes.data)
     return out, out_abs

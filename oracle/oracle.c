@@ -298,6 +298,31 @@ void orc_mttkrp(const orc_desc* d, int64_t nsel, const int64_t* sel, const float
     }
 }
 
+/* A[i][j][k] = sum_l [ (i, j, l) in set ] B[i][j][l] * C[k][l]
+ * (A(i,j,k) := B(i,j,l) * C(k,l), the tensor-times-matrix rule of the running example, Section 3).
+ * B_slabs[s] is the dense N x Q slab sel[s] of B; C is K x Q row-major; out[s] is the N x K slab. */
+void orc_ttm(const orc_desc* d, int64_t nsel, const int64_t* sel, const float* B_slabs, const float* C,
+             int64_t K, double* out, double* out_abs) {
+    const int64_t N = d->dims[1], Q = d->dims[2];
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        for (int64_t j = 0; j < N; ++j)
+            for (int64_t k = 0; k < K; ++k) {
+                double acc = 0.0, acc_abs = 0.0;
+                for (int64_t l = 0; l < Q; ++l) {
+                    int64_t idx[3] = {sel[s], j, l};
+                    if (in_domain(d, idx)) {
+                        double p = (double)B_slabs[(s * N + j) * Q + l] * (double)C[k * Q + l];
+                        acc += p;
+                        acc_abs += fabs(p);
+                    }
+                }
+                out[(s * N + j) * K + k] = acc;
+                out_abs[(s * N + j) * K + k] = acc_abs;
+            }
+    }
+}
+
 /* Thread count the contractions above will use. */
 #ifdef _OPENMP
 #include <omp.h>

@@ -363,3 +363,35 @@ def test_mttkrp():
     sel = np.array([11, 2])
     sub, _ = oracle.mttkrp(d, T[sel], B, C, sel=sel)
     assert np.array_equal(sub, out[sel])
+
+
+def test_ttm_upper_half_cube():
+    """Tensor-times-matrix of the paper's running example: A(i,j,k) = B(i,j,l) C(k,l), B nonzero for i <= j."""
+    M, N, Q, K = 5, 7, 4, 6
+    d = st.upper_half_cube(M, N, Q)
+    B = synth.dense(5, 0, (M, N, Q))
+    C = synth.dense(5, 1, (K, Q))
+    out, outa = oracle.ttm(d, B, C)
+    i, j, _ = np.indices((M, N, Q))
+    Bm = np.where(i <= j, B, 0).astype(np.float64)
+    ref = np.einsum("ijl,kl->ijk", Bm, C.astype(np.float64))
+    np.testing.assert_allclose(out, ref, atol=1e-13)
+    np.testing.assert_allclose(outa, np.einsum("ijl,kl->ijk", np.abs(Bm), np.abs(C).astype(np.float64)), rtol=1e-13)
+    # closed forms: all ones -> Q on the set, 0 elsewhere; C = identity returns the masked B itself
+    ones, _ = oracle.ttm(d, np.ones((M, N, Q), np.float32), np.ones((K, Q), np.float32))
+    ii, jj = np.indices((M, N))
+    assert np.array_equal(ones[:, :, 0], np.where(ii <= jj, Q, 0))
+    same, _ = oracle.ttm(d, B, np.eye(Q, dtype=np.float32))
+    assert np.array_equal(same, Bm)
+    # C is indexed (k, l): the transposed operand gives something else
+    Csq = synth.dense(5, 2, (Q, Q))
+    a1, _ = oracle.ttm(d, B, Csq)
+    a2, _ = oracle.ttm(d, B, np.ascontiguousarray(Csq.T))
+    assert np.abs(a1 - a2).max() > 1e-3
+    sel = np.array([4, 1])
+    sub, _ = oracle.ttm(d, B[sel], C, sel=sel)
+    assert np.array_equal(sub, out[sel])
+    # the packed result follows the output's own layout: same (i, j) set, trailing extent K
+    dA = st.upper_half_cube(M, N, K)
+    packedA = oracle.pack(dA, out)
+    assert packedA.shape == (oracle.count(dA),) and oracle.count(dA) == oracle.count(d) // Q * K
