@@ -141,7 +141,8 @@ dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype dtype, const
  * Contraction operand.
  *   structure == NULL: dense tensor, `rank` extents in dims, element strides in strides.
  *   structure != NULL: packed tensor of that structure (dims/strides ignored except that
- *                      batch instances are batch_stride elements apart).
+ *                      batch instances are batch_stride elements apart).  Outputs are dense except
+ *                      where the table of dastac_contract says otherwise.
  *   space: where `data` lives.  Host operands are staged through the workspace with asynchronous
  *          copies on `stream` (pinned memory recommended); a host output is valid after the
  *          caller synchronises the stream.
@@ -168,6 +169,9 @@ typedef struct {
  *   "ij,jc->ic"     band, padded diagonals              f32        C = A B
  *   "ij,jc->ic"     upper triangle (square)             bf16 -> f32 output, fp32 accumulation
  *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)
+ *   "ijl,kl->ijk"   upper half cube (i <= j, dense l)   f32        A = B x_3 C (tensor times matrix, the
+ *                   running example of Section 3); `out` is PACKED too: out->structure must be the
+ *                   upper half cube with the same first two extents and trailing extent K = rows of C
  * accumulate: 0 -> out = result (the library zero-fills where it needs to), 1 -> out += result.
  * workspace: device scratch of at least dastac_contract_workspace bytes, 256-byte aligned; may be
  *            NULL when that size is 0.  Its contents are undefined afterwards.

@@ -237,18 +237,19 @@ def _operand(t: torch.Tensor, structure: Optional[Structure], batch: int) -> _Op
     return op
 
 
-def _operands(s, packed, dense_inputs, out, batch):
+def _operands(s, packed, dense_inputs, out, batch, out_structure=None):
     ins = (_Operand * (1 + len(dense_inputs)))()
     ins[0] = _operand(packed, s, batch)
     for k, t in enumerate(dense_inputs):
         ins[1 + k] = _operand(t, None, batch)
-    o = _operand(out, None, batch)
+    o = _operand(out, out_structure, batch)
     return ins, o
 
 
 def contract_workspace(expr: str, s: Structure, packed: torch.Tensor,
-                       dense_inputs: Sequence[torch.Tensor], out: torch.Tensor, batch: int = 1) -> int:
-    ins, o = _operands(s, packed, dense_inputs, out, batch)
+                       dense_inputs: Sequence[torch.Tensor], out: torch.Tensor, batch: int = 1,
+                       out_structure: Optional[Structure] = None) -> int:
+    ins, o = _operands(s, packed, dense_inputs, out, batch, out_structure)
     nbytes = ctypes.c_size_t()
     _check(_lib.dastac_contract_workspace(expr.encode(), ins, len(ins), ctypes.byref(o),
                                           ctypes.byref(nbytes)), "dastac_contract_workspace")
@@ -257,10 +258,12 @@ def contract_workspace(expr: str, s: Structure, packed: torch.Tensor,
 
 def contract(expr: str, s: Structure, packed: torch.Tensor, dense_inputs: Sequence[torch.Tensor],
              out: torch.Tensor, accumulate: bool = False, workspace: Optional[torch.Tensor] = None,
-             err_word: Optional[torch.Tensor] = None, batch: int = 1) -> torch.Tensor:
+             err_word: Optional[torch.Tensor] = None, batch: int = 1,
+             out_structure: Optional[Structure] = None) -> torch.Tensor:
     """Evaluate ``expr`` with ``packed`` (structure ``s``) as first operand.  Tensors may live on
-    the device or in (pinned) host memory; host tensors are staged through ``workspace``."""
-    ins, o = _operands(s, packed, dense_inputs, out, batch)
+    the device or in (pinned) host memory; host tensors are staged through ``workspace``.
+    ``out_structure`` marks ``out`` as a packed buffer of that structure (rules with packed output)."""
+    ins, o = _operands(s, packed, dense_inputs, out, batch, out_structure)
     ws_ptr, ws_bytes = None, 0
     if workspace is not None:
         ws_ptr, ws_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()

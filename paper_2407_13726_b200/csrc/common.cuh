@@ -45,6 +45,8 @@ dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, i
 dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, int64_t ldb,
                             const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
                             int accumulate, cudaStream_t st);
+dastac_status launch_ttm(int64_t P, int64_t Q, int64_t K, const float* X, const float* C, int64_t ldc, float* Y,
+                         int accumulate, cudaStream_t st);
 size_t trimm_workspace_bytes(const IndexMap& m, int64_t ncols, int64_t ldb);
 dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B, int64_t ldb,
                                 float* C, int64_t ldc, int64_t ncols, int accumulate,

@@ -7,13 +7,14 @@
 namespace dastac {
 namespace {
 
-enum ExprClass { kMatVec, kMatMat, kMttkrp, kNoExpr };
+enum ExprClass { kMatVec, kMatMat, kMttkrp, kTtm, kNoExpr };
 
 ExprClass parse_expr(const char* e) {
     if (!e) return kNoExpr;
     if (!std::strcmp(e, "ij,j->i")) return kMatVec;
     if (!std::strcmp(e, "ij,jc->ic")) return kMatMat;
     if (!std::strcmp(e, "ijk,jr,kr->ir")) return kMttkrp;
+    if (!std::strcmp(e, "ijl,kl->ijk")) return kTtm;
     return kNoExpr;
 }
 
@@ -63,7 +64,7 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
     p.cls = parse_expr(expr);
     if (!in || !out || n_in < 1) return DASTAC_ERR_INVALID_ARG;
     if (p.cls == kNoExpr) return DASTAC_ERR_UNSUPPORTED_EXPR;
-    const int want_in = p.cls == kMttkrp ? 3 : 2;
+    const int want_in = p.cls == kMttkrp ? 3 : 2;  // the tensor-times-matrix rule has two inputs as well
     if (n_in != want_in) return DASTAC_ERR_INVALID_ARG;
     if (!in[0].structure) return DASTAC_ERR_UNSUPPORTED_EXPR;
     if (!(in[0].space == DASTAC_MEM_DEVICE || in[0].space == DASTAC_MEM_HOST))
@@ -72,7 +73,34 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
     p.map = &m;
     p.batch = batch_of(in[0]);
 
-    if (p.cls == kMatVec) {
+    if (out->structure && p.cls != kTtm) return DASTAC_ERR_UNSUPPORTED_EXPR;  // only this rule packs its output
+    if (p.cls == kTtm) {
+        // packed upper half cube in, packed upper half cube out: same (i, j) set, trailing extents Q and K
+        if (!out->structure) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        const IndexMap& mo = out->structure->map;
+        if (p.batch != 1 || batch_of(in[1]) != 1 || batch_of(*out) != 1) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        // classes whose trailing index is dense and contiguous (extents of 1 can close a half cube to
+        // the dense box or to the one-point tetrahedron: the same set, the same layout)
+        auto trailing_dense = [](const IndexMap& x) {
+            return x.kind == kEmpty || (x.rank == 3 && (x.kind == kUpper || x.kind == kDense ||
+                                                        (x.kind == kTetrahedron && x.dims[0] == 1)));
+        };
+        if (!trailing_dense(m) || !trailing_dense(mo)) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (in[0].dtype != DASTAC_F32 || in[1].dtype != DASTAC_F32 || out->dtype != DASTAC_F32)
+            return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (!dense_ok(in[1], 2)) return DASTAC_ERR_INVALID_ARG;
+        if (!(out->space == DASTAC_MEM_DEVICE || out->space == DASTAC_MEM_HOST)) return DASTAC_ERR_INVALID_ARG;
+        if (mo.dims[0] != m.dims[0] || mo.dims[1] != m.dims[1] || in[1].dims[0] != mo.dims[2] ||
+            in[1].dims[1] != m.dims[2])
+            return DASTAC_ERR_SHAPE;
+        if (m.dims[2] > 1 && in[1].strides[1] != 1) return DASTAC_ERR_SHAPE;
+        // the same (i, j) set on both sides
+        if ((m.dims[2] > 0 ? m.count / m.dims[2] : 0) != (mo.dims[2] > 0 ? mo.count / mo.dims[2] : 0) &&
+            m.dims[2] > 0 && mo.dims[2] > 0)
+            return DASTAC_ERR_SHAPE;
+        p.N = m.dims[2];   // Q
+        p.R = mo.dims[2];  // K
+    } else if (p.cls == kMatVec) {
         if (!(m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1]) && m.kind != kEmpty)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (in[0].dtype != DASTAC_F32 || in[1].dtype != DASTAC_F32 || out->dtype != DASTAC_F32)
@@ -191,6 +219,13 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
 
     if (m.kind == kEmpty || out_bytes == 0) {
         st = DASTAC_OK;
+        // an empty sum over l (Q = 0) still defines the packed output: zero
+        if (p.cls == kTtm && out_bytes > 0 && !accumulate &&
+            cudaMemsetAsync(dev_out, 0, (size_t)out_bytes, cs) != cudaSuccess)
+            st = DASTAC_ERR_CUDA;
+    } else if (p.cls == kTtm) {
+        st = launch_ttm(m.count / p.N, p.N, p.R, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0],
+                        (float*)dev_out, accumulate, cs);
     } else if (p.cls == kMatVec && !p.symmetric) {
         st = launch_trmv(m, (const float*)dev_in[0], (const float*)dev_in[1], (float*)dev_out,
                          p.batch, in[0].batch_stride, in[1].batch_stride, out->batch_stride,

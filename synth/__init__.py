@@ -43,6 +43,8 @@ def _load():
         lib.synth_fill_symmetric_row.restype = None
         lib.synth_stream_upper_triangle.argtypes = [u64, u64, cint, dbl, cint, u64, vp]
         lib.synth_stream_upper_triangle.restype = u64
+        lib.synth_stream_upper_half_cube.argtypes = [u64, u64, cint, dbl, u64, u64, u64, vp]
+        lib.synth_stream_upper_half_cube.restype = u64
         lib.synth_stream_tetrahedron.argtypes = [u64, u64, cint, dbl, cint, u64, vp]
         lib.synth_stream_tetrahedron.restype = u64
         lib.synth_stream_band_diagonals.argtypes = [u64, u64, cint, dbl, u64, u64, ctypes.c_uint32, vp]
@@ -90,6 +92,15 @@ def upper_triangle_stream(seed, tensor_id, N, dist=UNIFORM, scale=1.0, bf16=Fals
     got = _load().synth_stream_upper_triangle(seed, tensor_id, dist, scale, int(bf16), int(N), ptr)
     assert got == n
     return arr[:n]
+
+
+def upper_half_cube_stream(seed, tensor_id, M, N, Q, dist=UNIFORM, scale=1.0, out=None):
+    """Values of ``{(i, j, l): 0 <= i < M, i <= j < N, 0 <= l < Q}`` in (i, j, l) order."""
+    cnt = _load().synth_stream_upper_half_cube(seed, tensor_id, dist, scale, int(M), int(N), int(Q), None)
+    arr, ptr = _out(cnt, False, out)
+    got = _load().synth_stream_upper_half_cube(seed, tensor_id, dist, scale, int(M), int(N), int(Q), ptr)
+    assert got == cnt
+    return arr[:cnt]
 
 
 def tetrahedron_stream(seed, tensor_id, n, dist=UNIFORM, scale=1.0, out=None):

@@ -103,6 +103,27 @@ uint64_t synth_stream_upper_triangle(uint64_t seed, uint64_t tensor_id, int dist
     return total;
 }
 
+/* Upper half cube 0 <= i < M, i <= j < N, 0 <= l < Q of an M x N x Q tensor, emitted in (i, j, l)
+ * order.  Returns the number of values written (counted by the same walk when out == NULL). */
+uint64_t synth_stream_upper_half_cube(uint64_t seed, uint64_t tensor_id, int dist, double scale,
+                                      uint64_t M, uint64_t N, uint64_t Q, void* out) {
+    uint64_t key = tensor_key(seed, tensor_id);
+    uint64_t* start = (uint64_t*)malloc((M + 1) * sizeof(uint64_t));
+    if (!start) return 0;
+    start[0] = 0;
+    for (uint64_t i = 0; i < M; ++i) start[i + 1] = start[i] + (i < N ? (N - i) * Q : 0);
+    if (!out) { uint64_t c = start[M]; free(start); return c; }
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t i = 0; i < (int64_t)M; ++i)
+        for (uint64_t j = (uint64_t)i; j < N; ++j)
+            for (uint64_t l = 0; l < Q; ++l)
+                store_value(out, 0, (size_t)(start[i] + (j - (uint64_t)i) * Q + l),
+                            value_at(key, dist, scale, ((uint64_t)i * N + j) * Q + l));
+    uint64_t total = start[M];
+    free(start);
+    return total;
+}
+
 /* Tetrahedron 0 <= i <= j <= k < n of an n x n x n tensor, emitted in (i, j, k) order. */
 uint64_t synth_stream_tetrahedron(uint64_t seed, uint64_t tensor_id, int dist, double scale,
                                   int as_bf16, uint64_t n, void* out) {

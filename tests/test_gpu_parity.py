@@ -336,3 +336,41 @@ def test_empty_and_degenerate_inputs():
     out = torch.empty((16, 0), device="cuda")
     dastac.contract("ij,jc->ic", s, s.empty_packed(), [torch.empty((16, 0), device="cuda")], out)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("M,N,Q,K", [(1, 1, 1, 1), (5, 7, 4, 6), (7, 5, 3, 5), (33, 40, 32, 32), (64, 64, 20, 12),
+                                     (130, 130, 32, 64), (97, 97, 37, 33), (300, 300, 8, 40)])
+def test_ttm_upper_half_cube_packed_in_packed_out(M, N, Q, K):
+    """The paper's running example A(i,j,k) = B(i,j,l) C(k,l), i <= j: packed operand, packed result."""
+    dB, dA = st.upper_half_cube(M, N, Q), st.upper_half_cube(M, N, K)
+    sB, sA = dastac.Structure(dB), dastac.Structure(dA)
+    B = synth.dense(5, 0, (M, N, Q))
+    C = synth.dense(5, 1, (K, Q))
+    ref, ref_abs = oracle.ttm(dB, B, C)
+    exp, exp_abs = oracle.pack(dA, ref), oracle.pack(dA, ref_abs)
+    assert sA.nnz == exp.size
+    packedB = packed_dev(sB, synth.upper_half_cube_stream(5, 0, M, N, Q))
+    out = sA.empty_packed()
+    out.fill_(float("nan"))
+    dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out, out_structure=sA)
+    assert rel_err(out.cpu().numpy()[: sA.nnz], exp, exp_abs) <= TOL_F32
+    A0 = synth.dense(5, 2, (sA.nnz,))
+    out2 = sA.empty_packed()
+    out2[: sA.nnz] = dev(A0)
+    dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out2, accumulate=True, out_structure=sA)
+    assert rel_err(out2.cpu().numpy()[: sA.nnz], exp + A0, exp_abs + np.abs(A0)) <= TOL_F32
+    # a padded leading dimension of C
+    Cp = torch.zeros((K, Q + 3), device="cuda")[:, :Q]
+    Cp.copy_(dev(C))
+    out3 = sA.empty_packed()
+    dastac.contract("ijl,kl->ijk", sB, packedB, [Cp], out3, out_structure=sA)
+    assert rel_err(out3.cpu().numpy()[: sA.nnz], exp, exp_abs) <= TOL_F32
+    # the unpacked result is the dense rule on the set and zero off it
+    dense = dastac.unpack(sA, out).cpu().numpy()
+    ii, jj = np.indices((M, N))
+    assert (dense[ii > jj] == 0).all()
+    # shape errors are reported before anything runs
+    if K > 1:
+        with pytest.raises(dastac.DastacError) as e:
+            dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C[:-1])], out, out_structure=sA)
+        assert e.value.status == 4
