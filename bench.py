@@ -53,8 +53,8 @@ def peaks():
 
 def sizes(small: bool):
     if small:
-        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024)
-    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192)
+        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024, N6=128, Q6=32, K6=32)
+    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192, N6=1024, Q6=32, K6=32)
 
 
 def accounting(z):
@@ -62,6 +62,7 @@ def accounting(z):
     read once, the output written once) of every kernel of a step."""
     N1, b, N2, w, C2, N3, n4, R, N5 = (z[k] for k in ("N1", "batch", "N2", "w", "C2", "N3", "n4", "R", "N5"))
     nnz2 = (2 * w + 1) * N2 - w * (w + 1)
+    N6, Q6, K6 = z["N6"], z["Q6"], z["K6"]
     acc = {
         "trmv": dict(flops=2 * tri(N1), bytes=4 * (tri(N1) + 2 * N1), bound="hbm"),
         "trmv_batched": dict(flops=2 * tri(N1) * b, bytes=4 * (tri(N1) + 2 * N1) * b, bound="hbm"),
@@ -71,11 +72,13 @@ def accounting(z):
         "trimm_bf16": dict(flops=2 * tri(N5) * N5, bytes=2 * tri(N5) + 2 * N5 * N5 + 4 * N5 * N5, bound="tensor"),
         "pack_bf16": dict(flops=0, bytes=2 * (2 * tri(N5)), bound="hbm"),          # read the set, write it
         "unpack_bf16": dict(flops=0, bytes=2 * (tri(N5) + N5 * N5), bound="hbm"),  # read packed, write box
+        # widened row: tensor times matrix over the upper half cube, packed in and out (8 flop/B: HBM first)
+        "ttm_ut": dict(flops=2 * tri(N6) * Q6 * K6, bytes=4 * (tri(N6) * (Q6 + K6) + K6 * Q6), bound="hbm"),
     }
     return acc
 
 
-ORDER = ["trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
+ORDER = ["trmv", "trmv_batched", "bandmm", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
 
 
 def generate_host(z, pin, only=None):
@@ -132,11 +135,17 @@ def generate_host(z, pin, only=None):
         h["trimm_bf16"] = dict(desc=st.upper_triangle(N5), A=host(a5, True),
                                ins=[host(synth.dense(4, 1, (N5, N5), dist=synth.NORMAL, scale=sc, bf16=True), True)],
                                out=(N5, N5))
+    if want("ttm_ut"):
+        N6, Q6, K6 = z["N6"], z["Q6"], z["K6"]
+        a6 = np.zeros(cap(tri(N6) * Q6, 4), np.float32)
+        synth.upper_half_cube_stream(5, 0, N6, N6, Q6, out=a6)
+        h["ttm_ut"] = dict(desc=st.upper_half_cube(N6, N6, Q6), out_desc=st.upper_half_cube(N6, N6, K6), A=host(a6),
+                           ins=[host(synth.dense(5, 1, (K6, Q6)))], out=(cap(tri(N6) * K6, 4),))
     return h
 
 
 EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
-        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic"}
+        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk"}
 
 
 # ---- clocks ---------------------------------------------------------------------------------------------
@@ -244,8 +253,10 @@ def run_gpu(args):
         s = dastac.Structure(hw["desc"])
         structs[name] = s
         d = dict(A=hw["A"].cuda(), ins=[t.cuda() for t in hw["ins"]],
-                 out=torch.empty(hw["out"], dtype=torch.float32, device="cuda"), batch=hw.get("batch", 1))
-        n = dastac.contract_workspace(EXPR[name], s, d["A"], d["ins"], d["out"], batch=d["batch"])
+                 out=torch.empty(hw["out"], dtype=torch.float32, device="cuda"), batch=hw.get("batch", 1),
+                 out_s=dastac.Structure(hw["out_desc"]) if "out_desc" in hw else None)
+        n = dastac.contract_workspace(EXPR[name], s, d["A"], d["ins"], d["out"], batch=d["batch"],
+                                      out_structure=d["out_s"])
         d["ws"] = torch.empty(n, dtype=torch.uint8, device="cuda") if n else None
         devs[name] = d
     err_word = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -264,7 +275,7 @@ def run_gpu(args):
             dastac.unpack(structs["trimm_bf16"], d["A"], d["out"])
         else:
             dastac.contract(EXPR[name], structs[name], d["A"], d["ins"], d["out"], workspace=d["ws"],
-                            err_word=err_word, batch=d["batch"])
+                            err_word=err_word, batch=d["batch"], out_structure=d.get("out_s"))
 
     def run_kernel(name):
         run_kernel_on(name, devs[name])
@@ -377,7 +388,8 @@ def run_gpu(args):
             if name not in order:
                 continue
             out_h = torch.empty(hw["out"], dtype=torch.float32).pin_memory()
-            n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1))
+            n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1),
+                                          out_structure=devs[name]["out_s"])
             hd[name] = dict(out=out_h, ws=torch.empty(n, dtype=torch.uint8, device="cuda"))
             h2d += hw["A"].numel() * hw["A"].element_size() + sum(t.numel() * t.element_size() for t in hw["ins"])
             d2h += out_h.numel() * 4
@@ -387,7 +399,8 @@ def run_gpu(args):
                 if name in hd:
                     hw = host[name]
                     dastac.contract(EXPR[name], structs[name], hw["A"], hw["ins"], hd[name]["out"],
-                                    workspace=hd[name]["ws"], err_word=err_word, batch=hw.get("batch", 1))
+                                    workspace=hd[name]["ws"], err_word=err_word, batch=hw.get("batch", 1),
+                                    out_structure=devs[name]["out_s"])
 
         e2e_flops = sum(acct[n]["flops"] for n in hd)
         e_steps = max(1, min(args.steps, 3))
@@ -417,7 +430,8 @@ def run_gpu(args):
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
             "data": "synthetic",
-            "config": {"workload": "all five configs per step: " + json.dumps(z, separators=(",", ":")),
+            "config": {"workload": "all five configs per step, plus the tensor-times-matrix running example (N6,Q6,K6): "
+                                   + json.dumps(z, separators=(",", ":")),
                        "small": bool(args.small), "only": args.only or None,
                        "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
                              "(the 8.6 GB symmetric stream runs once per step)",
@@ -535,6 +549,13 @@ def oracle_sample(z, scale=1.0):
     secs += timed(lambda: oracle.matmat(st.upper_triangle(N5), A5, B5, sel=sel))
     flops += sum(2 * (N5 - int(i)) * N5 for i in sel)
     parts.append(f"cfg5 {len(sel)} rows x {N5} cols")
+    N6, Q6, K6 = z["N6"], z["Q6"], z["K6"]
+    sel = rows(N6, 48)
+    B6 = np.stack([synth.linear_slice(5, 0, int(i) * N6 * Q6, N6 * Q6).reshape(N6, Q6) for i in sel])
+    C6 = synth.dense(5, 1, (K6, Q6))
+    secs += timed(lambda: oracle.ttm(st.upper_half_cube(N6, N6, Q6), B6, C6, sel=sel))
+    flops += sum(2 * (N6 - int(i)) * Q6 * K6 for i in sel)
+    parts.append(f"ttm {len(sel)} slabs")
     return flops, secs, "rows spread evenly over the outer index: " + ", ".join(parts)
 
 
@@ -565,7 +586,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(tot_s / steps * 1e3, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "all five configs per step: " + json.dumps(z, separators=(",", ":")),
+        "config": {"workload": "all five configs per step, plus the tensor-times-matrix running example (N6,Q6,K6): "
+                               + json.dumps(z, separators=(",", ":")),
                    "sample": desc},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

@@ -149,3 +149,29 @@ def test_config5_triangular_bf16_n8192():
         assert np.array_equal(rows[r], exp)
     repacked = dastac.pack(s, dense)
     assert torch.equal(repacked.view(torch.int16)[: s.nnz], packed.view(torch.int16)[: s.nnz])
+
+
+def test_widened_row_ttm_n1024_q32_k32():
+    """The tensor-times-matrix running example at the size the benchmark times: sampled slabs i of
+    the packed result (slab i is the contiguous run of positions that starts at (i, i, 0))."""
+    N, Q, K = 1024, 32, 32
+    dB, dA = st.upper_half_cube(N, N, Q), st.upper_half_cube(N, N, K)
+    sB, sA = dastac.Structure(dB), dastac.Structure(dA)
+    assert sA.nnz == N * (N + 1) // 2 * K
+    C = synth.dense(5, 1, (K, Q))
+    packedB = _packed(sB, lambda h: synth.upper_half_cube_stream(5, 0, N, N, Q, out=h))
+    out = torch.full((sA.capacity(torch.float32),), float("nan"), device="cuda")
+    dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out, out_structure=sA)
+    got = out.cpu().numpy()[: sA.nnz]
+    assert np.isfinite(got).all()
+    sel = _rows(N, 12, extra=(1, 255, 256, 257, N - 2))
+    Bs = np.stack([synth.linear_slice(5, 0, int(i) * N * Q, N * Q).reshape(N, Q) for i in sel])
+    ref, ref_abs = oracle.ttm(dB, Bs, C, sel=sel)
+    # where slab i starts in the packed result: device and host maps must agree, the oracle counts it for two slabs
+    starts = dastac.rank_batch(sA, torch.tensor([[int(i), int(i), 0] for i in sel], dtype=torch.int32).cuda()).cpu().numpy()
+    for probe in (0, len(sel) // 2):
+        assert starts[probe] == oracle.rank_point(dA, (int(sel[probe]), int(sel[probe]), 0))
+    for s, i in enumerate(sel):
+        n_el = (N - int(i)) * K
+        seg = got[starts[s]: starts[s] + n_el]
+        assert rel_err(seg, ref[s, int(i):, :].reshape(-1), ref_abs[s, int(i):, :].reshape(-1)) <= TOL_F32
