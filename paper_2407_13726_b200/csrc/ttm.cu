@@ -65,9 +65,10 @@ ttm_kernel(int64_t P, int64_t Q, int64_t K, const float* __restrict__ X, const f
                 Xs[r][l] = (p < P && l0 + l < Q) ? __ldg(X + p * Q + l0 + l) : 0.f;
             }
         }
-        // C tile transposed: Cs[l][k] = C(k0 + k, l0 + l)
+        // C tile transposed: Cs[l][k] = C(k0 + k, l0 + l); lanes run along k so that the shared stores of a
+        // warp fall in 32 different banks (the tile is 4 KiB: the strided global reads do not matter)
         for (int item = tid; item < kKT * kLc; item += kThreads) {
-            const int k = item >> 5, l = item & 31;
+            const int k = item & 31, l = item >> 5;
             Cs[l][k] = (k0 + k < K && l0 + l < Q) ? __ldg(C + (k0 + k) * ldc + l0 + l) : 0.f;
         }
         __syncthreads();
