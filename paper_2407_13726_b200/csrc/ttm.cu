@@ -150,10 +150,11 @@ ttm_stream_kernel(int64_t P, int64_t Q, int64_t K, int64_t row_tiles, const floa
             const int64_t p = p0 + r;
             cp_async16(&sg.Xs[r][4 * c4], p < P ? X + p * Q + l0 + 4 * c4 : X, p < P ? 16 : 0);
         }
-        for (int item = tid; item < kKT * kLc; item += kThreads) {
-            const int k = item & 31, l = item >> 5;
-            sg.Cs[l][k] = (k0 + k < K) ? __ldg(C + (k0 + k) * ldc + l0 + l) : 0.f;
-        }
+        if (chunks > 1 || n < 2)  // with a single chunk the C tile never changes: fill each stage once
+            for (int item = tid; item < kKT * kLc; item += kThreads) {
+                const int k = item & 31, l = item >> 5;
+                sg.Cs[l][k] = (k0 + k < K) ? __ldg(C + (k0 + k) * ldc + l0 + l) : 0.f;
+            }
     };
 
     if (items > 0) request(0);
