@@ -374,3 +374,58 @@ def test_ttm_upper_half_cube_packed_in_packed_out(M, N, Q, K):
         with pytest.raises(dastac.DastacError) as e:
             dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C[:-1])], out, out_structure=sA)
         assert e.value.status == 4
+
+
+@pytest.mark.parametrize("N", [2047, 2048, 2049, 4097])
+def test_matvec_kernels_around_tile_edges(N):
+    """Sizes that straddle the kernels' own limits: 2048 is the last N of the quad TRMV kernel and one
+    column tile of the SYMV kernel, 4097 leaves a one-column last tile."""
+    U = synth.dense(12, 0, (N, N), dist=synth.NORMAL)
+    x = synth.dense(12, 1, (N,), dist=synth.NORMAL)
+    stream = synth.upper_triangle_stream(12, 0, N, dist=synth.NORMAL)
+    d = st.upper_triangle(N)
+    s = dastac.Structure(d)
+    ref, ref_abs = oracle.matvec(d, U, x)
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed_dev(s, stream), [dev(x)], y)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    ss = dastac.Structure(st.upper_triangle(N, symmetric=True))
+    ref, ref_abs = oracle.symv(U, x)
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", ss, packed_dev(ss, stream), [dev(x)], y)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+
+
+def test_matvec_does_not_read_values_beyond_the_rows():
+    """Non-finite values in a neighbouring row or in the padding behind the last row must not leak
+    into a result through the masked first / last quads."""
+    N = 203
+    d = st.upper_triangle(N)
+    s = dastac.Structure(d)
+    A = synth.dense(13, 0, (N, N))
+    A[5, 5:] = np.inf          # row 5 is all infinite: only y[5] may be non-finite
+    x = np.abs(synth.dense(13, 1, (N,))) + 0.5
+    packed = packed_dev(s, oracle.pack(d, A))      # tail of the buffer is NaN
+    y = torch.empty(N, device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y)
+    got = y.cpu().numpy()
+    assert np.isinf(got[5]) and np.isfinite(np.delete(got, 5)).all()
+    A[5, 5:] = 0
+    ref, ref_abs = oracle.matvec(d, A, x)
+    keep = np.arange(N) != 5
+    assert rel_err(got[keep], ref[keep], ref_abs[keep]) <= TOL_F32
+
+
+@pytest.mark.parametrize("desc", [st.tetrahedron(150), st.lower_triangle(1000), st.dense_box([3000]),
+                                  st.dense_box([40, 50, 60]), st.upper_triangle(2050)],
+                         ids=lambda d: f"{d.name}{d.dims}")
+def test_pack_unpack_larger_f32(desc):
+    s = dastac.Structure(desc)
+    bits = _bits(tuple(desc.dims), 17)
+    dense = torch.from_numpy(bits.view(np.int32)).cuda().view(torch.float32)
+    packed = dastac.pack(s, dense)
+    exp = oracle.pack(desc, bits)
+    assert np.array_equal(packed.view(torch.int32).cpu().numpy().view(np.uint32)[: s.nnz], exp)
+    out = torch.full(desc.dims, float("nan"), device="cuda")
+    dastac.unpack(s, packed, out)
+    assert np.array_equal(out.view(torch.int32).cpu().numpy().view(np.uint32), oracle.unpack(desc, exp))
