@@ -54,7 +54,8 @@ typedef enum {
     DASTAC_KIND_UPPER = 2,          /* 0<=i<M, i<=j<N, optional trailing dense extent Q (rank 3)   */
     DASTAC_KIND_LOWER = 3,          /* 0<=j<=i<N                                                   */
     DASTAC_KIND_BAND_DIAGONALS = 4, /* |i-j|<=w stored as 2w+1 diagonals of N slots                */
-    DASTAC_KIND_TETRAHEDRON = 5     /* 0<=i<=j<=k<n                                                */
+    DASTAC_KIND_TETRAHEDRON = 5,    /* 0<=i<=j<=k<n                                                */
+    DASTAC_KIND_BAND_EXACT = 6      /* |i-j|<=w, 2w+1<=N, rows packed back to back (no padding)    */
 } dastac_kind;
 
 #define DASTAC_LAYOUT_LEXICOGRAPHIC 0 /* exact pack in lexicographic order                         */
@@ -166,7 +167,7 @@ typedef struct {
  * Supported (expression, structure of in[0], dtypes):
  *   "ij,j->i"       upper triangle (square)             f32        y = A x         (batched)
  *   "ij,j->i"       upper triangle + swap (symmetric)   f32        y = S x
- *   "ij,jc->ic"     band, padded diagonals              f32        C = A B
+ *   "ij,jc->ic"     band, padded diagonals or exact     f32        C = A B
  *   "ij,jc->ic"     upper triangle (square)             bf16 -> f32 output, fp32 accumulation
  *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)
  *   "ijl,kl->ijk"   upper half cube (i <= j, dense l)   f32        A = B x_3 C (tensor times matrix, the

@@ -1,5 +1,6 @@
-// C = A B for a banded A (|i - j| <= w) stored as 2w+1 padded diagonals of N slots, B and C dense
-// row-major, fp32.  Slot (d, i) holds A(i, i + d - w): for a fixed diagonal consecutive rows are
+// C = A B for a banded A (|i - j| <= w), B and C dense row-major, fp32.  A is stored as 2w+1 padded
+// diagonals of N slots (described below), or packed exactly, row after row (then the band slice of a
+// row tile is gathered by the threads at rowbase(i) + j, everything else is the same).  Slot (d, i) holds A(i, i + d - w): for a fixed diagonal consecutive rows are
 // consecutive in memory and the position is the affine map d*N + i.  Padding slots are never read
 // into a result: a slot whose column i + d - w falls outside [0, N) is replaced by zero while the
 // band is staged, whatever it contains.
@@ -77,7 +78,7 @@ __device__ __forceinline__ void load_row(pair_t (&dst)[kPairs], const float* __r
 template <bool TMA_B>
 __global__ void __launch_bounds__(kThreads, 4)
 bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_a, int tma_a,
-              int64_t N, int64_t w, int64_t row_tile0,
+              int exact, int64_t N, int64_t w, int64_t row_tile0,
               const float* __restrict__ A, const float* __restrict__ B, int64_t ldb, float* __restrict__ C,
               int64_t ldc, int64_t ncols, int accumulate, int vec_c, int32_t* err_word) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -134,7 +135,9 @@ bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant_
             for (int t = tid; t < kChunk * kRows; t += kThreads) {
                 const int dl = t / kRows, r = t - dl * kRows;
                 const int64_t d = dc + dl, i = i0 + r, jj = i + d - w;
-                Ad[t] = (d < diagonals && i < N && jj >= 0 && jj < N) ? __ldg(A + d * N + i) : 0.f;
+                // padded diagonals: slot (d, i); exact rows: rowbase(i) + j with the row's hoisted base
+                const int64_t pos = exact ? band_row_start(N, w, i) - band_jlo(w, i) + jj : d * N + i;
+                Ad[t] = (d < diagonals && i < N && jj >= 0 && jj < N) ? __ldg(A + pos) : 0.f;
             }
         }
         if (TMA_B) {
@@ -276,7 +279,8 @@ dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, i
     CUtensorMap tmap_a;
     std::memset(&tmap_a, 0, sizeof(tmap_a));
     int tma_a = 0;
-    if (tma_b && (N % 4 == 0) && aligned16(A)) {
+    const int exact = m.kind == kBandExact;
+    if (!exact && tma_b && (N % 4 == 0) && aligned16(A)) {
         const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)(2 * m.w + 1)};
         const cuuint64_t strides[1] = {(cuuint64_t)N * 4};
         const cuuint32_t box[2] = {(cuuint32_t)kRows, (cuuint32_t)kChunk};
@@ -300,10 +304,10 @@ dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, i
         const int64_t ny = gy - y0 < 65535 ? gy - y0 : 65535;
         const dim3 grid((unsigned)gx, (unsigned)ny);
         if (tma_b)
-            bandmm_kernel<true><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, N, m.w, y0, A, B, ldb, C, ldc, ncols, accumulate,
+            bandmm_kernel<true><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, exact, N, m.w, y0, A, B, ldb, C, ldc, ncols, accumulate,
                                                               vec_c, err_word);
         else
-            bandmm_kernel<false><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, N, m.w, y0, A, B, ldb, C, ldc, ncols,
+            bandmm_kernel<false><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, exact, N, m.w, y0, A, B, ldb, C, ldc, ncols,
                                                                accumulate, vec_c, err_word);
         dastac_status s = launch_status();
         if (s != DASTAC_OK) return s;

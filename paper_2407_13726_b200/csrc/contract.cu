@@ -117,7 +117,7 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         if (p.batch != 1 || batch_of(in[1]) != 1 || batch_of(*out) != 1)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (!dense_ok(in[1], 2) || !dense_ok(*out, 2)) return DASTAC_ERR_INVALID_ARG;
-        const bool band = m.kind == kBandDiagonals && in[0].dtype == DASTAC_F32 &&
+        const bool band = (m.kind == kBandDiagonals || m.kind == kBandExact) && in[0].dtype == DASTAC_F32 &&
                           in[1].dtype == DASTAC_F32 && out->dtype == DASTAC_F32;
         const bool tri_bf16 = m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1] &&
                               !m.symmetric && in[0].dtype == DASTAC_BF16 &&
@@ -233,7 +233,7 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     } else if (p.cls == kMatVec) {
         st = launch_symv(m, (const float*)dev_in[0], (const float*)dev_in[1], (float*)dev_out,
                          accumulate, scratch, cs);
-    } else if (p.cls == kMatMat && m.kind == kBandDiagonals) {
+    } else if (p.cls == kMatMat && (m.kind == kBandDiagonals || m.kind == kBandExact)) {
         st = launch_bandmm(m, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0],
                            (float*)dev_out, out->strides[0], p.ncols, accumulate, err_word, cs);
     } else if (p.cls == kMatMat) {

@@ -27,7 +27,8 @@ enum Kind : int32_t {
     kUpper = 2,
     kLower = 3,
     kBandDiagonals = 4,
-    kTetrahedron = 5
+    kTetrahedron = 5,
+    kBandExact = 6  // |i - j| <= w packed row after row without padding (2w + 1 <= N)
 };
 
 // Plain data, passed to kernels by value.
@@ -66,6 +67,42 @@ DASTAC_HD int64_t tet_root(int64_t q) {
     return a;
 }
 
+// Exact band |i - j| <= w of an N x N matrix, 2w + 1 <= N, rows packed one after the other.  The
+// counting polynomial has three pieces (rows clipped on the left, full rows, rows clipped on the
+// right; Section 4, "Piecewise Polynomial Simplification" treats such piecewise results); written
+// with clamps it is one expression: every row holds 2w + 1 points minus the w - i it loses on the
+// left (rows i < w) and the i + w - (N - 1) it loses on the right (rows i > N - 1 - w).
+DASTAC_HD int64_t band_row_start(int64_t N, int64_t w, int64_t i) {
+    const int64_t a = i < w ? i : w;                      // rows before i that are clipped on the left
+    const int64_t b = i > N - w ? i - (N - w) : 0;        // rows before i that are clipped on the right
+    return i * (2 * w + 1) - (a * w - ((a * (a - 1)) >> 1)) - ((b * (b + 1)) >> 1);
+}
+DASTAC_HD int64_t band_jlo(int64_t w, int64_t i) { return i > w ? i - w : 0; }
+DASTAC_HD int64_t band_jhi(int64_t N, int64_t w, int64_t i) { return i + w < N - 1 ? i + w : N - 1; }  // inclusive
+// Row of position p (0 <= p < count): the clipped pieces are quadratic in i, the middle one linear.
+DASTAC_HD int64_t band_row_of(int64_t N, int64_t w, int64_t p) {
+    const int64_t top = band_row_start(N, w, w), mid_end = band_row_start(N, w, N - w);
+    int64_t i;
+    if (p < top) {  // rows 0 .. w-1: start(i) = i (w + 1) + i (i - 1) / 2
+        const double f = 2.0 * (double)w + 1.0;
+        i = (int64_t)((sqrt(f * f + 8.0 * (double)p) - f) * 0.5);
+        if (i < 0) i = 0;
+        while (i > 0 && band_row_start(N, w, i) > p) --i;
+        while (i + 1 < w && band_row_start(N, w, i + 1) <= p) ++i;
+    } else if (p < mid_end) {
+        i = w + (p - top) / (2 * w + 1);
+    } else {  // rows N-w .. N-1: the mirror image of the first piece
+        const int64_t q = band_row_start(N, w, N) - 1 - p;
+        const double f = 2.0 * (double)w + 1.0;
+        int64_t r = (int64_t)((sqrt(f * f + 8.0 * (double)q) - f) * 0.5);
+        if (r < 0) r = 0;
+        while (r > 0 && band_row_start(N, w, r) > q) --r;
+        while (r + 1 < w && band_row_start(N, w, r + 1) <= q) ++r;
+        i = N - 1 - r;
+    }
+    return i;
+}
+
 // Upper triangle / trapezoid: points before row i, in units of (j) positions.
 DASTAC_HD int64_t upper_row_start(int64_t N, int64_t i) { return i * N - ((i * (i - 1)) >> 1); }
 
@@ -99,6 +136,10 @@ DASTAC_HD bool in_set(const IndexMap& m, const int32_t* idx) {
             return d <= m.w && -d <= m.w;
         }
         case kTetrahedron: return idx[0] <= idx[1] && idx[1] <= idx[2];
+        case kBandExact: {
+            int64_t d = (int64_t)idx[1] - idx[0];
+            return d <= m.w && -d <= m.w;
+        }
         default: return false;
     }
 }
@@ -124,6 +165,7 @@ DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
             return tet(n) - tet(n - idx[0]) + tri(n - idx[0]) - tri(n - idx[1]) +
                    ((int64_t)idx[2] - idx[1]);
         }
+        case kBandExact: return band_row_start(m.N, m.w, idx[0]) + (idx[1] - band_jlo(m.w, idx[0]));
         default: return -1;
     }
 }
@@ -178,6 +220,12 @@ DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
             idx[2] = (int32_t)(n - 1 - c);
             return;
         }
+        case kBandExact: {
+            const int64_t i = band_row_of(m.N, m.w, p);
+            idx[0] = (int32_t)i;
+            idx[1] = (int32_t)(band_jlo(m.w, i) + (p - band_row_start(m.N, m.w, i)));
+            return;
+        }
         default: return;
     }
 }
@@ -220,6 +268,12 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
             pbase = tet(n) - tet(n - idx[0]) + tri(n - idx[0]) - tri(n - idx[1]) - idx[1];
             return true;
         }
+        case kBandExact: {
+            jlo = band_jlo(m.w, idx[0]);
+            jhi = band_jhi(m.N, m.w, idx[0]) + 1;
+            pbase = band_row_start(m.N, m.w, idx[0]) - jlo;
+            return true;
+        }
         default: return false;
     }
 }
@@ -260,6 +314,15 @@ DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {
                 idx[1] = idx[0];
             }
             idx[2] = idx[1];
+            return;
+        }
+        case kBandExact: {
+            if (idx[1] < band_jhi(m.N, m.w, idx[0])) {
+                ++idx[1];
+                return;
+            }
+            ++idx[0];
+            idx[1] = (int32_t)band_jlo(m.w, idx[0]);
             return;
         }
         default: return;

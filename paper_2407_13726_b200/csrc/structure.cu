@@ -224,6 +224,14 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
             m.count = (2 * m.w + 1) * m.N - m.w * (m.w + 1);
             m.slots = (2 * m.w + 1) * m.N;
             matched = true;
+        } else if (!padded && full0 && full1 && m.dims[0] == m.dims[1] && b.D[0][1] == b.D[1][0] && b.D[0][1] >= 0 &&
+                   2 * b.D[0][1] + 1 <= m.dims[0]) {
+            // the same band packed row after row with nothing in between (three-piece polynomial)
+            m.kind = kBandExact;
+            m.N = m.dims[0];
+            m.w = b.D[0][1];
+            m.count = (2 * m.w + 1) * m.N - m.w * (m.w + 1);
+            matched = true;
         }
     } else {  // rank 3
         const bool full = hi[0] == m.dims[0] - 1 && hi[1] == m.dims[1] - 1 && hi[2] == m.dims[2] - 1;

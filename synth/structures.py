@@ -82,6 +82,13 @@ def band(N: int, w: int, padded_diagonals: bool = True) -> Descriptor:
                       padded_diagonals=padded_diagonals, name="band", meta={"w": w})
 
 
+def band_exact(N: int, w: int) -> Descriptor:
+    """The same set {(i, j) : |i - j| <= w}, packed row after row without padding."""
+    d = band(N, w, padded_diagonals=False)
+    d.name = "band_exact"
+    return d
+
+
 def tetrahedron(n: int) -> Descriptor:
     """{(i, j, k) : 0 <= i <= j <= k < n}."""
     items = _box_rows(3, 1, [0, 0, 0]) + [[-1, 1, 0, 0, 0], [0, -1, 1, 0, 0]]

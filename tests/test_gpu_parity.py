@@ -20,7 +20,8 @@ dastac = pytest.importorskip("paper_2407_13726_b200") if torch.cuda.is_available
 INDEX_CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(97), st.upper_triangle(128, True),
                st.lower_triangle(61), st.tetrahedron(1), st.tetrahedron(2), st.tetrahedron(48),
                st.upper_half_cube(9, 14, 5), st.upper_half_cube(14, 9, 3), st.dense_box([5, 6, 7]),
-               st.band(50, 4), st.band(7, 0), st.upper_triangle(1000)]
+               st.band(50, 4), st.band(7, 0), st.upper_triangle(1000), st.band_exact(50, 4), st.band_exact(9, 4),
+               st.band_exact(300, 32)]
 
 
 @pytest.mark.parametrize("desc", INDEX_CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -107,7 +108,8 @@ def _bits(shape, seed, sixteen=False):
 PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33), st.upper_triangle(129),
               st.upper_triangle(1000), st.upper_triangle(130, True), st.lower_triangle(77),
               st.tetrahedron(2), st.tetrahedron(37), st.upper_half_cube(11, 17, 3),
-              st.upper_half_cube(17, 11, 6), st.dense_box([6, 10])]
+              st.upper_half_cube(17, 11, 6), st.dense_box([6, 10]), st.band_exact(11, 5), st.band_exact(130, 7),
+              st.band_exact(1000, 32)]
 
 
 @pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
@@ -429,3 +431,23 @@ def test_pack_unpack_larger_f32(desc):
     out = torch.full(desc.dims, float("nan"), device="cuda")
     dastac.unpack(s, packed, out)
     assert np.array_equal(out.view(torch.int32).cpu().numpy().view(np.uint32), oracle.unpack(desc, exp))
+
+
+@pytest.mark.parametrize("N,w,C", [(2, 0, 1), (7, 0, 3), (9, 4, 5), (300, 32, 256), (1000, 7, 130), (2048, 32, 64)])
+def test_band_matmat_exact_layout(N, w, C):
+    """The band packed row after row without padding (three-piece ranking polynomial)."""
+    desc = st.band_exact(N, w)
+    s = dastac.Structure(desc)
+    A = synth.dense(1, 0, (N, N))
+    B = synth.dense(1, 1, (N, C))
+    ref, ref_abs = oracle.matmat(desc, A, B)
+    packed = packed_dev(s, oracle.pack(desc, A))
+    out = torch.full((N, C), float("nan"), device="cuda")
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out)
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    C0 = synth.dense(1, 2, (N, C))
+    out2 = dev(C0)
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out2, accumulate=True)
+    assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_F32
+    # the library's own pack produces the same stream
+    assert np.array_equal(dastac.pack(s, dev(A)).cpu().numpy()[: s.nnz], oracle.pack(desc, A))

@@ -30,7 +30,9 @@ def test_library_exports_every_declared_symbol():
 CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(37), st.upper_triangle(12, True),
          st.lower_triangle(1), st.lower_triangle(23), st.tetrahedron(1), st.tetrahedron(2),
          st.tetrahedron(15), st.upper_half_cube(4, 6, 3), st.upper_half_cube(6, 4, 2),
-         st.upper_half_cube(5, 5, 1), st.dense_box([3, 4]), st.dense_box([2, 3, 4]), st.dense_box([7])]
+         st.upper_half_cube(5, 5, 1), st.dense_box([3, 4]), st.dense_box([2, 3, 4]), st.dense_box([7]),
+         st.band_exact(1, 0), st.band_exact(7, 0), st.band_exact(7, 3), st.band_exact(8, 3), st.band_exact(23, 4),
+         st.band_exact(40, 11)]
 
 
 @pytest.mark.parametrize("desc", CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -85,10 +87,10 @@ def test_recognition_is_independent_of_how_rows_are_written():
     with pytest.raises(dastac.DastacError) as e:
         dastac.Structure(strict)
     assert e.value.status == 2
-    # an equality row (diagonal) is a valid descriptor but not a supported class
-    with pytest.raises(dastac.DastacError) as e:
-        dastac.Structure(st.diagonal(5))
-    assert e.value.status == 2
+    # an equality row (diagonal) closes to the band of half width 0, packed exactly: N points, rank(i, i) = i
+    diag = dastac.Structure(st.diagonal(5))
+    assert (diag.kind, diag.nnz) == (dastac.KIND_BAND_EXACT, 5) and dastac.rank(diag, (3, 3)) == 3
+    assert oracle.count(st.diagonal(5)) == 5
     # a row coupling three indices is not a difference bound
     three = st.Descriptor([4, 4, 4], [4], np.array([[1, 1, -1, 0, 0]], dtype=np.int64), np.zeros(1, np.uint8))
     with pytest.raises(dastac.DastacError):
@@ -100,9 +102,10 @@ def test_recognition_is_independent_of_how_rows_are_written():
     assert oracle.count(empty) == 0
     # zero extent
     assert dastac.Structure(st.upper_triangle(0)).nnz == 0
-    # band without the padded layout, or as wide as the matrix, is refused
+    # band without the padded layout: the exact row-after-row pack; as wide as the matrix: refused
+    assert dastac.Structure(st.band(8, 2, padded_diagonals=False)).kind == dastac.KIND_BAND_EXACT
     with pytest.raises(dastac.DastacError):
-        dastac.Structure(st.band(8, 2, padded_diagonals=False))
+        dastac.Structure(st.band(8, 4, padded_diagonals=False))
     with pytest.raises(dastac.DastacError):
         dastac.Structure(st.band(8, 7))
     # symmetric swap only on a square upper triangle
@@ -201,3 +204,15 @@ def test_argument_errors_do_not_launch():
     ins[0].structure = t._h
     assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 3
     assert dastac.launch_count() == before
+
+
+def test_exact_band_limits_and_kind():
+    s = dastac.Structure(st.band_exact(9, 2))
+    assert s.kind == dastac.KIND_BAND_EXACT and s.nnz == s.slots == 5 * 9 - 2 * 3
+    with pytest.raises(dastac.DastacError) as e:       # 2w + 1 > N: the clipped pieces would overlap
+        dastac.Structure(st.band_exact(6, 3))
+    assert e.value.status == 2
+    big = dastac.Structure(st.band_exact(2 ** 20, 1000))
+    assert dastac.unrank(big, big.nnz - 1) == (2 ** 20 - 1, 2 ** 20 - 1)
+    for p in (0, 1, 500_500, 123_456_789, big.nnz - 2):
+        assert dastac.rank(big, dastac.unrank(big, p)) == p
