@@ -67,6 +67,8 @@ def accounting(z):
         "trmv": dict(flops=2 * tri(N1), bytes=4 * (tri(N1) + 2 * N1), bound="hbm"),
         "trmv_batched": dict(flops=2 * tri(N1) * b, bytes=4 * (tri(N1) + 2 * N1) * b, bound="hbm"),
         "bandmm": dict(flops=2 * nnz2 * C2, bytes=4 * ((2 * w + 1) * N2 + 2 * N2 * C2), bound="alu"),
+        # widened row: the same band product over the exact (un-padded) layout
+        "bandmm_exact": dict(flops=2 * nnz2 * C2, bytes=4 * (nnz2 + 2 * N2 * C2), bound="alu"),
         "symv": dict(flops=2 * N3 * N3, bytes=4 * (tri(N3) + 2 * N3), bound="hbm"),
         "mttkrp": dict(flops=3 * tet(n4) * R, bytes=4 * (tet(n4) + 3 * n4 * R), bound="alu"),
         "trimm_bf16": dict(flops=2 * tri(N5) * N5, bytes=2 * tri(N5) + 2 * N5 * N5 + 4 * N5 * N5, bound="tensor"),
@@ -78,7 +80,7 @@ def accounting(z):
     return acc
 
 
-ORDER = ["trmv", "trmv_batched", "bandmm", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
+ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
 
 
 def generate_host(z, pin, only=None):
@@ -115,6 +117,13 @@ def generate_host(z, pin, only=None):
         N2, w, C2 = z["N2"], z["w"], z["C2"]
         h["bandmm"] = dict(desc=st.band(N2, w), A=host(synth.band_diagonals_stream(1, 0, N2, w).reshape(-1)),
                            ins=[host(synth.dense(1, 1, (N2, C2)))], out=(N2, C2))
+    if want("bandmm_exact"):
+        N2, w, C2 = z["N2"], z["w"], z["C2"]
+        nnz2 = (2 * w + 1) * N2 - w * (w + 1)
+        ax = np.zeros(cap(nnz2, 4), np.float32)
+        synth.band_rows_stream(1, 0, N2, w, out=ax)
+        h["bandmm_exact"] = dict(desc=st.band_exact(N2, w), A=host(ax), ins=[host(synth.dense(1, 1, (N2, C2)))],
+                                 out=(N2, C2))
     if want("symv"):
         N3 = z["N3"]
         a3 = np.zeros(cap(tri(N3), 4), np.float32)
@@ -145,7 +154,8 @@ def generate_host(z, pin, only=None):
 
 
 EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
-        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk"}
+        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
+        "bandmm_exact": "ij,jc->ic"}
 
 
 # ---- clocks ---------------------------------------------------------------------------------------------
@@ -430,7 +440,7 @@ def run_gpu(args):
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
             "data": "synthetic",
-            "config": {"workload": "all five configs per step, plus the tensor-times-matrix running example (N6,Q6,K6): "
+            "config": {"workload": "all five configs per step, plus two widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6): "
                                    + json.dumps(z, separators=(",", ":")),
                        "small": bool(args.small), "only": args.only or None,
                        "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
@@ -587,7 +597,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(tot_s / steps * 1e3, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "all five configs per step, plus the tensor-times-matrix running example (N6,Q6,K6): "
+        "config": {"workload": "all five configs per step, plus two widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6): "
                                + json.dumps(z, separators=(",", ":")),
                    "sample": desc},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},

@@ -130,14 +130,19 @@ bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant_
                     : "memory");
         }
         if (!(TMA_B && tma_a)) {
-            // stage diagonals dc .. dc+kChunk-1 of rows i0 .. i0+63; zero outside the band / matrix
+            // stage diagonals dc .. dc+kChunk-1 of rows i0 .. i0+63; zero outside the band / matrix.
+            // kThreads is a multiple of kRows, so a thread keeps its row: the row's part of the position
+            // (the hoisted base of the ranking polynomial) is worked out once.
+            static_assert(kThreads % kRows == 0, "a thread must stay on one row of the slice");
+            const int r = tid % kRows;
+            const int64_t i = i0 + r;
+            // padded diagonals: slot (d, i) = d N + i; exact rows: rowbase(i) + j with j = i + d - w
+            const int64_t base = exact ? (i < N ? band_row_start(N, w, i) - band_jlo(w, i) + i - w : 0) : i;
+            const int64_t step = exact ? 1 : N;
 #pragma unroll 12
-            for (int t = tid; t < kChunk * kRows; t += kThreads) {
-                const int dl = t / kRows, r = t - dl * kRows;
-                const int64_t d = dc + dl, i = i0 + r, jj = i + d - w;
-                // padded diagonals: slot (d, i); exact rows: rowbase(i) + j with the row's hoisted base
-                const int64_t pos = exact ? band_row_start(N, w, i) - band_jlo(w, i) + jj : d * N + i;
-                Ad[t] = (d < diagonals && i < N && jj >= 0 && jj < N) ? __ldg(A + pos) : 0.f;
+            for (int dl = tid / kRows; dl < kChunk; dl += kThreads / kRows) {
+                const int64_t d = dc + dl, jj = i + d - w;
+                Ad[dl * kRows + r] = (d < diagonals && i < N && jj >= 0 && jj < N) ? __ldg(A + base + d * step) : 0.f;
             }
         }
         if (TMA_B) {

@@ -45,6 +45,8 @@ def _load():
         lib.synth_stream_upper_triangle.restype = u64
         lib.synth_stream_upper_half_cube.argtypes = [u64, u64, cint, dbl, u64, u64, u64, vp]
         lib.synth_stream_upper_half_cube.restype = u64
+        lib.synth_stream_band_rows.argtypes = [u64, u64, cint, dbl, u64, u64, vp]
+        lib.synth_stream_band_rows.restype = u64
         lib.synth_stream_tetrahedron.argtypes = [u64, u64, cint, dbl, cint, u64, vp]
         lib.synth_stream_tetrahedron.restype = u64
         lib.synth_stream_band_diagonals.argtypes = [u64, u64, cint, dbl, u64, u64, ctypes.c_uint32, vp]
@@ -99,6 +101,15 @@ def upper_half_cube_stream(seed, tensor_id, M, N, Q, dist=UNIFORM, scale=1.0, ou
     cnt = _load().synth_stream_upper_half_cube(seed, tensor_id, dist, scale, int(M), int(N), int(Q), None)
     arr, ptr = _out(cnt, False, out)
     got = _load().synth_stream_upper_half_cube(seed, tensor_id, dist, scale, int(M), int(N), int(Q), ptr)
+    assert got == cnt
+    return arr[:cnt]
+
+
+def band_rows_stream(seed, tensor_id, N, w, dist=UNIFORM, scale=1.0, out=None):
+    """Values of ``{(i, j): |i - j| <= w}`` row after row (j ascending), without padding."""
+    cnt = _load().synth_stream_band_rows(seed, tensor_id, dist, scale, int(N), int(w), None)
+    arr, ptr = _out(cnt, False, out)
+    got = _load().synth_stream_band_rows(seed, tensor_id, dist, scale, int(N), int(w), ptr)
     assert got == cnt
     return arr[:cnt]
 

@@ -124,6 +124,29 @@ uint64_t synth_stream_upper_half_cube(uint64_t seed, uint64_t tensor_id, int dis
     return total;
 }
 
+/* Band |i - j| <= w of an N x N matrix emitted row after row, j ascending, nothing in between. */
+uint64_t synth_stream_band_rows(uint64_t seed, uint64_t tensor_id, int dist, double scale, uint64_t N,
+                                uint64_t w, void* out) {
+    uint64_t key = tensor_key(seed, tensor_id);
+    uint64_t* start = (uint64_t*)malloc((N + 1) * sizeof(uint64_t));
+    if (!start) return 0;
+    start[0] = 0;
+    for (uint64_t i = 0; i < N; ++i) {
+        uint64_t lo = i > w ? i - w : 0, hi = i + w < N - 1 ? i + w : N - 1;
+        start[i + 1] = start[i] + (hi - lo + 1);
+    }
+    if (!out) { uint64_t c = start[N]; free(start); return c; }
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)N; ++i) {
+        uint64_t ui = (uint64_t)i, lo = ui > w ? ui - w : 0, hi = ui + w < N - 1 ? ui + w : N - 1;
+        for (uint64_t j = lo; j <= hi; ++j)
+            store_value(out, 0, (size_t)(start[i] + (j - lo)), value_at(key, dist, scale, ui * N + j));
+    }
+    uint64_t total = start[N];
+    free(start);
+    return total;
+}
+
 /* Tetrahedron 0 <= i <= j <= k < n of an n x n x n tensor, emitted in (i, j, k) order. */
 uint64_t synth_stream_tetrahedron(uint64_t seed, uint64_t tensor_id, int dist, double scale,
                                   int as_bf16, uint64_t n, void* out) {

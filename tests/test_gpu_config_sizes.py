@@ -175,3 +175,21 @@ def test_widened_row_ttm_n1024_q32_k32():
         n_el = (N - int(i)) * K
         seg = got[starts[s]: starts[s] + n_el]
         assert rel_err(seg, ref[s, int(i):, :].reshape(-1), ref_abs[s, int(i):, :].reshape(-1)) <= TOL_F32
+
+
+def test_widened_row_exact_band_n32768_w32_c256():
+    """Configuration 2's product over the exact (un-padded) band layout, on sampled rows."""
+    N, w, C = 32768, 32, 256
+    desc = st.band_exact(N, w)
+    s = dastac.Structure(desc)
+    assert s.nnz == 65 * N - 32 * 33 == s.slots
+    B = synth.dense(1, 1, (N, C))
+    packed = _packed(s, lambda h: synth.band_rows_stream(1, 0, N, w, out=h))
+    out = torch.full((N, C), float("nan"), device="cuda")
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out)
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    sel = np.union1d(_rows(N, 200, extra=range(0, 40)), np.arange(N - 40, N))
+    Ar = np.stack([synth.linear_slice(1, 0, int(i) * N, N) for i in sel])
+    ref, ref_abs = oracle.matmat(desc, Ar, B, sel=sel)
+    assert rel_err(got[sel], ref, ref_abs) <= TOL_F32

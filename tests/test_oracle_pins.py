@@ -224,6 +224,7 @@ def test_streams_match_oracle_pack():
     N, w = 23, 3
     A = synth.dense(7, 3, (N, N))
     assert np.array_equal(oracle.band_pack(N, w, A), synth.band_diagonals_stream(7, 3, N, w))
+    assert np.array_equal(oracle.pack(st.band_exact(N, w), A), synth.band_rows_stream(7, 3, N, w))
     for M, N, Q in ((6, 9, 5), (9, 6, 3)):
         H = synth.dense(10, 5, (M, N, Q))
         assert np.array_equal(oracle.pack(st.upper_half_cube(M, N, Q), H), synth.upper_half_cube_stream(10, 5, M, N, Q))
