@@ -34,6 +34,7 @@ constexpr int kPairs = 2;               // column pairs per lane: a lane owns 8 
 constexpr int kLaneCols = 2 * kPairs;
 constexpr int kCols = 16 * kLaneCols;   // 64 columns per CTA
 constexpr int kChunk = 72;              // diagonals per chunk (multiple of 8)
+constexpr int kPitchExact = 68;         // words per staged diagonal of the exact layout (68 = 4 mod 32, 16-byte rows)
 constexpr int kBRows = kRows + kChunk + 6;  // B rows a chunk touches: 64 + chunk - 1 + 7
 constexpr long long kWaitBudget = 4000000000LL;
 
@@ -75,15 +76,18 @@ __device__ __forceinline__ void load_row(pair_t (&dst)[kPairs], const float* __r
     }
 }
 
-template <bool TMA_B>
+// EXACT: A is packed row after row (no padding); its slice is staged with a row pitch of 68 words so
+// that the transposing stores below spread over all banks.
+template <bool TMA_B, bool EXACT>
 __global__ void __launch_bounds__(kThreads, 4)
 bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_a, int tma_a,
-              int exact, int64_t N, int64_t w, int64_t row_tile0,
+              int64_t N, int64_t w, int64_t row_tile0,
               const float* __restrict__ A, const float* __restrict__ B, int64_t ldb, float* __restrict__ C,
               int64_t ldc, int64_t ncols, int accumulate, int vec_c, int32_t* err_word) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     float* Bs = reinterpret_cast<float*>(smem_raw);                                   // [kBRows][kCols]
-    float* Ad = reinterpret_cast<float*>(smem_raw + (TMA_B ? kBRows * kCols * 4 : 0));  // [kChunk][kRows]
+    float* Ad = reinterpret_cast<float*>(smem_raw + (TMA_B ? kBRows * kCols * 4 : 0));  // [kChunk][kPitch]
+    constexpr int kPitch = EXACT ? kPitchExact : kRows;
     __shared__ __align__(8) uint64_t bar;
     __shared__ int failed;
 
@@ -129,20 +133,51 @@ bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant_
                     ::"r"(smem_u32(Ad)), "l"(&tmap_a), "r"((int)i0), "r"((int)dc), "r"(smem_u32(&bar))
                     : "memory");
         }
-        if (!(TMA_B && tma_a)) {
-            // stage diagonals dc .. dc+kChunk-1 of rows i0 .. i0+63; zero outside the band / matrix.
-            // kThreads is a multiple of kRows, so a thread keeps its row: the row's part of the position
-            // (the hoisted base of the ranking polynomial) is worked out once.
+        const int d_end = (int)((diagonals - dc < kChunk) ? diagonals - dc : kChunk);
+        if (EXACT) {
+            // A row's band entries are consecutive in memory (rowbase(i) + j, j = i + d - w).  A warp
+            // owns 16 rows and copies 4 rows x 8 consecutive diagonals per instruction (32-byte runs)
+            // with asynchronous 4-byte copies: all of a thread's copies are in flight at once and none
+            // holds a register.  Diagonals past d_end are not staged: the loop below never reads them.
+            const bool interior = i0 >= w && i0 + kRows - 1 + w < N;  // every row of the tile has all 2w+1 entries
+            const int dq = lane & 7;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int r = 16 * warp + 4 * b + (lane >> 3);
+                const int64_t i = i0 + r;
+                const float* src = A + (i < N ? band_row_start(N, w, i) - band_jlo(w, i) + i - w : 0) + dc + dq;
+                const uint32_t dst = smem_u32(&Ad[dq * kPitch + r]);
+                if (interior) {
+#pragma unroll
+                    for (int k = 0; k < kChunk / 8; ++k)
+                        if (8 * k + dq < d_end)
+                            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + k * 8 * kPitch * 4),
+                                         "l"(src + 8 * k)
+                                         : "memory");
+                } else {
+                    // first / last row tiles: entries whose column falls outside [0, N) are zero-filled
+                    // (source size 0 reads nothing)
+#pragma unroll
+                    for (int k = 0; k < kChunk / 8; ++k) {
+                        const int64_t jj = i + dc + dq + 8 * k - w;
+                        const bool in = 8 * k + dq < d_end && i < N && jj >= 0 && jj < N;
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst + k * 8 * kPitch * 4),
+                                     "l"(in ? src + 8 * k : A), "r"(in ? 4 : 0)
+                                     : "memory");
+                    }
+                }
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+        } else if (!(TMA_B && tma_a)) {
+            // stage diagonals dc .. dc+kChunk-1 of rows i0 .. i0+63 (slot (d, i) = d N + i); zero
+            // outside the band / matrix.  kThreads is a multiple of kRows, so a thread keeps its row.
             static_assert(kThreads % kRows == 0, "a thread must stay on one row of the slice");
             const int r = tid % kRows;
             const int64_t i = i0 + r;
-            // padded diagonals: slot (d, i) = d N + i; exact rows: rowbase(i) + j with j = i + d - w
-            const int64_t base = exact ? (i < N ? band_row_start(N, w, i) - band_jlo(w, i) + i - w : 0) : i;
-            const int64_t step = exact ? 1 : N;
 #pragma unroll 12
             for (int dl = tid / kRows; dl < kChunk; dl += kThreads / kRows) {
                 const int64_t d = dc + dl, jj = i + d - w;
-                Ad[dl * kRows + r] = (d < diagonals && i < N && jj >= 0 && jj < N) ? __ldg(A + base + d * step) : 0.f;
+                Ad[dl * kRows + r] = (d < diagonals && i < N && jj >= 0 && jj < N) ? __ldg(A + d * N + i) : 0.f;
             }
         }
         if (TMA_B) {
@@ -169,7 +204,7 @@ bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant_
         }
         __syncthreads();
         if (TMA_B && failed) return;
-        if (TMA_B && tma_a && (i0 < w || i0 + kRows - 1 + w >= N)) {
+        if (TMA_B && !EXACT && tma_a && (i0 < w || i0 + kRows - 1 + w >= N)) {
             // edge tile: the copied box contains padding slots (column i + d - w outside [0, N)); zero them
             for (int t = tid; t < kChunk * kRows; t += kThreads) {
                 const int dl = t / kRows, r = t - dl * kRows;
@@ -186,12 +221,11 @@ bandmm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant_
 #pragma unroll
         for (int q = 0; q < 7; ++q)
             load_row<TMA_B>(win[q], Bs, br0 + q, B, ldb, i_f + dc - w + q, N, c0, cl, ncols);
-        const int d_end = (int)((diagonals - dc < kChunk) ? diagonals - dc : kChunk);
         // one diagonal: slide the window down by one row of B, then 8 rows x 4 columns of multiply-adds
         auto step = [&](const int db, const int u) {
             load_row<TMA_B>(win[(u + 7) & 7], Bs, br0 + db + u + 7, B, ldb, i_f + dc + db + u - w + 7, N, c0, cl, ncols);
-            const float4 a_lo = *reinterpret_cast<const float4*>(&Ad[(db + u) * kRows + il]);
-            const float4 a_hi = *reinterpret_cast<const float4*>(&Ad[(db + u) * kRows + il + 4]);
+            const float4 a_lo = *reinterpret_cast<const float4*>(&Ad[(db + u) * kPitch + il]);
+            const float4 a_hi = *reinterpret_cast<const float4*>(&Ad[(db + u) * kPitch + il + 4]);
             const pair_t a2[8] = {pack2(a_lo.x, a_lo.x), pack2(a_lo.y, a_lo.y), pack2(a_lo.z, a_lo.z),
                                   pack2(a_lo.w, a_lo.w), pack2(a_hi.x, a_hi.x), pack2(a_hi.y, a_hi.y),
                                   pack2(a_hi.z, a_hi.z), pack2(a_hi.w, a_hi.w)};
@@ -296,24 +330,29 @@ dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, i
             return DASTAC_ERR_CUDA;
         tma_a = 1;
     }
+    if (exact) smem += (size_t)kChunk * (kPitchExact - kRows) * sizeof(float);
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
         const int big = (int)((size_t)kChunk * kRows * 4 + (size_t)kBRows * kCols * 4);
-        if (cudaFuncSetAttribute(bandmm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess)
+        const int big_exact = (int)((size_t)kChunk * kPitchExact * 4 + (size_t)kBRows * kCols * 4);
+        if (cudaFuncSetAttribute(bandmm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
+            cudaFuncSetAttribute(bandmm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_exact) != cudaSuccess)
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
     }
     for (int64_t y0 = 0; y0 < gy; y0 += 65535) {  // gridDim.y is limited to 65535
         const int64_t ny = gy - y0 < 65535 ? gy - y0 : 65535;
         const dim3 grid((unsigned)gx, (unsigned)ny);
-        if (tma_b)
-            bandmm_kernel<true><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, exact, N, m.w, y0, A, B, ldb, C, ldc, ncols, accumulate,
-                                                              vec_c, err_word);
-        else
-            bandmm_kernel<false><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, exact, N, m.w, y0, A, B, ldb, C, ldc, ncols,
-                                                               accumulate, vec_c, err_word);
+#define DASTAC_BANDMM_LAUNCH(TB, EX)                                                                              \
+    bandmm_kernel<TB, EX><<<grid, kThreads, smem, st>>>(tmap, tmap_a, tma_a, N, m.w, y0, A, B, ldb, C, ldc, ncols, \
+                                                        accumulate, vec_c, err_word)
+        if (tma_b && exact) DASTAC_BANDMM_LAUNCH(true, true);
+        else if (tma_b) DASTAC_BANDMM_LAUNCH(true, false);
+        else if (exact) DASTAC_BANDMM_LAUNCH(false, true);
+        else DASTAC_BANDMM_LAUNCH(false, false);
+#undef DASTAC_BANDMM_LAUNCH
         dastac_status s = launch_status();
         if (s != DASTAC_OK) return s;
     }

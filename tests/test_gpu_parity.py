@@ -433,7 +433,8 @@ def test_pack_unpack_larger_f32(desc):
     assert np.array_equal(out.view(torch.int32).cpu().numpy().view(np.uint32), oracle.unpack(desc, exp))
 
 
-@pytest.mark.parametrize("N,w,C", [(2, 0, 1), (7, 0, 3), (9, 4, 5), (300, 32, 256), (1000, 7, 130), (2048, 32, 64)])
+@pytest.mark.parametrize("N,w,C", [(2, 0, 1), (7, 0, 3), (9, 4, 5), (300, 32, 256), (1000, 7, 130), (2048, 32, 64),
+                                   (200, 40, 33), (513, 90, 64), (190, 94, 12)])
 def test_band_matmat_exact_layout(N, w, C):
     """The band packed row after row without padding (three-piece ranking polynomial)."""
     desc = st.band_exact(N, w)
