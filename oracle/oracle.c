@@ -323,6 +323,33 @@ void orc_ttm(const orc_desc* d, int64_t nsel, const int64_t* sel, const float* B
     }
 }
 
+/* A2[i1][i2] = sum_x [ (i1, i2) in set ] B[x][i1] * B[x][i2]
+ * (A^k(i_1..i_k) := B(x,i_1) * ... * B(x,i_k) with k = 2, Table 1 "Polynomial Regression"; the set is
+ * the unique part i1 <= i2 of the symmetric result, Section 2 "Redundancy map", and the output is
+ * stored compressed over it, Section 4 "Iteration space extraction").  B is M x n row-major, fp32 or
+ * bf16 bit patterns; out[s] is row sel[s] of the result as a dense row of n values, entries outside
+ * the set are 0. */
+void orc_moment2(const orc_desc* d, int is_bf16, int64_t nsel, const int64_t* sel, const void* B,
+                 int64_t M, double* out, double* out_abs) {
+    const int64_t n = d->dims[1];
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        for (int64_t i2 = 0; i2 < n; ++i2) {
+            double acc = 0.0, acc_abs = 0.0;
+            int64_t idx[2] = {sel[s], i2};
+            if (in_domain(d, idx)) {
+                for (int64_t x = 0; x < M; ++x) {
+                    double p = widen(B, x * n + sel[s], is_bf16) * widen(B, x * n + i2, is_bf16);
+                    acc += p;
+                    acc_abs += fabs(p);
+                }
+            }
+            out[s * n + i2] = acc;
+            out_abs[s * n + i2] = acc_abs;
+        }
+    }
+}
+
 /* Thread count the contractions above will use. */
 #ifdef _OPENMP
 #include <omp.h>

@@ -399,3 +399,44 @@ def test_ttm_upper_half_cube():
     dA = st.upper_half_cube(M, N, K)
     packedA = oracle.pack(dA, out)
     assert packedA.shape == (oracle.count(dA),) and oracle.count(dA) == oracle.count(d) // Q * K
+
+
+def test_moment2_packed_symmetric_output():
+    """Degree-2 moments of polynomial regression: A2(i1,i2) = sum_x B(x,i1) B(x,i2), kept on i1 <= i2."""
+    M, n = 37, 9
+    d = st.upper_triangle(n, symmetric=True)
+    B = synth.dense(6, 0, (M, n))
+    out, outa = oracle.moment2(d, B)
+    B64 = B.astype(np.float64)
+    gram = B64.T @ B64                                   # library routine, all n x n entries
+    np.testing.assert_allclose(out, np.triu(gram), atol=1e-12)
+    np.testing.assert_allclose(outa, np.triu(np.abs(B64).T @ np.abs(B64)), rtol=1e-13)
+    assert (out[np.tril_indices(n, -1)] == 0).all()      # outside the unique set nothing is computed
+    # closed forms: a single sample gives the outer product; all ones gives M on the set;
+    # the diagonal holds the squared column norms; orthonormal columns give the identity
+    one, _ = oracle.moment2(d, B[:1])
+    assert np.array_equal(one, np.triu(np.outer(B64[0], B64[0])))
+    ones, _ = oracle.moment2(d, np.ones((M, n), np.float32))
+    assert np.array_equal(ones, np.triu(np.full((n, n), float(M))))
+    np.testing.assert_allclose(np.diag(out), (B64 ** 2).sum(0), rtol=1e-13)
+    q, _ = np.linalg.qr(np.random.default_rng(0).standard_normal((M, n)))
+    eye, _ = oracle.moment2(d, q.astype(np.float32))
+    np.testing.assert_allclose(eye, np.eye(n), atol=1e-6)
+    # the sum runs over the first index of B (samples): a square B and its transpose differ
+    Bs = synth.dense(6, 1, (n, n))
+    a1, _ = oracle.moment2(d, Bs)
+    a2, _ = oracle.moment2(d, np.ascontiguousarray(Bs.T))
+    assert np.abs(a1 - a2).max() > 1e-3
+    # selected rows, and bf16 bit patterns widened exactly
+    sel = np.array([7, 0, 3])
+    sub, _ = oracle.moment2(d, B, sel=sel)
+    assert np.array_equal(sub, out[sel])
+    bits = synth.dense(6, 2, (M, n), bf16=True)
+    wide = (bits.astype(np.uint32) << 16).view(np.float32)
+    o16, _ = oracle.moment2(d, bits)
+    o32, _ = oracle.moment2(d, wide)
+    assert np.array_equal(o16, o32)
+    # the stored result is the packed upper triangle: position of (i1, i2) = number of kept entries before it
+    packed = oracle.pack(d, out)
+    assert packed.shape == (n * (n + 1) // 2,)
+    assert packed[oracle.rank_point(d, (2, 5))] == out[2, 5] and packed[n] == out[1, 1]
