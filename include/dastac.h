@@ -163,7 +163,8 @@ typedef struct {
 } dastac_operand;
 
 /*
- * Evaluate a sum-of-products rule (Section 3, "Input"; Table 1) whose first operand is packed.
+ * Evaluate a sum-of-products rule (Section 3, "Input"; Table 1) whose first operand is packed
+ * (one rule, the last of the table, packs its output instead).
  * Supported (expression, structure of in[0], dtypes):
  *   "ij,j->i"       upper triangle (square)             f32        y = A x         (batched)
  *   "ij,j->i"       upper triangle + swap (symmetric)   f32        y = S x
@@ -173,6 +174,13 @@ typedef struct {
  *   "ijl,kl->ijk"   upper half cube (i <= j, dense l)   f32        A = B x_3 C (tensor times matrix, the
  *                   running example of Section 3); `out` is PACKED too: out->structure must be the
  *                   upper half cube with the same first two extents and trailing extent K = rows of C
+ *   "xi,xj->ij"     in[0] = in[1] = dense B (M x n)     bf16 -> f32  A2 = B^T B, the degree-2 moments of
+ *                   polynomial regression (Table 1, A^k(i_1..i_k) := B(x,i_1) ... B(x,i_k), k = 2).  This
+ *                   rule has no packed input: both inputs must be the same dense tensor (same data,
+ *                   extents and strides, unit stride along i) and `out` is PACKED: out->structure is the
+ *                   n x n upper triangle (the unique part i <= j of the symmetric result, Section 2;
+ *                   with or without the redundancy swap), fp32 accumulation.  Positions of the packed
+ *                   buffer beyond the set's count are not written.
  * accumulate: 0 -> out = result (the library zero-fills where it needs to), 1 -> out += result.
  * workspace: device scratch of at least dastac_contract_workspace bytes, 256-byte aligned; may be
  *            NULL when that size is 0.  Its contents are undefined afterwards.

@@ -262,7 +262,9 @@ def contract(expr: str, s: Structure, packed: torch.Tensor, dense_inputs: Sequen
              out_structure: Optional[Structure] = None) -> torch.Tensor:
     """Evaluate ``expr`` with ``packed`` (structure ``s``) as first operand.  Tensors may live on
     the device or in (pinned) host memory; host tensors are staged through ``workspace``.
-    ``out_structure`` marks ``out`` as a packed buffer of that structure (rules with packed output)."""
+    ``out_structure`` marks ``out`` as a packed buffer of that structure (rules with packed output).
+    For the rule without a packed input (``"xi,xj->ij"``) pass ``s=None`` and the dense tensor itself
+    as ``packed`` and again as the only entry of ``dense_inputs``."""
     ins, o = _operands(s, packed, dense_inputs, out, batch, out_structure)
     ws_ptr, ws_bytes = None, 0
     if workspace is not None:

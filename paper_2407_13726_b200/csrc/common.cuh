@@ -51,5 +51,8 @@ size_t trimm_workspace_bytes(const IndexMap& m, int64_t ncols, int64_t ldb);
 dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B, int64_t ldb,
                                 float* C, int64_t ldc, int64_t ncols, int accumulate,
                                 void* workspace, int32_t* err_word, cudaStream_t st);
+size_t moment2_workspace_bytes(int64_t M, int64_t n, int64_t ldb);
+dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
+                                  int accumulate, void* workspace, int32_t* err_word, cudaStream_t st);
 
 }  // namespace dastac

@@ -141,6 +141,7 @@ struct Params {
     const uint8_t* tiles;        // staged tile images, 16 KiB each
     float* C;
     int64_t N, ncols, ldc;
+    int64_t M;           // second-moment form only: number of samples (rows of B)
     int64_t cap_elems;   // capacity of the packed buffer in elements (multiple of 8)
     int32_t row_blocks, col_blocks, k_blocks;
     int32_t accumulate;
@@ -245,6 +246,15 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
         : "memory");
 }
 
+//
+// MOMENT2 (the degree-2 moments A2(i1,i2) = sum_x B(x,i1) B(x,i2) of polynomial regression, Table 1,
+// kept on i1 <= i2 and stored packed): the same pipeline with both operands read from B.  The "A"
+// operand is B transposed, which the tensor core takes directly as an M-major operand: CTA r copies
+// the 64 x 128 block of B at columns 128 (2P + r) with the same two swizzled boxes it uses for its
+// half of the "B" operand, and the instruction descriptor marks A as M-major.  Tiles are the
+// 256 x 256 blocks (P, J) with J >= P, every one with the full K loop over the samples; the
+// epilogue writes element (i1, i2) at rowbase(i1) + i2 of the packed triangle and skips i2 < i1.
+template <bool MOMENT2>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
 trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const Params p) {
@@ -292,7 +302,24 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // Tile t = (pair P, column block J), P ascending = K length descending, dealt to the clusters in
     // boustrophedon order.
     const int pair_blocks = (p.row_blocks + 1) >> 1;
-    const int64_t tiles = (int64_t)pair_blocks * p.col_blocks;
+    const int64_t tiles = MOMENT2 ? (int64_t)pair_blocks * (pair_blocks + 1) / 2 : (int64_t)pair_blocks * p.col_blocks;
+    // tile index -> (row-block pair P, column block J); MOMENT2: row P of the block triangle holds J = P ..
+    auto decode = [&](int64_t t, int& P, int& J) {
+        if (MOMENT2) {
+            int r = 0;
+            while (t >= pair_blocks - r) {
+                t -= pair_blocks - r;
+                ++r;
+            }
+            P = r;
+            J = r + (int)t;
+        } else {
+            P = (int)(t / p.col_blocks);
+            J = (int)(t - (int64_t)P * p.col_blocks);
+        }
+    };
+    auto kb_first = [&](int P) { return MOMENT2 ? 0 : 4 * P; };
+    constexpr uint32_t kIdesc = MOMENT2 ? (kPIdesc | (1u << 15)) : kPIdesc;  // A operand M-major
     const int64_t G = gridDim.x >> 1, cid = blockIdx.x >> 1;
     auto tile_of = [&](uint32_t n) -> int64_t { return (int64_t)n * G + ((n & 1) ? (G - 1 - cid) : cid); };
     const uint32_t rounds = (uint32_t)((tiles + G - 1) / G);
@@ -306,12 +333,13 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (uint32_t n = 0; n < rounds && ok; ++n) {
                 const int64_t t = tile_of(n);
                 if (t >= tiles) continue;
-                const int P = (int)(t / p.col_blocks), J = (int)(t - (int64_t)P * p.col_blocks);
+                int P, J;
+                decode(t, P, J);
                 const int I = 2 * P + (int)rank;
                 // staged tile (I, kb) sits at tile index tile_base + kb; a row block past the end of
                 // the matrix has no tiles and its loads are out of range of the map: zero fill
                 const int64_t tile_base = (I < p.row_blocks) ? tile_offset(I, p.k_blocks) - 4 * P : (int64_t)1 << 22;
-                for (int kb = 4 * P; kb < p.k_blocks; ++kb, ++it) {
+                for (int kb = kb_first(P); kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kPStages;
                     if (it >= kPStages &&
                         !mbar_wait(empty(s), ((it / kPStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty)) {
@@ -321,7 +349,13 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t dst = smem_base + s * kPStageBytes;
                     if (leader) mbar_arrive_expect_tx(full(s), 2 * kPStageBytes);  // both CTAs' bytes
                     const uint32_t bar = full0 + 8u * s;
-                    tma_load_2d_pair(dst, &tmap_a, 0, (int)((tile_base + kb) * kTileM), bar);
+                    if (MOMENT2) {
+#pragma unroll
+                        for (int q = 0; q < kTileM / 64; ++q)
+                            tma_load_2d_pair(dst + q * (kBlockK * 128), &tmap_b, I * kTileM + q * 64, kb * kBlockK, bar);
+                    } else {
+                        tma_load_2d_pair(dst, &tmap_a, 0, (int)((tile_base + kb) * kTileM), bar);
+                    }
 #pragma unroll
                     for (int q = 0; q < kTileN / 128; ++q)
                         tma_load_2d_pair(dst + kABytes + q * (kBlockK * 128), &tmap_b,
@@ -343,7 +377,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (uint32_t n = 0; n < rounds && ok; ++n) {
                 const int64_t t = tile_of(n);
                 if (t >= tiles) continue;
-                const int P = (int)(t / p.col_blocks);
+                int P, J;
+                decode(t, P, J);
                 const int acc = tile_n & 1;
                 if (tile_n >= 2 &&
                     !mbar_wait_cluster(tmem_empty(acc), ((tile_n >> 1) - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
@@ -352,7 +387,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileN;
-                for (int kb = 4 * P; kb < p.k_blocks; ++kb, ++it) {
+                for (int kb = kb_first(P); kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kPStages;
                     if (!mbar_wait_cluster(full(s), (it / kPStages) & 1, abort_flag, p.err_word, kErrFull)) {
                         ok = false;
@@ -363,9 +398,10 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
                     for (int k16 = 0; k16 < kBlockK / 16; ++k16) {
-                        const uint64_t da = smem_desc(a_addr + k16 * 32, 16, 1024);
+                        const uint64_t da = MOMENT2 ? smem_desc(a_addr + k16 * 2048, kBlockK * 128, 1024)
+                                                    : smem_desc(a_addr + k16 * 32, 16, 1024);
                         const uint64_t db = smem_desc(b_addr + k16 * 2048, kBlockK * 128, 1024);
-                        umma_bf16_pair(d_tmem, da, db, kPIdesc, (kb > 4 * P || k16 > 0) ? 1u : 0u);
+                        umma_bf16_pair(d_tmem, da, db, kIdesc, (kb > kb_first(P) || k16 > 0) ? 1u : 0u);
                     }
                     umma_commit_pair(empty(s));
                 }
@@ -387,7 +423,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (uint32_t n = 0; n < rounds && ok; ++n) {
             const int64_t t = tile_of(n);
             if (t >= tiles) continue;
-            const int P = (int)(t / p.col_blocks), J = (int)(t - (int64_t)P * p.col_blocks);
+            int P, J;
+            decode(t, P, J);
             const int I = 2 * P + (int)rank;
             const int acc = tile_n & 1;
             if (!mbar_wait_warp(tmem_full(acc), (tile_n >> 1) & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
@@ -397,8 +434,33 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             tc_fence_after();
             const int64_t i = (int64_t)I * kTileM + warp * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + acc * kTileN;
-            float* crow = p.C + i * p.ldc + (int64_t)J * kTileN;
-            if (I < p.row_blocks) {
+            float* crow = MOMENT2 ? p.C : p.C + i * p.ldc + (int64_t)J * kTileN;
+            if (MOMENT2) {
+                // packed triangle: (i, j) sits at rowbase(i) + j; keep i <= j < n.  A lane's 32 values
+                // are consecutive in memory but only 4-byte aligned: scalar stores.
+                if (I < p.row_blocks) {
+                    float* prow = p.C + (i < p.N ? upper_row_base(p.N, i) : 0);
+#pragma unroll 1
+                    for (int cc = 0; cc < kTileN / 32; ++cc) {
+                        const int64_t col0 = (int64_t)J * kTileN + cc * 32;
+                        if (col0 + 32 <= (int64_t)I * kTileM + warp * 32 || col0 >= p.N) continue;  // warp-uniform: nothing kept
+                        uint32_t r[32];
+                        tmem_ld32(taddr + cc * 32, r);
+                        tmem_ld_wait();
+                        if (i < p.N) {
+#pragma unroll
+                            for (int v = 0; v < 32; ++v) {
+                                const int64_t j = col0 + v;
+                                if (j >= i && j < p.N) {
+                                    float o = __uint_as_float(r[v]);
+                                    if (p.accumulate) o += prow[j];
+                                    prow[j] = o;
+                                }
+                            }
+                        }
+                    }
+                }
+            } else if (I < p.row_blocks) {
 #pragma unroll 1
                 for (int cc = 0; cc < kTileN / 32; ++cc) {
                     uint32_t r[32];
@@ -585,6 +647,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     p.N = N;
     p.ncols = ncols;
     p.ldc = ldc;
+    p.M = 0;
     p.cap_elems = round_up(m.slots, 8);
     p.row_blocks = (int32_t)((N + kTileM - 1) / kTileM);
     p.col_blocks = (int32_t)((ncols + kTileN - 1) / kTileN);
@@ -609,7 +672,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(trimm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(trimm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kPSmemBytes) != cudaSuccess)
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
@@ -621,7 +684,79 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     const int64_t n_tiles = (int64_t)((p.row_blocks + 1) / 2) * p.col_blocks;  // pairs of row blocks x column blocks
     const int64_t max_clusters = sm_count() / 2;
     const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-    trimm_pair_kernel<<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, p);
+    trimm_pair_kernel<false><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, p);
+    return launch_status();
+}
+
+// ---- degree-2 moments: A2 = B^T B on the unique part i1 <= i2, packed output ---------------------------
+// Workspace: only when B's row pitch is not a multiple of 16 bytes (a re-pitched copy of B).
+size_t moment2_workspace_bytes(int64_t M, int64_t n, int64_t ldb) {
+    if (M == 0 || n == 0 || ldb % 8 == 0) return 0;
+    return (size_t)(M * round_up(n, 8) * 2);
+}
+
+dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
+                                  int accumulate, void* workspace, int32_t* err_word, cudaStream_t st) {
+    const int64_t n = mo.N;
+    if (n == 0) return DASTAC_OK;
+    if (M == 0) {  // an empty sum: the packed result is zero
+        if (!accumulate && cudaMemsetAsync(out, 0, (size_t)mo.count * sizeof(float), st) != cudaSuccess)
+            return DASTAC_ERR_CUDA;
+        return DASTAC_OK;
+    }
+    if (!aligned16(B)) return DASTAC_ERR_ALIGNMENT;
+    if (M > 0x7fffffffLL - kBlockK || n > 0x7fffffffLL - 2 * kTileN) return DASTAC_ERR_OVERFLOW;
+    if (ldb % 8 != 0) {
+        if (!workspace) return DASTAC_ERR_WORKSPACE;
+        const int64_t ldd = round_up(n, 8);
+        int64_t blocks = (M * ldd + 255) / 256;
+        if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
+        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, (uint16_t*)workspace, ldd, M, n);
+        dastac_status rs = launch_status();
+        if (rs != DASTAC_OK) return rs;
+        B = workspace;
+        ldb = ldd;
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return DASTAC_ERR_CUDA;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBlockK};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DASTAC_ERR_CUDA;
+    Params p;
+    p.A = nullptr;
+    p.tiles = nullptr;
+    p.C = out;
+    p.N = n;
+    p.ncols = n;
+    p.ldc = 0;
+    p.M = M;
+    p.cap_elems = 0;
+    p.row_blocks = (int32_t)((n + kTileM - 1) / kTileM);
+    p.col_blocks = (int32_t)((n + kTileN - 1) / kTileN);
+    p.k_blocks = (int32_t)((M + kBlockK - 1) / kBlockK);
+    p.accumulate = accumulate;
+    p.vector_store = 0;
+    p.err_word = err_word;
+    static bool attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(trimm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kPSmemBytes) != cudaSuccess)
+            return DASTAC_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const int64_t pb = (p.row_blocks + 1) / 2;
+    const int64_t n_tiles = pb * (pb + 1) / 2;
+    const int64_t max_clusters = sm_count() / 2;
+    const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
+    trimm_pair_kernel<true><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap, tmap, p);  // the first map is not used
     return launch_status();
 }
 

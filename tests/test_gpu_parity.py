@@ -452,3 +452,80 @@ def test_band_matmat_exact_layout(N, w, C):
     assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_F32
     # the library's own pack produces the same stream
     assert np.array_equal(dastac.pack(s, dev(A)).cpu().numpy()[: s.nnz], oracle.pack(desc, A))
+
+
+@pytest.mark.parametrize("M,n", [(1, 1), (5, 8), (64, 128), (100, 200), (257, 300), (700, 520), (130, 1030),
+                                 (2000, 256), (63, 77)])
+@pytest.mark.parametrize("symmetric", [False, True], ids=["plain", "swap"])
+def test_moment2_packed_symmetric_output(M, n, symmetric):
+    """Degree-2 moments A2(i1,i2) = sum_x B(x,i1) B(x,i2) on i1 <= i2, packed (Table 1, polynomial regression)."""
+    desc = st.upper_triangle(n, symmetric=symmetric)
+    sA = dastac.Structure(desc)
+    B = synth.dense(6, 0, (M, n), dist=synth.NORMAL, bf16=True)
+    ref, ref_abs = oracle.moment2(desc, B)
+    exp, exp_abs = oracle.pack(desc, ref), oracle.pack(desc, ref_abs)
+    Bd = dev(B, "bf16")
+    out = sA.empty_packed()
+    out.fill_(float("nan"))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    nws = dastac.contract_workspace("xi,xj->ij", None, Bd, [Bd], out, out_structure=sA)
+    assert (nws == 0) == (n % 8 == 0)          # a row pitch that is not a multiple of 16 bytes needs a re-pitched copy
+    ws = torch.empty(max(nws, 1), dtype=torch.uint8, device="cuda")
+    dastac.contract("xi,xj->ij", None, Bd, [Bd], out, out_structure=sA, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    got = out.cpu().numpy()
+    assert rel_err(got[: sA.nnz], exp, exp_abs) <= TOL_BF16
+    assert rel_err(got[: sA.nnz], exp, exp_abs) <= 1e-5     # exact products, fp32 sums: far inside the bf16 bar
+    assert np.isnan(got[sA.nnz:]).all()                      # nothing is written beyond the set's count
+    A0 = synth.dense(6, 1, (sA.nnz,))
+    out2 = sA.empty_packed()
+    out2[: sA.nnz] = dev(A0)
+    dastac.contract("xi,xj->ij", None, Bd, [Bd], out2, accumulate=True, out_structure=sA, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out2.cpu().numpy()[: sA.nnz], exp + A0, exp_abs + np.abs(A0)) <= 1e-5
+    # a padded row pitch (multiple of 8 elements: read in place)
+    Bp = torch.zeros((M, n + 8 - n % 8 + 8), dtype=torch.bfloat16, device="cuda")[:, :n]
+    Bp.copy_(Bd)
+    out3 = sA.empty_packed()
+    dastac.contract("xi,xj->ij", None, Bp, [Bp], out3, out_structure=sA, err_word=err)
+    assert rel_err(out3.cpu().numpy()[: sA.nnz], exp, exp_abs) <= 1e-5
+    if symmetric:
+        full = dastac.unpack(sA, out3).cpu().numpy()
+        assert np.array_equal(full, full.T)
+    # two different tensors, a dense output, fp32 inputs: refused before anything runs
+    other = Bd.clone()
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.contract("xi,xj->ij", None, Bd, [other], out3, out_structure=sA)
+    assert e.value.status == 3
+    with pytest.raises(dastac.DastacError):
+        dastac.contract("xi,xj->ij", None, Bd, [Bd], torch.zeros((n, n), device="cuda"))
+    Bf = Bd.float()
+    with pytest.raises(dastac.DastacError):
+        dastac.contract("xi,xj->ij", None, Bf, [Bf], out3, out_structure=sA)
+    if n > 1:
+        with pytest.raises(dastac.DastacError) as e:
+            dastac.contract("xi,xj->ij", None, Bd, [Bd], out3, out_structure=dastac.Structure(st.upper_triangle(n - 1)))
+        assert e.value.status == 4
+
+
+def test_moment2_empty_sum_and_host_operands():
+    n = 40
+    desc = st.upper_triangle(n, symmetric=True)
+    sA = dastac.Structure(desc)
+    out = sA.empty_packed()
+    out.fill_(float("nan"))
+    B0 = torch.zeros((0, n), dtype=torch.bfloat16, device="cuda")
+    dastac.contract("xi,xj->ij", None, B0, [B0], out, out_structure=sA)
+    assert (out[: sA.nnz] == 0).all()
+    # pinned host operands in and out, staged once through the workspace
+    M = 300
+    B = synth.dense(6, 3, (M, n), dist=synth.NORMAL, bf16=True)
+    ref, ref_abs = oracle.moment2(desc, B)
+    hB = torch.from_numpy(B).view(torch.int16).view(torch.bfloat16).pin_memory()
+    hout = torch.full((sA.capacity(torch.float32),), float("nan")).pin_memory()
+    nws = dastac.contract_workspace("xi,xj->ij", None, hB, [hB], hout, out_structure=sA)
+    assert nws >= M * n * 2 + sA.nnz * 4
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    dastac.contract("xi,xj->ij", None, hB, [hB], hout, out_structure=sA, workspace=ws)
+    torch.cuda.synchronize()
+    assert rel_err(hout.numpy()[: sA.nnz], oracle.pack(desc, ref), oracle.pack(desc, ref_abs)) <= 1e-5
