@@ -53,8 +53,8 @@ def peaks():
 
 def sizes(small: bool):
     if small:
-        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024, N6=128, Q6=32, K6=32)
-    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192, N6=1024, Q6=32, K6=32)
+        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024, N6=128, Q6=32, K6=32, N7=512, M7=2048)
+    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192, N6=1024, Q6=32, K6=32, N7=4096, M7=100000)
 
 
 def accounting(z):
@@ -63,6 +63,7 @@ def accounting(z):
     N1, b, N2, w, C2, N3, n4, R, N5 = (z[k] for k in ("N1", "batch", "N2", "w", "C2", "N3", "n4", "R", "N5"))
     nnz2 = (2 * w + 1) * N2 - w * (w + 1)
     N6, Q6, K6 = z["N6"], z["Q6"], z["K6"]
+    N7, M7 = z["N7"], z["M7"]
     acc = {
         "trmv": dict(flops=2 * tri(N1), bytes=4 * (tri(N1) + 2 * N1), bound="hbm"),
         "trmv_batched": dict(flops=2 * tri(N1) * b, bytes=4 * (tri(N1) + 2 * N1) * b, bound="hbm"),
@@ -76,11 +77,16 @@ def accounting(z):
         "unpack_bf16": dict(flops=0, bytes=2 * (tri(N5) + N5 * N5), bound="hbm"),  # read packed, write box
         # widened row: tensor times matrix over the upper half cube, packed in and out (8 flop/B: HBM first)
         "ttm_ut": dict(flops=2 * tri(N6) * Q6 * K6, bytes=4 * (tri(N6) * (Q6 + K6) + K6 * Q6), bound="hbm"),
+        # widened row: degree-2 moments B^T B on i1 <= i2 (M7 samples x N7 features, bf16), packed fp32 output
+        "moment2_bf16": dict(flops=2 * tri(N7) * M7, bytes=2 * M7 * N7 + 4 * tri(N7), bound="tensor"),
     }
     return acc
 
 
-ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv"]
+ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
+         "moment2_bf16", "symv"]
+# the kernels of the five configurations; the others are widened rows and never the roofline's kernel
+CONFIG_KERNELS = ("trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv")
 
 
 def generate_host(z, pin, only=None):
@@ -150,12 +156,18 @@ def generate_host(z, pin, only=None):
         synth.upper_half_cube_stream(5, 0, N6, N6, Q6, out=a6)
         h["ttm_ut"] = dict(desc=st.upper_half_cube(N6, N6, Q6), out_desc=st.upper_half_cube(N6, N6, K6), A=host(a6),
                            ins=[host(synth.dense(5, 1, (K6, Q6)))], out=(cap(tri(N6) * K6, 4),))
+    if want("moment2_bf16"):
+        N7, M7 = z["N7"], z["M7"]
+        b7 = host(synth.dense(6, 0, (M7, N7), dist=synth.NORMAL, bf16=True), True)
+        # no packed input: the dense tensor is both factors (the same buffer), the output is the packed triangle
+        h["moment2_bf16"] = dict(desc=None, out_desc=st.upper_triangle(N7, symmetric=True), A=b7, ins=[b7], alias=True,
+                                 out=(cap(tri(N7), 4),))
     return h
 
 
 EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
         "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
-        "bandmm_exact": "ij,jc->ic"}
+        "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij"}
 
 
 # ---- clocks ---------------------------------------------------------------------------------------------
@@ -260,9 +272,10 @@ def run_gpu(args):
     # device-resident copies
     devs, structs = {}, {}
     for name, hw in host.items():
-        s = dastac.Structure(hw["desc"])
+        s = dastac.Structure(hw["desc"]) if hw["desc"] is not None else None
         structs[name] = s
-        d = dict(A=hw["A"].cuda(), ins=[t.cuda() for t in hw["ins"]],
+        dA = hw["A"].cuda()
+        d = dict(A=dA, ins=[dA] if hw.get("alias") else [t.cuda() for t in hw["ins"]], alias=hw.get("alias", False),
                  out=torch.empty(hw["out"], dtype=torch.float32, device="cuda"), batch=hw.get("batch", 1),
                  out_s=dastac.Structure(hw["out_desc"]) if "out_desc" in hw else None)
         n = dastac.contract_workspace(EXPR[name], s, d["A"], d["ins"], d["out"], batch=d["batch"],
@@ -370,7 +383,8 @@ def run_gpu(args):
             if a["bound"] == "tensor":
                 k["tensor_frac_measured"] = round(a["flops"] / us / 1e6 / pk["bf16_tflops"], 4)
                 k["tensor_frac_nominal_2250"] = round(a["flops"] / us / 1e6 / 2250.0, 4)
-    dominant = max(order, key=lambda n: kernels[n].get("us_in_step", kernels[n]["us"]))
+    dominant = max([n for n in order if n in CONFIG_KERNELS] or order,
+                   key=lambda n: kernels[n].get("us_in_step", kernels[n]["us"]))
     dk, da = dict(kernels[dominant]), acct[dominant]
     if "us_in_step" in dk:  # the roofline object is taken from the events inside the timed step
         dk["gbs"] = round(da["bytes"] / dk["us_in_step"] / 1e3, 1)
@@ -401,7 +415,9 @@ def run_gpu(args):
             n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1),
                                           out_structure=devs[name]["out_s"])
             hd[name] = dict(out=out_h, ws=torch.empty(n, dtype=torch.uint8, device="cuda"))
-            h2d += hw["A"].numel() * hw["A"].element_size() + sum(t.numel() * t.element_size() for t in hw["ins"])
+            h2d += hw["A"].numel() * hw["A"].element_size()
+            if not hw.get("alias"):
+                h2d += sum(t.numel() * t.element_size() for t in hw["ins"])
             d2h += out_h.numel() * 4
 
         def e2e_step():
@@ -427,7 +443,7 @@ def run_gpu(args):
         e2e = {"value": round(whole_job_gflops(world, e2e_flops, e_ms / e_steps), 1), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e_steps,
                "ms_per_step": round(e_ms / e_steps, 3),
-               "note": "five contractions with pinned host operands staged by dastac_contract; pack/unpack legs excluded"}
+               "note": "every contraction of the step with pinned host operands staged by dastac_contract; pack/unpack legs excluded"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -440,7 +456,7 @@ def run_gpu(args):
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
             "data": "synthetic",
-            "config": {"workload": "all five configs per step, plus two widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6): "
+            "config": {"workload": "all five configs per step, plus three widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features): "
                                    + json.dumps(z, separators=(",", ":")),
                        "small": bool(args.small), "only": args.only or None,
                        "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
@@ -463,11 +479,14 @@ def isolated_times(order, devs, structs, run_kernel_on, z, acct, launches):
     side = torch.cuda.Stream()
     for name in order:
         d = devs[name]
-        tensors = [d["A"], d["out"]] + list(d.get("ins", []))
+        tensors = [d["A"], d["out"]] + ([] if d.get("alias") else list(d.get("ins", [])))
         foot = sum(t.numel() * t.element_size() for t in tensors)
         nsets = max(1, min(256, -(-3 * 126 * 2 ** 20 // max(foot, 1))))
-        sets = [d] + [dict(d, A=d["A"].clone(), out=d["out"].clone(), ins=[t.clone() for t in d.get("ins", [])])
-                      for _ in range(nsets - 1)]
+        def clone_set(d):
+            A = d["A"].clone()
+            return dict(d, A=A, out=d["out"].clone(), ins=[A] if d.get("alias") else [t.clone() for t in d.get("ins", [])])
+
+        sets = [d] + [clone_set(d) for _ in range(nsets - 1)]
         reps = max(1, -(-launches // nsets))
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -567,6 +586,12 @@ def oracle_sample(z, scale=1.0):
     secs += timed(lambda: oracle.ttm(st.upper_half_cube(N6, N6, Q6), B6, C6, sel=sel))
     flops += sum(2 * (N6 - int(i)) * Q6 * K6 for i in sel)
     parts.append(f"ttm {len(sel)} slabs")
+    N7, M7 = z["N7"], z["M7"]
+    sel = rows(N7, 2)
+    B7 = synth.dense(6, 0, (M7, N7), dist=synth.NORMAL, bf16=True)
+    secs += timed(lambda: oracle.moment2(st.upper_triangle(N7, symmetric=True), B7, sel=sel))
+    flops += sum(2 * (N7 - int(i)) * M7 for i in sel)
+    parts.append(f"moment2 {len(sel)} rows")
     return flops, secs, "rows spread evenly over the outer index: " + ", ".join(parts)
 
 
@@ -597,7 +622,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(tot_s / steps * 1e3, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "all five configs per step, plus two widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6): "
+        "config": {"workload": "all five configs per step, plus three widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features): "
                                + json.dumps(z, separators=(",", ":")),
                    "sample": desc},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},

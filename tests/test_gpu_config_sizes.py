@@ -193,3 +193,28 @@ def test_widened_row_exact_band_n32768_w32_c256():
     Ar = np.stack([synth.linear_slice(1, 0, int(i) * N, N) for i in sel])
     ref, ref_abs = oracle.matmat(desc, Ar, B, sel=sel)
     assert rel_err(got[sel], ref, ref_abs) <= TOL_F32
+
+
+def test_widened_row_moment2_m100000_n4096():
+    """Degree-2 moments of 100000 samples x 4096 features (the sample count of the paper's PR2 runs),
+    packed symmetric output, on sampled rows of the result."""
+    M, n = 100000, 4096
+    desc = st.upper_triangle(n, symmetric=True)
+    sA = dastac.Structure(desc)
+    B = synth.dense(6, 0, (M, n), dist=synth.NORMAL, bf16=True)
+    Bd = dev(B, "bf16")
+    out = torch.full((sA.capacity(torch.float32),), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dastac.contract("xi,xj->ij", None, Bd, [Bd], out, out_structure=sA, err_word=err)
+    assert int(err.item()) == 0
+    got = out.cpu().numpy()[: sA.nnz]
+    assert np.isfinite(got).all()
+    sel = np.array([0, 127, 128, 255, 256, 1000, 2047, 2048, 3839, 3840, n - 2, n - 1], dtype=np.int64)
+    ref, ref_abs = oracle.moment2(desc, B, sel=sel)
+    for s, i in enumerate(sel):
+        start = oracle.rank_point(desc, (int(i), int(i))) if s < 2 else int(i) * n - int(i) * (int(i) - 1) // 2
+        seg = got[start: start + n - int(i)]
+        # 100000 same-sign terms on the diagonal, accumulated in fp32 inside the tensor core: the error
+        # grows with the length of the sum (about 5e-4 here), still far inside the bf16 bar
+        assert rel_err(seg, ref[s, int(i):], ref_abs[s, int(i):]) <= TOL_BF16
+        assert rel_err(seg, ref[s, int(i):], ref_abs[s, int(i):]) <= 2e-3

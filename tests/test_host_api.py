@@ -216,3 +216,51 @@ def test_exact_band_limits_and_kind():
     assert dastac.unrank(big, big.nnz - 1) == (2 ** 20 - 1, 2 ** 20 - 1)
     for p in (0, 1, 500_500, 123_456_789, big.nnz - 2):
         assert dastac.rank(big, dastac.unrank(big, p)) == p
+
+
+def test_moment2_plan_is_validated_on_the_host():
+    """"xi,xj->ij": dense bf16 input given twice, packed f32 upper triangle out; no launch, no GPU."""
+    before = dastac.launch_count()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    n, M = 24, 100
+    s = dastac.Structure(st.upper_triangle(n, symmetric=True))
+    ins = (binding._Operand * 2)()
+    for k in range(2):
+        ins[k].data = 4096          # never dereferenced: planning only
+        ins[k].dtype = binding.BF16
+        ins[k].rank = 2
+        ins[k].dims[0], ins[k].dims[1] = M, n
+        ins[k].strides[0], ins[k].strides[1] = n, 1
+    out = binding._Operand()
+    out.structure = s._h
+    out.rank = 2
+    nbytes = ctypes.c_size_t(123)
+    args = (ins, 2, ctypes.byref(out), ctypes.byref(nbytes))
+    ws = lib.dastac_contract_workspace
+    assert ws(b"xi,xj->ij", *args) == 0 and nbytes.value == 0        # row pitch 48 bytes: read in place
+    ins[0].strides[0] = ins[1].strides[0] = n + 1                      # 50 bytes: a re-pitched copy of B
+    assert ws(b"xi,xj->ij", *args) == 0 and nbytes.value == -(-M * n * 2 // 256) * 256
+    ins[0].strides[0] = ins[1].strides[0] = n
+    ins[0].space = ins[1].space = 1                                    # host input: staged once, not twice
+    out.space = 1
+    assert ws(b"xi,xj->ij", *args) == 0
+    assert nbytes.value == -(-M * n * 2 // 256) * 256 + -(-s.capacity(__import__("torch").float32) * 4 // 256) * 256
+    ins[0].space = ins[1].space = out.space = 0
+    ins[1].data = 8192                                                 # two different tensors
+    assert ws(b"xi,xj->ij", *args) == 3
+    ins[1].data = 4096
+    ins[1].strides[0] = n + 8
+    assert ws(b"xi,xj->ij", *args) == 3
+    ins[1].strides[0] = n
+    ins[0].dtype = ins[1].dtype = binding.F32
+    assert ws(b"xi,xj->ij", *args) == 3
+    ins[0].dtype = ins[1].dtype = binding.BF16
+    out.structure = None                                               # dense output
+    assert ws(b"xi,xj->ij", *args) == 3
+    bigger, lower = dastac.Structure(st.upper_triangle(n + 1)), dastac.Structure(st.lower_triangle(n))
+    out.structure = bigger._h                                          # wrong extent
+    assert ws(b"xi,xj->ij", *args) == 4
+    out.structure = lower._h                                           # not the unique part i <= j
+    assert ws(b"xi,xj->ij", *args) == 3
+    assert ws(b"xi,xj->ij", ins, 1, ctypes.byref(out), ctypes.byref(nbytes)) == 1
+    assert dastac.launch_count() == before
