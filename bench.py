@@ -522,6 +522,8 @@ TRAFFIC = {
     "trimm_bf16": int(855.178240e6 + 215.225600e6 + 67.129856e6 + 28.432640e6),  # main kernel + tile staging
     "bandmm": int(42.104320e6 + 3.751424e6),   # outputs of this size stay in L2 past the end of the launch
     "ttm_ut": int(67.207424e6 + 18.528000e6),
+    "bandmm_exact": int(42.108160e6 + 2.613248e6),
+    "moment2_bf16": int(1.410541e9 + 22.173440e6),   # full size, DRAM counters only (one pass)
     "pack_bf16": int(67.683584e6 + 27.079680e6),
     "unpack_bf16": int(67.140864e6 + 78.835712e6),
 }
