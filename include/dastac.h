@@ -55,7 +55,9 @@ typedef enum {
     DASTAC_KIND_LOWER = 3,          /* 0<=j<=i<N                                                   */
     DASTAC_KIND_BAND_DIAGONALS = 4, /* |i-j|<=w stored as 2w+1 diagonals of N slots                */
     DASTAC_KIND_TETRAHEDRON = 5,    /* 0<=i<=j<=k<n                                                */
-    DASTAC_KIND_BAND_EXACT = 6      /* |i-j|<=w, 2w+1<=N, rows packed back to back (no padding)    */
+    DASTAC_KIND_BAND_EXACT = 6,     /* |i-j|<=w, 2w+1<=N, rows packed back to back (no padding)    */
+    DASTAC_KIND_UPPER_SHIFTED = 7   /* j-i>=c, c>=1, square: the size N-c triangle in the top right corner
+                                       (the sub-triangular structure of Section 6.4)               */
 } dastac_kind;
 
 #define DASTAC_LAYOUT_LEXICOGRAPHIC 0 /* exact pack in lexicographic order                         */
@@ -168,6 +170,8 @@ typedef struct {
  * Supported (expression, structure of in[0], dtypes):
  *   "ij,j->i"       upper triangle (square)             f32        y = A x         (batched)
  *   "ij,j->i"       upper triangle + swap (symmetric)   f32        y = S x
+ *   "ij,j->i"       sub-triangle j - i >= c             f32        y = A x         (batched); rows N-c .. N-1 of
+ *                   y have no stored element and are set to 0 (left unchanged when accumulating)
  *   "ij,jc->ic"     band, padded diagonals or exact     f32        C = A B
  *   "ij,jc->ic"     upper triangle (square)             bf16 -> f32 output, fp32 accumulation
  *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)

@@ -131,7 +131,8 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         p.N = m.dims[2];   // Q
         p.R = mo.dims[2];  // K
     } else if (p.cls == kMatVec) {
-        if (!(m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1]) && m.kind != kEmpty)
+        if (!(m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1]) && m.kind != kEmpty &&
+            m.kind != kUpperShifted)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (in[0].dtype != DASTAC_F32 || in[1].dtype != DASTAC_F32 || out->dtype != DASTAC_F32)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
@@ -265,6 +266,19 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     } else if (p.cls == kTtm) {
         st = launch_ttm(m.count / p.N, p.N, p.R, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0],
                         (float*)dev_out, accumulate, cs);
+    } else if (p.cls == kMatVec && m.kind == kUpperShifted) {
+        // The sub-triangle is the size-M upper triangle applied to x shifted by c; rows M .. N-1 of y
+        // have no stored element: they are zero (or left alone when accumulating).
+        IndexMap t = m;
+        t.kind = kUpper;
+        t.N = t.dims[0] = t.dims[1] = m.M;
+        t.w = 0;
+        st = launch_trmv(t, (const float*)dev_in[0], (const float*)dev_in[1] + m.w, (float*)dev_out, p.batch,
+                         in[0].batch_stride, in[1].batch_stride, out->batch_stride, accumulate, cs);
+        if (st == DASTAC_OK && !accumulate &&
+            cudaMemset2DAsync((float*)dev_out + m.M, (size_t)(p.batch > 1 ? out->batch_stride : m.N) * sizeof(float), 0,
+                              (size_t)m.w * sizeof(float), (size_t)p.batch, cs) != cudaSuccess)
+            st = DASTAC_ERR_CUDA;
     } else if (p.cls == kMatVec && !p.symmetric) {
         st = launch_trmv(m, (const float*)dev_in[0], (const float*)dev_in[1], (float*)dev_out,
                          p.batch, in[0].batch_stride, in[1].batch_stride, out->batch_stride,

@@ -28,7 +28,11 @@ enum Kind : int32_t {
     kLower = 3,
     kBandDiagonals = 4,
     kTetrahedron = 5,
-    kBandExact = 6  // |i - j| <= w packed row after row without padding (2w + 1 <= N)
+    kBandExact = 6,  // |i - j| <= w packed row after row without padding (2w + 1 <= N)
+    // j - i >= c in an N x N box (c >= 1): the upper triangle of size M = N - c sitting in the top
+    // right corner (the sub-triangular structure of Section 6.4, "Density and Compression", with
+    // c = N - k).  Row i < M holds columns i + c .. N-1; the shift c is kept in `w`.
+    kUpperShifted = 7
 };
 
 // Plain data, passed to kernels by value.
@@ -140,6 +144,7 @@ DASTAC_HD bool in_set(const IndexMap& m, const int32_t* idx) {
             int64_t d = (int64_t)idx[1] - idx[0];
             return d <= m.w && -d <= m.w;
         }
+        case kUpperShifted: return (int64_t)idx[1] - idx[0] >= m.w;
         default: return false;
     }
 }
@@ -166,6 +171,7 @@ DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
                    ((int64_t)idx[2] - idx[1]);
         }
         case kBandExact: return band_row_start(m.N, m.w, idx[0]) + (idx[1] - band_jlo(m.w, idx[0]));
+        case kUpperShifted: return upper_row_base(m.M, idx[0]) + (idx[1] - m.w);  // the size-M triangle at column j - c
         default: return -1;
     }
 }
@@ -226,6 +232,12 @@ DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
             idx[1] = (int32_t)(band_jlo(m.w, i) + (p - band_row_start(m.N, m.w, i)));
             return;
         }
+        case kUpperShifted: {
+            const int64_t i = upper_row_of(m.M, p);
+            idx[0] = (int32_t)i;
+            idx[1] = (int32_t)(m.w + i + (p - upper_row_start(m.M, i)));
+            return;
+        }
         default: return;
     }
 }
@@ -272,6 +284,13 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
             jlo = band_jlo(m.w, idx[0]);
             jhi = band_jhi(m.N, m.w, idx[0]) + 1;
             pbase = band_row_start(m.N, m.w, idx[0]) - jlo;
+            return true;
+        }
+        case kUpperShifted: {
+            if (idx[0] >= m.M) return false;
+            jlo = idx[0] + m.w;
+            jhi = m.N;
+            pbase = upper_row_base(m.M, idx[0]) - m.w;
             return true;
         }
         default: return false;
@@ -323,6 +342,12 @@ DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {
             }
             ++idx[0];
             idx[1] = (int32_t)band_jlo(m.w, idx[0]);
+            return;
+        }
+        case kUpperShifted: {
+            if (++idx[1] < m.N) return;
+            ++idx[0];
+            idx[1] = (int32_t)(idx[0] + m.w);
             return;
         }
         default: return;

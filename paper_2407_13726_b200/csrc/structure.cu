@@ -177,6 +177,19 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
         lo[k] = -b.D[O][k];
         hi[k] = b.D[k][O];
     }
+    // The sub-triangle j - i >= c (c >= 1) of a square box: its closure moves the lower bound of j
+    // to c and the upper bound of i to N - 1 - c; nothing else relates the two indices.
+    if (rank == 2 && desc->layout != DASTAC_LAYOUT_PADDED_DIAGONALS && m.dims[0] == m.dims[1] && b.D[0][1] < 0 &&
+        lo[0] == 0 && lo[1] == -b.D[0][1] && hi[1] == m.dims[1] - 1 && hi[0] == m.dims[0] - 1 + b.D[0][1] &&
+        b.D[1][0] == hi[1] - lo[0]) {
+        if (desc->mirror && !(desc->mirror[0] == 0 && desc->mirror[1] == 1)) return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
+        m.kind = kUpperShifted;
+        m.N = m.dims[1];
+        m.w = -b.D[0][1];
+        m.M = m.N - m.w;
+        m.count = m.slots = tri(m.M);
+        return finish();
+    }
     // Every class below starts at the origin of the box in every index.
     for (int k = 0; k < rank; ++k)
         if (lo[k] != 0) return DASTAC_ERR_UNSUPPORTED_STRUCTURE;

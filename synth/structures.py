@@ -109,3 +109,11 @@ def diagonal(N: int) -> Descriptor:
     eq = np.zeros(len(items), np.uint8)
     eq[-1] = 1
     return Descriptor([N, N], [N], _rows(2, 1, items), eq, name="diagonal")
+
+
+def sub_triangle(N: int, k: int) -> Descriptor:
+    """{(i, j) : 0 <= i < N, 0 <= j < N, j - i >= N - k}: the triangle of size k in the top right
+    corner of the N x N box; params = (N, k)."""
+    items = _box_rows(2, 2, [0, 0]) + [[-1, 1, -1, 1, 0]]
+    return Descriptor([N, N], [N, k], _rows(2, 2, items), np.zeros(len(items), np.uint8),
+                      name="sub_triangle", meta={"k": k})

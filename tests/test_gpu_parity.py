@@ -21,7 +21,7 @@ INDEX_CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(97)
                st.lower_triangle(61), st.tetrahedron(1), st.tetrahedron(2), st.tetrahedron(48),
                st.upper_half_cube(9, 14, 5), st.upper_half_cube(14, 9, 3), st.dense_box([5, 6, 7]),
                st.band(50, 4), st.band(7, 0), st.upper_triangle(1000), st.band_exact(50, 4), st.band_exact(9, 4),
-               st.band_exact(300, 32)]
+               st.band_exact(300, 32), st.sub_triangle(60, 13), st.sub_triangle(9, 1), st.sub_triangle(300, 299)]
 
 
 @pytest.mark.parametrize("desc", INDEX_CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -109,7 +109,7 @@ PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33),
               st.upper_triangle(1000), st.upper_triangle(130, True), st.lower_triangle(77),
               st.tetrahedron(2), st.tetrahedron(37), st.upper_half_cube(11, 17, 3),
               st.upper_half_cube(17, 11, 6), st.dense_box([6, 10]), st.band_exact(11, 5), st.band_exact(130, 7),
-              st.band_exact(1000, 32)]
+              st.band_exact(1000, 32), st.sub_triangle(11, 4), st.sub_triangle(130, 77), st.sub_triangle(1000, 333)]
 
 
 @pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
@@ -179,6 +179,41 @@ def test_trmv(N):
     y2 = dev(y0)
     dastac.contract("ij,j->i", s, packed, [dev(x)], y2, accumulate=True)
     assert rel_err(y2.cpu().numpy(), ref + y0, ref_abs + np.abs(y0)) <= TOL_F32
+
+
+@pytest.mark.parametrize("N,k", [(2, 1), (9, 4), (64, 64), (100, 33), (1000, 128), (1024, 1000), (4096, 512), (3000, 2500)])
+def test_trmv_sub_triangle(N, k):
+    """y = A x for the sub-triangular structure j - i >= N - k (Section 6.4): rows k .. N-1 of y are zero."""
+    desc = st.sub_triangle(N, k)
+    s = dastac.Structure(desc)
+    A = synth.dense(0, 0, (N, N))
+    x = synth.dense(0, 1, (N,))
+    ref, ref_abs = oracle.matvec(desc, A, x)
+    packed = packed_dev(s, oracle.pack(desc, A))
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    y0 = synth.dense(0, 2, (N,))
+    y2 = dev(y0)
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y2, accumulate=True)
+    assert rel_err(y2.cpu().numpy(), ref + y0, ref_abs + np.abs(y0)) <= TOL_F32
+    assert np.array_equal(y2.cpu().numpy()[k:], y0[k:])          # rows without stored elements are left alone
+    # the library's own pack gives the same stream; batched instances with strided operands
+    assert np.array_equal(dastac.pack(s, dev(A)).cpu().numpy()[: s.nnz], oracle.pack(desc, A))
+    batch = 3
+    cap = s.capacity(torch.float32)
+    pk = torch.full((batch, cap + 4), float("nan"), device="cuda")[:, :cap]
+    xs = torch.empty((batch, N + 2), device="cuda")[:, :N]
+    ys = torch.full((batch, N + 1), float("nan"), device="cuda")[:, :N]
+    refs = []
+    for b in range(batch):
+        Ab, xb = synth.dense(30 + b, 0, (N, N)), synth.dense(30 + b, 1, (N,))
+        pk[b, : s.nnz] = dev(oracle.pack(desc, Ab))
+        xs[b] = dev(xb)
+        refs.append(oracle.matvec(desc, Ab, xb))
+    dastac.contract("ij,j->i", s, pk, [xs], ys, batch=batch)
+    for b in range(batch):
+        assert rel_err(ys[b].cpu().numpy(), refs[b][0], refs[b][1]) <= TOL_F32
 
 
 def test_trmv_closed_forms():

@@ -32,7 +32,8 @@ CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(37), st.u
          st.tetrahedron(15), st.upper_half_cube(4, 6, 3), st.upper_half_cube(6, 4, 2),
          st.upper_half_cube(5, 5, 1), st.dense_box([3, 4]), st.dense_box([2, 3, 4]), st.dense_box([7]),
          st.band_exact(1, 0), st.band_exact(7, 0), st.band_exact(7, 3), st.band_exact(8, 3), st.band_exact(23, 4),
-         st.band_exact(40, 11)]
+         st.band_exact(40, 11), st.sub_triangle(7, 3), st.sub_triangle(6, 1), st.sub_triangle(9, 8),
+         st.sub_triangle(40, 17), st.sub_triangle(5, 5)]
 
 
 @pytest.mark.parametrize("desc", CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -82,10 +83,13 @@ def test_recognition_is_independent_of_how_rows_are_written():
     d2 = st.Descriptor([N, N], [N], rows, np.zeros(len(rows), np.uint8))
     s1, s2 = dastac.Structure(base), dastac.Structure(d2)
     assert (s1.kind, s1.nnz) == (s2.kind, s2.nnz) == (binding.KIND_UPPER, N * (N + 1) // 2)
-    # strict inequality written as i - j + 1 <= 0 is a different set (strictly upper): not a class
+    # strict inequality written as i - j + 1 <= 0 is a different set: strictly upper = the sub-triangle with shift 1
     strict = st.Descriptor([N, N], [N], np.array([[-1, 1, 0, -1]], dtype=np.int64), np.zeros(1, np.uint8))
+    ss = dastac.Structure(strict)
+    assert (ss.kind, ss.nnz) == (dastac.KIND_UPPER_SHIFTED, N * (N - 1) // 2) and oracle.count(strict) == ss.nnz
+    # a lower bound on i alone (i >= 2) is not a recognised class
     with pytest.raises(dastac.DastacError) as e:
-        dastac.Structure(strict)
+        dastac.Structure(st.Descriptor([N, N], [N], np.array([[1, 0, 0, -2]], dtype=np.int64), np.zeros(1, np.uint8)))
     assert e.value.status == 2
     # an equality row (diagonal) closes to the band of half width 0, packed exactly: N points, rank(i, i) = i
     diag = dastac.Structure(st.diagonal(5))
@@ -204,6 +208,23 @@ def test_argument_errors_do_not_launch():
     ins[0].structure = t._h
     assert lib.dastac_contract_workspace(b"ij,j->i", *args) == 3
     assert dastac.launch_count() == before
+
+
+def test_sub_triangle_kind_and_limits():
+    """j - i >= N - k: the size-k triangle in the top right corner (Section 6.4, density experiment)."""
+    s = dastac.Structure(st.sub_triangle(16, 5))
+    assert s.kind == dastac.KIND_UPPER_SHIFTED and s.nnz == s.slots == 15
+    assert dastac.rank(s, (0, 11)) == 0 and dastac.rank(s, (4, 15)) == 14 and dastac.unrank(s, 5) == (1, 12)
+    assert dastac.Structure(st.sub_triangle(16, 16)).kind == dastac.KIND_UPPER       # k = N: the whole upper triangle
+    assert dastac.Structure(st.sub_triangle(16, 0)).nnz == 0                          # k = 0: empty
+    big = dastac.Structure(st.sub_triangle(2 ** 16, 2 ** 14))
+    assert big.nnz == 2 ** 14 * (2 ** 14 + 1) // 2
+    for p in (0, 1, 12345678, big.nnz - 1):
+        assert dastac.rank(big, dastac.unrank(big, p)) == p
+    sym = st.sub_triangle(8, 3)
+    sym.mirror = [1, 0]
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(sym)
 
 
 def test_exact_band_limits_and_kind():
