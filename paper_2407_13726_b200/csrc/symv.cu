@@ -24,7 +24,8 @@ constexpr int kThreads = 256;
 constexpr int kQ = 2;                       // quads per thread and row
 constexpr int kTileQuads = kThreads * kQ;   // 512 quads
 constexpr int kTileCols = 4 * kTileQuads;   // 2048 columns
-constexpr int kTileRows = 128;
+// Rows per tile: 128 for the largest matrices; fewer when 128-row tiles would give the GPU only a
+// wave or two of CTAs (the tiles left of the diagonal return at once), chosen by the host.
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -111,6 +112,7 @@ __device__ __forceinline__ void tile_rows(const int N, const int64_t cap_quads, 
     }
 }
 
+template <int kTileRows>
 __global__ void __launch_bounds__(kThreads, 4)
 symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, const float* __restrict__ A,
                  const float* __restrict__ x, float* __restrict__ y) {
@@ -172,10 +174,21 @@ dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, flo
     if (!accumulate && cudaMemsetAsync(y, 0, (size_t)N * sizeof(float), st) != cudaSuccess)
         return DASTAC_ERR_CUDA;
     const int64_t quads_per_row = (N + 2) / 4 + 1;  // quads that can hold a column < N for some alignment
-    const int64_t row_tiles = (N + kTileRows - 1) / kTileRows, col_tiles = (quads_per_row + kTileQuads - 1) / kTileQuads;
+    const int64_t col_tiles = (quads_per_row + kTileQuads - 1) / kTileQuads;
+    // about half of the tiles do work; aim at six or more waves of 4 CTAs per SM
+    const int64_t want = (int64_t)sm_count() * 4 * 6;
+    int rows = 128;
+    while (rows > 32 && ((N + rows - 1) / rows) * col_tiles / 2 < want) rows >>= 1;
+    const int64_t row_tiles = (N + rows - 1) / rows;
     if (row_tiles * col_tiles > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
     const int64_t cap_quads = (m.count + 3) / 4;
-    symv_quad_kernel<<<(unsigned)(row_tiles * col_tiles), kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
+    const unsigned grid = (unsigned)(row_tiles * col_tiles);
+    if (rows == 128)
+        symv_quad_kernel<128><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
+    else if (rows == 64)
+        symv_quad_kernel<64><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
+    else
+        symv_quad_kernel<32><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
     return launch_status();
 }
 
