@@ -56,8 +56,11 @@ typedef enum {
     DASTAC_KIND_BAND_DIAGONALS = 4, /* |i-j|<=w stored as 2w+1 diagonals of N slots                */
     DASTAC_KIND_TETRAHEDRON = 5,    /* 0<=i<=j<=k<n                                                */
     DASTAC_KIND_BAND_EXACT = 6,     /* |i-j|<=w, 2w+1<=N, rows packed back to back (no padding)    */
-    DASTAC_KIND_UPPER_SHIFTED = 7   /* j-i>=c, c>=1, square: the size N-c triangle in the top right corner
+    DASTAC_KIND_UPPER_SHIFTED = 7,  /* j-i>=c, c>=1, square: the size N-c triangle in the top right corner
                                        (the sub-triangular structure of Section 6.4)               */
+    DASTAC_KIND_BAND_OFFSETS = 8    /* lo<=j-i<=hi, square, any lo<=hi: rows packed back to back.  One
+                                       off-diagonal (lo=hi=s) is a per-summand buffer of the strided band
+                                       of Section 6.4; chosen when no class above applies           */
 } dastac_kind;
 
 #define DASTAC_LAYOUT_LEXICOGRAPHIC 0 /* exact pack in lexicographic order                         */
@@ -170,6 +173,11 @@ typedef struct {
  * Supported (expression, structure of in[0], dtypes):
  *   "ij,j->i"       upper triangle (square)             f32        y = A x         (batched)
  *   "ij,j->i"       upper triangle + swap (symmetric)   f32        y = S x
+ *   "ij,j->i"       dense box, lower triangle, exact    f32        y = A x         (batched); rows without a
+ *                   band, offset band                                 stored element give 0.  A rule with
+ *                   several summands (strided band: three diagonals; Leslie matrix: first row +
+ *                   sub-diagonal) is evaluated summand by summand, each with its own packed buffer
+ *                   (Section 4, one buffer per summand), the later calls with accumulate = 1
  *   "ij,j->i"       sub-triangle j - i >= c             f32        y = A x         (batched); rows N-c .. N-1 of
  *                   y have no stored element and are set to 0 (left unchanged when accumulating)
  *   "ij,jc->ic"     band, padded diagonals or exact     f32        C = A B

@@ -37,6 +37,10 @@ int sm_count();
 dastac_status launch_trmv(const IndexMap& m, const float* A, const float* x, float* y, int batch,
                           int64_t a_stride, int64_t x_stride, int64_t y_stride, int accumulate,
                           cudaStream_t st);
+bool rowspan_mv_supports(const IndexMap& m);
+dastac_status launch_rowspan_mv(const IndexMap& m, const float* A, const float* x, float* y, int batch,
+                                int64_t a_stride, int64_t x_stride, int64_t y_stride, int accumulate,
+                                cudaStream_t st);
 size_t symv_workspace_bytes(const IndexMap& m);
 dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, float* y,
                           int accumulate, void* workspace, cudaStream_t st);

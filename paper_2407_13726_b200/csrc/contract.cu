@@ -132,7 +132,7 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         p.R = mo.dims[2];  // K
     } else if (p.cls == kMatVec) {
         if (!(m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1]) && m.kind != kEmpty &&
-            m.kind != kUpperShifted)
+            m.kind != kUpperShifted && !rowspan_mv_supports(m))
             return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (in[0].dtype != DASTAC_F32 || in[1].dtype != DASTAC_F32 || out->dtype != DASTAC_F32)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
@@ -279,6 +279,9 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
             cudaMemset2DAsync((float*)dev_out + m.M, (size_t)(p.batch > 1 ? out->batch_stride : m.N) * sizeof(float), 0,
                               (size_t)m.w * sizeof(float), (size_t)p.batch, cs) != cudaSuccess)
             st = DASTAC_ERR_CUDA;
+    } else if (p.cls == kMatVec && rowspan_mv_supports(m)) {
+        st = launch_rowspan_mv(m, (const float*)dev_in[0], (const float*)dev_in[1], (float*)dev_out, p.batch,
+                               in[0].batch_stride, in[1].batch_stride, out->batch_stride, accumulate, cs);
     } else if (p.cls == kMatVec && !p.symmetric) {
         st = launch_trmv(m, (const float*)dev_in[0], (const float*)dev_in[1], (float*)dev_out,
                          p.batch, in[0].batch_stride, in[1].batch_stride, out->batch_stride,

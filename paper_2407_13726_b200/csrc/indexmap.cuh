@@ -32,7 +32,12 @@ enum Kind : int32_t {
     // j - i >= c in an N x N box (c >= 1): the upper triangle of size M = N - c sitting in the top
     // right corner (the sub-triangular structure of Section 6.4, "Density and Compression", with
     // c = N - k).  Row i < M holds columns i + c .. N-1; the shift c is kept in `w`.
-    kUpperShifted = 7
+    kUpperShifted = 7,
+    // lo_off <= j - i <= hi_off inside an N x N box, any lo_off <= hi_off: rows packed back to back.
+    // One diagonal at distance s (lo_off = hi_off = s) is the per-summand buffer of a strided band
+    // (Section 6.4, "Distance of Elements and Compression"); asymmetric bands, strictly lower
+    // triangles and the like fall out of the same counting function.
+    kBandOffsets = 8
 };
 
 // Plain data, passed to kernels by value.
@@ -48,6 +53,7 @@ struct IndexMap {
     int64_t w;        // kBand: half width
     int64_t count;    // points of the set
     int64_t slots;    // elements of the packed vector (count, or (2w+1)N with padding)
+    int64_t lo_off, hi_off;  // kBandOffsets: bounds of j - i
 };
 
 DASTAC_HD int64_t tri(int64_t m) { return (m * (m + 1)) >> 1; }
@@ -107,6 +113,36 @@ DASTAC_HD int64_t band_row_of(int64_t N, int64_t w, int64_t p) {
     return i;
 }
 
+// General offset band lo <= j - i <= hi of an N x N box.  Row t holds hi - lo + 1 points minus the
+// max(0, -lo - t) it loses at column 0 and the max(0, t + hi - (N-1)) it loses at column N-1, for
+// rows t in [first, last] = [max(0, -hi), min(N-1, N-1-lo)].  The points before row i are therefore
+// a linear term minus two arithmetic series, each switched on by a clamp: a piecewise quadratic
+// (Section 4, "Access domain linearization") written as one expression.
+DASTAC_HD int64_t oband_first_row(int64_t hi) { return hi < 0 ? -hi : 0; }
+DASTAC_HD int64_t oband_last_row(int64_t N, int64_t lo) { return lo > 0 ? N - 1 - lo : N - 1; }
+DASTAC_HD int64_t oband_jlo(int64_t lo, int64_t i) { return i + lo > 0 ? i + lo : 0; }
+DASTAC_HD int64_t oband_jhi(int64_t N, int64_t hi, int64_t i) { return i + hi < N - 1 ? i + hi : N - 1; }  // inclusive
+// valid for first <= i <= last + 1
+DASTAC_HD int64_t oband_row_start(int64_t N, int64_t lo, int64_t hi, int64_t i) {
+    const int64_t f = oband_first_row(hi);
+    int64_t total = (i - f) * (hi - lo + 1);
+    const int64_t tl = i < -lo ? i : -lo;  // rows f .. tl-1 are clipped at column 0 by -lo - t
+    if (tl > f) total -= (((-lo - f) + (-lo - (tl - 1))) * (tl - f)) >> 1;
+    const int64_t tr = f > N - hi ? f : N - hi;  // rows tr .. i-1 are clipped at column N-1 by t + hi - N + 1
+    if (i > tr) total -= (((tr + hi - N + 1) + (i + hi - N)) * (i - tr)) >> 1;
+    return total;
+}
+// Row of position p: the starts are increasing in i, so bisection over the closed form is exact.
+DASTAC_HD int64_t oband_row_of(int64_t N, int64_t lo, int64_t hi, int64_t p) {
+    int64_t a = oband_first_row(hi), b = oband_last_row(N, lo);
+    while (a < b) {
+        const int64_t mid = (a + b + 1) >> 1;
+        if (oband_row_start(N, lo, hi, mid) <= p) a = mid;
+        else b = mid - 1;
+    }
+    return a;
+}
+
 // Upper triangle / trapezoid: points before row i, in units of (j) positions.
 DASTAC_HD int64_t upper_row_start(int64_t N, int64_t i) { return i * N - ((i * (i - 1)) >> 1); }
 
@@ -145,6 +181,10 @@ DASTAC_HD bool in_set(const IndexMap& m, const int32_t* idx) {
             return d <= m.w && -d <= m.w;
         }
         case kUpperShifted: return (int64_t)idx[1] - idx[0] >= m.w;
+        case kBandOffsets: {
+            int64_t d = (int64_t)idx[1] - idx[0];
+            return d >= m.lo_off && d <= m.hi_off;
+        }
         default: return false;
     }
 }
@@ -172,6 +212,8 @@ DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
         }
         case kBandExact: return band_row_start(m.N, m.w, idx[0]) + (idx[1] - band_jlo(m.w, idx[0]));
         case kUpperShifted: return upper_row_base(m.M, idx[0]) + (idx[1] - m.w);  // the size-M triangle at column j - c
+        case kBandOffsets:
+            return oband_row_start(m.N, m.lo_off, m.hi_off, idx[0]) + (idx[1] - oband_jlo(m.lo_off, idx[0]));
         default: return -1;
     }
 }
@@ -238,6 +280,12 @@ DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
             idx[1] = (int32_t)(m.w + i + (p - upper_row_start(m.M, i)));
             return;
         }
+        case kBandOffsets: {
+            const int64_t i = oband_row_of(m.N, m.lo_off, m.hi_off, p);
+            idx[0] = (int32_t)i;
+            idx[1] = (int32_t)(oband_jlo(m.lo_off, i) + (p - oband_row_start(m.N, m.lo_off, m.hi_off, i)));
+            return;
+        }
         default: return;
     }
 }
@@ -291,6 +339,13 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
             jlo = idx[0] + m.w;
             jhi = m.N;
             pbase = upper_row_base(m.M, idx[0]) - m.w;
+            return true;
+        }
+        case kBandOffsets: {
+            if (idx[0] < oband_first_row(m.hi_off) || idx[0] > oband_last_row(m.N, m.lo_off)) return false;
+            jlo = oband_jlo(m.lo_off, idx[0]);
+            jhi = oband_jhi(m.N, m.hi_off, idx[0]) + 1;
+            pbase = oband_row_start(m.N, m.lo_off, m.hi_off, idx[0]) - jlo;
             return true;
         }
         default: return false;
@@ -348,6 +403,15 @@ DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {
             if (++idx[1] < m.N) return;
             ++idx[0];
             idx[1] = (int32_t)(idx[0] + m.w);
+            return;
+        }
+        case kBandOffsets: {
+            if (idx[1] < oband_jhi(m.N, m.hi_off, idx[0])) {
+                ++idx[1];
+                return;
+            }
+            ++idx[0];
+            idx[1] = (int32_t)oband_jlo(m.lo_off, idx[0]);
             return;
         }
         default: return;

@@ -323,7 +323,7 @@ unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ d
 
 bool row_path(const IndexMap& m) {
     return (m.kind == kDense || (m.kind == kUpper && m.rank == 2) || m.kind == kLower || m.kind == kTetrahedron ||
-            m.kind == kBandExact || m.kind == kUpperShifted) &&
+            m.kind == kBandExact || m.kind == kUpperShifted || m.kind == kBandOffsets) &&
            !m.symmetric;
 }
 

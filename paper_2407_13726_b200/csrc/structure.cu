@@ -190,9 +190,29 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
         m.count = m.slots = tri(m.M);
         return finish();
     }
+    // General offset band lo_off <= j - i <= hi_off of a square box, tried when none of the special
+    // classes (which have faster kernels) applies: the closure must carry nothing but the two
+    // difference bounds and the index ranges they imply.
+    auto offset_band = [&]() -> bool {
+        if (rank != 2 || desc->layout == DASTAC_LAYOUT_PADDED_DIAGONALS || m.dims[0] != m.dims[1]) return false;
+        const int64_t N = m.dims[0], a = -b.D[0][1], c = b.D[1][0];
+        if (a > c) return false;
+        if (lo[0] != oband_first_row(c) || hi[0] != oband_last_row(N, a)) return false;
+        if (lo[1] != (a > 0 ? a : 0) || hi[1] != (c < 0 ? N - 1 + c : N - 1)) return false;
+        if (desc->mirror && !(desc->mirror[0] == 0 && desc->mirror[1] == 1)) return false;
+        m.kind = kBandOffsets;
+        m.N = N;
+        m.lo_off = a;
+        m.hi_off = c;
+        m.count = m.slots = oband_row_start(N, a, c, oband_last_row(N, a) + 1);
+        return true;
+    };
     // Every class below starts at the origin of the box in every index.
     for (int k = 0; k < rank; ++k)
-        if (lo[k] != 0) return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
+        if (lo[k] != 0) {
+            if (offset_band()) return finish();
+            return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
+        }
     auto free_pair = [&](int p, int q) {  // no constraint between p and q beyond the box
         return b.D[p][q] == hi[p] - lo[q] && b.D[q][p] == hi[q] - lo[p];
     };
@@ -272,6 +292,7 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
             matched = true;
         }
     }
+    if (!matched && offset_band()) return finish();
     if (!matched) return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
     if (m.kind != kBandDiagonals) m.slots = m.count;
 

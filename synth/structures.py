@@ -117,3 +117,11 @@ def sub_triangle(N: int, k: int) -> Descriptor:
     items = _box_rows(2, 2, [0, 0]) + [[-1, 1, -1, 1, 0]]
     return Descriptor([N, N], [N, k], _rows(2, 2, items), np.zeros(len(items), np.uint8),
                       name="sub_triangle", meta={"k": k})
+
+
+def offset_band(N: int, lo: int, hi: int) -> Descriptor:
+    """{(i, j) : lo <= j - i <= hi} inside the N x N box (a single diagonal at distance s when
+    lo = hi = s); params = (N,)."""
+    items = _box_rows(2, 1, [0, 0]) + [[-1, 1, 0, -lo], [1, -1, 0, hi]]
+    return Descriptor([N, N], [N], _rows(2, 1, items), np.zeros(len(items), np.uint8),
+                      name="offset_band", meta={"lo": lo, "hi": hi})

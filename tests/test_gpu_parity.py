@@ -21,7 +21,8 @@ INDEX_CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(97)
                st.lower_triangle(61), st.tetrahedron(1), st.tetrahedron(2), st.tetrahedron(48),
                st.upper_half_cube(9, 14, 5), st.upper_half_cube(14, 9, 3), st.dense_box([5, 6, 7]),
                st.band(50, 4), st.band(7, 0), st.upper_triangle(1000), st.band_exact(50, 4), st.band_exact(9, 4),
-               st.band_exact(300, 32), st.sub_triangle(60, 13), st.sub_triangle(9, 1), st.sub_triangle(300, 299)]
+               st.band_exact(300, 32), st.sub_triangle(60, 13), st.sub_triangle(9, 1), st.sub_triangle(300, 299),
+               st.offset_band(50, 7, 7), st.offset_band(50, -20, 3), st.offset_band(33, -30, 28), st.offset_band(200, -199, -1)]
 
 
 @pytest.mark.parametrize("desc", INDEX_CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -109,7 +110,8 @@ PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33),
               st.upper_triangle(1000), st.upper_triangle(130, True), st.lower_triangle(77),
               st.tetrahedron(2), st.tetrahedron(37), st.upper_half_cube(11, 17, 3),
               st.upper_half_cube(17, 11, 6), st.dense_box([6, 10]), st.band_exact(11, 5), st.band_exact(130, 7),
-              st.band_exact(1000, 32), st.sub_triangle(11, 4), st.sub_triangle(130, 77), st.sub_triangle(1000, 333)]
+              st.band_exact(1000, 32), st.sub_triangle(11, 4), st.sub_triangle(130, 77), st.sub_triangle(1000, 333),
+              st.offset_band(40, 9, 9), st.offset_band(130, -50, 7), st.offset_band(1000, -3, 40), st.offset_band(90, -85, 80)]
 
 
 @pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
@@ -214,6 +216,101 @@ def test_trmv_sub_triangle(N, k):
     dastac.contract("ij,j->i", s, pk, [xs], ys, batch=batch)
     for b in range(batch):
         assert rel_err(ys[b].cpu().numpy(), refs[b][0], refs[b][1]) <= TOL_F32
+
+
+def _trapezoid(M, N):
+    """{(i, j) : 0 <= i < M, i <= j < N} with M < N."""
+    rows = np.array([[1, 0, 0, 0, 0], [-1, 0, 1, 0, -1], [0, 1, 0, 0, 0], [0, -1, 0, 1, -1], [-1, 1, 0, 0, 0]], dtype=np.int64)
+    return st.Descriptor([M, N], [M, N], rows, np.zeros(len(rows), np.uint8), name="trapezoid")
+
+
+ROWSPAN_CASES = [st.dense_box([1, 1]), st.dense_box([7, 13]), st.dense_box([1, 50]), _trapezoid(20, 70), st.dense_box([300, 70]), st.dense_box([64, 1000]),
+                 st.lower_triangle(1), st.lower_triangle(33), st.lower_triangle(600), st.band_exact(9, 4),
+                 st.band_exact(500, 32), st.band_exact(2000, 1), st.offset_band(100, 17, 17), st.offset_band(100, -99, -99),
+                 st.offset_band(1000, -30, 200), st.offset_band(700, -699, -1), st.offset_band(257, -200, 190),
+                 st.offset_band(4096, 1024, 1024)]
+
+
+@pytest.mark.parametrize("desc", ROWSPAN_CASES, ids=lambda d: f"{d.name}{d.dims}{sorted(d.meta.items()) if d.meta else ''}")
+def test_matvec_row_contiguous_classes(desc):
+    """y = A x for the classes whose rows are stored contiguously: dense, lower, exact and offset bands."""
+    s = dastac.Structure(desc)
+    M, N = desc.dims
+    A = synth.dense(0, 0, (M, N))
+    x = synth.dense(0, 1, (N,))
+    ref, ref_abs = oracle.matvec(desc, A, x)
+    packed = packed_dev(s, oracle.pack(desc, A))
+    y = torch.full((M,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    y0 = synth.dense(0, 2, (M,))
+    y2 = dev(y0)
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y2, accumulate=True)
+    assert rel_err(y2.cpu().numpy(), ref + y0, ref_abs + np.abs(y0)) <= TOL_F32
+    batch = 3
+    cap = s.capacity(torch.float32)
+    pk = torch.full((batch, cap + 4), float("nan"), device="cuda")[:, :cap]
+    xs = torch.empty((batch, N + 2), device="cuda")[:, :N]
+    ys = torch.full((batch, M + 1), float("nan"), device="cuda")[:, :M]
+    refs = []
+    for b in range(batch):
+        Ab, xb = synth.dense(40 + b, 0, (M, N)), synth.dense(40 + b, 1, (N,))
+        pk[b, : s.nnz] = dev(oracle.pack(desc, Ab))
+        xs[b] = dev(xb)
+        refs.append(oracle.matvec(desc, Ab, xb))
+    dastac.contract("ij,j->i", s, pk, [xs], ys, batch=batch)
+    for b in range(batch):
+        assert rel_err(ys[b].cpu().numpy(), refs[b][0], refs[b][1]) <= TOL_F32
+
+
+@pytest.mark.parametrize("N,sdist", [(64, 1), (1000, 37), (4096, 512), (5000, 4999)])
+def test_strided_band_one_buffer_per_summand(N, sdist):
+    """The strided band of Section 6.4, B_U = (j = i) + (j - i = s) + (i - j = s): three summands, each with
+    its own packed buffer, evaluated one after the other into the same y."""
+    A = synth.dense(7, 0, (N, N))
+    x = synth.dense(7, 1, (N,))
+    y = torch.full((N,), float("nan"), device="cuda")
+    ref = np.zeros(N)
+    ref_abs = np.zeros(N)
+    total = 0
+    for k, (lo, hi) in enumerate([(0, 0), (sdist, sdist), (-sdist, -sdist)]):
+        desc = st.offset_band(N, lo, hi)
+        s = dastac.Structure(desc)
+        total += s.nnz
+        packed = dastac.pack(s, dev(A))
+        assert np.array_equal(packed.cpu().numpy()[: s.nnz], oracle.pack(desc, A))
+        dastac.contract("ij,j->i", s, packed, [dev(x)], y, accumulate=k > 0)
+        r, ra = oracle.matvec(desc, A, x)
+        ref += r
+        ref_abs += ra
+    assert total == N + 2 * (N - sdist)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    # the same numbers from the dense definition of the three diagonals
+    i = np.arange(N)
+    dense_ref = A[i, i].astype(np.float64) * x
+    dense_ref[: N - sdist] += A[i[: N - sdist], i[: N - sdist] + sdist].astype(np.float64) * x[sdist:]
+    dense_ref[sdist:] += A[i[sdist:], i[sdist:] - sdist].astype(np.float64) * x[: N - sdist]
+    np.testing.assert_allclose(ref, dense_ref, rtol=1e-12, atol=1e-12)
+
+
+def test_leslie_matrix_first_row_plus_subdiagonal():
+    """A Leslie matrix (Table 1, SpMV_L): a dense first row and the sub-diagonal, as two summands."""
+    N = 3000
+    A = synth.dense(8, 0, (N, N))
+    x = synth.dense(8, 1, (N,))
+    y = torch.zeros(N, device="cuda")
+    first = st.dense_box([1, N])
+    s1 = dastac.Structure(first)
+    dastac.contract("ij,j->i", s1, packed_dev(s1, A[0]), [dev(x)], y[:1])
+    sub = st.offset_band(N, -1, -1)
+    s2 = dastac.Structure(sub)
+    dastac.contract("ij,j->i", s2, packed_dev(s2, oracle.pack(sub, A)), [dev(x)], y, accumulate=True)
+    r1, a1 = oracle.matvec(first, A[:1], x)
+    r2, a2 = oracle.matvec(sub, A, x)
+    ref, ref_abs = r2.copy(), a2.copy()
+    ref[0] += r1[0]
+    ref_abs[0] += a1[0]
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
 
 
 def test_trmv_closed_forms():

@@ -33,7 +33,10 @@ CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(37), st.u
          st.upper_half_cube(5, 5, 1), st.dense_box([3, 4]), st.dense_box([2, 3, 4]), st.dense_box([7]),
          st.band_exact(1, 0), st.band_exact(7, 0), st.band_exact(7, 3), st.band_exact(8, 3), st.band_exact(23, 4),
          st.band_exact(40, 11), st.sub_triangle(7, 3), st.sub_triangle(6, 1), st.sub_triangle(9, 8),
-         st.sub_triangle(40, 17), st.sub_triangle(5, 5)]
+         st.sub_triangle(40, 17), st.sub_triangle(5, 5), st.offset_band(9, 3, 3), st.offset_band(9, -4, -4),
+         st.offset_band(12, -2, 5), st.offset_band(12, -9, 1), st.offset_band(7, -6, -1), st.offset_band(10, -8, 8),
+         st.offset_band(11, 2, 6), st.offset_band(6, -5, 4), st.offset_band(1, 0, 0), st.offset_band(8, -7, -7),
+         st.band_exact(6, 3), st.band_exact(9, 7)]
 
 
 @pytest.mark.parametrize("desc", CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -106,10 +109,10 @@ def test_recognition_is_independent_of_how_rows_are_written():
     assert oracle.count(empty) == 0
     # zero extent
     assert dastac.Structure(st.upper_triangle(0)).nnz == 0
-    # band without the padded layout: the exact row-after-row pack; as wide as the matrix: refused
+    # band without the padded layout: the exact row-after-row pack; wider than half the matrix: the general
+    # offset band (same layout rule); in the padded layout a band as wide as the matrix is refused
     assert dastac.Structure(st.band(8, 2, padded_diagonals=False)).kind == dastac.KIND_BAND_EXACT
-    with pytest.raises(dastac.DastacError):
-        dastac.Structure(st.band(8, 4, padded_diagonals=False))
+    assert dastac.Structure(st.band(8, 4, padded_diagonals=False)).kind == dastac.KIND_BAND_OFFSETS
     with pytest.raises(dastac.DastacError):
         dastac.Structure(st.band(8, 7))
     # symmetric swap only on a square upper triangle
@@ -227,12 +230,40 @@ def test_sub_triangle_kind_and_limits():
         dastac.Structure(sym)
 
 
+def test_offset_band_kinds_and_large_sizes():
+    """lo <= j - i <= hi: a single off-diagonal is a per-summand buffer of the strided band (Section 6.4)."""
+    N, sdist = 2 ** 16, 2 ** 12
+    up = dastac.Structure(st.offset_band(N, sdist, sdist))
+    dn = dastac.Structure(st.offset_band(N, -sdist, -sdist))
+    assert up.kind == dn.kind == dastac.KIND_BAND_OFFSETS and up.nnz == dn.nnz == N - sdist
+    assert dastac.rank(up, (5, 5 + sdist)) == 5 and dastac.rank(dn, (sdist + 7, 7)) == 7
+    assert dastac.unrank(dn, 0) == (sdist, 0) and dastac.unrank(up, N - sdist - 1) == (N - sdist - 1, N - 1)
+    # classes with faster kernels keep their kind: the symmetric band, the diagonal, the sub-triangle, the triangles
+    assert dastac.Structure(st.offset_band(64, -3, 3)).kind == dastac.KIND_BAND_EXACT
+    assert dastac.Structure(st.offset_band(64, 0, 0)).kind == dastac.KIND_BAND_EXACT
+    assert dastac.Structure(st.offset_band(64, 5, 63)).kind == dastac.KIND_UPPER_SHIFTED
+    assert dastac.Structure(st.offset_band(64, 0, 63)).kind == dastac.KIND_UPPER
+    assert dastac.Structure(st.offset_band(64, -63, 0)).kind == dastac.KIND_LOWER
+    assert dastac.Structure(st.offset_band(64, -63, 63)).kind == dastac.KIND_DENSE
+    assert dastac.Structure(st.offset_band(64, 70, 80)).nnz == 0
+    strictly_lower = dastac.Structure(st.offset_band(64, -63, -1))
+    assert strictly_lower.kind == dastac.KIND_BAND_OFFSETS and strictly_lower.nnz == 64 * 63 // 2
+    big = dastac.Structure(st.offset_band(2 ** 20, -1000, 37))
+    assert big.nnz == oracle_count_offset_band(2 ** 20, -1000, 37)
+    for p in (0, 1, 500_500, 123_456_789, big.nnz - 1):
+        assert dastac.rank(big, dastac.unrank(big, p)) == p
+
+
+def oracle_count_offset_band(N, lo, hi):
+    """Points of lo <= j - i <= hi in the N x N box, one diagonal at a time (diagonal d has N - |d| points)."""
+    return sum(N - abs(d) for d in range(lo, hi + 1) if abs(d) < N)
+
+
 def test_exact_band_limits_and_kind():
     s = dastac.Structure(st.band_exact(9, 2))
     assert s.kind == dastac.KIND_BAND_EXACT and s.nnz == s.slots == 5 * 9 - 2 * 3
-    with pytest.raises(dastac.DastacError) as e:       # 2w + 1 > N: the clipped pieces would overlap
-        dastac.Structure(st.band_exact(6, 3))
-    assert e.value.status == 2
+    wide = dastac.Structure(st.band_exact(6, 3))        # 2w + 1 > N: rows clipped on both sides -> the general offset band
+    assert wide.kind == dastac.KIND_BAND_OFFSETS and wide.nnz == 7 * 6 - 3 * 4
     big = dastac.Structure(st.band_exact(2 ** 20, 1000))
     assert dastac.unrank(big, big.nnz - 1) == (2 ** 20 - 1, 2 ** 20 - 1)
     for p in (0, 1, 500_500, 123_456_789, big.nnz - 2):
