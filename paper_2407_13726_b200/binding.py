@@ -140,7 +140,7 @@ class Structure:
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
-        if h:
+        if h and _lib is not None:  # module globals are already cleared at interpreter shutdown
             _lib.dastac_structure_destroy(h)
 
     def capacity(self, dtype: torch.dtype) -> int:

@@ -28,11 +28,21 @@ rowspan_mv_kernel(const IndexMap m, const float* __restrict__ A, const float* __
         if (row_span(m, idx, jlo, jhi, pbase)) {
             const float* a = A + pbase;  // a[j] = A(row, j)
             int64_t j = jlo + sub;
-            for (; j + L < jhi; j += 2 * L) {
-                acc0 = fmaf(__ldg(a + j), __ldg(x + j), acc0);
-                acc1 = fmaf(__ldg(a + j + L), __ldg(x + j + L), acc1);
+            // eight independent loads of each operand per lane keep enough bytes in flight for long rows
+            for (; j + 7 * L < jhi; j += 8 * L) {
+                float av[8], xv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    av[u] = __ldg(a + j + u * L);
+                    xv[u] = __ldg(x + j + u * L);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; u += 2) {
+                    acc0 = fmaf(av[u], xv[u], acc0);
+                    acc1 = fmaf(av[u + 1], xv[u + 1], acc1);
+                }
             }
-            if (j < jhi) acc0 = fmaf(__ldg(a + j), __ldg(x + j), acc0);
+            for (; j < jhi; j += L) acc0 = fmaf(__ldg(a + j), __ldg(x + j), acc0);
         }
     }
     float acc = acc0 + acc1;
