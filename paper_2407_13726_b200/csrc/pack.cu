@@ -200,9 +200,29 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
         const int64_t ps = pbase + jlo, pe = pbase + jhi;              // the row's span in the packed stream
         const T* drow = dense + dense_row_offset(m, st, idx) - pbase;  // drow[p]: element stored at position p
         const int64_t c_first = ps / E;
+        // A packed chunk is 16-byte aligned and every chunk is 16 bytes, so the dense source of all
+        // chunks of a row has the same misalignment: one shift and one aligned base per item.
+        const uintptr_t d_first = reinterpret_cast<uintptr_t>(drow + c_first * E);
+        const uint32_t sh_row = (uint32_t)(d_first & 15);
+        const uint4* srcq = reinterpret_cast<const uint4*>(d_first - sh_row);  // srcq[c - c_first]: granule under chunk c
+        uint4* dstq = reinterpret_cast<uint4*>(packed) + c_first;
         for (int win = grp * windows_per_group; win < (grp + 1) * windows_per_group; ++win) {
             const int64_t c0 = c_first + (int64_t)win * (32 * kUnroll) + lane;
             if ((c0 - lane) * E >= pe) break;
+            if ((c0 - lane) * E >= ps && (c0 - lane + 32 * kUnroll) * E <= pe) {
+                // the whole window lies inside the row: no per-chunk tests, addresses are one pointer plus constants
+                const uint4* sp = srcq + (int64_t)win * (32 * kUnroll) + lane;
+                uint4* dp = dstq + (int64_t)win * (32 * kUnroll) + lane;
+                uint4 lo[kUnroll], hi[kUnroll];
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    lo[u] = __ldg(sp + 32 * u);
+                    hi[u] = sh_row ? __ldg(sp + 32 * u + 1) : zero4;
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) dp[32 * u] = realign16(lo[u], hi[u], sh_row);
+                continue;
+            }
             uint4 lo[kUnroll], hi[kUnroll];
             uint32_t sh[kUnroll];
 #pragma unroll
@@ -279,6 +299,30 @@ unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ d
         for (int win = grp * windows_per_group; win < (grp + 1) * windows_per_group; ++win) {
             const int jfirst = (win * (32 * kUnroll) + lane) * E;
             if (win * (32 * kUnroll) * E >= inner) break;
+            const int wlo = win * (32 * kUnroll) * E, whi = wlo + 32 * kUnroll * E;  // columns of the window
+            if (whi <= inner && (whi <= jlo || wlo >= jhi)) {
+                // nothing of the set in this window: plain zero fill
+                uint4* dp = reinterpret_cast<uint4*>(drow + jfirst);
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) dp[32 * u] = zero4;
+                continue;
+            }
+            if (wlo >= jlo && whi <= jhi && whi <= inner && whi - E <= jsafe) {
+                // the whole window is stored: one shift per row, addresses are one pointer plus constants
+                const uintptr_t paddr = reinterpret_cast<uintptr_t>(prow + jfirst);
+                const uint32_t shw = (uint32_t)(paddr & 15);
+                const uint4* sp = reinterpret_cast<const uint4*>(paddr - shw);
+                uint4* dp = reinterpret_cast<uint4*>(drow + jfirst);
+                uint4 lo[kUnroll], hi[kUnroll];
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    lo[u] = __ldg(sp + 32 * u);
+                    hi[u] = shw ? __ldg(sp + 32 * u + 1) : zero4;
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) dp[32 * u] = realign16(lo[u], hi[u], shw);
+                continue;
+            }
             uint4 lo[kUnroll], hi[kUnroll];
             uint32_t sh[kUnroll];
 #pragma unroll
