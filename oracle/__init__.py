@@ -66,10 +66,11 @@ def _load():
         lib.orc_mttkrp.argtypes = [P, i64, vp, vp, vp, vp, i64, vp, vp]
         lib.orc_ttm.argtypes = [P, i64, vp, vp, vp, i64, vp, vp]
         lib.orc_moment2.argtypes = [P, ctypes.c_int, i64, vp, vp, i64, vp, vp]
+        lib.orc_moment3.argtypes = [P, ctypes.c_int, i64, vp, vp, i64, vp, vp]
         lib.orc_num_threads.restype = ctypes.c_int
         for name in ("orc_rank_table", "orc_unrank_table", "orc_pack", "orc_unpack", "orc_band_pack",
                      "orc_band_unpack", "orc_band_slot_table", "orc_matvec", "orc_symv",
-                     "orc_matmat", "orc_mttkrp", "orc_ttm", "orc_moment2"):
+                     "orc_matmat", "orc_mttkrp", "orc_ttm", "orc_moment2", "orc_moment3"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -270,5 +271,21 @@ def moment2(desc, B, sel=None):
     assert B.ndim == 2 and B.shape[1] == n and int(h.dims[0]) == n
     out, out_abs = np.empty((len(sel), n)), np.empty((len(sel), n))
     _load().orc_moment2(h.ref, int(is_bf16), len(sel), sel.ctypes.data, B.ctypes.data, B.shape[0],
+                        out.ctypes.data, out_abs.ctypes.data)
+    return out, out_abs
+
+
+def moment3(desc, B, sel=None):
+    """``A3[i1][i2][i3] = sum_x [(i1,i2,i3) in set] B[x][i1] B[x][i2] B[x][i3]`` for the slabs ``i1`` in
+    ``sel``; B is ``M x n`` (fp32, or uint16 holding bf16 bit patterns).  Returns ``[len(sel), n, n]``
+    arrays (dense slabs, zero outside the set)."""
+    h = _Held(desc)
+    sel = _sel(sel, int(h.dims[0]))
+    is_bf16 = B.dtype == np.uint16
+    B = np.ascontiguousarray(B) if is_bf16 else _f32(B)
+    n = int(h.dims[1])
+    assert B.ndim == 2 and B.shape[1] == n and int(h.dims[0]) == n and int(h.dims[2]) == n
+    out, out_abs = np.empty((len(sel), n, n)), np.empty((len(sel), n, n))
+    _load().orc_moment3(h.ref, int(is_bf16), len(sel), sel.ctypes.data, B.ctypes.data, B.shape[0],
                         out.ctypes.data, out_abs.ctypes.data)
     return out, out_abs

@@ -350,6 +350,34 @@ void orc_moment2(const orc_desc* d, int is_bf16, int64_t nsel, const int64_t* se
     }
 }
 
+/* A3[i1][i2][i3] = sum_x [ (i1, i2, i3) in set ] B[x][i1] * B[x][i2] * B[x][i3]
+ * (A^k(i_1..i_k) := B(x,i_1) * ... * B(x,i_k) with k = 3, Table 1 "Polynomial Regression"; the set is
+ * the unique part i1 <= i2 <= i3 of the fully symmetric result, the hyper-triangular domain of
+ * Section 1).  out[s] is slab sel[s] of the result as a dense n x n array, zero outside the set. */
+void orc_moment3(const orc_desc* d, int is_bf16, int64_t nsel, const int64_t* sel, const void* B,
+                 int64_t M, double* out, double* out_abs) {
+    const int64_t n = d->dims[1];
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        for (int64_t i2 = 0; i2 < n; ++i2) {
+            for (int64_t i3 = 0; i3 < n; ++i3) {
+                double acc = 0.0, acc_abs = 0.0;
+                int64_t idx[3] = {sel[s], i2, i3};
+                if (in_domain(d, idx)) {
+                    for (int64_t x = 0; x < M; ++x) {
+                        double p = widen(B, x * n + sel[s], is_bf16) * widen(B, x * n + i2, is_bf16) *
+                                   widen(B, x * n + i3, is_bf16);
+                        acc += p;
+                        acc_abs += fabs(p);
+                    }
+                }
+                out[(s * n + i2) * n + i3] = acc;
+                out_abs[(s * n + i2) * n + i3] = acc_abs;
+            }
+        }
+    }
+}
+
 /* Thread count the contractions above will use. */
 #ifdef _OPENMP
 #include <omp.h>

@@ -440,3 +440,45 @@ def test_moment2_packed_symmetric_output():
     packed = oracle.pack(d, out)
     assert packed.shape == (n * (n + 1) // 2,)
     assert packed[oracle.rank_point(d, (2, 5))] == out[2, 5] and packed[n] == out[1, 1]
+
+
+def test_moment3_packed_tetrahedral_output():
+    """Degree-3 moments: A3(i1,i2,i3) = sum_x B(x,i1) B(x,i2) B(x,i3), kept on i1 <= i2 <= i3."""
+    M, n = 23, 7
+    d = st.tetrahedron(n)
+    B = synth.dense(9, 0, (M, n))
+    out, outa = oracle.moment3(d, B)
+    B64 = B.astype(np.float64)
+    full = np.einsum("xi,xj,xk->ijk", B64, B64, B64)          # library routine, all n^3 entries
+    i, j, k = np.indices((n, n, n))
+    keep = (i <= j) & (j <= k)
+    np.testing.assert_allclose(out, np.where(keep, full, 0), atol=1e-12)
+    np.testing.assert_allclose(outa, np.where(keep, np.einsum("xi,xj,xk->ijk", *(np.abs(B64),) * 3), 0), rtol=1e-13)
+    assert (out[~keep] == 0).all()
+    # closed forms: one sample gives the triple outer product; all ones give M on the set;
+    # the body diagonal holds the sums of cubes; a constant third factor reduces it to the degree-2 moments
+    one, _ = oracle.moment3(d, B[:1])
+    assert np.array_equal(one, np.where(keep, np.einsum("i,j,k->ijk", B64[0], B64[0], B64[0]), 0))
+    ones, _ = oracle.moment3(d, np.ones((M, n), np.float32))
+    assert np.array_equal(ones, np.where(keep, float(M), 0.0))
+    np.testing.assert_allclose(out[np.arange(n), np.arange(n), np.arange(n)], (B64 ** 3).sum(0), rtol=1e-13)
+    Bc = B.copy()
+    Bc[:, n - 1] = 1.0                                           # last feature = the constant 1
+    o3, _ = oracle.moment3(d, Bc)
+    o2, _ = oracle.moment2(st.upper_triangle(n, symmetric=True), Bc)
+    np.testing.assert_allclose(o3[:, :, n - 1], o2, atol=1e-12)
+    # the sum runs over the first index of B
+    Bs = synth.dense(9, 1, (n, n))
+    a1, _ = oracle.moment3(d, Bs)
+    a2, _ = oracle.moment3(d, np.ascontiguousarray(Bs.T))
+    assert np.abs(a1 - a2).max() > 1e-3
+    # selected slabs; bf16 bit patterns widened exactly; packed order of the result
+    sel = np.array([5, 0, 2])
+    sub, _ = oracle.moment3(d, B, sel=sel)
+    assert np.array_equal(sub, out[sel])
+    bits = synth.dense(9, 2, (M, n), bf16=True)
+    wide = (bits.astype(np.uint32) << 16).view(np.float32)
+    assert np.array_equal(oracle.moment3(d, bits)[0], oracle.moment3(d, wide)[0])
+    packed = oracle.pack(d, out)
+    assert packed.shape == (n * (n + 1) * (n + 2) // 6,)
+    assert packed[oracle.rank_point(d, (1, 3, 4))] == out[1, 3, 4] and packed[0] == out[0, 0, 0]
