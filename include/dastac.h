@@ -193,6 +193,11 @@ typedef struct {
  *                   n x n upper triangle (the unique part i <= j of the symmetric result, Section 2;
  *                   with or without the redundancy swap), fp32 accumulation.  Positions of the packed
  *                   buffer beyond the set's count are not written.
+ *   "xi,xj,xk->ijk" in[0] = in[1] = in[2] = dense B     bf16 -> f32  A3, the degree-3 moments (k = 3 of the same
+ *                   rule); `out` is PACKED: out->structure is the n x n x n tetrahedron i <= j <= k (the
+ *                   hyper-triangular domain of Section 1).  The pairwise products B(x,i) B(x,j) are
+ *                   rounded to bf16 once before they meet the third factor on the tensor cores
+ *                   (relative error 2^-9 per term); accumulation is fp32.  Needs workspace.
  * accumulate: 0 -> out = result (the library zero-fills where it needs to), 1 -> out += result.
  * workspace: device scratch of at least dastac_contract_workspace bytes, 256-byte aligned; may be
  *            NULL when that size is 0.  Its contents are undefined afterwards.

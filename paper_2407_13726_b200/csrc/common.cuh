@@ -58,5 +58,8 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
 size_t moment2_workspace_bytes(int64_t M, int64_t n, int64_t ldb);
 dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
                                   int accumulate, void* workspace, int32_t* err_word, cudaStream_t st);
+size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb);
+dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
+                                  int accumulate, void* workspace, int32_t* err_word, cudaStream_t st);
 
 }  // namespace dastac

@@ -7,7 +7,7 @@
 namespace dastac {
 namespace {
 
-enum ExprClass { kMatVec, kMatMat, kMttkrp, kTtm, kMoment2, kNoExpr };
+enum ExprClass { kMatVec, kMatMat, kMttkrp, kTtm, kMoment2, kMoment3, kNoExpr };
 
 ExprClass parse_expr(const char* e) {
     if (!e) return kNoExpr;
@@ -16,6 +16,7 @@ ExprClass parse_expr(const char* e) {
     if (!std::strcmp(e, "ijk,jr,kr->ir")) return kMttkrp;
     if (!std::strcmp(e, "ijl,kl->ijk")) return kTtm;
     if (!std::strcmp(e, "xi,xj->ij")) return kMoment2;
+    if (!std::strcmp(e, "xi,xj,xk->ijk")) return kMoment3;
     return kNoExpr;
 }
 
@@ -65,20 +66,23 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
     p.cls = parse_expr(expr);
     if (!in || !out || n_in < 1) return DASTAC_ERR_INVALID_ARG;
     if (p.cls == kNoExpr) return DASTAC_ERR_UNSUPPORTED_EXPR;
-    const int want_in = p.cls == kMttkrp ? 3 : 2;  // the tensor-times-matrix rule has two inputs as well
+    const int want_in = (p.cls == kMttkrp || p.cls == kMoment3) ? 3 : 2;  // the tensor-times-matrix rule has two inputs as well
     if (n_in != want_in) return DASTAC_ERR_INVALID_ARG;
-    if (p.cls == kMoment2) {
-        // dense B (samples x features) twice, packed unique part of the symmetric result out
-        if (!dense_ok(in[0], 2) || !dense_ok(in[1], 2)) return DASTAC_ERR_INVALID_ARG;
+    if (p.cls == kMoment2 || p.cls == kMoment3) {
+        // dense B (samples x features) as every factor, packed unique part of the symmetric result out
+        for (int k = 0; k < n_in; ++k)
+            if (!dense_ok(in[k], 2)) return DASTAC_ERR_INVALID_ARG;
         if (!out->structure) return DASTAC_ERR_UNSUPPORTED_EXPR;
-        // both factors are the same tensor: only then is the result symmetric
-        if (in[0].data != in[1].data || in[0].space != in[1].space || in[0].dtype != in[1].dtype ||
-            in[0].dims[0] != in[1].dims[0] || in[0].dims[1] != in[1].dims[1] ||
-            in[0].strides[0] != in[1].strides[0] || in[0].strides[1] != in[1].strides[1])
-            return DASTAC_ERR_UNSUPPORTED_EXPR;
+        // all factors are the same tensor: only then is the result symmetric
+        for (int k = 1; k < n_in; ++k)
+            if (in[0].data != in[k].data || in[0].space != in[k].space || in[0].dtype != in[k].dtype ||
+                in[0].dims[0] != in[k].dims[0] || in[0].dims[1] != in[k].dims[1] ||
+                in[0].strides[0] != in[k].strides[0] || in[0].strides[1] != in[k].strides[1])
+                return DASTAC_ERR_UNSUPPORTED_EXPR;
         const IndexMap& mo = out->structure->map;
-        if (!(mo.kind == kUpper && mo.rank == 2 && mo.dims[0] == mo.dims[1]) && mo.kind != kEmpty)
+        if (p.cls == kMoment2 && !(mo.kind == kUpper && mo.rank == 2 && mo.dims[0] == mo.dims[1]) && mo.kind != kEmpty)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (p.cls == kMoment3 && mo.kind != kTetrahedron && mo.kind != kEmpty) return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (in[0].dtype != DASTAC_BF16 || out->dtype != DASTAC_F32) return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (batch_of(in[0]) != 1 || batch_of(*out) != 1) return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (!(out->space == DASTAC_MEM_DEVICE || out->space == DASTAC_MEM_HOST)) return DASTAC_ERR_INVALID_ARG;
@@ -87,9 +91,10 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         p.map = &mo;
         p.N = mo.dims[0];
         p.R = in[0].dims[0];  // samples
-        p.scratch = moment2_workspace_bytes(p.R, p.N, in[0].strides[0]);
+        p.scratch = p.cls == kMoment3 ? moment3_workspace_bytes(p.R, p.N, in[0].strides[0])
+                                      : moment2_workspace_bytes(p.R, p.N, in[0].strides[0]);
         size_t off = (size_t)round_up((int64_t)p.scratch, 256);
-        p.stage_off[0] = p.stage_off[1] = off;  // one staged copy serves both factors
+        p.stage_off[0] = p.stage_off[1] = p.stage_off[2] = off;  // one staged copy serves every factor
         if (in[0].space == DASTAC_MEM_HOST) off += (size_t)round_up(total_bytes(in[0]), 256);
         p.stage_off[3] = off;
         if (out->space == DASTAC_MEM_HOST) off += (size_t)round_up(total_bytes(*out), 256);
@@ -224,8 +229,8 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     // Resolve device pointers (staging host operands).
     const void* dev_in[3] = {nullptr, nullptr, nullptr};
     for (int k = 0; k < n_in; ++k) {
-        if (p.cls == kMoment2 && k == 1) {  // the same tensor as in[0]
-            dev_in[1] = dev_in[0];
+        if ((p.cls == kMoment2 || p.cls == kMoment3) && k >= 1) {  // the same tensor as in[0]
+            dev_in[k] = dev_in[0];
             continue;
         }
         const int64_t bytes = total_bytes(in[k]);
@@ -252,7 +257,12 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     if (out_bytes > 0 && !aligned16(dev_out)) return DASTAC_ERR_ALIGNMENT;
     void* scratch = p.scratch ? workspace : nullptr;
 
-    if (p.cls == kMoment2) {
+    if (p.cls == kMoment3) {
+        st = (m.kind == kEmpty || out_bytes == 0)
+                 ? DASTAC_OK
+                 : launch_moment3_bf16(m, dev_in[0], in[0].strides[0], p.R, (float*)dev_out, accumulate, scratch,
+                                       err_word, cs);
+    } else if (p.cls == kMoment2) {
         st = (m.kind == kEmpty || out_bytes == 0)
                  ? DASTAC_OK
                  : launch_moment2_bf16(m, dev_in[0], in[0].strides[0], p.R, (float*)dev_out, accumulate, scratch,

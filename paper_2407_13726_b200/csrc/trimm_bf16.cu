@@ -141,7 +141,11 @@ struct Params {
     const uint8_t* tiles;        // staged tile images, 16 KiB each
     float* C;
     int64_t N, ncols, ldc;
-    int64_t M;           // second-moment form only: number of samples (rows of B)
+    int64_t M;           // moment forms only: number of samples (rows of B)
+    // degree-3 moments only: slabs i1 = i1_first .. i1_first + slots - 1 are computed by this launch; the
+    // products Z(x, slot, i2) = B(x, i1) B(x, i2) sit in a matrix with slot_pitch columns per slot
+    int32_t i1_first, slots, slot_pitch;
+    int64_t tiles_total;
     int64_t cap_elems;   // capacity of the packed buffer in elements (multiple of 8)
     int32_t row_blocks, col_blocks, k_blocks;
     int32_t accumulate;
@@ -254,7 +258,17 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // half of the "B" operand, and the instruction descriptor marks A as M-major.  Tiles are the
 // 256 x 256 blocks (P, J) with J >= P, every one with the full K loop over the samples; the
 // epilogue writes element (i1, i2) at rowbase(i1) + i2 of the packed triangle and skips i2 < i1.
-template <bool MOMENT2>
+//
+// MODE 2 (degree-3 moments A3(i1,i2,i3) = sum_x B(x,i1) B(x,i2) B(x,i3) on i1 <= i2 <= i3, the
+// hyper-triangular domain of Section 1, stored as the packed tetrahedron): for a fixed i1 the slab is
+// the degree-2 product of Z_i1(x, i2) = B(x,i1) B(x,i2) with B, kept on i1 <= i2 <= i3.  A launch
+// covers a run of slabs; the "A" operand comes from the matrix of products Z (one column block
+// per slab, written by a small kernel beforehand), the "B" operand from B; tiles are (slab, P, J)
+// with P from the block that holds row i1 and J >= P; the epilogue writes at the tetrahedral
+// position pbase(i1, i2) + i3.
+enum PairMode : int { kModeTrimm = 0, kModeMoment2 = 1, kModeMoment3 = 2 };
+
+template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
 trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const Params p) {
@@ -302,11 +316,24 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // Tile t = (pair P, column block J), P ascending = K length descending, dealt to the clusters in
     // boustrophedon order.
     const int pair_blocks = (p.row_blocks + 1) >> 1;
-    const int64_t tiles = MOMENT2 ? (int64_t)pair_blocks * (pair_blocks + 1) / 2 : (int64_t)pair_blocks * p.col_blocks;
-    // tile index -> (row-block pair P, column block J); MOMENT2: row P of the block triangle holds J = P ..
-    auto decode = [&](int64_t t, int& P, int& J) {
+    constexpr bool MOMENT2 = MODE != kModeTrimm;  // both moment forms share the operand handling of degree 2
+    const int64_t tiles = MODE == kModeMoment3 ? p.tiles_total
+                          : MOMENT2            ? (int64_t)pair_blocks * (pair_blocks + 1) / 2
+                                               : (int64_t)pair_blocks * p.col_blocks;
+    // tile index -> (slab, row-block pair P, column block J); moments: row P of the block triangle holds J = P ..
+    auto decode = [&](int64_t t, int& P, int& J, int& slot) {
+        slot = 0;
         if (MOMENT2) {
             int r = 0;
+            if (MODE == kModeMoment3) {
+                for (;;) {  // slabs in order; slab i1 uses the block rows from the one that holds row i1
+                    r = (p.i1_first + slot) / (2 * kTileM);
+                    const int64_t cnt = (int64_t)(pair_blocks - r) * (pair_blocks - r + 1) / 2;
+                    if (t < cnt || slot + 1 >= p.slots) break;
+                    t -= cnt;
+                    ++slot;
+                }
+            }
             while (t >= pair_blocks - r) {
                 t -= pair_blocks - r;
                 ++r;
@@ -333,8 +360,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (uint32_t n = 0; n < rounds && ok; ++n) {
                 const int64_t t = tile_of(n);
                 if (t >= tiles) continue;
-                int P, J;
-                decode(t, P, J);
+                int P, J, slot;
+                decode(t, P, J, slot);
                 const int I = 2 * P + (int)rank;
                 // staged tile (I, kb) sits at tile index tile_base + kb; a row block past the end of
                 // the matrix has no tiles and its loads are out of range of the map: zero fill
@@ -350,9 +377,12 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (leader) mbar_arrive_expect_tx(full(s), 2 * kPStageBytes);  // both CTAs' bytes
                     const uint32_t bar = full0 + 8u * s;
                     if (MOMENT2) {
+                        // degree 2: columns of B itself; degree 3: the slab's column block of the products
+                        const int xa = (MODE == kModeMoment3 ? slot * p.slot_pitch : 0) + I * kTileM;
 #pragma unroll
                         for (int q = 0; q < kTileM / 64; ++q)
-                            tma_load_2d_pair(dst + q * (kBlockK * 128), &tmap_b, I * kTileM + q * 64, kb * kBlockK, bar);
+                            tma_load_2d_pair(dst + q * (kBlockK * 128), MODE == kModeMoment3 ? &tmap_a : &tmap_b,
+                                             xa + q * 64, kb * kBlockK, bar);
                     } else {
                         tma_load_2d_pair(dst, &tmap_a, 0, (int)((tile_base + kb) * kTileM), bar);
                     }
@@ -377,8 +407,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (uint32_t n = 0; n < rounds && ok; ++n) {
                 const int64_t t = tile_of(n);
                 if (t >= tiles) continue;
-                int P, J;
-                decode(t, P, J);
+                int P, J, slot;
+                decode(t, P, J, slot);
                 const int acc = tile_n & 1;
                 if (tile_n >= 2 &&
                     !mbar_wait_cluster(tmem_empty(acc), ((tile_n >> 1) - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
@@ -423,8 +453,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (uint32_t n = 0; n < rounds && ok; ++n) {
             const int64_t t = tile_of(n);
             if (t >= tiles) continue;
-            int P, J;
-            decode(t, P, J);
+            int P, J, slot;
+            decode(t, P, J, slot);
             const int I = 2 * P + (int)rank;
             const int acc = tile_n & 1;
             if (!mbar_wait_warp(tmem_full(acc), (tile_n >> 1) & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
@@ -439,7 +469,17 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // packed triangle: (i, j) sits at rowbase(i) + j; keep i <= j < n.  A lane's 32 values
                 // are consecutive in memory but only 4-byte aligned: scalar stores.
                 if (I < p.row_blocks) {
-                    float* prow = p.C + (i < p.N ? upper_row_base(p.N, i) : 0);
+                    // degree 2: row i of the packed triangle.  degree 3: row (i1, i) of the packed
+                    // tetrahedron, whose hoisted base is tet(n) - tet(n-i1) + tri(n-i1) - tri(n-i) - i;
+                    // rows above i1 are not part of the slab.
+                    const int64_t i1 = p.i1_first + slot;
+                    const bool row_live = i < p.N && (MODE != kModeMoment3 || i >= i1);
+                    int64_t rb = 0;
+                    if (row_live)
+                        rb = MODE == kModeMoment3
+                                 ? tet(p.N) - tet(p.N - i1) + tri(p.N - i1) - tri(p.N - i) - i
+                                 : upper_row_base(p.N, i);
+                    float* prow = p.C + rb;
 #pragma unroll 1
                     for (int cc = 0; cc < kTileN / 32; ++cc) {
                         const int64_t col0 = (int64_t)J * kTileN + cc * 32;
@@ -447,7 +487,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         uint32_t r[32];
                         tmem_ld32(taddr + cc * 32, r);
                         tmem_ld_wait();
-                        if (i < p.N) {
+                        if (row_live) {
 #pragma unroll
                             for (int v = 0; v < 32; ++v) {
                                 const int64_t j = col0 + v;
@@ -648,6 +688,8 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     p.ncols = ncols;
     p.ldc = ldc;
     p.M = 0;
+    p.i1_first = p.slots = p.slot_pitch = 0;
+    p.tiles_total = 0;
     p.cap_elems = round_up(m.slots, 8);
     p.row_blocks = (int32_t)((N + kTileM - 1) / kTileM);
     p.col_blocks = (int32_t)((ncols + kTileN - 1) / kTileN);
@@ -672,7 +714,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(trimm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(trimm_pair_kernel<kModeTrimm>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kPSmemBytes) != cudaSuccess)
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
@@ -684,7 +726,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     const int64_t n_tiles = (int64_t)((p.row_blocks + 1) / 2) * p.col_blocks;  // pairs of row blocks x column blocks
     const int64_t max_clusters = sm_count() / 2;
     const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-    trimm_pair_kernel<false><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, p);
+    trimm_pair_kernel<kModeTrimm><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, p);
     return launch_status();
 }
 
@@ -736,6 +778,8 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
     p.ncols = n;
     p.ldc = 0;
     p.M = M;
+    p.i1_first = p.slots = p.slot_pitch = 0;
+    p.tiles_total = 0;
     p.cap_elems = 0;
     p.row_blocks = (int32_t)((n + kTileM - 1) / kTileM);
     p.col_blocks = (int32_t)((n + kTileN - 1) / kTileN);
@@ -747,7 +791,7 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(trimm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(trimm_pair_kernel<kModeMoment2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kPSmemBytes) != cudaSuccess)
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
@@ -756,8 +800,147 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
     const int64_t n_tiles = pb * (pb + 1) / 2;
     const int64_t max_clusters = sm_count() / 2;
     const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-    trimm_pair_kernel<true><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap, tmap, p);  // the first map is not used
+    trimm_pair_kernel<kModeMoment2><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap, tmap, p);  // the first map is not used
     return launch_status();
+}
+
+// ---- degree-3 moments: A3 on i1 <= i2 <= i3, packed tetrahedron out ------------------------------------
+// Z(x, slot * pitch + i2) = bf16(B(x, i1) * B(x, i2)) for i2 >= i1 = i1_first + slot, zero elsewhere in the
+// slot (columns below i1 and the padding up to the pitch).  The product of two bf16 values has 16
+// significant bits; it is rounded to bf16 once, to nearest even.
+__global__ void moment3_products_kernel(const __nv_bfloat16* __restrict__ B, int64_t ldb, int64_t M, int n,
+                                        int i1_first, int slots, int pitch, __nv_bfloat16* __restrict__ Z) {
+    const int chunks = pitch / 8;  // 16-byte chunks per slot
+    const int64_t total = M * slots * (int64_t)chunks;
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(t % chunks);
+        const int64_t q = t / chunks;
+        const int slot = (int)(q % slots);
+        const int64_t x = q / slots;
+        const int i1 = i1_first + slot;
+        const float b1 = __bfloat162float(B[x * ldb + i1]);
+        union {
+            uint4 v;
+            __nv_bfloat16 e[8];
+        } out;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int i2 = 8 * c + e;
+            out.e[e] = (i2 >= i1 && i2 < n) ? __float2bfloat16_rn(b1 * __bfloat162float(B[x * ldb + i2])) : __float2bfloat16_rn(0.f);
+        }
+        *reinterpret_cast<uint4*>(Z + (x * slots + slot) * (int64_t)pitch + 8 * c) = out.v;
+    }
+}
+
+// Slabs computed per launch: as many as keep the matrix of products within kMoment3ZBytes.
+constexpr int64_t kMoment3ZBytes = (int64_t)512 << 20;
+static int64_t moment3_slots(int64_t M, int64_t n) {
+    const int64_t pitch = round_up(n, 128);
+    int64_t s = kMoment3ZBytes / (M * pitch * 2);
+    if (s < 1) s = 1;
+    return s < n ? s : n;
+}
+size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb) {
+    if (M == 0 || n == 0) return 0;
+    size_t bytes = (size_t)round_up(M * moment3_slots(M, n) * round_up(n, 128) * 2, 256);
+    if (ldb % 8 != 0) bytes += (size_t)(M * round_up(n, 8) * 2);
+    return bytes;
+}
+
+dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
+                                  int accumulate, void* workspace, int32_t* err_word, cudaStream_t st) {
+    const int64_t n = mo.N;
+    if (n == 0) return DASTAC_OK;
+    if (M == 0) {
+        if (!accumulate && cudaMemsetAsync(out, 0, (size_t)mo.count * sizeof(float), st) != cudaSuccess)
+            return DASTAC_ERR_CUDA;
+        return DASTAC_OK;
+    }
+    if (!aligned16(B)) return DASTAC_ERR_ALIGNMENT;
+    if (!workspace) return DASTAC_ERR_WORKSPACE;
+    const int64_t pitch = round_up(n, 128), slots_max = moment3_slots(M, n);
+    if (M > 0x7fffffffLL - kBlockK || slots_max * pitch > 0x7fffffffLL - 2 * kTileN) return DASTAC_ERR_OVERFLOW;
+    __nv_bfloat16* Z = (__nv_bfloat16*)workspace;
+    if (ldb % 8 != 0) {
+        uint16_t* copy = (uint16_t*)((uint8_t*)workspace + round_up(M * slots_max * pitch * 2, 256));
+        const int64_t ldd = round_up(n, 8);
+        int64_t blocks = (M * ldd + 255) / 256;
+        if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
+        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, copy, ldd, M, n);
+        dastac_status rs = launch_status();
+        if (rs != DASTAC_OK) return rs;
+        B = copy;
+        ldb = ldd;
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return DASTAC_ERR_CUDA;
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBlockK};
+    const cuuint32_t estr[2] = {1, 1};
+    CUtensorMap tmap_b;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)M};
+        const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
+        if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DASTAC_ERR_CUDA;
+    }
+    static bool attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(trimm_pair_kernel<kModeMoment3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kPSmemBytes) != cudaSuccess)
+            return DASTAC_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    Params p;
+    p.A = nullptr;
+    p.tiles = nullptr;
+    p.C = out;
+    p.N = n;
+    p.ncols = n;
+    p.ldc = 0;
+    p.M = M;
+    p.cap_elems = 0;
+    p.row_blocks = (int32_t)((n + kTileM - 1) / kTileM);
+    p.col_blocks = (int32_t)((n + kTileN - 1) / kTileN);
+    p.k_blocks = (int32_t)((M + kBlockK - 1) / kBlockK);
+    p.accumulate = accumulate;
+    p.vector_store = 0;
+    p.err_word = err_word;
+    p.slot_pitch = (int32_t)pitch;
+    const int64_t pb = (p.row_blocks + 1) / 2;
+    for (int64_t i1 = 0; i1 < n; i1 += slots_max) {
+        const int64_t slots = n - i1 < slots_max ? n - i1 : slots_max;
+        int64_t blocks = (M * slots * (pitch / 8) + 255) / 256;
+        if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
+        moment3_products_kernel<<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)B, ldb, M, (int)n, (int)i1,
+                                                                 (int)slots, (int)pitch, Z);
+        dastac_status rs = launch_status();
+        if (rs != DASTAC_OK) return rs;
+        CUtensorMap tmap_z;
+        const cuuint64_t dims[2] = {(cuuint64_t)(slots * pitch), (cuuint64_t)M};
+        const cuuint64_t strides[1] = {(cuuint64_t)(slots * pitch) * 2};
+        if (enc(&tmap_z, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Z, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DASTAC_ERR_CUDA;
+        p.i1_first = (int32_t)i1;
+        p.slots = (int32_t)slots;
+        int64_t n_tiles = 0;
+        for (int64_t s = 0; s < slots; ++s) {
+            const int64_t r = (i1 + s) / (2 * kTileM);
+            n_tiles += (pb - r) * (pb - r + 1) / 2;
+        }
+        p.tiles_total = n_tiles;
+        const int64_t max_clusters = sm_count() / 2;
+        const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
+        trimm_pair_kernel<kModeMoment3><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_z, tmap_b, p);
+        rs = launch_status();
+        if (rs != DASTAC_OK) return rs;
+    }
+    return DASTAC_OK;
 }
 
 }  // namespace dastac

@@ -661,3 +661,40 @@ def test_moment2_empty_sum_and_host_operands():
     dastac.contract("xi,xj->ij", None, hB, [hB], hout, out_structure=sA, workspace=ws)
     torch.cuda.synchronize()
     assert rel_err(hout.numpy()[: sA.nnz], oracle.pack(desc, ref), oracle.pack(desc, ref_abs)) <= 1e-5
+
+
+@pytest.mark.parametrize("M,n", [(1, 1), (5, 8), (64, 100), (100, 260), (300, 130), (40, 300), (1000, 77)])
+def test_moment3_packed_tetrahedral_output(M, n):
+    """Degree-3 moments A3(i1,i2,i3) = sum_x B(x,i1) B(x,i2) B(x,i3) on i1 <= i2 <= i3, packed tetrahedron."""
+    desc = st.tetrahedron(n)
+    sA = dastac.Structure(desc)
+    B = synth.dense(9, 0, (M, n), dist=synth.NORMAL, bf16=True)
+    ref, ref_abs = oracle.moment3(desc, B)
+    exp, exp_abs = oracle.pack(desc, ref), oracle.pack(desc, ref_abs)
+    Bd = dev(B, "bf16")
+    out = sA.empty_packed()
+    out.fill_(float("nan"))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    nws = dastac.contract_workspace("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
+    assert nws >= M * n * 2
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    got = out.cpu().numpy()
+    # the pairwise product is rounded to bf16 (2^-9 relative) before the third factor: 4e-3 covers it
+    assert rel_err(got[: sA.nnz], exp, exp_abs) <= 4e-3 <= TOL_BF16
+    assert np.isnan(got[sA.nnz:]).all()
+    A0 = synth.dense(9, 1, (sA.nnz,))
+    out2 = sA.empty_packed()
+    out2[: sA.nnz] = dev(A0)
+    dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out2, accumulate=True, out_structure=sA, workspace=ws, err_word=err)
+    assert rel_err(out2.cpu().numpy()[: sA.nnz], exp + A0, exp_abs + np.abs(A0)) <= 4e-3
+    # refused before anything runs: different tensors, wrong output structure, missing workspace
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd.clone()], out, out_structure=sA, workspace=ws)
+    assert e.value.status == 3
+    with pytest.raises(dastac.DastacError):
+        dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=dastac.Structure(st.upper_triangle(n)), workspace=ws)
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
+    assert e.value.status == 7
