@@ -53,8 +53,8 @@ def peaks():
 
 def sizes(small: bool):
     if small:
-        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024, N6=128, Q6=32, K6=32, N7=512, M7=2048)
-    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192, N6=1024, Q6=32, K6=32, N7=4096, M7=100000)
+        return dict(N1=1024, batch=8, N2=4096, w=32, C2=256, N3=4096, n4=128, R=32, N5=1024, N6=128, Q6=32, K6=32, N7=512, M7=2048, N8=64, M8=512)
+    return dict(N1=1024, batch=512, N2=32768, w=32, C2=256, N3=65536, n4=512, R=32, N5=8192, N6=1024, Q6=32, K6=32, N7=4096, M7=100000, N8=256, M8=10000)
 
 
 def accounting(z):
@@ -64,6 +64,7 @@ def accounting(z):
     nnz2 = (2 * w + 1) * N2 - w * (w + 1)
     N6, Q6, K6 = z["N6"], z["Q6"], z["K6"]
     N7, M7 = z["N7"], z["M7"]
+    N8, M8 = z["N8"], z["M8"]
     acc = {
         "trmv": dict(flops=2 * tri(N1), bytes=4 * (tri(N1) + 2 * N1), bound="hbm"),
         "trmv_batched": dict(flops=2 * tri(N1) * b, bytes=4 * (tri(N1) + 2 * N1) * b, bound="hbm"),
@@ -79,12 +80,14 @@ def accounting(z):
         "ttm_ut": dict(flops=2 * tri(N6) * Q6 * K6, bytes=4 * (tri(N6) * (Q6 + K6) + K6 * Q6), bound="hbm"),
         # widened row: degree-2 moments B^T B on i1 <= i2 (M7 samples x N7 features, bf16), packed fp32 output
         "moment2_bf16": dict(flops=2 * tri(N7) * M7, bytes=2 * M7 * N7 + 4 * tri(N7), bound="tensor"),
+        # widened row: degree-3 moments on i1 <= i2 <= i3 (two multiplies and an add per term), packed tetrahedron out
+        "moment3_bf16": dict(flops=3 * tet(N8) * M8, bytes=2 * M8 * N8 + 4 * tet(N8), bound="tensor"),
     }
     return acc
 
 
 ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
-         "moment2_bf16", "symv"]
+         "moment2_bf16", "moment3_bf16", "symv"]
 # the kernels of the five configurations; the others are widened rows and never the roofline's kernel
 CONFIG_KERNELS = ("trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv")
 
@@ -162,12 +165,17 @@ def generate_host(z, pin, only=None):
         # no packed input: the dense tensor is both factors (the same buffer), the output is the packed triangle
         h["moment2_bf16"] = dict(desc=None, out_desc=st.upper_triangle(N7, symmetric=True), A=b7, ins=[b7], alias=True,
                                  out=(cap(tri(N7), 4),))
+    if want("moment3_bf16"):
+        N8, M8 = z["N8"], z["M8"]
+        b8 = host(synth.dense(9, 0, (M8, N8), dist=synth.NORMAL, bf16=True), True)
+        h["moment3_bf16"] = dict(desc=None, out_desc=st.tetrahedron(N8), A=b8, ins=[b8, b8], alias=True,
+                                 out=(cap(tet(N8), 4),))
     return h
 
 
 EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
         "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
-        "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij"}
+        "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij", "moment3_bf16": "xi,xj,xk->ijk"}
 
 
 # ---- clocks ---------------------------------------------------------------------------------------------
@@ -275,7 +283,7 @@ def run_gpu(args):
         s = dastac.Structure(hw["desc"]) if hw["desc"] is not None else None
         structs[name] = s
         dA = hw["A"].cuda()
-        d = dict(A=dA, ins=[dA] if hw.get("alias") else [t.cuda() for t in hw["ins"]], alias=hw.get("alias", False),
+        d = dict(A=dA, ins=[dA] * len(hw["ins"]) if hw.get("alias") else [t.cuda() for t in hw["ins"]], alias=hw.get("alias", False),
                  out=torch.empty(hw["out"], dtype=torch.float32, device="cuda"), batch=hw.get("batch", 1),
                  out_s=dastac.Structure(hw["out_desc"]) if "out_desc" in hw else None)
         n = dastac.contract_workspace(EXPR[name], s, d["A"], d["ins"], d["out"], batch=d["batch"],
@@ -456,7 +464,7 @@ def run_gpu(args):
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
             "data": "synthetic",
-            "config": {"workload": "all five configs per step, plus three widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features): "
+            "config": {"workload": "all five configs per step, plus four widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features; degree-3 moments of M8 x N8): "
                                    + json.dumps(z, separators=(",", ":")),
                        "small": bool(args.small), "only": args.only or None,
                        "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
@@ -484,7 +492,8 @@ def isolated_times(order, devs, structs, run_kernel_on, z, acct, launches):
         nsets = max(1, min(256, -(-3 * 126 * 2 ** 20 // max(foot, 1))))
         def clone_set(d):
             A = d["A"].clone()
-            return dict(d, A=A, out=d["out"].clone(), ins=[A] if d.get("alias") else [t.clone() for t in d.get("ins", [])])
+            return dict(d, A=A, out=d["out"].clone(),
+                        ins=[A] * len(d["ins"]) if d.get("alias") else [t.clone() for t in d.get("ins", [])])
 
         sets = [d] + [clone_set(d) for _ in range(nsets - 1)]
         reps = max(1, -(-launches // nsets))
@@ -594,6 +603,12 @@ def oracle_sample(z, scale=1.0):
     secs += timed(lambda: oracle.moment2(st.upper_triangle(N7, symmetric=True), B7, sel=sel))
     flops += sum(2 * (N7 - int(i)) * M7 for i in sel)
     parts.append(f"moment2 {len(sel)} rows")
+    N8, M8 = z["N8"], z["M8"]
+    sel = rows(N8, 2)
+    B8 = synth.dense(9, 0, (M8, N8), dist=synth.NORMAL, bf16=True)
+    secs += timed(lambda: oracle.moment3(st.tetrahedron(N8), B8, sel=sel))
+    flops += sum(3 * tri(N8 - int(i)) * M8 for i in sel)
+    parts.append(f"moment3 {len(sel)} slabs")
     return flops, secs, "rows spread evenly over the outer index: " + ", ".join(parts)
 
 
@@ -624,7 +639,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(tot_s / steps * 1e3, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "all five configs per step, plus three widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features): "
+        "config": {"workload": "all five configs per step, plus four widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features; degree-3 moments of M8 x N8): "
                                + json.dumps(z, separators=(",", ":")),
                    "sample": desc},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},

@@ -142,9 +142,8 @@ struct Params {
     float* C;
     int64_t N, ncols, ldc;
     int64_t M;           // moment forms only: number of samples (rows of B)
-    // degree-3 moments only: slabs i1 = i1_first .. i1_first + slots - 1 are computed by this launch; the
-    // products Z(x, slot, i2) = B(x, i1) B(x, i2) sit in a matrix with slot_pitch columns per slot
-    int32_t i1_first, slots, slot_pitch;
+    // degree-3 moments only: slabs i1 = i1_first .. i1_first + slots - 1 are computed by this launch
+    int32_t i1_first, slots;
     int64_t tiles_total;
     int64_t cap_elems;   // capacity of the packed buffer in elements (multiple of 8)
     int32_t row_blocks, col_blocks, k_blocks;
@@ -224,6 +223,13 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// Tensor copy into this CTA's shared memory, completing on a barrier of this CTA.
+__device__ __forceinline__ void tma_load_2d_local(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
 }
@@ -261,27 +267,38 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 //
 // MODE 2 (degree-3 moments A3(i1,i2,i3) = sum_x B(x,i1) B(x,i2) B(x,i3) on i1 <= i2 <= i3, the
 // hyper-triangular domain of Section 1, stored as the packed tetrahedron): for a fixed i1 the slab is
-// the degree-2 product of Z_i1(x, i2) = B(x,i1) B(x,i2) with B, kept on i1 <= i2 <= i3.  A launch
-// covers a run of slabs; the "A" operand comes from the matrix of products Z (one column block
-// per slab, written by a small kernel beforehand), the "B" operand from B; tiles are (slab, P, J)
-// with P from the block that holds row i1 and J >= P; the epilogue writes at the tetrahedral
-// position pbase(i1, i2) + i3.
+// the degree-2 product of Z_i1(x, i2) = B(x,i1) B(x,i2) with B, kept on i1 <= i2 <= i3.  Z is never
+// stored.  The producer copies the plain 64 x 128 block of B into the stage exactly as for degree 2,
+// plus a 64 x 8 box that contains column i1, both completing on a barrier of the CTA itself; eight
+// extra warps then scale the block in place, row x by B(x, i1), with packed bf16 multiplies (the
+// product of two bf16 values rounded once, to nearest even), issue a proxy fence so that the
+// tensor core sees the generic-proxy writes, and arrive on the leader's full barrier (3 arrivals:
+// one product warp of each CTA plus the producer's expect-tx for the "B" operand).
+// Everything the product warps wait for arrives asynchronously: they never have a global load
+// outstanding when they execute the fence.  Tiles are (slab, P, J) with P from the block that holds
+// row i1 and J >= P; the epilogue writes at the tetrahedral position pbase(i1, i2) + i3.
 enum PairMode : int { kModeTrimm = 0, kModeMoment2 = 1, kModeMoment3 = 2 };
+constexpr int kScaleWarps = kPStages, kPWarpScale0 = 6;  // one product warp per stage
+constexpr int kPThreadsFused = kPThreads + 32 * kScaleWarps;  // 384
+constexpr int kCxBytes = kBlockK * 16;                         // 64 x 8 bf16 box around column i1, per stage
+constexpr size_t kPSmemBytesFused = kPSmemBytes + (size_t)kPStages * kCxBytes;
 
 template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == kModeMoment3 ? kPThreadsFused : kPThreads, 1)
 trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = (uint64_t*)(smem + (size_t)kPStages * kPStageBytes);
-    // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2], drain
+    uint8_t* cxbuf = smem + (size_t)kPStages * kPStageBytes;  // degree 3 only
+    uint64_t* bars = (uint64_t*)(cxbuf + (MODE == kModeMoment3 ? kPStages * kCxBytes : 0));
+    // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2], drain, (tmem slot, abort flag), rawfull[s]
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (kPStages + s); };
     auto tmem_full = [&](int a) { return bar0 + 8u * (2 * kPStages + a); };
     auto tmem_empty = [&](int a) { return bar0 + 8u * (2 * kPStages + 2 + a); };
     auto drain_bar = [&]() { return bar0 + 8u * (2 * kPStages + 4); };
+    auto rawfull = [&](int s) { return bar0 + 8u * (2 * kPStages + 6 + s); };  // degree 3: this CTA's plain block has landed
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * kPStages + 5);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
@@ -292,8 +309,9 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPStages; ++s) {
-            mbar_init(full(s), 1);
+            mbar_init(full(s), MODE == kModeMoment3 ? 1 + 2 : 1);  // degree 3: one product warp of each CTA as well
             mbar_init(empty(s), 1);
+            if (MODE == kModeMoment3) mbar_init(rawfull(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
@@ -326,13 +344,18 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (MOMENT2) {
             int r = 0;
             if (MODE == kModeMoment3) {
-                for (;;) {  // slabs in order; slab i1 uses the block rows from the one that holds row i1
-                    r = (p.i1_first + slot) / (2 * kTileM);
-                    const int64_t cnt = (int64_t)(pair_blocks - r) * (pair_blocks - r + 1) / 2;
-                    if (t < cnt || slot + 1 >= p.slots) break;
-                    t -= cnt;
-                    ++slot;
+                // slabs in order; the 256 slabs whose i1 lies in block row r all use block rows r .. and
+                // have the same number of tiles
+                for (r = 0; r + 1 < pair_blocks; ++r) {
+                    const int64_t per_slab = (int64_t)(pair_blocks - r) * (pair_blocks - r + 1) / 2;
+                    const int64_t in_block = per_slab * (2 * kTileM);
+                    if (t < in_block) break;
+                    t -= in_block;
+                    slot += 2 * kTileM;
                 }
+                const int64_t per_slab = (int64_t)(pair_blocks - r) * (pair_blocks - r + 1) / 2;
+                slot += (int)(t / per_slab);
+                t %= per_slab;
             }
             while (t >= pair_blocks - r) {
                 t -= pair_blocks - r;
@@ -374,15 +397,20 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         break;
                     }
                     const uint32_t dst = smem_base + s * kPStageBytes;
-                    if (leader) mbar_arrive_expect_tx(full(s), 2 * kPStageBytes);  // both CTAs' bytes
+                    // both CTAs' bytes; degree 3: only the "B" operand comes by TMA
+                    if (leader) mbar_arrive_expect_tx(full(s), MODE == kModeMoment3 ? 2 * kPBBytes : 2 * kPStageBytes);
                     const uint32_t bar = full0 + 8u * s;
-                    if (MOMENT2) {
-                        // degree 2: columns of B itself; degree 3: the slab's column block of the products
-                        const int xa = (MODE == kModeMoment3 ? slot * p.slot_pitch : 0) + I * kTileM;
+                    if (MODE == kModeMoment3) {
+                        // the plain block of B and the box around column i1, for this CTA's product warps
+                        mbar_arrive_expect_tx(rawfull(s), kABytes + kCxBytes);
 #pragma unroll
                         for (int q = 0; q < kTileM / 64; ++q)
-                            tma_load_2d_pair(dst + q * (kBlockK * 128), MODE == kModeMoment3 ? &tmap_a : &tmap_b,
-                                             xa + q * 64, kb * kBlockK, bar);
+                            tma_load_2d_local(dst + q * (kBlockK * 128), &tmap_b, I * kTileM + q * 64, kb * kBlockK, rawfull(s));
+                        tma_load_2d_local(smem_u32(cxbuf) + s * kCxBytes, &tmap_a, slot & ~7, kb * kBlockK, rawfull(s));
+                    } else if (MOMENT2) {
+#pragma unroll
+                        for (int q = 0; q < kTileM / 64; ++q)
+                            tma_load_2d_pair(dst + q * (kBlockK * 128), &tmap_b, I * kTileM + q * 64, kb * kBlockK, bar);
                     } else {
                         tma_load_2d_pair(dst, &tmap_a, 0, (int)((tile_base + kb) * kTileM), bar);
                     }
@@ -397,6 +425,56 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const long long t0 = clock64();
                 while (clock64() - t0 < 2000000) {
                 }
+            }
+        }
+    } else if (MODE == kModeMoment3 && warp >= kPWarpScale0) {
+        // ---- product warps (both CTAs): scale this CTA's 64 x 128 block of B by column i1, in place --------
+        // Warp w owns stage w: the proxy fence costs about as much as a copy in flight, so a warp pays
+        // it once per six K blocks and all six stages can be in the scaling step at once.  (A warp
+        // that owned varying stages could wait on a barrier two phases ahead of it, which a parity
+        // wait cannot tell from one phase behind.)  A lane owns one 16-byte chunk column c of the block and
+        // walks the rows r = (lane >> 4) + 2 j.
+        const int w = warp - kPWarpScale0;
+        const int c = lane & 15, r0 = lane >> 4;
+        const uint32_t full0 = map_to_cta(full(0), 0);
+        uint32_t it = 0;
+        bool ok = true;
+        for (uint32_t n = 0; n < rounds && ok; ++n) {
+            const int64_t t = tile_of(n);
+            if (t >= tiles) continue;
+            int P, J, slot;
+            decode(t, P, J, slot);
+            const uint32_t cx_col = (uint32_t)((slot & 7) * 2);  // B(x, i1) inside the 64 x 8 box: row r at r * 16
+            for (int kb = 0; kb < p.k_blocks && ok; ++kb, ++it) {
+                const int s = it % kPStages;
+                if (s != w) continue;
+                if (!mbar_wait_warp(rawfull(s), (it / kPStages) & 1, abort_flag, p.err_word, kErrFull, lane)) {
+                    ok = false;
+                    break;
+                }
+                uint8_t* stage = smem + s * kPStageBytes;
+                const uint8_t* cxs = cxbuf + s * kCxBytes + cx_col;
+#pragma unroll 4
+                for (int j = 0; j < kBlockK / 2; ++j) {
+                    const int r = r0 + 2 * j;
+                    // 128-byte swizzle of an M-major tile: two 64-column halves of 8 KiB, row r at r * 128,
+                    // chunk index xor (r mod 8)
+                    const uint32_t off = (uint32_t)((c >> 3) * (kBlockK * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+                    const __nv_bfloat16 c1 = *reinterpret_cast<const __nv_bfloat16*>(cxs + r * 16);
+                    const __nv_bfloat162 c2 = __halves2bfloat162(c1, c1);
+                    union {
+                        uint4 v;
+                        __nv_bfloat162 h[4];
+                    } ch;
+                    ch.v = *reinterpret_cast<const uint4*>(stage + off);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) ch.h[e] = __hmul2(ch.h[e], c2);
+                    *reinterpret_cast<uint4*>(stage + off) = ch.v;
+                }
+                // make the generic-proxy writes visible to the tensor core's reads, then publish
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(full0 + 8u * s);
             }
         }
     } else if (warp == kPWarpMma) {
@@ -445,7 +523,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
         }
-    } else {
+    } else if (warp < 4) {
         // ---- epilogue (both CTAs): this CTA's 128 rows of the tile ------------------------------------
         const uint32_t empty0 = map_to_cta(tmem_empty(0), 0);
         uint32_t tile_n = 0;
@@ -688,7 +766,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     p.ncols = ncols;
     p.ldc = ldc;
     p.M = 0;
-    p.i1_first = p.slots = p.slot_pitch = 0;
+    p.i1_first = p.slots = 0;
     p.tiles_total = 0;
     p.cap_elems = round_up(m.slots, 8);
     p.row_blocks = (int32_t)((N + kTileM - 1) / kTileM);
@@ -778,7 +856,7 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
     p.ncols = n;
     p.ldc = 0;
     p.M = M;
-    p.i1_first = p.slots = p.slot_pitch = 0;
+    p.i1_first = p.slots = 0;
     p.tiles_total = 0;
     p.cap_elems = 0;
     p.row_blocks = (int32_t)((n + kTileM - 1) / kTileM);
@@ -805,47 +883,8 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
 }
 
 // ---- degree-3 moments: A3 on i1 <= i2 <= i3, packed tetrahedron out ------------------------------------
-// Z(x, slot * pitch + i2) = bf16(B(x, i1) * B(x, i2)) for i2 >= i1 = i1_first + slot, zero elsewhere in the
-// slot (columns below i1 and the padding up to the pitch).  The product of two bf16 values has 16
-// significant bits; it is rounded to bf16 once, to nearest even.
-__global__ void moment3_products_kernel(const __nv_bfloat16* __restrict__ B, int64_t ldb, int64_t M, int n,
-                                        int i1_first, int slots, int pitch, __nv_bfloat16* __restrict__ Z) {
-    const int chunks = pitch / 8;  // 16-byte chunks per slot
-    const int64_t total = M * slots * (int64_t)chunks;
-    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
-        const int c = (int)(t % chunks);
-        const int64_t q = t / chunks;
-        const int slot = (int)(q % slots);
-        const int64_t x = q / slots;
-        const int i1 = i1_first + slot;
-        const float b1 = __bfloat162float(B[x * ldb + i1]);
-        union {
-            uint4 v;
-            __nv_bfloat16 e[8];
-        } out;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int i2 = 8 * c + e;
-            out.e[e] = (i2 >= i1 && i2 < n) ? __float2bfloat16_rn(b1 * __bfloat162float(B[x * ldb + i2])) : __float2bfloat16_rn(0.f);
-        }
-        *reinterpret_cast<uint4*>(Z + (x * slots + slot) * (int64_t)pitch + 8 * c) = out.v;
-    }
-}
-
-// Slabs computed per launch: as many as keep the matrix of products within kMoment3ZBytes.
-constexpr int64_t kMoment3ZBytes = (int64_t)512 << 20;
-static int64_t moment3_slots(int64_t M, int64_t n) {
-    const int64_t pitch = round_up(n, 128);
-    int64_t s = kMoment3ZBytes / (M * pitch * 2);
-    if (s < 1) s = 1;
-    return s < n ? s : n;
-}
-size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb) {
-    if (M == 0 || n == 0) return 0;
-    size_t bytes = (size_t)round_up(M * moment3_slots(M, n) * round_up(n, 128) * 2, 256);
-    if (ldb % 8 != 0) bytes += (size_t)(M * round_up(n, 8) * 2);
-    return bytes;
-}
+// Workspace: only when B's row pitch is not a multiple of 16 bytes (a re-pitched copy of B).
+size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb) { return moment2_workspace_bytes(M, n, ldb); }
 
 dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
                                   int accumulate, void* workspace, int32_t* err_word, cudaStream_t st) {
@@ -857,40 +896,42 @@ dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb
         return DASTAC_OK;
     }
     if (!aligned16(B)) return DASTAC_ERR_ALIGNMENT;
-    if (!workspace) return DASTAC_ERR_WORKSPACE;
-    const int64_t pitch = round_up(n, 128), slots_max = moment3_slots(M, n);
-    if (M > 0x7fffffffLL - kBlockK || slots_max * pitch > 0x7fffffffLL - 2 * kTileN) return DASTAC_ERR_OVERFLOW;
-    __nv_bfloat16* Z = (__nv_bfloat16*)workspace;
+    if (M > 0x7fffffffLL - kBlockK || n > 0x7fffffffLL - 2 * kTileN) return DASTAC_ERR_OVERFLOW;
     if (ldb % 8 != 0) {
-        uint16_t* copy = (uint16_t*)((uint8_t*)workspace + round_up(M * slots_max * pitch * 2, 256));
+        if (!workspace) return DASTAC_ERR_WORKSPACE;
         const int64_t ldd = round_up(n, 8);
         int64_t blocks = (M * ldd + 255) / 256;
         if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
-        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, copy, ldd, M, n);
+        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, (uint16_t*)workspace, ldd, M, n);
         dastac_status rs = launch_status();
         if (rs != DASTAC_OK) return rs;
-        B = copy;
+        B = workspace;
         ldb = ldd;
     }
     EncodeTiledFn enc = encode_fn();
     if (!enc) return DASTAC_ERR_CUDA;
+    CUtensorMap tmap_b;
+    const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)kBlockK};
     const cuuint32_t estr[2] = {1, 1};
-    CUtensorMap tmap_b;
-    {
-        const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)M};
-        const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
-        if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DASTAC_ERR_CUDA;
-    }
+    if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DASTAC_ERR_CUDA;
+    // 64 rows x 8 columns around column i1 (16 bytes per row, no swizzle): the factor B(x, i1) of a K block
+    CUtensorMap tmap_c;
+    const cuuint32_t cbox[2] = {8, (cuuint32_t)kBlockK};
+    if (enc(&tmap_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, cbox, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DASTAC_ERR_CUDA;
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
         if (cudaFuncSetAttribute(trimm_pair_kernel<kModeMoment3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kPSmemBytes) != cudaSuccess)
+                                 (int)kPSmemBytesFused) != cudaSuccess)
             return DASTAC_ERR_CUDA;
         attr_set[dev] = true;
     }
@@ -909,38 +950,19 @@ dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb
     p.accumulate = accumulate;
     p.vector_store = 0;
     p.err_word = err_word;
-    p.slot_pitch = (int32_t)pitch;
+    p.i1_first = 0;
+    p.slots = (int32_t)n;
     const int64_t pb = (p.row_blocks + 1) / 2;
-    for (int64_t i1 = 0; i1 < n; i1 += slots_max) {
-        const int64_t slots = n - i1 < slots_max ? n - i1 : slots_max;
-        int64_t blocks = (M * slots * (pitch / 8) + 255) / 256;
-        if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
-        moment3_products_kernel<<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)B, ldb, M, (int)n, (int)i1,
-                                                                 (int)slots, (int)pitch, Z);
-        dastac_status rs = launch_status();
-        if (rs != DASTAC_OK) return rs;
-        CUtensorMap tmap_z;
-        const cuuint64_t dims[2] = {(cuuint64_t)(slots * pitch), (cuuint64_t)M};
-        const cuuint64_t strides[1] = {(cuuint64_t)(slots * pitch) * 2};
-        if (enc(&tmap_z, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Z, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DASTAC_ERR_CUDA;
-        p.i1_first = (int32_t)i1;
-        p.slots = (int32_t)slots;
-        int64_t n_tiles = 0;
-        for (int64_t s = 0; s < slots; ++s) {
-            const int64_t r = (i1 + s) / (2 * kTileM);
-            n_tiles += (pb - r) * (pb - r + 1) / 2;
-        }
-        p.tiles_total = n_tiles;
-        const int64_t max_clusters = sm_count() / 2;
-        const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-        trimm_pair_kernel<kModeMoment3><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_z, tmap_b, p);
-        rs = launch_status();
-        if (rs != DASTAC_OK) return rs;
+    int64_t n_tiles = 0;
+    for (int64_t i1 = 0; i1 < n; ++i1) {
+        const int64_t r = i1 / (2 * kTileM);
+        n_tiles += (pb - r) * (pb - r + 1) / 2;
     }
-    return DASTAC_OK;
+    p.tiles_total = n_tiles;
+    const int64_t max_clusters = sm_count() / 2;
+    const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
+    trimm_pair_kernel<kModeMoment3><<<2 * clusters, kPThreadsFused, kPSmemBytesFused, st>>>(tmap_c, tmap_b, p);
+    return launch_status();
 }
 
 }  // namespace dastac

@@ -218,3 +218,32 @@ def test_widened_row_moment2_m100000_n4096():
         # grows with the length of the sum (about 5e-4 here), still far inside the bf16 bar
         assert rel_err(seg, ref[s, int(i):], ref_abs[s, int(i):]) <= TOL_BF16
         assert rel_err(seg, ref[s, int(i):], ref_abs[s, int(i):]) <= 2e-3
+
+
+@pytest.mark.parametrize("M,n", [(10000, 256), (60000, 200)], ids=["m10000_n256", "m60000_n200"])
+def test_widened_row_moment3(M, n):
+    """Degree-3 moments of 10000 samples (the sample count of the paper's PR3 runs) x 256 features, and
+    a taller, narrower case with an odd number of K blocks and a ragged last row block; sampled slabs
+    of the packed tetrahedron."""
+    desc = st.tetrahedron(n)
+    sA = dastac.Structure(desc)
+    B = synth.dense(9, 0, (M, n), dist=synth.NORMAL, bf16=True)
+    Bd = dev(B, "bf16")
+    out = torch.full((sA.capacity(torch.float32),), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    nws = dastac.contract_workspace("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
+    ws = torch.empty(max(nws, 1), dtype=torch.uint8, device="cuda")
+    dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    got = out.cpu().numpy()[: sA.nnz]
+    assert np.isfinite(got).all()
+    sel = np.array([0, 1, 51, 52, 103, 104, 127, 128, n - 2, n - 1] if n == 256 else [0, 51, 52, 155, 156, n - 1], dtype=np.int64)
+    ref, ref_abs = oracle.moment3(desc, B, sel=sel)
+    for s, i in enumerate(sel):
+        i = int(i)
+        start = oracle.rank_point(desc, (i, i, i))
+        m = n - i
+        exp = np.concatenate([ref[s, j, j:] for j in range(i, n)])
+        exp_abs = np.concatenate([ref_abs[s, j, j:] for j in range(i, n)])
+        assert exp.size == m * (m + 1) // 2
+        assert rel_err(got[start: start + exp.size], exp, exp_abs) <= 4e-3 <= TOL_BF16
