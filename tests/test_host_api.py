@@ -316,3 +316,39 @@ def test_moment2_plan_is_validated_on_the_host():
     assert ws(b"xi,xj->ij", *args) == 3
     assert ws(b"xi,xj->ij", ins, 1, ctypes.byref(out), ctypes.byref(nbytes)) == 1
     assert dastac.launch_count() == before
+
+
+def test_moment3_plan_is_validated_on_the_host():
+    """"xi,xj,xk->ijk": the same dense bf16 tensor three times, packed f32 tetrahedron out; planning only."""
+    before = dastac.launch_count()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    n, M = 24, 100
+    tet = dastac.Structure(st.tetrahedron(n))
+    ins = (binding._Operand * 3)()
+    for k in range(3):
+        ins[k].data = 4096
+        ins[k].dtype = binding.BF16
+        ins[k].rank = 2
+        ins[k].dims[0], ins[k].dims[1] = M, n
+        ins[k].strides[0], ins[k].strides[1] = n, 1
+    out = binding._Operand()
+    out.structure = tet._h
+    out.rank = 3
+    nbytes = ctypes.c_size_t(123)
+    ws = lib.dastac_contract_workspace
+    args = (ins, 3, ctypes.byref(out), ctypes.byref(nbytes))
+    assert ws(b"xi,xj,xk->ijk", *args) == 0 and nbytes.value == 0
+    ins[0].strides[0] = ins[1].strides[0] = ins[2].strides[0] = n + 3     # 54-byte pitch: re-pitched copy
+    assert ws(b"xi,xj,xk->ijk", *args) == 0 and nbytes.value == -(-M * n * 2 // 256) * 256
+    ins[0].strides[0] = ins[1].strides[0] = ins[2].strides[0] = n
+    ins[2].data = 8192                                                     # third factor is another tensor
+    assert ws(b"xi,xj,xk->ijk", *args) == 3
+    ins[2].data = 4096
+    tri2 = dastac.Structure(st.upper_triangle(n, symmetric=True))
+    out.structure = tri2._h                                                # degree-2 output structure
+    assert ws(b"xi,xj,xk->ijk", *args) == 3
+    other = dastac.Structure(st.tetrahedron(n + 1))
+    out.structure = other._h
+    assert ws(b"xi,xj,xk->ijk", *args) == 4
+    assert ws(b"xi,xj,xk->ijk", ins, 2, ctypes.byref(out), ctypes.byref(nbytes)) == 1
+    assert dastac.launch_count() == before
