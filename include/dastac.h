@@ -197,7 +197,8 @@ typedef struct {
  *                   rule); `out` is PACKED: out->structure is the n x n x n tetrahedron i <= j <= k (the
  *                   hyper-triangular domain of Section 1).  The pairwise products B(x,i) B(x,j) are
  *                   rounded to bf16 once before they meet the third factor on the tensor cores
- *                   (relative error 2^-9 per term); accumulation is fp32.
+ *                   (relative error 2^-9 per term); accumulation is fp32.  Needs workspace (a transposed
+ *                   copy of B).
  * accumulate: 0 -> out = result (the library zero-fills where it needs to), 1 -> out += result.
  * workspace: device scratch of at least dastac_contract_workspace bytes, 256-byte aligned; may be
  *            NULL when that size is 0.  Its contents are undefined afterwards.

@@ -112,6 +112,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr)
         : "memory");
 }
+// 32 consecutive 32-bit columns of this thread's lane, from registers.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -248,6 +260,16 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc,
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the A operand in tensor memory (K-major: lane = row, two bf16 per 32-bit column).
+__device__ __forceinline__ void umma_bf16_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // Arrive on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far retire.
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
     asm volatile(
@@ -268,25 +290,30 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // MODE 2 (degree-3 moments A3(i1,i2,i3) = sum_x B(x,i1) B(x,i2) B(x,i3) on i1 <= i2 <= i3, the
 // hyper-triangular domain of Section 1, stored as the packed tetrahedron): for a fixed i1 the slab is
 // the degree-2 product of Z_i1(x, i2) = B(x,i1) B(x,i2) with B, kept on i1 <= i2 <= i3.  Z is never
-// stored.  The producer copies the plain 64 x 128 block of B into the stage exactly as for degree 2,
-// plus a 64 x 8 box that contains column i1, both completing on a barrier of the CTA itself; eight
-// extra warps then scale the block in place, row x by B(x, i1), with packed bf16 multiplies (the
-// product of two bf16 values rounded once, to nearest even), issue a proxy fence so that the
-// tensor core sees the generic-proxy writes, and arrive on the leader's full barrier (3 arrivals:
-// one product warp of each CTA plus the producer's expect-tx for the "B" operand).
-// Everything the product warps wait for arrives asynchronously: they never have a global load
-// outstanding when they execute the fence.  Tiles are (slab, P, J) with P from the block that holds
-// row i1 and J >= P; the epilogue writes at the tetrahedral position pbase(i1, i2) + i3.
+// stored: the "A" operand of the MMAs lives in tensor memory and four extra warps write it.  The
+// host transposes B once (Bt, n x M, a few MB), so that row i2 of a K block is 128 contiguous bytes:
+// the producer copies the 128 x 64 block of Bt (128-byte swizzle) and the 64 values Bt(i1, x) of the
+// slab's own column into the stage, completing on a barrier of the CTA itself; thread m of the
+// product warps reads row m of the block (eight 128-bit loads), multiplies it by the column with
+// packed bf16 multiplies (the product of two bf16 values rounded once, to nearest even) and stores
+// the 64 products to lane m of the stage's 32 tensor-memory columns with tcgen05.st.  No generic
+// write to shared memory is involved, hence no proxy fence (an earlier form that scaled the block
+// in shared memory spent most of its time in fence.proxy.async).  One arrive per warp on the
+// leader's full barrier (9 arrivals: 8 warps of the pair plus the producer's expect-tx for the "B"
+// operand, which comes from B by TMA as for degree 2) publishes the stage.  Tensor memory holds one
+// 256-column accumulator and six 32-column A stages.  Tiles are (slab, P, J) with P from the block
+// that holds row i1 and J >= P; the epilogue writes at the tetrahedral position pbase(i1, i2) + i3.
 enum PairMode : int { kModeTrimm = 0, kModeMoment2 = 1, kModeMoment3 = 2 };
-constexpr int kScaleWarps = kPStages, kPWarpScale0 = 6;  // one product warp per stage
-constexpr int kPThreadsFused = kPThreads + 32 * kScaleWarps;  // 384
-constexpr int kCxBytes = kBlockK * 16;                         // 64 x 8 bf16 box around column i1, per stage
+constexpr int kScaleWarps = 4, kPWarpScale0 = 8;  // product warps 8..11: warp w writes tensor-memory lanes 32 (w mod 4) ..
+constexpr int kPThreadsFused = 32 * (kPWarpScale0 + kScaleWarps);  // 384 (warps 6 and 7 idle)
+constexpr int kCxBytes = kBlockK * 2;                          // the 64 values B(x, i1) of a K block, per stage
+constexpr int kTmemAStage0 = kTileN, kTmemAStageCols = kBlockK / 2;  // A stages behind the single accumulator
 constexpr size_t kPSmemBytesFused = kPSmemBytes + (size_t)kPStages * kCxBytes;
 
 template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == kModeMoment3 ? kPThreadsFused : kPThreads, 1)
 trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                  const Params p) {
+                  const __grid_constant__ CUtensorMap tmap_c, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* cxbuf = smem + (size_t)kPStages * kPStageBytes;  // degree 3 only
@@ -309,7 +336,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPStages; ++s) {
-            mbar_init(full(s), MODE == kModeMoment3 ? 1 + 2 : 1);  // degree 3: one product warp of each CTA as well
+            mbar_init(full(s), MODE == kModeMoment3 ? 1 + 2 * kScaleWarps : 1);  // degree 3: the product warps of both CTAs as well
             mbar_init(empty(s), 1);
             if (MODE == kModeMoment3) mbar_init(rawfull(s), 1);
         }
@@ -401,12 +428,10 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (leader) mbar_arrive_expect_tx(full(s), MODE == kModeMoment3 ? 2 * kPBBytes : 2 * kPStageBytes);
                     const uint32_t bar = full0 + 8u * s;
                     if (MODE == kModeMoment3) {
-                        // the plain block of B and the box around column i1, for this CTA's product warps
+                        // the 128 x 64 block of Bt and the slab's own column, for this CTA's product warps
                         mbar_arrive_expect_tx(rawfull(s), kABytes + kCxBytes);
-#pragma unroll
-                        for (int q = 0; q < kTileM / 64; ++q)
-                            tma_load_2d_local(dst + q * (kBlockK * 128), &tmap_b, I * kTileM + q * 64, kb * kBlockK, rawfull(s));
-                        tma_load_2d_local(smem_u32(cxbuf) + s * kCxBytes, &tmap_a, slot & ~7, kb * kBlockK, rawfull(s));
+                        tma_load_2d_local(dst, &tmap_a, kb * kBlockK, I * kTileM, rawfull(s));
+                        tma_load_2d_local(smem_u32(cxbuf) + s * kCxBytes, &tmap_c, kb * kBlockK, p.i1_first + slot, rawfull(s));
                     } else if (MOMENT2) {
 #pragma unroll
                         for (int q = 0; q < kTileM / 64; ++q)
@@ -428,51 +453,43 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
     } else if (MODE == kModeMoment3 && warp >= kPWarpScale0) {
-        // ---- product warps (both CTAs): scale this CTA's 64 x 128 block of B by column i1, in place --------
-        // Warp w owns stage w: the proxy fence costs about as much as a copy in flight, so a warp pays
-        // it once per six K blocks and all six stages can be in the scaling step at once.  (A warp
-        // that owned varying stages could wait on a barrier two phases ahead of it, which a parity
-        // wait cannot tell from one phase behind.)  A lane owns one 16-byte chunk column c of the block and
-        // walks the rows r = (lane >> 4) + 2 j.
-        const int w = warp - kPWarpScale0;
-        const int c = lane & 15, r0 = lane >> 4;
+        // ---- product warps (both CTAs): rows of the block times the slab's column, into tensor memory -----
+        const int m = 32 * (warp - kPWarpScale0) + lane;  // row of the block = tensor-memory lane
         const uint32_t full0 = map_to_cta(full(0), 0);
         uint32_t it = 0;
         bool ok = true;
         for (uint32_t n = 0; n < rounds && ok; ++n) {
             const int64_t t = tile_of(n);
             if (t >= tiles) continue;
-            int P, J, slot;
-            decode(t, P, J, slot);
-            const uint32_t cx_col = (uint32_t)((slot & 7) * 2);  // B(x, i1) inside the 64 x 8 box: row r at r * 16
             for (int kb = 0; kb < p.k_blocks && ok; ++kb, ++it) {
                 const int s = it % kPStages;
-                if (s != w) continue;
+                // the copies into stage s are only issued once the MMAs that read tensor-memory stage s
+                // have retired, so their arrival also says that the stage may be overwritten
                 if (!mbar_wait_warp(rawfull(s), (it / kPStages) & 1, abort_flag, p.err_word, kErrFull, lane)) {
                     ok = false;
                     break;
                 }
-                uint8_t* stage = smem + s * kPStageBytes;
-                const uint8_t* cxs = cxbuf + s * kCxBytes + cx_col;
-#pragma unroll 4
-                for (int j = 0; j < kBlockK / 2; ++j) {
-                    const int r = r0 + 2 * j;
-                    // 128-byte swizzle of an M-major tile: two 64-column halves of 8 KiB, row r at r * 128,
-                    // chunk index xor (r mod 8)
-                    const uint32_t off = (uint32_t)((c >> 3) * (kBlockK * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4));
-                    const __nv_bfloat16 c1 = *reinterpret_cast<const __nv_bfloat16*>(cxs + r * 16);
-                    const __nv_bfloat162 c2 = __halves2bfloat162(c1, c1);
-                    union {
-                        uint4 v;
-                        __nv_bfloat162 h[4];
-                    } ch;
-                    ch.v = *reinterpret_cast<const uint4*>(stage + off);
+                const uint8_t* row = smem + s * kPStageBytes + m * 128;  // 128-byte swizzle: chunk j sits at j xor (m mod 8)
+                const uint4* cx = reinterpret_cast<const uint4*>(cxbuf + s * kCxBytes);
+                uint32_t v[32];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) ch.h[e] = __hmul2(ch.h[e], c2);
-                    *reinterpret_cast<uint4*>(stage + off) = ch.v;
+                for (int j = 0; j < 8; ++j) {
+                    union {
+                        uint4 q;
+                        __nv_bfloat162 h[4];
+                        uint32_t u[4];
+                    } a, c;
+                    a.q = *reinterpret_cast<const uint4*>(row + ((j ^ (m & 7)) << 4));
+                    c.q = cx[j];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        a.h[e] = __hmul2(a.h[e], c.h[e]);
+                        v[4 * j + e] = a.u[e];
+                    }
                 }
-                // make the generic-proxy writes visible to the tensor core's reads, then publish
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                tmem_st32(tmem_base + ((uint32_t)(32 * (warp - kPWarpScale0)) << 16) + kTmemAStage0 + s * kTmemAStageCols, v);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(full0 + 8u * s);
             }
@@ -487,9 +504,11 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (t >= tiles) continue;
                 int P, J, slot;
                 decode(t, P, J, slot);
-                const int acc = tile_n & 1;
-                if (tile_n >= 2 &&
-                    !mbar_wait_cluster(tmem_empty(acc), ((tile_n >> 1) - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
+                // degree 3 has a single accumulator (the other half of tensor memory holds the A stages)
+                const int acc = MODE == kModeMoment3 ? 0 : (tile_n & 1);
+                const uint32_t use = MODE == kModeMoment3 ? tile_n : (tile_n >> 1);  // how often this buffer was used before
+                if (use >= 1 &&
+                    !mbar_wait_cluster(tmem_empty(acc), (use - 1) & 1, abort_flag, p.err_word, kErrTmemEmpty)) {
                     ok = false;
                     break;
                 }
@@ -509,7 +528,11 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const uint64_t da = MOMENT2 ? smem_desc(a_addr + k16 * 2048, kBlockK * 128, 1024)
                                                     : smem_desc(a_addr + k16 * 32, 16, 1024);
                         const uint64_t db = smem_desc(b_addr + k16 * 2048, kBlockK * 128, 1024);
-                        umma_bf16_pair(d_tmem, da, db, kIdesc, (kb > kb_first(P) || k16 > 0) ? 1u : 0u);
+                        if (MODE == kModeMoment3)
+                            umma_bf16_pair_ts(d_tmem, tmem_base + kTmemAStage0 + s * kTmemAStageCols + k16 * 8, db, kPIdesc,
+                                              (kb > 0 || k16 > 0) ? 1u : 0u);
+                        else
+                            umma_bf16_pair(d_tmem, da, db, kIdesc, (kb > kb_first(P) || k16 > 0) ? 1u : 0u);
                     }
                     umma_commit_pair(empty(s));
                 }
@@ -534,8 +557,9 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             int P, J, slot;
             decode(t, P, J, slot);
             const int I = 2 * P + (int)rank;
-            const int acc = tile_n & 1;
-            if (!mbar_wait_warp(tmem_full(acc), (tile_n >> 1) & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
+            const int acc = MODE == kModeMoment3 ? 0 : (tile_n & 1);
+            const uint32_t use = MODE == kModeMoment3 ? tile_n : (tile_n >> 1);
+            if (!mbar_wait_warp(tmem_full(acc), use & 1, abort_flag, p.err_word, kErrTmemFull, lane)) {
                 ok = false;
                 break;
             }
@@ -804,7 +828,7 @@ dastac_status launch_trimm_bf16(const IndexMap& m, const void* A, const void* B,
     const int64_t n_tiles = (int64_t)((p.row_blocks + 1) / 2) * p.col_blocks;  // pairs of row blocks x column blocks
     const int64_t max_clusters = sm_count() / 2;
     const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-    trimm_pair_kernel<kModeTrimm><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, p);
+    trimm_pair_kernel<kModeTrimm><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap_a, tmap, tmap, p);  // the third map is not used
     return launch_status();
 }
 
@@ -878,13 +902,33 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
     const int64_t n_tiles = pb * (pb + 1) / 2;
     const int64_t max_clusters = sm_count() / 2;
     const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-    trimm_pair_kernel<kModeMoment2><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap, tmap, p);  // the first map is not used
+    trimm_pair_kernel<kModeMoment2><<<2 * clusters, kPThreads, kPSmemBytes, st>>>(tmap, tmap, tmap, p);  // only the second map is used
     return launch_status();
 }
 
 // ---- degree-3 moments: A3 on i1 <= i2 <= i3, packed tetrahedron out ------------------------------------
-// Workspace: only when B's row pitch is not a multiple of 16 bytes (a re-pitched copy of B).
-size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb) { return moment2_workspace_bytes(M, n, ldb); }
+// Bt[i][x] = B[x][i], row pitch ldt elements.
+__global__ void transpose_bf16_kernel(const uint16_t* __restrict__ B, int64_t ldb, int64_t M, int64_t n,
+                                      uint16_t* __restrict__ Bt, int64_t ldt) {
+    __shared__ uint16_t tile[32][33];
+    const int64_t x0 = blockIdx.x * 32LL, i0 = blockIdx.y * 32LL;
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int64_t x = x0 + r, i = i0 + threadIdx.x;
+        tile[r][threadIdx.x] = (x < M && i < n) ? B[x * ldb + i] : (uint16_t)0;
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int64_t i = i0 + r, x = x0 + threadIdx.x;
+        if (i < n && x < M) Bt[i * ldt + x] = tile[threadIdx.x][r];
+    }
+}
+
+// Workspace: the transposed copy of B (n rows of round_up(M, 8) elements), then, only when B's row pitch
+// is not a multiple of 16 bytes, a re-pitched copy of B.
+size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb) {
+    if (M == 0 || n == 0) return 0;
+    return (size_t)round_up(n * round_up(M, 8) * 2, 256) + moment2_workspace_bytes(M, n, ldb);
+}
 
 dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
                                   int accumulate, void* workspace, int32_t* err_word, cudaStream_t st) {
@@ -896,36 +940,55 @@ dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb
         return DASTAC_OK;
     }
     if (!aligned16(B)) return DASTAC_ERR_ALIGNMENT;
+    if (!workspace) return DASTAC_ERR_WORKSPACE;
     if (M > 0x7fffffffLL - kBlockK || n > 0x7fffffffLL - 2 * kTileN) return DASTAC_ERR_OVERFLOW;
+    const int64_t ldt = round_up(M, 8);
+    uint16_t* Bt = (uint16_t*)workspace;
+    {
+        const int64_t gx = (M + 31) / 32, gy = (n + 31) / 32;
+        if (gy > 65535) return DASTAC_ERR_OVERFLOW;
+        transpose_bf16_kernel<<<dim3((unsigned)gx, (unsigned)gy), dim3(32, 8), 0, st>>>((const uint16_t*)B, ldb, M, n, Bt, ldt);
+        dastac_status rs = launch_status();
+        if (rs != DASTAC_OK) return rs;
+    }
     if (ldb % 8 != 0) {
-        if (!workspace) return DASTAC_ERR_WORKSPACE;
+        uint16_t* copy = (uint16_t*)((uint8_t*)workspace + round_up(n * ldt * 2, 256));
         const int64_t ldd = round_up(n, 8);
         int64_t blocks = (M * ldd + 255) / 256;
         if (blocks > (int64_t)sm_count() * 32) blocks = (int64_t)sm_count() * 32;
-        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, (uint16_t*)workspace, ldd, M, n);
+        repitch_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)B, ldb, copy, ldd, M, n);
         dastac_status rs = launch_status();
         if (rs != DASTAC_OK) return rs;
-        B = workspace;
+        B = copy;
         ldb = ldd;
     }
     EncodeTiledFn enc = encode_fn();
     if (!enc) return DASTAC_ERR_CUDA;
-    CUtensorMap tmap_b;
-    const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kBlockK};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return DASTAC_ERR_CUDA;
-    // 64 rows x 8 columns around column i1 (16 bytes per row, no swizzle): the factor B(x, i1) of a K block
-    CUtensorMap tmap_c;
-    const cuuint32_t cbox[2] = {8, (cuuint32_t)kBlockK};
-    if (enc(&tmap_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, cbox, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return DASTAC_ERR_CUDA;
+    CUtensorMap tmap_b, tmap_t, tmap_c;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)M};
+        const cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)kBlockK};
+        if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DASTAC_ERR_CUDA;
+    }
+    {
+        // Bt: 128 rows (features) x 64 samples per box, rows of 128 bytes, swizzled; and one row of 64 samples
+        const cuuint64_t dims[2] = {(cuuint64_t)M, (cuuint64_t)n};
+        const cuuint64_t strides[1] = {(cuuint64_t)ldt * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM};
+        const cuuint32_t cbox[2] = {(cuuint32_t)kBlockK, 1};
+        if (enc(&tmap_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            enc(&tmap_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt, dims, strides, cbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DASTAC_ERR_CUDA;
+    }
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -961,7 +1024,7 @@ dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb
     p.tiles_total = n_tiles;
     const int64_t max_clusters = sm_count() / 2;
     const int clusters = (int)(n_tiles < max_clusters ? n_tiles : max_clusters);
-    trimm_pair_kernel<kModeMoment3><<<2 * clusters, kPThreadsFused, kPSmemBytesFused, st>>>(tmap_c, tmap_b, p);
+    trimm_pair_kernel<kModeMoment3><<<2 * clusters, kPThreadsFused, kPSmemBytesFused, st>>>(tmap_t, tmap_b, tmap_c, p);
     return launch_status();
 }
 

@@ -676,8 +676,8 @@ def test_moment3_packed_tetrahedral_output(M, n):
     out.fill_(float("nan"))
     err = torch.zeros(1, dtype=torch.int32, device="cuda")
     nws = dastac.contract_workspace("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
-    assert (nws == 0) == (n % 8 == 0)          # only a row pitch that is not a multiple of 16 bytes needs scratch
-    ws = torch.empty(max(nws, 1), dtype=torch.uint8, device="cuda")
+    assert nws >= n * M * 2                     # the transposed copy of B
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
     dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA, workspace=ws, err_word=err)
     assert int(err.item()) == 0
     got = out.cpu().numpy()
@@ -689,13 +689,12 @@ def test_moment3_packed_tetrahedral_output(M, n):
     out2[: sA.nnz] = dev(A0)
     dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out2, accumulate=True, out_structure=sA, workspace=ws, err_word=err)
     assert rel_err(out2.cpu().numpy()[: sA.nnz], exp + A0, exp_abs + np.abs(A0)) <= 4e-3
-    # refused before anything runs: different tensors, wrong output structure, missing scratch for an odd row pitch
+    # refused before anything runs: different tensors, wrong output structure, missing workspace
     with pytest.raises(dastac.DastacError) as e:
         dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd.clone()], out, out_structure=sA, workspace=ws)
     assert e.value.status == 3
     with pytest.raises(dastac.DastacError):
         dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=dastac.Structure(st.upper_triangle(n)), workspace=ws)
-    if n % 8:
-        with pytest.raises(dastac.DastacError) as e:
-            dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
-        assert e.value.status == 7
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
+    assert e.value.status == 7

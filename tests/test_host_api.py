@@ -337,9 +337,10 @@ def test_moment3_plan_is_validated_on_the_host():
     nbytes = ctypes.c_size_t(123)
     ws = lib.dastac_contract_workspace
     args = (ins, 3, ctypes.byref(out), ctypes.byref(nbytes))
-    assert ws(b"xi,xj,xk->ijk", *args) == 0 and nbytes.value == 0
-    ins[0].strides[0] = ins[1].strides[0] = ins[2].strides[0] = n + 3     # 54-byte pitch: re-pitched copy
-    assert ws(b"xi,xj,xk->ijk", *args) == 0 and nbytes.value == -(-M * n * 2 // 256) * 256
+    bt = -(-n * (-(-M // 8) * 8) * 2 // 256) * 256                          # transposed copy of B, rows padded to 16 bytes
+    assert ws(b"xi,xj,xk->ijk", *args) == 0 and nbytes.value == bt
+    ins[0].strides[0] = ins[1].strides[0] = ins[2].strides[0] = n + 3     # 54-byte pitch: re-pitched copy as well
+    assert ws(b"xi,xj,xk->ijk", *args) == 0 and nbytes.value == -(-(bt + M * n * 2) // 256) * 256
     ins[0].strides[0] = ins[1].strides[0] = ins[2].strides[0] = n
     ins[2].data = 8192                                                     # third factor is another tensor
     assert ws(b"xi,xj,xk->ijk", *args) == 3
