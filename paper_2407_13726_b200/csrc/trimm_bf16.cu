@@ -290,9 +290,10 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // MODE 2 (degree-3 moments A3(i1,i2,i3) = sum_x B(x,i1) B(x,i2) B(x,i3) on i1 <= i2 <= i3, the
 // hyper-triangular domain of Section 1, stored as the packed tetrahedron): for a fixed i1 the slab is
 // the degree-2 product of Z_i1(x, i2) = B(x,i1) B(x,i2) with B, kept on i1 <= i2 <= i3.  Z is never
-// stored: the "A" operand of the MMAs lives in tensor memory and four extra warps write it.  The
+// stored: the "A" operand of the MMAs lives in tensor memory and extra warps write it (six sets of four
+// warps, one set per stage, so that the waits inside one K block's work overlap with the others').  The
 // host transposes B once (Bt, n x M, a few MB), so that row i2 of a K block is 128 contiguous bytes:
-// the producer copies the 128 x 64 block of Bt (128-byte swizzle) and the 64 values Bt(i1, x) of the
+// a second producer copies the 128 x 64 block of Bt (128-byte swizzle) and the 64 values Bt(i1, x) of the
 // slab's own column into the stage, completing on a barrier of the CTA itself; thread m of the
 // product warps reads row m of the block (eight 128-bit loads), multiplies it by the column with
 // packed bf16 multiplies (the product of two bf16 values rounded once, to nearest even) and stores
@@ -304,8 +305,8 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // 256-column accumulator and six 32-column A stages.  Tiles are (slab, P, J) with P from the block
 // that holds row i1 and J >= P; the epilogue writes at the tetrahedral position pbase(i1, i2) + i3.
 enum PairMode : int { kModeTrimm = 0, kModeMoment2 = 1, kModeMoment3 = 2 };
-constexpr int kScaleWarps = 4, kPWarpScale0 = 8;  // product warps 8..11: warp w writes tensor-memory lanes 32 (w mod 4) ..
-constexpr int kPThreadsFused = 32 * (kPWarpScale0 + kScaleWarps);  // 384 (warps 6 and 7 idle)
+constexpr int kScaleWarps = 4, kScaleSets = 6, kPWarpScale0 = 8, kPWarpRaw = 6;  // six sets of four product warps: one set per stage  // product warps 8..11: warp w writes tensor-memory lanes 32 (w mod 4) ..
+constexpr int kPThreadsFused = 32 * (kPWarpScale0 + kScaleWarps * kScaleSets);  // 1024 (warp 6: second producer, warp 7 idle)
 constexpr int kCxBytes = kBlockK * 2;                          // the 64 values B(x, i1) of a K block, per stage
 constexpr int kTmemAStage0 = kTileN, kTmemAStageCols = kBlockK / 2;  // A stages behind the single accumulator
 constexpr size_t kPSmemBytesFused = kPSmemBytes + (size_t)kPStages * kCxBytes;
@@ -325,7 +326,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     auto tmem_full = [&](int a) { return bar0 + 8u * (2 * kPStages + a); };
     auto tmem_empty = [&](int a) { return bar0 + 8u * (2 * kPStages + 2 + a); };
     auto drain_bar = [&]() { return bar0 + 8u * (2 * kPStages + 4); };
-    auto rawfull = [&](int s) { return bar0 + 8u * (2 * kPStages + 6 + s); };  // degree 3: this CTA's plain block has landed
+    auto rawfull = [&](int s) { return bar0 + 8u * (2 * kPStages + 6 + s); };   // degree 3: this CTA's block of Bt has landed
+    auto rawempty = [&](int s) { return bar0 + 8u * (3 * kPStages + 6 + s); };  // ... and has been read by the product warps
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * kPStages + 5);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
@@ -338,7 +340,10 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int s = 0; s < kPStages; ++s) {
             mbar_init(full(s), MODE == kModeMoment3 ? 1 + 2 * kScaleWarps : 1);  // degree 3: the product warps of both CTAs as well
             mbar_init(empty(s), 1);
-            if (MODE == kModeMoment3) mbar_init(rawfull(s), 1);
+            if (MODE == kModeMoment3) {
+                mbar_init(rawfull(s), 1);
+                mbar_init(rawempty(s), kScaleWarps);
+            }
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
@@ -428,10 +433,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (leader) mbar_arrive_expect_tx(full(s), MODE == kModeMoment3 ? 2 * kPBBytes : 2 * kPStageBytes);
                     const uint32_t bar = full0 + 8u * s;
                     if (MODE == kModeMoment3) {
-                        // the 128 x 64 block of Bt and the slab's own column, for this CTA's product warps
-                        mbar_arrive_expect_tx(rawfull(s), kABytes + kCxBytes);
-                        tma_load_2d_local(dst, &tmap_a, kb * kBlockK, I * kTileM, rawfull(s));
-                        tma_load_2d_local(smem_u32(cxbuf) + s * kCxBytes, &tmap_c, kb * kBlockK, p.i1_first + slot, rawfull(s));
+                        // the block of Bt for the product warps has its own producer (below)
                     } else if (MOMENT2) {
 #pragma unroll
                         for (int q = 0; q < kTileM / 64; ++q)
@@ -452,9 +454,45 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
         }
+    } else if (MODE == kModeMoment3 && warp == kPWarpRaw) {
+        // ---- second producer, degree 3 (both CTAs): the 128 x 64 block of Bt and the slab's own column for this
+        // CTA's product warps.  Its ring is released by the product warps as soon as they have read a
+        // block, not by the MMAs, so these copies run ahead of the tensor-memory stages.
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (uint32_t n = 0; n < rounds && ok; ++n) {
+                const int64_t t = tile_of(n);
+                if (t >= tiles) continue;
+                int P, J, slot;
+                decode(t, P, J, slot);
+                const int I = 2 * P + (int)rank;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kPStages;
+                    if (it >= kPStages &&
+                        !mbar_wait(rawempty(s), ((it / kPStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_arrive_expect_tx(rawfull(s), kABytes + kCxBytes);
+                    tma_load_2d_local(smem_base + s * kPStageBytes, &tmap_a, kb * kBlockK, I * kTileM, rawfull(s));
+                    tma_load_2d_local(smem_u32(cxbuf) + s * kCxBytes, &tmap_c, kb * kBlockK, p.i1_first + slot, rawfull(s));
+                }
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < 2000000) {
+                }
+            }
+        }
     } else if (MODE == kModeMoment3 && warp >= kPWarpScale0) {
         // ---- product warps (both CTAs): rows of the block times the slab's column, into tensor memory -----
-        const int m = 32 * (warp - kPWarpScale0) + lane;  // row of the block = tensor-memory lane
+        // A set of four warps handles every kScaleSets-th K block, so that the waits inside one
+        // block's work (the copy, the free stage, the tensor-memory store) overlap with the other
+        // set's.  A stage is always served by the same set (the stage count is a multiple of the sets).
+        static_assert(kPStages % kScaleSets == 0, "a stage must stay with one set of product warps");
+        const int set = (warp - kPWarpScale0) / kScaleWarps, quarter = (warp - kPWarpScale0) % kScaleWarps;
+        const int m = 32 * quarter + lane;  // row of the block = tensor-memory lane
         const uint32_t full0 = map_to_cta(full(0), 0);
         uint32_t it = 0;
         bool ok = true;
@@ -462,9 +500,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int64_t t = tile_of(n);
             if (t >= tiles) continue;
             for (int kb = 0; kb < p.k_blocks && ok; ++kb, ++it) {
+                if ((int)(it % kScaleSets) != set) continue;
                 const int s = it % kPStages;
-                // the copies into stage s are only issued once the MMAs that read tensor-memory stage s
-                // have retired, so their arrival also says that the stage may be overwritten
                 if (!mbar_wait_warp(rawfull(s), (it / kPStages) & 1, abort_flag, p.err_word, kErrFull, lane)) {
                     ok = false;
                     break;
@@ -487,7 +524,17 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         v[4 * j + e] = a.u[e];
                     }
                 }
-                tmem_st32(tmem_base + ((uint32_t)(32 * (warp - kPWarpScale0)) << 16) + kTmemAStage0 + s * kTmemAStageCols, v);
+                // the block has been read: its shared-memory slot may be refilled
+                __syncwarp();
+                if (lane == 0) mbar_arrive(rawempty(s));
+                // tensor-memory stage s is free once the MMAs that read it six K blocks ago have retired
+                if (it >= kPStages &&
+                    !mbar_wait_warp(empty(s), ((it / kPStages) - 1) & 1, abort_flag, p.err_word, kErrEmpty, lane)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                tmem_st32(tmem_base + ((uint32_t)(32 * quarter) << 16) + kTmemAStage0 + s * kTmemAStageCols, v);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
