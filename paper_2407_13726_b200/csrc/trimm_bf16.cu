@@ -305,7 +305,8 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // 256-column accumulator and six 32-column A stages.  Tiles are (slab, P, J) with P from the block
 // that holds row i1 and J >= P; the epilogue writes at the tetrahedral position pbase(i1, i2) + i3.
 enum PairMode : int { kModeTrimm = 0, kModeMoment2 = 1, kModeMoment3 = 2 };
-constexpr int kScaleWarps = 4, kScaleSets = 6, kPWarpScale0 = 8, kPWarpRaw = 6;  // six sets of four product warps: one set per stage  // product warps 8..11: warp w writes tensor-memory lanes 32 (w mod 4) ..
+// product warps 8..31: six sets of four, one set per stage; warp w writes tensor-memory lanes 32 (w mod 4) ..
+constexpr int kScaleWarps = 4, kScaleSets = 6, kPWarpScale0 = 8, kPWarpRaw = 6;
 constexpr int kPThreadsFused = 32 * (kPWarpScale0 + kScaleWarps * kScaleSets);  // 1024 (warp 6: second producer, warp 7 idle)
 constexpr int kCxBytes = kBlockK * 2;                          // the 64 values B(x, i1) of a K block, per stage
 constexpr int kTmemAStage0 = kTileN, kTmemAStageCols = kBlockK / 2;  // A stages behind the single accumulator
