@@ -365,6 +365,148 @@ unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ d
     }
 }
 
+// pack through shared memory: the source windows arrive by bulk asynchronous copies (one request of
+// up to 4 KiB per window instead of 2 x 256 separate 16-byte loads), so a warp always has a whole
+// window in flight while it realigns and stores the previous one.  A warp owns two window buffers
+// and two mbarriers; nothing is shared between warps.  Per window: the packed chunks that lie
+// wholly inside the row are served from the buffer (two aligned 128-bit shared loads around the
+// chunk's source bytes, the same word select + funnel shift as above, one 128-bit store); the at
+// most two chunks a row shares with its neighbours are written element by element from global
+// memory.  The source may be read up to the end of the 16-byte granule that holds a needed element.
+constexpr int kBulkWin = 256;                          // chunks (16 bytes each) per window
+constexpr int kBulkBufBytes = kBulkWin * 16 + 16;      // + the granule after the last chunk
+constexpr int kBulkSmemBytes = kWarpsPerBlock * 2 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;
+constexpr long long kBulkWaitBudget = 2000000000LL;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+template <typename T>
+__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
+pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed, int64_t rows,
+                 int windows_per_row) {
+    constexpr int E = 16 / sizeof(T);
+    extern __shared__ __align__(128) uint8_t bulk_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* buf0 = bulk_smem + warp * 2 * kBulkBufBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * 2 * kBulkBufBytes) + warp * 2;
+    if (lane == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+
+    // what a window needs, worked out by every lane (uniform in the warp)
+    struct Win {
+        int64_t ps, pe;          // the row's span in the packed stream
+        int64_t c_lo, c_hi;      // chunks of the window that lie wholly inside the row: [c_lo, c_hi)
+        int64_t c0;              // first chunk of the window
+        const T* drow;           // drow[p] = element stored at position p
+        uintptr_t g0;            // aligned source address under chunk c_lo
+        uint32_t sh, bytes;      // misalignment of the source (bytes), size of the bulk copy
+        bool live;
+    };
+    const int64_t items = rows * windows_per_row;
+    const int64_t warps = (int64_t)gridDim.x * kWarpsPerBlock;
+    auto describe = [&](int64_t item, Win& w) {
+        w.live = false;
+        w.bytes = 0;
+        w.sh = 0;
+        w.g0 = 0;
+        w.c_lo = w.c_hi = 0;
+        if (item >= items) return;
+        const int64_t row = item / windows_per_row;
+        const int win = (int)(item - row * windows_per_row);
+        int32_t idx[3] = {0, 0, 0};
+        if (m.rank == 2) {
+            idx[0] = (int32_t)row;
+        } else if (m.rank == 3) {
+            const int64_t q = row / m.dims[1];
+            idx[1] = (int32_t)(row - q * m.dims[1]);
+            idx[0] = (int32_t)q;
+        }
+        int64_t jlo = 0, jhi = 0, pbase = 0;
+        if (!row_span(m, idx, jlo, jhi, pbase)) return;
+        w.ps = pbase + jlo;
+        w.pe = pbase + jhi;
+        w.c0 = w.ps / E + (int64_t)win * kBulkWin;
+        if (w.c0 * E >= w.pe) return;
+        w.live = true;
+        w.drow = dense + dense_row_offset(m, st, idx) - pbase;
+        const int64_t first_in = (w.ps + E - 1) / E, last_in = w.pe / E;  // chunks wholly inside: [first_in, last_in)
+        w.c_lo = w.c0 > first_in ? w.c0 : first_in;
+        w.c_hi = w.c0 + kBulkWin < last_in ? w.c0 + kBulkWin : last_in;
+        if (w.c_hi > w.c_lo) {
+            const uintptr_t a = reinterpret_cast<uintptr_t>(w.drow + w.c_lo * E);
+            w.sh = (uint32_t)(a & 15);
+            w.g0 = a - w.sh;
+            w.bytes = (uint32_t)(w.c_hi - w.c_lo) * 16 + (w.sh ? 16u : 0u);
+        }
+    };
+    auto issue = [&](const Win& w, int b) {
+        if (w.bytes == 0 || lane != 0) return;
+        const uint32_t bar = smem_addr(&bars[b]);
+        // the warp's earlier generic-proxy reads of this buffer come before the async-proxy overwrite
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(w.bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_addr(buf0 + b * kBulkBufBytes)),
+                     "l"(w.g0), "r"(w.bytes), "r"(bar)
+                     : "memory");
+    };
+
+    Win cur, nxt;
+    int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + warp;
+    describe(item, cur);
+    issue(cur, 0);
+    uint32_t phases = 0;  // bit b: parity of the next completion of buffer b
+    int b = 0;
+    for (; item < items; item += warps, b ^= 1) {
+        describe(item + warps, nxt);
+        // the other buffer was consumed one iteration ago (all lanes passed the __syncwarp below)
+        issue(nxt, b ^ 1);
+        if (cur.live) {
+            if (cur.bytes) {
+                const uint32_t bar = smem_addr(&bars[b]);
+                const long long t0 = clock64();
+                uint32_t done = 0;
+                while (!done) {
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t"
+                        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                        "selp.u32 %0, 1, 0, p;\n\t}"
+                        : "=r"(done)
+                        : "r"(bar), "r"((phases >> b) & 1u)
+                        : "memory");
+                    if (!done && clock64() - t0 > kBulkWaitBudget) break;  // never expected; gives up instead of spinning
+                }
+                phases ^= 1u << b;
+                const uint8_t* src = buf0 + b * kBulkBufBytes;
+                const uint4 zero4 = make_uint4(0, 0, 0, 0);
+                for (int64_t c = cur.c_lo + lane; c < cur.c_hi; c += 32) {
+                    const uint4* g = reinterpret_cast<const uint4*>(src + (c - cur.c_lo) * 16);
+                    const uint4 lo = g[0];
+                    const uint4 hi = cur.sh ? g[1] : zero4;
+                    *reinterpret_cast<uint4*>(packed + c * E) = realign16(lo, hi, cur.sh);
+                }
+            }
+            // chunks of this window that the row shares with a neighbour (or the tail of the stream)
+            for (int side = 0; side < 2; ++side) {
+                const int64_t c = side == 0 ? cur.ps / E : cur.pe / E;
+                const bool mine = c >= cur.c0 && c < cur.c0 + kBulkWin && (c < cur.c_lo || c >= cur.c_hi) &&
+                                  !(side == 1 && c == cur.ps / E) && c * E < cur.pe;
+                if (mine && lane < E) {
+                    const int64_t p = c * E + lane;
+                    if (p >= cur.ps && p < cur.pe) packed[p] = cur.drow[p];
+                    else if (p >= m.count) packed[p] = T(0);
+                }
+            }
+        }
+        __syncwarp();
+        cur = nxt;
+    }
+}
+
 bool row_path(const IndexMap& m) {
     return (m.kind == kDense || (m.kind == kUpper && m.rank == 2) || m.kind == kLower || m.kind == kTetrahedron ||
             m.kind == kBandExact || m.kind == kUpperShifted || m.kind == kBandOffsets) &&
@@ -429,6 +571,32 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
         if (gpr > wpr) gpr = wpr;
         const int64_t wpg = (wpr + gpr - 1) / gpr;
         gpr = (wpr + wpg - 1) / wpg;
+        if (aligned16(dense)) {
+            // windows arrive by bulk copies into shared memory
+            static bool attr_set[64];
+            int dev = 0;
+            cudaGetDevice(&dev);
+            if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+                if (cudaFuncSetAttribute(pack_bulk_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kBulkSmemBytes) != cudaSuccess ||
+                    cudaFuncSetAttribute(pack_bulk_kernel<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kBulkSmemBytes) != cudaSuccess)
+                    return DASTAC_ERR_CUDA;
+                attr_set[dev] = true;
+            }
+            const int64_t bwpr = ((m.dims[m.rank - 1] + E - 1) / E + 2 + kBulkWin - 1) / kBulkWin;
+            const int64_t items = rows * bwpr;
+            int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
+            if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
+            if (bwpr > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
+            if (dtype == DASTAC_F32)
+                pack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                    m, (const uint32_t*)dense, st, (uint32_t*)packed, rows, (int)bwpr);
+            else
+                pack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                    m, (const uint16_t*)dense, st, (uint16_t*)packed, rows, (int)bwpr);
+            return launch_status();
+        }
         const int grid = grid_for(rows * gpr * 32, 32 * kWarpsPerBlock);
         if (dtype == DASTAC_F32)
             pack_stream_kernel<uint32_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
