@@ -507,6 +507,145 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
     }
 }
 
+// unpack through shared memory, the mirror image: a window is 256 aligned chunks of a dense row; the
+// packed elements it needs are one contiguous run, fetched by one bulk copy; chunks wholly inside
+// the set are realigned from the buffer, chunks wholly outside are zero stores, the at most two
+// chunks that straddle an end of the row's interval are assembled element by element.
+template <typename T>
+__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
+unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st, int64_t rows,
+                   int windows_per_row) {
+    constexpr int E = 16 / sizeof(T);
+    extern __shared__ __align__(128) uint8_t bulk_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* buf0 = bulk_smem + warp * 2 * kBulkBufBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * 2 * kBulkBufBytes) + warp * 2;
+    if (lane == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const int inner = (int)(m.rank == 3 ? m.dims[2] : m.rank == 2 ? m.dims[1] : m.dims[0]);
+
+    struct Win {
+        int jlo, jhi;        // the row's interval of stored columns
+        int wlo, whi;        // columns of the window (whi clipped to the row)
+        int c_lo, c_hi;      // columns [c_lo, c_hi): chunks wholly inside the interval, multiples of E
+        T* drow;
+        const T* prow;       // prow[j] = stored element (row, j)
+        uintptr_t g0;        // aligned source address under column c_lo
+        uint32_t sh, bytes;
+        bool live;
+    };
+    const int64_t items = rows * windows_per_row;
+    const int64_t warps = (int64_t)gridDim.x * kWarpsPerBlock;
+    auto describe = [&](int64_t item, Win& w) {
+        w.live = false;
+        w.bytes = 0;
+        w.sh = 0;
+        w.g0 = 0;
+        w.c_lo = w.c_hi = 0;
+        if (item >= items) return;
+        const int64_t row = item / windows_per_row;
+        const int win = (int)(item - row * windows_per_row);
+        w.wlo = win * kBulkWin * E;
+        if (w.wlo >= inner) return;
+        w.whi = w.wlo + kBulkWin * E < inner ? w.wlo + kBulkWin * E : inner;
+        w.live = true;
+        int32_t idx[3] = {0, 0, 0};
+        if (m.rank == 2) {
+            idx[0] = (int32_t)row;
+        } else if (m.rank == 3) {
+            const int64_t q = row / m.dims[1];
+            idx[1] = (int32_t)(row - q * m.dims[1]);
+            idx[0] = (int32_t)q;
+        }
+        int64_t jlo64 = 0, jhi64 = 0, pbase = 0;
+        if (!row_span(m, idx, jlo64, jhi64, pbase)) jlo64 = jhi64 = 0;
+        w.jlo = (int)jlo64;
+        w.jhi = (int)jhi64;
+        w.drow = dense + dense_row_offset(m, st, idx);
+        w.prow = packed + pbase;
+        // whole chunks inside both the interval and the window
+        int lo = w.jlo > w.wlo ? w.jlo : w.wlo, hi = w.jhi < w.whi ? w.jhi : w.whi;
+        lo = (lo + E - 1) / E * E;
+        hi = hi / E * E;
+        if (hi > lo) {
+            w.c_lo = lo;
+            w.c_hi = hi;
+            const uintptr_t a = reinterpret_cast<uintptr_t>(w.prow + lo);
+            w.sh = (uint32_t)(a & 15);
+            w.g0 = a - w.sh;
+            w.bytes = (uint32_t)((hi - lo) / E) * 16 + (w.sh ? 16u : 0u);
+        }
+    };
+    auto issue = [&](const Win& w, int b) {
+        if (w.bytes == 0 || lane != 0) return;
+        const uint32_t bar = smem_addr(&bars[b]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(w.bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_addr(buf0 + b * kBulkBufBytes)),
+                     "l"(w.g0), "r"(w.bytes), "r"(bar)
+                     : "memory");
+    };
+    union Chunk {
+        uint4 v;
+        T e[E];
+    };
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+
+    Win cur, nxt;
+    int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + warp;
+    describe(item, cur);
+    issue(cur, 0);
+    uint32_t phases = 0;
+    int b = 0;
+    for (; item < items; item += warps, b ^= 1) {
+        describe(item + warps, nxt);
+        issue(nxt, b ^ 1);
+        if (cur.live) {
+            if (cur.bytes) {
+                const uint32_t bar = smem_addr(&bars[b]);
+                const long long t0 = clock64();
+                uint32_t done = 0;
+                while (!done) {
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t"
+                        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                        "selp.u32 %0, 1, 0, p;\n\t}"
+                        : "=r"(done)
+                        : "r"(bar), "r"((phases >> b) & 1u)
+                        : "memory");
+                    if (!done && clock64() - t0 > kBulkWaitBudget) break;
+                }
+                phases ^= 1u << b;
+            }
+            const uint8_t* src = buf0 + b * kBulkBufBytes;
+            for (int j0 = cur.wlo + lane * E; j0 < cur.whi; j0 += 32 * E) {
+                Chunk out;
+                out.v = zero4;
+                if (j0 >= cur.c_lo && j0 + E <= cur.c_hi) {
+                    const uint4* g = reinterpret_cast<const uint4*>(src + (size_t)(j0 - cur.c_lo) / E * 16);
+                    out.v = realign16(g[0], cur.sh ? g[1] : zero4, cur.sh);
+                } else if (j0 + E > cur.jlo && j0 < cur.jhi) {  // straddles an end of the interval
+#pragma unroll
+                    for (int e = 0; e < E; ++e)
+                        if (j0 + e >= cur.jlo && j0 + e < cur.jhi) out.e[e] = cur.prow[j0 + e];
+                }
+                if (j0 + E <= inner) {
+                    *reinterpret_cast<uint4*>(cur.drow + j0) = out.v;
+                } else {
+                    for (int e = 0; e < E && j0 + e < inner; ++e) cur.drow[j0 + e] = out.e[e];
+                }
+            }
+        }
+        __syncwarp();
+        cur = nxt;
+    }
+}
+
 bool row_path(const IndexMap& m) {
     return (m.kind == kDense || (m.kind == kUpper && m.rank == 2) || m.kind == kLower || m.kind == kTetrahedron ||
             m.kind == kBandExact || m.kind == kUpperShifted || m.kind == kBandOffsets) &&
@@ -646,6 +785,32 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
         if (gpr > wpr) gpr = wpr;
         const int64_t wpg = (wpr + gpr - 1) / gpr;
         gpr = (wpr + wpg - 1) / wpg;
+        {
+            static bool attr_set[64];
+            int dev = 0;
+            cudaGetDevice(&dev);
+            if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+                if (cudaFuncSetAttribute(unpack_bulk_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kBulkSmemBytes) != cudaSuccess ||
+                    cudaFuncSetAttribute(unpack_bulk_kernel<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kBulkSmemBytes) != cudaSuccess)
+                    return DASTAC_ERR_CUDA;
+                attr_set[dev] = true;
+            }
+            const int64_t bwpr = (chunks_per_row + kBulkWin - 1) / kBulkWin;
+            const int64_t items = rows * bwpr;
+            int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
+            if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
+            if (bwpr <= 0x7fffffffLL && m.dims[m.rank - 1] < (int64_t(1) << 30)) {
+                if (dtype == DASTAC_F32)
+                    unpack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                        m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)bwpr);
+                else
+                    unpack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                        m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)bwpr);
+                return launch_status();
+            }
+        }
         const int grid = grid_for(rows * gpr * 32, 32 * kWarpsPerBlock);
         if (dtype == DASTAC_F32)
             unpack_stream_kernel<uint32_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
