@@ -533,8 +533,8 @@ TRAFFIC = {
     "ttm_ut": int(67.207424e6 + 18.528000e6),
     "bandmm_exact": int(42.108160e6 + 2.613248e6),
     "moment2_bf16": int(1.410541e9 + 22.173440e6),   # full size, DRAM counters only (one pass)
-    "pack_bf16": int(67.683584e6 + 27.079680e6),
-    "unpack_bf16": int(67.140864e6 + 78.835712e6),
+    "pack_bf16": int(67.666432e6 + 18.678784e6),
+    "unpack_bf16": int(67.146496e6 + 76.666112e6),
 }
 
 

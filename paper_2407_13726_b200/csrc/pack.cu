@@ -1,17 +1,18 @@
 // Index-map batch kernels and compress / decompress (Section 3, "Data Layout Compression":
 // iterate over the accessed indices and copy the data in and out of the packed buffer).
 //
-// Stream kernels (the fast path, unit inner stride): for fixed outer indices the innermost indices
-// of the set are one interval [jlo, jhi) stored contiguously at pbase + j, with pbase the hoisted
-// part of the ranking polynomial.
-//   pack    a lane owns 16-byte aligned chunks of the PACKED span of a row.  The matching dense
-//           elements start at an arbitrary element offset, so the lane loads the two aligned
-//           16-byte granules that cover them and shifts them into place in registers.  Chunks that
-//           a row shares with its neighbour (first and last of the row) are written element by
-//           element by both rows.
-//   unpack  a lane owns 16-byte aligned chunks of a DENSE row; the packed source is realigned the
-//           same way, elements outside [jlo, jhi) become zero, and the zero fill of the rest of the
-//           box is the same pass.
+// Row kernels (the fast path, unit inner stride): for fixed outer indices the innermost indices of
+// the set are one interval [jlo, jhi) stored contiguously at pbase + j, with pbase the hoisted part
+// of the ranking polynomial.  Source and destination of a row differ in their alignment modulo 16
+// bytes by a constant, so data moves in aligned 16-byte chunks of the DESTINATION and every chunk
+// is cut out of the two aligned source granules that cover it (word select + funnel shift).
+//   pack    destination = aligned chunks of the packed span of a row.  Chunks that a row shares
+//           with its neighbour (first and last of the row) are written element by element by both.
+//   unpack  destination = aligned chunks of a dense row; elements outside [jlo, jhi) become zero,
+//           so the zero fill of the rest of the box is the same pass.
+// In both, a warp fetches the source of a whole window (256 chunks) with one bulk asynchronous
+// copy into its own shared-memory buffer and works on the previous window meanwhile; pack keeps a
+// register-only form for dense tensors whose base is not 16-byte aligned.
 // Generic kernels (any strides, the padded-diagonal layout, the redundancy swap): pack walks the
 // packed stream, a thread unranks the first of its positions and steps with index increments;
 // unpack walks the dense box and ranks every point.
@@ -250,115 +251,6 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
                         if (p >= ps && p < pe) packed[p] = drow[p];
                         else if (p >= m.count) packed[p] = T(0);
                     }
-                }
-            }
-        }
-    }
-}
-
-// unpack: a warp item is a run of windows (32 * kUnroll chunks each) of one dense row, so the row's
-// span and base are worked out once per item; the zero fill outside the set and the copy are the
-// same pass.
-template <typename T>
-__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
-unpack_stream_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st,
-                     int64_t rows, int groups_per_row, int windows_per_group) {
-    constexpr int E = 16 / sizeof(T);
-    const int lane = threadIdx.x & 31;
-    const int inner = (int)(m.rank == 3 ? m.dims[2] : m.rank == 2 ? m.dims[1] : m.dims[0]);
-    const int64_t cap = (m.count + E - 1) / E * E;
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    union Chunk {
-        uint4 v;
-        T e[E];
-    };
-    const int64_t warps = (int64_t)gridDim.x * kWarpsPerBlock;
-    for (int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + (threadIdx.x >> 5); item < rows * groups_per_row;
-         item += warps) {
-        int64_t row = item;
-        int grp = 0;
-        if (groups_per_row > 1) {
-            row = item / groups_per_row;
-            grp = (int)(item - row * groups_per_row);
-        }
-        int32_t idx[3] = {0, 0, 0};
-        if (m.rank == 2) {
-            idx[0] = (int32_t)row;
-        } else if (m.rank == 3) {
-            const int64_t q = row / m.dims[1];
-            idx[1] = (int32_t)(row - q * m.dims[1]);
-            idx[0] = (int32_t)q;
-        }
-        int64_t jlo64 = 0, jhi64 = 0, pbase = 0;
-        if (!row_span(m, idx, jlo64, jhi64, pbase)) jlo64 = jhi64 = 0;
-        const int jlo = (int)jlo64, jhi = (int)jhi64;
-        T* drow = dense + dense_row_offset(m, st, idx);
-        const T* prow = packed + pbase;  // prow[j] = stored element (row, j)
-        // the vector path reads the two aligned granules around a chunk: both must lie inside the buffer
-        const int jsafe = (int)((cap - pbase - 2 * E < (int64_t)inner) ? cap - pbase - 2 * E : (int64_t)inner);
-        for (int win = grp * windows_per_group; win < (grp + 1) * windows_per_group; ++win) {
-            const int jfirst = (win * (32 * kUnroll) + lane) * E;
-            if (win * (32 * kUnroll) * E >= inner) break;
-            const int wlo = win * (32 * kUnroll) * E, whi = wlo + 32 * kUnroll * E;  // columns of the window
-            if (whi <= inner && (whi <= jlo || wlo >= jhi)) {
-                // nothing of the set in this window: plain zero fill
-                uint4* dp = reinterpret_cast<uint4*>(drow + jfirst);
-#pragma unroll
-                for (int u = 0; u < kUnroll; ++u) dp[32 * u] = zero4;
-                continue;
-            }
-            if (wlo >= jlo && whi <= jhi && whi <= inner && whi - E <= jsafe) {
-                // the whole window is stored: one shift per row, addresses are one pointer plus constants
-                const uintptr_t paddr = reinterpret_cast<uintptr_t>(prow + jfirst);
-                const uint32_t shw = (uint32_t)(paddr & 15);
-                const uint4* sp = reinterpret_cast<const uint4*>(paddr - shw);
-                uint4* dp = reinterpret_cast<uint4*>(drow + jfirst);
-                uint4 lo[kUnroll], hi[kUnroll];
-#pragma unroll
-                for (int u = 0; u < kUnroll; ++u) {
-                    lo[u] = __ldg(sp + 32 * u);
-                    hi[u] = shw ? __ldg(sp + 32 * u + 1) : zero4;
-                }
-#pragma unroll
-                for (int u = 0; u < kUnroll; ++u) dp[32 * u] = realign16(lo[u], hi[u], shw);
-                continue;
-            }
-            uint4 lo[kUnroll], hi[kUnroll];
-            uint32_t sh[kUnroll];
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int j0 = jfirst + 32 * u * E;
-                sh[u] = 0xffffffffu;  // no vector load for this chunk
-                if (j0 < inner && j0 + E > jlo && j0 < jhi && j0 <= jsafe) {
-                    const uintptr_t addr = reinterpret_cast<uintptr_t>(prow + j0);
-                    sh[u] = (uint32_t)(addr & 15);
-                    const uint4* src = reinterpret_cast<const uint4*>(addr - sh[u]);
-                    lo[u] = __ldg(src);
-                    hi[u] = sh[u] ? __ldg(src + 1) : zero4;
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int j0 = jfirst + 32 * u * E;
-                if (j0 >= inner) break;
-                Chunk out;
-                out.v = zero4;
-                if (sh[u] != 0xffffffffu) {
-                    out.v = realign16(lo[u], hi[u], sh[u]);
-                    if (j0 < jlo || j0 + E > jhi) {
-#pragma unroll
-                        for (int e = 0; e < E; ++e)
-                            if (j0 + e < jlo || j0 + e >= jhi) out.e[e] = T(0);
-                    }
-                } else if (j0 + E > jlo && j0 < jhi) {  // the last granules of the packed buffer
-#pragma unroll
-                    for (int e = 0; e < E; ++e)
-                        if (j0 + e >= jlo && j0 + e < jhi) out.e[e] = prow[j0 + e];
-                }
-                if (j0 + E <= inner) {
-                    *reinterpret_cast<uint4*>(drow + j0) = out.v;
-                } else {
-                    for (int e = 0; e < E && j0 + e < inner; ++e) drow[j0 + e] = out.e[e];
                 }
             }
         }
@@ -778,13 +670,6 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
     if (row_path(m) && vector_ok) {
         const int64_t rows = box / m.dims[m.rank - 1];
         const int64_t chunks_per_row = (m.dims[m.rank - 1] + E - 1) / E;
-        const int64_t wpr = (chunks_per_row + 32 * kUnroll - 1) / (32 * kUnroll);
-        // a warp takes a whole row unless there are too few rows to fill the GPU
-        const int64_t want_items = (int64_t)sm_count() * 3 * kWarpsPerBlock * 4;
-        int64_t gpr = rows >= want_items ? 1 : (want_items + rows - 1) / rows;
-        if (gpr > wpr) gpr = wpr;
-        const int64_t wpg = (wpr + gpr - 1) / gpr;
-        gpr = (wpr + wpg - 1) / wpg;
         {
             static bool attr_set[64];
             int dev = 0;
@@ -801,24 +686,15 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
             const int64_t items = rows * bwpr;
             int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
             if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
-            if (bwpr <= 0x7fffffffLL && m.dims[m.rank - 1] < (int64_t(1) << 30)) {
-                if (dtype == DASTAC_F32)
-                    unpack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
-                        m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)bwpr);
-                else
-                    unpack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
-                        m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)bwpr);
-                return launch_status();
-            }
+            if (bwpr > 0x7fffffffLL || m.dims[m.rank - 1] > (int64_t(1) << 30)) return DASTAC_ERR_OVERFLOW;
+            if (dtype == DASTAC_F32)
+                unpack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                    m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)bwpr);
+            else
+                unpack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                    m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)bwpr);
+            return launch_status();
         }
-        const int grid = grid_for(rows * gpr * 32, 32 * kWarpsPerBlock);
-        if (dtype == DASTAC_F32)
-            unpack_stream_kernel<uint32_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
-                m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)gpr, (int)wpg);
-        else
-            unpack_stream_kernel<uint16_t><<<grid, 32 * kWarpsPerBlock, 0, (cudaStream_t)stream>>>(
-                m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)gpr, (int)wpg);
-        return launch_status();
     }
     const int last = m.rank - 1;
     int64_t rows = box / m.dims[last];
