@@ -111,7 +111,9 @@ PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33),
               st.tetrahedron(2), st.tetrahedron(37), st.upper_half_cube(11, 17, 3),
               st.upper_half_cube(17, 11, 6), st.dense_box([6, 10]), st.band_exact(11, 5), st.band_exact(130, 7),
               st.band_exact(1000, 32), st.sub_triangle(11, 4), st.sub_triangle(130, 77), st.sub_triangle(1000, 333),
-              st.offset_band(40, 9, 9), st.offset_band(130, -50, 7), st.offset_band(1000, -3, 40), st.offset_band(90, -85, 80)]
+              st.offset_band(40, 9, 9), st.offset_band(130, -50, 7), st.offset_band(1000, -3, 40), st.offset_band(90, -85, 80),
+              st.dense_box([7]), st.dense_box([5000]), st.dense_box([3, 4, 5]), st.dense_box([2, 3, 2100]), st.tetrahedron(130),
+              st.lower_triangle(2100), st.upper_triangle(4100)]
 
 
 @pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
