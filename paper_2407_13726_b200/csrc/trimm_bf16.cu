@@ -24,6 +24,10 @@
 //     swizzle copies verbatim.
 //  2. trimm_pair: warp-specialised pipeline (details at the kernel).
 //
+// The same CTA-pair pipeline also evaluates the polynomial-regression moments of Table 1 (degree 2:
+// B^T B on i1 <= i2 with packed output; degree 3: the packed tetrahedron i1 <= i2 <= i3, with the
+// scaled operand in tensor memory); their differences are described at the kernel.
+//
 // Every wait on an mbarrier is bounded by a clock budget; on expiry the thread records a code in
 // the error word and the CTA drains: nothing can spin forever.
 #include <cuda.h>
