@@ -3,8 +3,12 @@
 
 One step = one pass over every kernel of the path on seeded synthetic inputs of the five
 configurations: upper-triangular matrix-vector (single and 512-instance batch), band x dense,
-symmetric matrix-vector, tetrahedral MTTKRP, bf16 triangular x dense, plus pack and unpack of the
-bf16 triangle.  Prints one JSON line (see README/DESIGN for the keys).
+symmetric matrix-vector, tetrahedral MTTKRP, bf16 triangular x dense, pack and unpack of the bf16
+triangle, plus four further rules (band x dense over the exact band layout, tensor times matrix
+over the half cube, degree-2 and degree-3 polynomial-regression moments).  Prints one JSON line:
+whole-step throughput, per-kernel times (inside the step and alone in steady state), the roofline
+object of the largest configuration kernel, end-to-end throughput with host operands, the CPU
+oracle's throughput on a bounded sample, clocks during the timed region.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--small]
 """
