@@ -67,10 +67,11 @@ def _load():
         lib.orc_ttm.argtypes = [P, i64, vp, vp, vp, i64, vp, vp]
         lib.orc_moment2.argtypes = [P, ctypes.c_int, i64, vp, vp, i64, vp, vp]
         lib.orc_moment3.argtypes = [P, ctypes.c_int, i64, vp, vp, i64, vp, vp]
+        lib.orc_hadamard.argtypes = [P, vp, vp, vp, vp]
         lib.orc_num_threads.restype = ctypes.c_int
         for name in ("orc_rank_table", "orc_unrank_table", "orc_pack", "orc_unpack", "orc_band_pack",
                      "orc_band_unpack", "orc_band_slot_table", "orc_matvec", "orc_symv",
-                     "orc_matmat", "orc_mttkrp", "orc_ttm", "orc_moment2", "orc_moment3"):
+                     "orc_matmat", "orc_mttkrp", "orc_ttm", "orc_moment2", "orc_moment3", "orc_hadamard"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -288,4 +289,16 @@ def moment3(desc, B, sel=None):
     out, out_abs = np.empty((len(sel), n, n)), np.empty((len(sel), n, n))
     _load().orc_moment3(h.ref, int(is_bf16), len(sel), sel.ctypes.data, B.ctypes.data, B.shape[0],
                         out.ctypes.data, out_abs.ctypes.data)
+    return out, out_abs
+
+
+def hadamard(desc, B, C):
+    """``A[idx] = [idx in set] B[idx] C[idx]`` over the whole box (dense fp32 arrays in, dense fp64
+    arrays out, zero outside the set)."""
+    h = _Held(desc)
+    B, C = _f32(B), _f32(C)
+    shape = tuple(int(v) for v in h.dims)
+    assert B.shape == shape and C.shape == shape
+    out, out_abs = np.empty(shape), np.empty(shape)
+    _load().orc_hadamard(h.ref, B.ctypes.data, C.ctypes.data, out.ctypes.data, out_abs.ctypes.data)
     return out, out_abs

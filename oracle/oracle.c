@@ -378,6 +378,25 @@ void orc_moment3(const orc_desc* d, int is_bf16, int64_t nsel, const int64_t* se
     }
 }
 
+/* A[idx] = [ idx in set ] B[idx] * C[idx]   (A(i,j,k) := B(i,j,k) * C(i,j,k), Table 1 "THP", the tensor
+ * Hadamard product with a structured B and a dense C; any rank up to 3).  B, C and out are dense
+ * arrays over the box; outside the set the result is 0. */
+void orc_hadamard(const orc_desc* d, const float* B, const float* C, double* out, double* out_abs) {
+    int64_t total = 1;
+    for (int k = 0; k < d->rank; ++k) total *= d->dims[k];
+    for (int64_t t = 0; t < total; ++t) out[t] = out_abs[t] = 0.0;
+    if (box_empty(d)) return;
+    int64_t idx[ORC_MAX_RANK] = {0, 0, 0, 0};
+    do {
+        if (in_domain(d, idx)) {
+            const int64_t lin = dense_linear(d, idx);
+            const double p = (double)B[lin] * (double)C[lin];
+            out[lin] = p;
+            out_abs[lin] = fabs(p);
+        }
+    } while (box_next(d, idx));
+}
+
 /* Thread count the contractions above will use. */
 #ifdef _OPENMP
 #include <omp.h>

@@ -482,3 +482,22 @@ def test_moment3_packed_tetrahedral_output():
     packed = oracle.pack(d, out)
     assert packed.shape == (n * (n + 1) * (n + 2) // 6,)
     assert packed[oracle.rank_point(d, (1, 3, 4))] == out[1, 3, 4] and packed[0] == out[0, 0, 0]
+
+
+def test_hadamard_structured_times_dense():
+    """Tensor Hadamard product A(i,j,k) = B(i,j,k) C(i,j,k) with a structured B (Table 1, THP)."""
+    for desc in (st.upper_half_cube(5, 7, 3), st.tetrahedron(6), st.upper_triangle(9), st.band_exact(8, 2), st.dense_box([4])):
+        shape = tuple(desc.dims)
+        B = synth.dense(10, 0, shape)
+        C = synth.dense(10, 1, shape)
+        out, outa = oracle.hadamard(desc, B, C)
+        mask = oracle.rank_table(desc) >= 0
+        ref = np.where(mask, B.astype(np.float64) * C.astype(np.float64), 0.0)   # plain definition in numpy
+        assert np.array_equal(out, ref) and np.array_equal(outa, np.abs(ref))
+        # closed forms: C = 1 returns the masked B; both all ones give the indicator of the set
+        same, _ = oracle.hadamard(desc, B, np.ones(shape, np.float32))
+        assert np.array_equal(same, np.where(mask, B, 0).astype(np.float64))
+        ones, _ = oracle.hadamard(desc, np.ones(shape, np.float32), np.ones(shape, np.float32))
+        assert ones.sum() == oracle.count(desc)
+        # the packed result is the element-wise product of the two packed operands
+        assert np.array_equal(oracle.pack(desc, out), oracle.pack(desc, B).astype(np.float64) * oracle.pack(desc, C))
