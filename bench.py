@@ -4,8 +4,8 @@
 One step = one pass over every kernel of the path on seeded synthetic inputs of the five
 configurations: upper-triangular matrix-vector (single and 512-instance batch), band x dense,
 symmetric matrix-vector, tetrahedral MTTKRP, bf16 triangular x dense, pack and unpack of the bf16
-triangle, plus four further rules (band x dense over the exact band layout, tensor times matrix
-over the half cube, degree-2 and degree-3 polynomial-regression moments).  Prints one JSON line:
+triangle, plus five further rules (band x dense over the exact band layout, tensor times matrix and
+tensor Hadamard product over the half cube, degree-2 and degree-3 polynomial-regression moments).  Prints one JSON line:
 whole-step throughput, per-kernel times (inside the step and alone in steady state), the roofline
 object of the largest configuration kernel, end-to-end throughput with host operands, the CPU
 oracle's throughput on a bounded sample, clocks during the timed region.
@@ -86,12 +86,14 @@ def accounting(z):
         "moment2_bf16": dict(flops=2 * tri(N7) * M7, bytes=2 * M7 * N7 + 4 * tri(N7), bound="tensor"),
         # widened row: degree-3 moments on i1 <= i2 <= i3 (two multiplies and an add per term), packed tetrahedron out
         "moment3_bf16": dict(flops=3 * tet(N8) * M8, bytes=2 * M8 * N8 + 4 * tet(N8), bound="tensor"),
+        # widened row: tensor Hadamard product over the upper half cube: packed B, the set's part of dense C, packed out
+        "thp_ut": dict(flops=tri(N6) * Q6, bytes=4 * 3 * tri(N6) * Q6, bound="hbm"),
     }
     return acc
 
 
 ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
-         "moment2_bf16", "moment3_bf16", "symv"]
+         "moment2_bf16", "moment3_bf16", "thp_ut", "symv"]
 # the kernels of the five configurations; the others are widened rows and never the roofline's kernel
 CONFIG_KERNELS = ("trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv")
 
@@ -163,6 +165,13 @@ def generate_host(z, pin, only=None):
         synth.upper_half_cube_stream(5, 0, N6, N6, Q6, out=a6)
         h["ttm_ut"] = dict(desc=st.upper_half_cube(N6, N6, Q6), out_desc=st.upper_half_cube(N6, N6, K6), A=host(a6),
                            ins=[host(synth.dense(5, 1, (K6, Q6)))], out=(cap(tri(N6) * K6, 4),))
+    if want("thp_ut"):
+        N6, Q6 = z["N6"], z["Q6"]
+        a9 = np.zeros(cap(tri(N6) * Q6, 4), np.float32)
+        synth.upper_half_cube_stream(10, 0, N6, N6, Q6, out=a9)
+        dh = st.upper_half_cube(N6, N6, Q6)
+        h["thp_ut"] = dict(desc=dh, out_desc=dh, A=host(a9), ins=[host(synth.dense(10, 1, (N6, N6, Q6)))],
+                           out=(cap(tri(N6) * Q6, 4),))
     if want("moment2_bf16"):
         N7, M7 = z["N7"], z["M7"]
         b7 = host(synth.dense(6, 0, (M7, N7), dist=synth.NORMAL, bf16=True), True)
@@ -179,7 +188,7 @@ def generate_host(z, pin, only=None):
 
 EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
         "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
-        "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij", "moment3_bf16": "xi,xj,xk->ijk"}
+        "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij", "moment3_bf16": "xi,xj,xk->ijk", "thp_ut": "ijk,ijk->ijk"}
 
 
 # ---- clocks ---------------------------------------------------------------------------------------------
@@ -468,7 +477,7 @@ def run_gpu(args):
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 (configs 1-4), bf16 inputs with f32 accumulate (config 5)",
             "data": "synthetic",
-            "config": {"workload": "all five configs per step, plus four widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features; degree-3 moments of M8 x N8): "
+            "config": {"workload": "all five configs per step, plus five widened rows (band x dense over the exact band layout; tensor times matrix and tensor Hadamard product N6,Q6,K6; degree-2 moments of M7 samples x N7 features; degree-3 moments of M8 x N8): "
                                    + json.dumps(z, separators=(",", ":")),
                        "small": bool(args.small), "only": args.only or None,
                        "l2": "step working set ~10 GB >> 126 MB L2: every operand is evicted between its uses "
@@ -643,7 +652,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(tot_s / steps * 1e3, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "all five configs per step, plus four widened rows (band x dense over the exact band layout; tensor times matrix N6,Q6,K6; degree-2 moments of M7 samples x N7 features; degree-3 moments of M8 x N8): "
+        "config": {"workload": "all five configs per step, plus five widened rows (band x dense over the exact band layout; tensor times matrix and tensor Hadamard product N6,Q6,K6; degree-2 moments of M7 samples x N7 features; degree-3 moments of M8 x N8): "
                                + json.dumps(z, separators=(",", ":")),
                    "sample": desc},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},

@@ -186,6 +186,10 @@ typedef struct {
  *   "ijl,kl->ijk"   upper half cube (i <= j, dense l)   f32        A = B x_3 C (tensor times matrix, the
  *                   running example of Section 3); `out` is PACKED too: out->structure must be the
  *                   upper half cube with the same first two extents and trailing extent K = rows of C
+ *   "ij,ij->ij"     any structure (also "i,i->i",       f32        A = B o C, the tensor Hadamard product (Table 1,
+ *                   "ijk,ijk->ijk" by rank)                            THP) of a packed structured B and a dense C of the
+ *                   same box; `out` is PACKED with the same structure as B (a structure created from the
+ *                   same descriptor): out[P(idx)] = B[P(idx)] * C[idx]
  *   "xi,xj->ij"     in[0] = in[1] = dense B (M x n)     bf16 -> f32  A2 = B^T B, the degree-2 moments of
  *                   polynomial regression (Table 1, A^k(i_1..i_k) := B(x,i_1) ... B(x,i_k), k = 2).  This
  *                   rule has no packed input: both inputs must be the same dense tensor (same data,

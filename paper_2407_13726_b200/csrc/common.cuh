@@ -61,5 +61,7 @@ dastac_status launch_moment2_bf16(const IndexMap& mo, const void* B, int64_t ldb
 size_t moment3_workspace_bytes(int64_t M, int64_t n, int64_t ldb);
 dastac_status launch_moment3_bf16(const IndexMap& mo, const void* B, int64_t ldb, int64_t M, float* out,
                                   int accumulate, void* workspace, int32_t* err_word, cudaStream_t st);
+dastac_status launch_hadamard(const IndexMap& m, const float* Bp, const float* C, const int64_t* c_strides,
+                              float* out, int accumulate, cudaStream_t stream);
 
 }  // namespace dastac

@@ -7,7 +7,7 @@
 namespace dastac {
 namespace {
 
-enum ExprClass { kMatVec, kMatMat, kMttkrp, kTtm, kMoment2, kMoment3, kNoExpr };
+enum ExprClass { kMatVec, kMatMat, kMttkrp, kTtm, kMoment2, kMoment3, kHadamard, kNoExpr };
 
 ExprClass parse_expr(const char* e) {
     if (!e) return kNoExpr;
@@ -17,6 +17,7 @@ ExprClass parse_expr(const char* e) {
     if (!std::strcmp(e, "ijl,kl->ijk")) return kTtm;
     if (!std::strcmp(e, "xi,xj->ij")) return kMoment2;
     if (!std::strcmp(e, "xi,xj,xk->ijk")) return kMoment3;
+    if (!std::strcmp(e, "i,i->i") || !std::strcmp(e, "ij,ij->ij") || !std::strcmp(e, "ijk,ijk->ijk")) return kHadamard;
     return kNoExpr;
 }
 
@@ -108,8 +109,25 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
     p.map = &m;
     p.batch = batch_of(in[0]);
 
-    if (out->structure && p.cls != kTtm) return DASTAC_ERR_UNSUPPORTED_EXPR;  // only this rule packs its output
-    if (p.cls == kTtm) {
+    if (p.cls == kHadamard) {
+        // packed structured operand times a dense one of the same box; the result has the same structure
+        const int want_rank = (int)(std::strchr(expr, ',') - expr);
+        if (m.rank != want_rank && m.kind != kEmpty) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (!out->structure) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        const IndexMap& mo = out->structure->map;
+        if (std::memcmp(&mo, &m, sizeof(IndexMap)) != 0) return DASTAC_ERR_SHAPE;  // the same structure on both sides
+        if (in[0].dtype != DASTAC_F32 || in[1].dtype != DASTAC_F32 || out->dtype != DASTAC_F32)
+            return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (p.batch != 1 || batch_of(in[1]) != 1 || batch_of(*out) != 1) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (!dense_ok(in[1], m.rank)) return DASTAC_ERR_INVALID_ARG;
+        if (!(out->space == DASTAC_MEM_DEVICE || out->space == DASTAC_MEM_HOST)) return DASTAC_ERR_INVALID_ARG;
+        for (int k = 0; k < m.rank; ++k)
+            if (in[1].dims[k] != m.dims[k]) return DASTAC_ERR_SHAPE;
+    } else if (out->structure && p.cls != kTtm) {
+        return DASTAC_ERR_UNSUPPORTED_EXPR;  // no other rule with a packed first operand packs its output
+    }
+    if (p.cls == kHadamard) {
+    } else if (p.cls == kTtm) {
         // packed upper half cube in, packed upper half cube out: same (i, j) set, trailing extents Q and K
         if (!out->structure) return DASTAC_ERR_UNSUPPORTED_EXPR;
         const IndexMap& mo = out->structure->map;
@@ -257,7 +275,12 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     if (out_bytes > 0 && !aligned16(dev_out)) return DASTAC_ERR_ALIGNMENT;
     void* scratch = p.scratch ? workspace : nullptr;
 
-    if (p.cls == kMoment3) {
+    if (p.cls == kHadamard) {
+        st = (m.kind == kEmpty || out_bytes == 0)
+                 ? DASTAC_OK
+                 : launch_hadamard(m, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides, (float*)dev_out,
+                                   accumulate, cs);
+    } else if (p.cls == kMoment3) {
         st = (m.kind == kEmpty || out_bytes == 0)
                  ? DASTAC_OK
                  : launch_moment3_bf16(m, dev_in[0], in[0].strides[0], p.R, (float*)dev_out, accumulate, scratch,

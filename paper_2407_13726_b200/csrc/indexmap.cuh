@@ -308,10 +308,12 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
             return jhi > 0;
         }
         case kUpper: {
+            // Q > 1 with rank 2: the half cube seen as a matrix of rows i and columns j Q + l (used by
+            // the copy kernels when the two inner dense strides are compact)
             if (m.rank != 2 || idx[0] >= m.M) return false;
-            jlo = idx[0];
-            jhi = m.N;
-            pbase = upper_row_base(m.N, idx[0]);
+            jlo = idx[0] * m.Q;
+            jhi = m.N * m.Q;
+            pbase = upper_row_base(m.N, idx[0]) * m.Q;
             return true;
         }
         case kLower: {

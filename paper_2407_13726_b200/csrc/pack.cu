@@ -56,9 +56,18 @@ struct Vec16 {
     T v[kElems];
 };
 
-template <typename T>
+// Element of the Hadamard form: the gathered dense value times the packed factor, optionally added
+// to what the output holds (values are fp32 carried in the 32-bit copy type).
+__device__ __forceinline__ uint32_t mul_acc(uint32_t gathered, uint32_t factor, uint32_t old, bool accumulate) {
+    const float v = __uint_as_float(gathered) * __uint_as_float(factor);
+    return __float_as_uint(accumulate ? v + __uint_as_float(old) : v);
+}
+__device__ __forceinline__ uint16_t mul_acc(uint16_t g, uint16_t, uint16_t, bool) { return g; }  // copy type only
+
+// MUL: packed[p] = dense[idx(p)] * factor[p] (+ packed[p]) instead of a plain copy.
+template <typename T, bool MUL = false>
 __global__ void pack_kernel(IndexMap m, const T* __restrict__ dense, Strides st,
-                            T* __restrict__ packed) {
+                            T* __restrict__ packed, const T* __restrict__ factor = nullptr, int accumulate = 0) {
     constexpr int E = Vec16<T>::kElems;
     const int64_t groups = (m.slots + E - 1) / E;
     for (int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; g < groups;
@@ -72,7 +81,10 @@ __global__ void pack_kernel(IndexMap m, const T* __restrict__ dense, Strides st,
                 T val = T(0);
                 if (p0 + e < m.slots) {
                     int64_t j = i + d - m.w;
-                    if (j >= 0 && j < m.N) val = dense[i * st.s[0] + j * st.s[1]];
+                    if (j >= 0 && j < m.N) {
+                        val = dense[i * st.s[0] + j * st.s[1]];
+                        if (MUL) val = mul_acc(val, factor[p0 + e], packed[p0 + e], accumulate != 0);
+                    }
                     if (++i == m.N) {
                         i = 0;
                         ++d;
@@ -88,6 +100,7 @@ __global__ void pack_kernel(IndexMap m, const T* __restrict__ dense, Strides st,
                 T val = T(0);
                 if (p0 + e < m.count) {
                     val = dense[idx[0] * st.s[0] + idx[1] * st.s[1] + idx[2] * st.s[2]];
+                    if (MUL) val = mul_acc(val, factor[p0 + e], packed[p0 + e], accumulate != 0);
                     advance(m, idx);
                 }
                 out.v[e] = val;
@@ -272,10 +285,10 @@ constexpr long long kBulkWaitBudget = 2000000000LL;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-template <typename T>
+template <typename T, bool MUL = false>
 __global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
 pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed, int64_t rows,
-                 int windows_per_row) {
+                 int windows_per_row, const T* __restrict__ factor = nullptr, int accumulate = 0) {
     constexpr int E = 16 / sizeof(T);
     extern __shared__ __align__(128) uint8_t bulk_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -375,11 +388,22 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
                 phases ^= 1u << b;
                 const uint8_t* src = buf0 + b * kBulkBufBytes;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
+#pragma unroll 4
                 for (int64_t c = cur.c_lo + lane; c < cur.c_hi; c += 32) {
                     const uint4* g = reinterpret_cast<const uint4*>(src + (c - cur.c_lo) * 16);
                     const uint4 lo = g[0];
                     const uint4 hi = cur.sh ? g[1] : zero4;
-                    *reinterpret_cast<uint4*>(packed + c * E) = realign16(lo, hi, cur.sh);
+                    uint4 v = realign16(lo, hi, cur.sh);
+                    if (MUL) {  // fp32: four elements per chunk
+                        const uint4 f = *reinterpret_cast<const uint4*>(factor + c * E);
+                        uint4 old = zero4;
+                        if (accumulate) old = *reinterpret_cast<const uint4*>(packed + c * E);
+                        v.x = mul_acc((T)v.x, (T)f.x, (T)old.x, accumulate != 0);
+                        v.y = mul_acc((T)v.y, (T)f.y, (T)old.y, accumulate != 0);
+                        v.z = mul_acc((T)v.z, (T)f.z, (T)old.z, accumulate != 0);
+                        v.w = mul_acc((T)v.w, (T)f.w, (T)old.w, accumulate != 0);
+                    }
+                    *reinterpret_cast<uint4*>(packed + c * E) = v;
                 }
             }
             // chunks of this window that the row shares with a neighbour (or the tail of the stream)
@@ -389,8 +413,10 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
                                   !(side == 1 && c == cur.ps / E) && c * E < cur.pe;
                 if (mine && lane < E) {
                     const int64_t p = c * E + lane;
-                    if (p >= cur.ps && p < cur.pe) packed[p] = cur.drow[p];
-                    else if (p >= m.count) packed[p] = T(0);
+                    if (p >= cur.ps && p < cur.pe)
+                        packed[p] = MUL ? mul_acc(cur.drow[p], factor[p], packed[p], accumulate != 0) : cur.drow[p];
+                    else if (p >= m.count && !(MUL && accumulate))
+                        packed[p] = T(0);
                 }
             }
         }
@@ -538,6 +564,20 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
     }
 }
 
+// The upper half cube (i <= j, dense l) with compact inner strides is, for copying, a matrix whose
+// row i holds the columns j Q + l, j >= i: one long contiguous interval per row instead of N - i short
+// ones.  Rewrites the map and the strides in place when that view applies.
+void collapse_half_cube(IndexMap& m, Strides& st) {
+    if (m.kind == kUpper && m.rank == 3 && m.Q > 1 && st.s[2] == 1 && st.s[1] == m.Q &&
+        m.N * m.Q < (int64_t(1) << 30)) {
+        m.rank = 2;
+        m.dims[1] = m.N * m.Q;
+        m.dims[2] = 0;
+        st.s[1] = 1;
+        st.s[2] = 0;
+    }
+}
+
 bool row_path(const IndexMap& m) {
     return (m.kind == kDense || (m.kind == kUpper && m.rank == 2) || m.kind == kLower || m.kind == kTetrahedron ||
             m.kind == kBandExact || m.kind == kUpperShifted || m.kind == kBandOffsets) &&
@@ -559,6 +599,48 @@ bool strides_ok(const IndexMap& m, const int64_t* s) {
 }
 
 }  // namespace
+
+// out[p] = Bp[p] * C[idx(p)] (+ out[p]) over the packed positions of a structure: the tensor Hadamard
+// product with a structured first operand (A(i,j,k) := B(i,j,k) * C(i,j,k), Table 1 "THP").  The dense
+// factor is gathered exactly as pack gathers it, so this is pack with one multiply per element.
+dastac_status launch_hadamard(const IndexMap& m, const float* Bp, const float* C, const int64_t* c_strides,
+                              float* out, int accumulate, cudaStream_t stream) {
+    if (m.slots == 0) return DASTAC_OK;
+    Strides st{{0, 0, 0}};
+    for (int k = 0; k < m.rank; ++k) st.s[k] = c_strides[k];
+    constexpr int E = 4;
+    const uint32_t* Cq = reinterpret_cast<const uint32_t*>(C);
+    const uint32_t* Bq = reinterpret_cast<const uint32_t*>(Bp);
+    uint32_t* Oq = reinterpret_cast<uint32_t*>(out);
+    IndexMap mc = m;
+    if (aligned16(C)) collapse_half_cube(mc, st);
+    if (mc.rank != m.rank) return launch_hadamard(mc, Bp, C, st.s, out, accumulate, stream);
+    if (row_path(m) && st.s[m.rank - 1] == 1 && aligned16(C)) {
+        int64_t rows = 1;
+        for (int k = 0; k + 1 < m.rank; ++k) rows *= m.dims[k];
+        static bool attr_set[64];
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+            if (cudaFuncSetAttribute(pack_bulk_kernel<uint32_t, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kBulkSmemBytes) != cudaSuccess)
+                return DASTAC_ERR_CUDA;
+            attr_set[dev] = true;
+        }
+        const int64_t bwpr = ((m.dims[m.rank - 1] + E - 1) / E + 2 + kBulkWin - 1) / kBulkWin;
+        if (bwpr > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
+        const int64_t items = rows * bwpr;
+        int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
+        if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
+        pack_bulk_kernel<uint32_t, true><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, stream>>>(
+            m, Cq, st, Oq, rows, (int)bwpr, Bq, accumulate);
+        return launch_status();
+    }
+    const int grid = grid_for((m.slots + E - 1) / E, 256);
+    pack_kernel<uint32_t, true><<<grid, 256, 0, stream>>>(m, Cq, st, Oq, Bq, accumulate);
+    return launch_status();
+}
+
 }  // namespace dastac
 
 using namespace dastac;
@@ -584,7 +666,7 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
                                      void* stream) {
     if (!s || !dense_strides) return DASTAC_ERR_INVALID_ARG;
     if (dtype != DASTAC_F32 && dtype != DASTAC_BF16) return DASTAC_ERR_INVALID_ARG;
-    const IndexMap& m = s->map;
+    IndexMap m = s->map;
     if (!strides_ok(m, dense_strides)) return DASTAC_ERR_INVALID_ARG;
     if (m.slots == 0) return DASTAC_OK;
     if (!dense || !packed) return DASTAC_ERR_INVALID_ARG;
@@ -592,6 +674,8 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
     Strides st{{0, 0, 0}};
     for (int k = 0; k < m.rank; ++k) st.s[k] = dense_strides[k];
     const int E = 16 / elt_size(dtype);
+    // (the row kernels below only use the row intervals, which the collapsed view provides)
+    if ((reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) collapse_half_cube(m, st);
     if (row_path(m) && st.s[m.rank - 1] == 1 && (reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) {
         int64_t rows = 1;
         for (int k = 0; k + 1 < m.rank; ++k) rows *= m.dims[k];
@@ -652,7 +736,7 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
                                        const int64_t* dense_strides, void* stream) {
     if (!s || !dense_strides) return DASTAC_ERR_INVALID_ARG;
     if (dtype != DASTAC_F32 && dtype != DASTAC_BF16) return DASTAC_ERR_INVALID_ARG;
-    const IndexMap& m = s->map;
+    IndexMap m = s->map;
     if (!strides_ok(m, dense_strides)) return DASTAC_ERR_INVALID_ARG;
     int64_t box = 1;
     for (int k = 0; k < m.rank; ++k) box *= m.dims[k];
@@ -667,6 +751,7 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
     // every row start on a 16-byte boundary.
     int vector_ok = st.s[m.rank - 1] == 1 && aligned16(dense);
     for (int k = 0; k + 1 < m.rank; ++k) vector_ok = vector_ok && (st.s[k] % E == 0);
+    if (vector_ok) collapse_half_cube(m, st);  // the row kernel only uses the row intervals
     if (row_path(m) && vector_ok) {
         const int64_t rows = box / m.dims[m.rank - 1];
         const int64_t chunks_per_row = (m.dims[m.rank - 1] + E - 1) / E;

@@ -113,7 +113,8 @@ PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33),
               st.band_exact(1000, 32), st.sub_triangle(11, 4), st.sub_triangle(130, 77), st.sub_triangle(1000, 333),
               st.offset_band(40, 9, 9), st.offset_band(130, -50, 7), st.offset_band(1000, -3, 40), st.offset_band(90, -85, 80),
               st.dense_box([7]), st.dense_box([5000]), st.dense_box([3, 4, 5]), st.dense_box([2, 3, 2100]), st.tetrahedron(130),
-              st.lower_triangle(2100), st.upper_triangle(4100)]
+              st.lower_triangle(2100), st.upper_triangle(4100), st.upper_half_cube(40, 64, 32), st.upper_half_cube(20, 33, 8),
+              st.upper_half_cube(33, 20, 4), st.upper_half_cube(9, 9, 1)]
 
 
 @pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
@@ -700,3 +701,60 @@ def test_moment3_packed_tetrahedral_output(M, n):
     with pytest.raises(dastac.DastacError) as e:
         dastac.contract("xi,xj,xk->ijk", None, Bd, [Bd, Bd], out, out_structure=sA)
     assert e.value.status == 7
+
+
+HADAMARD_CASES = [st.upper_half_cube(5, 7, 3), st.upper_half_cube(40, 64, 32), st.tetrahedron(37), st.upper_triangle(130),
+                  st.upper_triangle(1000), st.lower_triangle(77), st.band_exact(300, 7), st.band(50, 4), st.dense_box([9]),
+                  st.dense_box([6, 10, 33]), st.sub_triangle(90, 31), st.offset_band(64, -5, 20), st.upper_triangle(64, True)]
+
+
+@pytest.mark.parametrize("desc", HADAMARD_CASES, ids=lambda d: f"{d.name}{d.dims}")
+def test_hadamard_structured_times_dense(desc):
+    """A(idx) = B(idx) C(idx) on the set: packed structured B, dense C, packed result (Table 1, THP)."""
+    s = dastac.Structure(desc)
+    shape = tuple(desc.dims)
+    expr = {1: "i,i->i", 2: "ij,ij->ij", 3: "ijk,ijk->ijk"}[len(shape)]
+    B = synth.dense(10, 0, shape)
+    C = synth.dense(10, 1, shape)
+    ref, ref_abs = oracle.hadamard(desc, B, C)
+    if desc.name == "band":
+        N, w = desc.dims[0], desc.meta["w"]
+        packedB = packed_dev(s, oracle.band_pack(N, w, B), poison_tail=False)
+        exp, exp_abs = oracle.band_pack(N, w, ref).reshape(-1), oracle.band_pack(N, w, ref_abs).reshape(-1)
+        live = oracle.band_pack(N, w, np.ones(shape, np.float32)).reshape(-1) != 0   # padding slots are don't-care
+    else:
+        packedB = packed_dev(s, oracle.pack(desc, B))
+        exp, exp_abs = oracle.pack(desc, ref), oracle.pack(desc, ref_abs)
+        live = np.ones(exp.shape, bool)
+    n = exp.size
+    out = s.empty_packed()
+    out.fill_(float("nan"))
+    dastac.contract(expr, s, packedB, [dev(C)], out, out_structure=s)
+    got = out.cpu().numpy()[:n]
+    # one fp32 multiply per element: exactly the rounded product
+    assert np.array_equal(got[live], (exp.astype(np.float32))[live])
+    assert rel_err(got[live], exp[live], exp_abs[live]) <= TOL_F32
+    # accumulate, and a dense factor with padded strides (generic gather)
+    A0 = synth.dense(10, 2, (n,))
+    out2 = s.empty_packed()
+    out2[:n] = dev(A0)
+    L = (shape[-1] + 3) // 4 * 4 + 8                       # padded pitches; the view's first element stays 16-byte aligned
+    big = torch.zeros([d + 2 for d in shape[:-1]] + [L], device="cuda")
+    view = big[tuple(slice(1, 1 + d) for d in shape[:-1]) + (slice(4, 4 + shape[-1]),)]
+    assert view.data_ptr() % 16 == 0 and not view.is_contiguous() or len(shape) == 1
+    view.copy_(dev(C))
+    dastac.contract(expr, s, packedB, [view], out2, accumulate=True, out_structure=s)
+    strided = torch.zeros(shape[:-1] + (2 * shape[-1],), device="cuda")[..., ::2]   # inner stride 2: the generic gather
+    strided.copy_(dev(C))
+    out4 = s.empty_packed()
+    dastac.contract(expr, s, packedB, [strided], out4, out_structure=s)
+    assert np.array_equal(out4.cpu().numpy()[:n][live], exp.astype(np.float32)[live])
+    assert rel_err(out2.cpu().numpy()[:n][live], (exp + A0)[live], (exp_abs + np.abs(A0))[live]) <= TOL_F32
+    # a second structure object made from the same descriptor is the same structure; another one is not
+    out3 = s.empty_packed()
+    dastac.contract(expr, s, packedB, [dev(C)], out3, out_structure=dastac.Structure(desc))
+    assert torch.equal(out3[:n][torch.from_numpy(live).cuda()], out[:n][torch.from_numpy(live).cuda()])
+    with pytest.raises(dastac.DastacError):
+        dastac.contract(expr, s, packedB, [dev(C)], out3, out_structure=dastac.Structure(st.dense_box(list(shape))) if desc.name != "dense" else None)
+    with pytest.raises(dastac.DastacError):
+        dastac.contract(expr, s, packedB, [dev(C)[..., :-1] if shape[-1] > 1 else torch.zeros([d + 1 for d in shape], device="cuda")], out3, out_structure=s)

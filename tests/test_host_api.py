@@ -353,3 +353,39 @@ def test_moment3_plan_is_validated_on_the_host():
     assert ws(b"xi,xj,xk->ijk", *args) == 4
     assert ws(b"xi,xj,xk->ijk", ins, 2, ctypes.byref(out), ctypes.byref(nbytes)) == 1
     assert dastac.launch_count() == before
+
+
+def test_hadamard_plan_is_validated_on_the_host():
+    """"ijk,ijk->ijk": packed structured operand, dense operand of the same box, packed result of the same structure."""
+    before = dastac.launch_count()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    d = st.upper_half_cube(6, 8, 4)
+    s, same, other = dastac.Structure(d), dastac.Structure(d), dastac.Structure(st.upper_half_cube(6, 8, 5))
+    ins = (binding._Operand * 2)()
+    ins[0].structure = s._h
+    ins[0].rank = 3
+    ins[1].rank = 3
+    for k, (n, stv) in enumerate(zip((6, 8, 4), (32, 4, 1))):
+        ins[1].dims[k], ins[1].strides[k] = n, stv
+    out = binding._Operand()
+    out.structure = same._h
+    out.rank = 3
+    nbytes = ctypes.c_size_t(1)
+    ws = lib.dastac_contract_workspace
+    args = (ins, 2, ctypes.byref(out), ctypes.byref(nbytes))
+    assert ws(b"ijk,ijk->ijk", *args) == 0 and nbytes.value == 0
+    assert ws(b"ij,ij->ij", *args) == 3                 # rank of the expression and of the structure differ
+    out.structure = other._h
+    assert ws(b"ijk,ijk->ijk", *args) == 4              # the result must have the structure of the packed operand
+    out.structure = None
+    assert ws(b"ijk,ijk->ijk", *args) == 3              # dense result: not this rule
+    out.structure = same._h
+    ins[1].dims[2] = 5
+    assert ws(b"ijk,ijk->ijk", *args) == 4
+    ins[1].dims[2] = 4
+    ins[1].dtype = binding.BF16
+    assert ws(b"ijk,ijk->ijk", *args) == 3
+    ins[1].dtype = binding.F32
+    ins[1].space = 1                                    # host dense operand: staged through the workspace
+    assert ws(b"ijk,ijk->ijk", *args) == 0 and nbytes.value == 768
+    assert dastac.launch_count() == before
