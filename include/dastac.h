@@ -58,9 +58,12 @@ typedef enum {
     DASTAC_KIND_BAND_EXACT = 6,     /* |i-j|<=w, 2w+1<=N, rows packed back to back (no padding)    */
     DASTAC_KIND_UPPER_SHIFTED = 7,  /* j-i>=c, c>=1, square: the size N-c triangle in the top right corner
                                        (the sub-triangular structure of Section 6.4)               */
-    DASTAC_KIND_BAND_OFFSETS = 8    /* lo<=j-i<=hi, square, any lo<=hi: rows packed back to back.  One
+    DASTAC_KIND_BAND_OFFSETS = 8,   /* lo<=j-i<=hi, square, any lo<=hi: rows packed back to back.  One
                                        off-diagonal (lo=hi=s) is a per-summand buffer of the strided band
                                        of Section 6.4; chosen when no class above applies           */
+    DASTAC_KIND_PLANE = 9           /* one index fixed (idx_a = c) or equal to an earlier one (idx_b = idx_a),
+                                       everything else dense: "Fixed i", "Fixed j", "Diagonal (plane)" of
+                                       Table 1; packed as the dense box over the free indices        */
 } dastac_kind;
 
 #define DASTAC_LAYOUT_LEXICOGRAPHIC 0 /* exact pack in lexicographic order                         */
@@ -185,7 +188,9 @@ typedef struct {
  *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)
  *   "ijl,kl->ijk"   upper half cube (i <= j, dense l)   f32        A = B x_3 C (tensor times matrix, the
  *                   running example of Section 3); `out` is PACKED too: out->structure must be the
- *                   upper half cube with the same first two extents and trailing extent K = rows of C
+ *                   upper half cube with the same first two extents and trailing extent K = rows of C.
+ *                   The same rule runs on the plane structures whose trailing index is dense
+ *                   (i = j, fixed i, fixed j: TTM_DP, TTM_J of Table 1), `out` being the same plane
  *   "ij,ij->ij"     any structure (also "i,i->i",       f32        A = B o C, the tensor Hadamard product (Table 1,
  *                   "ijk,ijk->ijk" by rank)                            THP) of a packed structured B and a dense C of the
  *                   same box; `out` is PACKED with the same structure as B (a structure created from the

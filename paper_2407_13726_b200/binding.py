@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libdastac.so")
 F32, BF16 = 0, 1
 MEM_DEVICE, MEM_HOST = 0, 1
 (KIND_EMPTY, KIND_DENSE, KIND_UPPER, KIND_LOWER, KIND_BAND_DIAGONALS, KIND_TETRAHEDRON, KIND_BAND_EXACT,
- KIND_UPPER_SHIFTED, KIND_BAND_OFFSETS) = range(9)
+ KIND_UPPER_SHIFTED, KIND_BAND_OFFSETS, KIND_PLANE) = range(10)
 LAYOUT_LEXICOGRAPHIC, LAYOUT_PADDED_DIAGONALS = 0, 1
 
 EXPORTS = [

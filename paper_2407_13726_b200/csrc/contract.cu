@@ -136,6 +136,7 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         // the dense box or to the one-point tetrahedron: the same set, the same layout)
         auto trailing_dense = [](const IndexMap& x) {
             return x.kind == kEmpty || (x.rank == 3 && (x.kind == kUpper || x.kind == kDense ||
+                                                        (x.kind == kPlane && x.w != 2) ||
                                                         (x.kind == kTetrahedron && x.dims[0] == 1)));
         };
         if (!trailing_dense(m) || !trailing_dense(mo)) return DASTAC_ERR_UNSUPPORTED_EXPR;
@@ -150,6 +151,10 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         // the same (i, j) set on both sides
         if ((m.dims[2] > 0 ? m.count / m.dims[2] : 0) != (mo.dims[2] > 0 ? mo.count / mo.dims[2] : 0) &&
             m.dims[2] > 0 && mo.dims[2] > 0)
+            return DASTAC_ERR_SHAPE;
+        // planes: the same determined index on both sides
+        if ((m.kind == kPlane || mo.kind == kPlane) &&
+            !(m.kind == mo.kind && m.w == mo.w && m.lo_off == mo.lo_off && m.hi_off == mo.hi_off))
             return DASTAC_ERR_SHAPE;
         p.N = m.dims[2];   // Q
         p.R = mo.dims[2];  // K

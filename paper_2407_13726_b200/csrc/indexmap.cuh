@@ -37,7 +37,13 @@ enum Kind : int32_t {
     // One diagonal at distance s (lo_off = hi_off = s) is the per-summand buffer of a strided band
     // (Section 6.4, "Distance of Elements and Compression"); asymmetric bands, strictly lower
     // triangles and the like fall out of the same counting function.
-    kBandOffsets = 8
+    kBandOffsets = 8,
+    // One index is determined by the rest: idx[dep] = idx[src] (a diagonal plane such as i = j) or
+    // idx[dep] = c (a fixed index), everything else dense: the structures "Diagonal (plane)",
+    // "Fixed i", "Fixed j" of Table 1.  The packed layout is the dense box over the free indices
+    // in their own order.  dep is kept in `w`, src (or -1) in `lo_off`, c in `hi_off`; M and Q hold
+    // the extents of the first and second free index.
+    kPlane = 9
 };
 
 // Plain data, passed to kernels by value.
@@ -143,6 +149,16 @@ DASTAC_HD int64_t oband_row_of(int64_t N, int64_t lo, int64_t hi, int64_t p) {
     return a;
 }
 
+// kPlane helpers: the k-th free index (k = 0, 1) of a map with dependent index dep.
+DASTAC_HD int plane_free(int dep, int k) { return k + (k >= dep ? 1 : 0); }
+// Element k of a 3-index array without a dynamically indexed access (keeps the array in registers).
+DASTAC_HD int32_t pick3(const int32_t* v, int k) { return k == 0 ? v[0] : k == 1 ? v[1] : v[2]; }
+DASTAC_HD void put3(int32_t* v, int k, int32_t x) {
+    if (k == 0) v[0] = x;
+    else if (k == 1) v[1] = x;
+    else v[2] = x;
+}
+
 // Upper triangle / trapezoid: points before row i, in units of (j) positions.
 DASTAC_HD int64_t upper_row_start(int64_t N, int64_t i) { return i * N - ((i * (i - 1)) >> 1); }
 
@@ -185,6 +201,15 @@ DASTAC_HD bool in_set(const IndexMap& m, const int32_t* idx) {
             int64_t d = (int64_t)idx[1] - idx[0];
             return d >= m.lo_off && d <= m.hi_off;
         }
+        case kPlane: {
+            const int dep = (int)m.w;
+            const int64_t want = m.lo_off >= 0 ? (m.lo_off == 0 ? idx[0] : m.lo_off == 1 ? idx[1] : idx[2]) : m.hi_off;
+            const int64_t have = dep == 0 ? idx[0] : dep == 1 ? idx[1] : idx[2];
+            if (have != want) return false;
+            // a free index that is the source of an equality is limited by the smaller extent
+            const int64_t f0 = plane_free(dep, 0) == 0 ? idx[0] : idx[1];
+            return f0 < m.M && (m.rank == 2 || (plane_free(dep, 1) == 1 ? idx[1] : idx[2]) < m.Q);
+        }
         default: return false;
     }
 }
@@ -214,6 +239,13 @@ DASTAC_HD int64_t rank_of(const IndexMap& m, const int32_t* idx) {
         case kUpperShifted: return upper_row_base(m.M, idx[0]) + (idx[1] - m.w);  // the size-M triangle at column j - c
         case kBandOffsets:
             return oband_row_start(m.N, m.lo_off, m.hi_off, idx[0]) + (idx[1] - oband_jlo(m.lo_off, idx[0]));
+        case kPlane: {
+            const int dep = (int)m.w;
+            const int64_t f0 = plane_free(dep, 0) == 0 ? idx[0] : idx[1];
+            if (m.rank == 2) return f0;
+            const int64_t f1 = plane_free(dep, 1) == 1 ? idx[1] : idx[2];
+            return f0 * m.Q + f1;
+        }
         default: return -1;
     }
 }
@@ -286,6 +318,22 @@ DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
             idx[1] = (int32_t)(oband_jlo(m.lo_off, i) + (p - oband_row_start(m.N, m.lo_off, m.hi_off, i)));
             return;
         }
+        case kPlane: {
+            const int dep = (int)m.w;
+            int64_t f0 = p, f1 = 0;
+            if (m.rank == 3) {
+                f0 = p / m.Q;
+                f1 = p - f0 * m.Q;
+            }
+            int32_t v[3] = {0, 0, 0};
+            put3(v, plane_free(dep, 0), (int32_t)f0);
+            if (m.rank == 3) put3(v, plane_free(dep, 1), (int32_t)f1);
+            put3(v, dep, m.lo_off >= 0 ? pick3(v, (int)m.lo_off) : (int32_t)m.hi_off);
+#pragma unroll
+            for (int k = 0; k < 3; ++k)
+                if (k < m.rank) idx[k] = v[k];
+            return;
+        }
         default: return;
     }
 }
@@ -342,6 +390,24 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
             jhi = m.N;
             pbase = upper_row_base(m.M, idx[0]) - m.w;
             return true;
+        }
+        case kPlane: {
+            // contiguous along the innermost index only when that index is free
+            const int dep = (int)m.w, last = m.rank - 1;
+            if (dep == last) return false;
+            const int64_t want = m.lo_off >= 0 ? (m.lo_off == 0 ? idx[0] : idx[1]) : m.hi_off;
+            if ((dep == 0 ? idx[0] : idx[1]) != want) return false;
+            jlo = 0;
+            if (m.rank == 2) {  // dep = 0: the single stored row
+                jhi = m.M;
+                pbase = 0;
+            } else {
+                const int64_t f0 = plane_free(dep, 0) == 0 ? idx[0] : idx[1];
+                if (f0 >= m.M) return false;
+                jhi = m.Q;
+                pbase = f0 * m.Q;
+            }
+            return jhi > 0;
         }
         case kBandOffsets: {
             if (idx[0] < oband_first_row(m.hi_off) || idx[0] > oband_last_row(m.N, m.lo_off)) return false;
@@ -405,6 +471,23 @@ DASTAC_HD void advance(const IndexMap& m, int32_t* idx) {
             if (++idx[1] < m.N) return;
             ++idx[0];
             idx[1] = (int32_t)(idx[0] + m.w);
+            return;
+        }
+        case kPlane: {
+            const int dep = (int)m.w;
+            const int a = plane_free(dep, 0), b = plane_free(dep, 1);
+            int32_t v[3] = {idx[0], m.rank > 1 ? idx[1] : 0, m.rank > 2 ? idx[2] : 0};
+            bool carry = true;
+            if (m.rank == 3) {
+                const int32_t nb = pick3(v, b) + 1;
+                carry = nb >= m.Q;
+                put3(v, b, carry ? 0 : nb);
+            }
+            if (carry) put3(v, a, pick3(v, a) + 1);
+            if (m.lo_off >= 0) put3(v, dep, pick3(v, (int)m.lo_off));
+#pragma unroll
+            for (int k = 0; k < 3; ++k)
+                if (k < m.rank) idx[k] = v[k];
             return;
         }
         case kBandOffsets: {

@@ -61,6 +61,7 @@ static int64_t longest_row(const IndexMap& m) {
         case kUpper: return m.dims[0] != m.dims[1] ? m.N : -1;  // trapezoids (a box of one row closes to this class)
         case kLower: return m.N;
         case kBandExact: return 2 * m.w + 1;
+        case kPlane: return m.w == 0 ? m.M : -1;  // one stored row (a fixed first index)
         case kBandOffsets: {
             const int64_t len = m.hi_off - m.lo_off + 1;
             return len < m.N ? len : m.N;

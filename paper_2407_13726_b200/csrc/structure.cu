@@ -207,15 +207,67 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
         m.count = m.slots = oband_row_start(N, a, c, oband_last_row(N, a) + 1);
         return true;
     };
+    auto free_pair = [&](int p, int q) {  // no constraint between p and q beyond the box
+        return b.D[p][q] == hi[p] - lo[q] && b.D[q][p] == hi[q] - lo[p];
+    };
+    // One index determined by the rest (fixed, or equal to an earlier index), the others dense: the
+    // "Fixed i / Fixed j / Diagonal (plane)" structures of Table 1.
+    auto plane = [&]() -> bool {
+        if (rank < 2 || desc->layout == DASTAC_LAYOUT_PADDED_DIAGONALS) return false;
+        if (desc->mirror)
+            for (int k = 0; k < rank; ++k)
+                if (desc->mirror[k] != k) return false;
+        int dep = -1, src = -1;
+        int64_t cval = 0;
+        for (int a = 0; a < rank; ++a)  // a fixed index
+            if (lo[a] == hi[a] && m.dims[a] > 1) {
+                if (dep >= 0) return false;
+                dep = a;
+                cval = lo[a];
+            }
+        if (dep < 0) {  // an equality between two indices: the later one is the dependent one
+            for (int a = 0; a < rank; ++a)
+                for (int c = a + 1; c < rank; ++c)
+                    if (b.D[a][c] == 0 && b.D[c][a] == 0) {
+                        if (dep >= 0) return false;
+                        dep = c;
+                        src = a;
+                    }
+            if (dep < 0) return false;
+        }
+        int64_t ext[3] = {0, 0, 0};
+        for (int k = 0; k < rank; ++k) {
+            if (k == dep) continue;
+            if (lo[k] != 0) return false;
+            const int64_t full = (k == src) ? (m.dims[src] < m.dims[dep] ? m.dims[src] : m.dims[dep]) : m.dims[k];
+            if (hi[k] != full - 1) return false;
+            ext[k] = full;
+        }
+        if (src >= 0 && (lo[dep] != 0 || hi[dep] != hi[src])) return false;
+        // nothing else relates the indices
+        for (int p = 0; p < rank; ++p)
+            for (int q = p + 1; q < rank; ++q) {
+                if ((p == src && q == dep)) continue;
+                if (!free_pair(p, q)) return false;
+            }
+        m.kind = kPlane;
+        m.w = dep;
+        m.lo_off = src;
+        m.hi_off = cval;
+        const int f0 = dep == 0 ? 1 : 0, f1 = dep == 2 ? 1 : 2;
+        m.M = ext[f0];
+        m.Q = rank == 3 ? ext[f1] : 1;
+        m.N = m.dims[rank - 1];
+        m.count = m.slots = m.M * m.Q;
+        return true;
+    };
     // Every class below starts at the origin of the box in every index.
     for (int k = 0; k < rank; ++k)
         if (lo[k] != 0) {
             if (offset_band()) return finish();
+            if (plane()) return finish();
             return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
         }
-    auto free_pair = [&](int p, int q) {  // no constraint between p and q beyond the box
-        return b.D[p][q] == hi[p] - lo[q] && b.D[q][p] == hi[q] - lo[p];
-    };
     // p <= q is the only relation between p and q:  D[p][q] == 0 and D[q][p] is the box value.
     auto ordered_pair = [&](int p, int q) { return b.D[p][q] == 0 && b.D[q][p] == hi[q] - lo[p]; };
 
@@ -293,6 +345,7 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
         }
     }
     if (!matched && offset_band()) return finish();
+    if (!matched && plane()) return finish();
     if (!matched) return DASTAC_ERR_UNSUPPORTED_STRUCTURE;
     if (m.kind != kBandDiagonals) m.slots = m.count;
 

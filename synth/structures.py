@@ -125,3 +125,30 @@ def offset_band(N: int, lo: int, hi: int) -> Descriptor:
     items = _box_rows(2, 1, [0, 0]) + [[-1, 1, 0, -lo], [1, -1, 0, hi]]
     return Descriptor([N, N], [N], _rows(2, 1, items), np.zeros(len(items), np.uint8),
                       name="offset_band", meta={"lo": lo, "hi": hi})
+
+
+def fixed_index(dims: Sequence[int], axis: int, value: int) -> Descriptor:
+    """{idx : idx[axis] = value} inside the box ``dims`` (the "Fixed i" / "Fixed j" structures)."""
+    rank = len(dims)
+    items = _box_rows(rank, rank, list(range(rank)))
+    row = [0] * (2 * rank + 1)
+    row[axis] = 1
+    row[-1] = -value
+    items.append(row)
+    eq = np.zeros(len(items), np.uint8)
+    eq[-1] = 1
+    return Descriptor(list(dims), list(dims), _rows(rank, rank, items), eq, name="fixed_index",
+                      meta={"axis": axis, "value": value})
+
+
+def equal_indices(dims: Sequence[int], a: int, b: int) -> Descriptor:
+    """{idx : idx[a] = idx[b]} inside the box ``dims`` (a diagonal plane such as i = j)."""
+    rank = len(dims)
+    items = _box_rows(rank, rank, list(range(rank)))
+    row = [0] * (2 * rank + 1)
+    row[a], row[b] = 1, -1
+    items.append(row)
+    eq = np.zeros(len(items), np.uint8)
+    eq[-1] = 1
+    return Descriptor(list(dims), list(dims), _rows(rank, rank, items), eq, name="equal_indices",
+                      meta={"a": a, "b": b})

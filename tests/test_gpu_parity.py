@@ -22,7 +22,10 @@ INDEX_CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(97)
                st.upper_half_cube(9, 14, 5), st.upper_half_cube(14, 9, 3), st.dense_box([5, 6, 7]),
                st.band(50, 4), st.band(7, 0), st.upper_triangle(1000), st.band_exact(50, 4), st.band_exact(9, 4),
                st.band_exact(300, 32), st.sub_triangle(60, 13), st.sub_triangle(9, 1), st.sub_triangle(300, 299),
-               st.offset_band(50, 7, 7), st.offset_band(50, -20, 3), st.offset_band(33, -30, 28), st.offset_band(200, -199, -1)]
+               st.offset_band(50, 7, 7), st.offset_band(50, -20, 3), st.offset_band(33, -30, 28), st.offset_band(200, -199, -1),
+               st.fixed_index([9, 11, 5], 0, 4), st.fixed_index([9, 11, 5], 1, 10), st.fixed_index([9, 11, 5], 2, 2),
+               st.equal_indices([12, 12, 6], 0, 1), st.equal_indices([7, 9, 9], 1, 2), st.equal_indices([8, 5, 11], 0, 2),
+               st.fixed_index([13, 40], 0, 5), st.fixed_index([13, 40], 1, 39), st.equal_indices([10, 31], 0, 1)]
 
 
 @pytest.mark.parametrize("desc", INDEX_CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -114,7 +117,10 @@ PACK_CASES = [st.upper_triangle(1), st.upper_triangle(3), st.upper_triangle(33),
               st.offset_band(40, 9, 9), st.offset_band(130, -50, 7), st.offset_band(1000, -3, 40), st.offset_band(90, -85, 80),
               st.dense_box([7]), st.dense_box([5000]), st.dense_box([3, 4, 5]), st.dense_box([2, 3, 2100]), st.tetrahedron(130),
               st.lower_triangle(2100), st.upper_triangle(4100), st.upper_half_cube(40, 64, 32), st.upper_half_cube(20, 33, 8),
-              st.upper_half_cube(33, 20, 4), st.upper_half_cube(9, 9, 1)]
+              st.upper_half_cube(33, 20, 4), st.upper_half_cube(9, 9, 1), st.fixed_index([9, 11, 8], 0, 4),
+              st.fixed_index([9, 11, 8], 1, 3), st.fixed_index([9, 11, 5], 2, 2), st.equal_indices([40, 40, 32], 0, 1),
+              st.equal_indices([7, 9, 9], 1, 2), st.equal_indices([8, 5, 11], 0, 2), st.fixed_index([13, 2100], 0, 5),
+              st.fixed_index([13, 40], 1, 39)]
 
 
 @pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
@@ -705,7 +711,9 @@ def test_moment3_packed_tetrahedral_output(M, n):
 
 HADAMARD_CASES = [st.upper_half_cube(5, 7, 3), st.upper_half_cube(40, 64, 32), st.tetrahedron(37), st.upper_triangle(130),
                   st.upper_triangle(1000), st.lower_triangle(77), st.band_exact(300, 7), st.band(50, 4), st.dense_box([9]),
-                  st.dense_box([6, 10, 33]), st.sub_triangle(90, 31), st.offset_band(64, -5, 20), st.upper_triangle(64, True)]
+                  st.dense_box([6, 10, 33]), st.sub_triangle(90, 31), st.offset_band(64, -5, 20), st.upper_triangle(64, True),
+                  st.equal_indices([50, 50, 16], 0, 1), st.fixed_index([20, 30, 12], 0, 7), st.fixed_index([20, 30, 12], 1, 29),
+                  st.fixed_index([20, 30, 12], 2, 11), st.equal_indices([9, 14, 14], 1, 2)]
 
 
 @pytest.mark.parametrize("desc", HADAMARD_CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -758,3 +766,42 @@ def test_hadamard_structured_times_dense(desc):
         dastac.contract(expr, s, packedB, [dev(C)], out3, out_structure=dastac.Structure(st.dense_box(list(shape))) if desc.name != "dense" else None)
     with pytest.raises(dastac.DastacError):
         dastac.contract(expr, s, packedB, [dev(C)[..., :-1] if shape[-1] > 1 else torch.zeros([d + 1 for d in shape], device="cuda")], out3, out_structure=s)
+
+
+@pytest.mark.parametrize("which", ["diagonal_plane", "fixed_j", "fixed_i"])
+def test_ttm_over_plane_structures(which):
+    """TTM_DP / TTM_J of Table 1: A(i,j,k) = B(i,j,l) C(k,l) with B on a plane; packed in, packed out."""
+    N, Q, K = 33, 32, 24
+    mk = {"diagonal_plane": lambda L: st.equal_indices([N, N, L], 0, 1), "fixed_j": lambda L: st.fixed_index([N, N, L], 1, 5),
+          "fixed_i": lambda L: st.fixed_index([N, N, L], 0, 17)}[which]
+    dB, dA = mk(Q), mk(K)
+    sB, sA = dastac.Structure(dB), dastac.Structure(dA)
+    assert sB.kind == sA.kind == dastac.KIND_PLANE and sA.nnz == sB.nnz // Q * K
+    B = synth.dense(11, 0, (N, N, Q))
+    C = synth.dense(11, 1, (K, Q))
+    ref, ref_abs = oracle.ttm(dB, B, C)
+    exp, exp_abs = oracle.pack(dA, ref), oracle.pack(dA, ref_abs)
+    packedB = dastac.pack(sB, dev(B))
+    assert np.array_equal(packedB.cpu().numpy()[: sB.nnz], oracle.pack(dB, B))
+    out = sA.empty_packed()
+    out.fill_(float("nan"))
+    dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out, out_structure=sA)
+    assert rel_err(out.cpu().numpy()[: sA.nnz], exp, exp_abs) <= TOL_F32
+    dense = dastac.unpack(sA, out).cpu().numpy()
+    assert np.array_equal(dense != 0, (oracle.rank_table(dA) >= 0) & (dense != 0))     # nothing off the plane
+    # a plane on one side and a different plane on the other: refused
+    with pytest.raises(dastac.DastacError):
+        dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out, out_structure=dastac.Structure(st.fixed_index([N, N, K], 1, 6)))
+
+
+def test_matvec_single_stored_row():
+    """A matrix whose only stored row is i = c (the dense first row of a Leslie matrix inside the N x N box)."""
+    N, c = 700, 0
+    desc = st.fixed_index([N, N], 0, c)
+    s = dastac.Structure(desc)
+    A = synth.dense(12, 0, (N, N))
+    x = synth.dense(12, 1, (N,))
+    ref, ref_abs = oracle.matvec(desc, A, x)
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed_dev(s, oracle.pack(desc, A)), [dev(x)], y)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32 and (y[1:] == 0).all()

@@ -36,7 +36,10 @@ CASES = [st.upper_triangle(1), st.upper_triangle(2), st.upper_triangle(37), st.u
          st.sub_triangle(40, 17), st.sub_triangle(5, 5), st.offset_band(9, 3, 3), st.offset_band(9, -4, -4),
          st.offset_band(12, -2, 5), st.offset_band(12, -9, 1), st.offset_band(7, -6, -1), st.offset_band(10, -8, 8),
          st.offset_band(11, 2, 6), st.offset_band(6, -5, 4), st.offset_band(1, 0, 0), st.offset_band(8, -7, -7),
-         st.band_exact(6, 3), st.band_exact(9, 7)]
+         st.band_exact(6, 3), st.band_exact(9, 7), st.fixed_index([5, 7, 3], 0, 2), st.fixed_index([5, 7, 3], 1, 6),
+         st.fixed_index([5, 7, 3], 2, 0), st.equal_indices([6, 6, 4], 0, 1), st.equal_indices([4, 6, 3], 0, 1),
+         st.equal_indices([7, 5, 2], 0, 1), st.equal_indices([5, 4, 4], 1, 2), st.equal_indices([5, 3, 5], 0, 2),
+         st.fixed_index([6, 9], 0, 3), st.fixed_index([6, 9], 1, 8), st.equal_indices([4, 7], 0, 1)]
 
 
 @pytest.mark.parametrize("desc", CASES, ids=lambda d: f"{d.name}{d.dims}")
@@ -257,6 +260,27 @@ def test_offset_band_kinds_and_large_sizes():
 def oracle_count_offset_band(N, lo, hi):
     """Points of lo <= j - i <= hi in the N x N box, one diagonal at a time (diagonal d has N - |d| points)."""
     return sum(N - abs(d) for d in range(lo, hi + 1) if abs(d) < N)
+
+
+def test_plane_structures_kind_and_refusals():
+    """One index fixed or equal to an earlier one (Table 1: fixed i, fixed j, diagonal plane)."""
+    s = dastac.Structure(st.equal_indices([100, 100, 8], 0, 1))
+    assert s.kind == dastac.KIND_PLANE and s.nnz == s.slots == 800 and dastac.rank(s, (7, 7, 3)) == 59
+    f = dastac.Structure(st.fixed_index([100, 50, 8], 1, 49))
+    assert f.kind == dastac.KIND_PLANE and f.nnz == 800 and dastac.unrank(f, 17) == (2, 49, 1)
+    assert dastac.Structure(st.fixed_index([100, 50, 8], 1, 50)).nnz == 0        # outside the box: empty
+    assert dastac.Structure(st.equal_indices([9, 9], 0, 1)).kind == dastac.KIND_BAND_EXACT   # square matrix: the w = 0 band
+    # two determined indices (a line) and an equality combined with an order are not classes
+    two = st.fixed_index([5, 6, 7], 0, 1)
+    two.rows = np.vstack([two.rows, [0, 1, 0, 0, 0, 0, -2]])
+    two.is_eq = np.append(two.is_eq, 1).astype(np.uint8)
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(two)
+    mixed = st.equal_indices([6, 6, 6], 0, 1)
+    mixed.rows = np.vstack([mixed.rows, [0, -1, 1, 0, 0, 0, 0]])                  # j <= k as well
+    mixed.is_eq = np.append(mixed.is_eq, 0).astype(np.uint8)
+    with pytest.raises(dastac.DastacError):
+        dastac.Structure(mixed)
 
 
 def test_exact_band_limits_and_kind():
