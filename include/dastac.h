@@ -186,6 +186,8 @@ typedef struct {
  *   "ij,jc->ic"     band, padded diagonals or exact     f32        C = A B
  *   "ij,jc->ic"     upper triangle (square)             bf16 -> f32 output, fp32 accumulation
  *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)
+ *   "ijk,jr,kr->ir" dense box, upper half cube, plane   f32        the same rule over the other rank-3 structures
+ *                   with a free trailing index                         whose fibres (i, j, :) are contiguous (slower kernel)
  *   "ijl,kl->ijk"   upper half cube (i <= j, dense l)   f32        A = B x_3 C (tensor times matrix, the
  *                   running example of Section 3); `out` is PACKED too: out->structure must be the
  *                   upper half cube with the same first two extents and trailing extent K = rows of C.

@@ -46,6 +46,7 @@ dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, flo
                           int accumulate, void* workspace, cudaStream_t st);
 dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, int64_t ldb, float* C,
                             int64_t ldc, int64_t ncols, int accumulate, int32_t* err_word, cudaStream_t st);
+bool mttkrp_supports(const IndexMap& m);
 dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, int64_t ldb,
                             const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
                             int accumulate, cudaStream_t st);

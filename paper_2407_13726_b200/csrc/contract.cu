@@ -191,7 +191,7 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
     } else {
         if (p.batch != 1 || batch_of(in[1]) != 1 || batch_of(in[2]) != 1 || batch_of(*out) != 1)
             return DASTAC_ERR_UNSUPPORTED_EXPR;
-        if (m.kind != kTetrahedron && m.kind != kEmpty) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        if (!mttkrp_supports(m) && m.kind != kEmpty) return DASTAC_ERR_UNSUPPORTED_EXPR;
         if (in[0].dtype != DASTAC_F32 || in[1].dtype != DASTAC_F32 || in[2].dtype != DASTAC_F32 ||
             out->dtype != DASTAC_F32)
             return DASTAC_ERR_UNSUPPORTED_EXPR;

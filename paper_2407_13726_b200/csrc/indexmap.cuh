@@ -341,8 +341,7 @@ DASTAC_HD void unrank_of(const IndexMap& m, int64_t p, int32_t* idx) {
 // For fixed outer indices idx[0 .. rank-2], the innermost indices of the set form one interval
 // [jlo, jhi) and the point (outer, j) is stored at pbase + j: pbase is the loop-invariant part of
 // the ranking polynomial, hoisted out of the innermost loop.  Returns false when the interval is
-// empty or the layout is not contiguous along the innermost index (padded diagonals, or the
-// trailing-extent form of the upper triangle, which is handled by position instead).
+// empty or the layout is not contiguous along the innermost index (padded diagonals).
 DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int64_t& jhi, int64_t& pbase) {
     switch (m.kind) {
         case kDense: {
@@ -358,7 +357,14 @@ DASTAC_HD bool row_span(const IndexMap& m, const int32_t* idx, int64_t& jlo, int
         case kUpper: {
             // Q > 1 with rank 2: the half cube seen as a matrix of rows i and columns j Q + l (used by
             // the copy kernels when the two inner dense strides are compact)
-            if (m.rank != 2 || idx[0] >= m.M) return false;
+            if (m.rank == 3) {  // half cube: the trailing index of fibre (i, j), j >= i
+                if (idx[0] >= m.M || idx[1] < idx[0]) return false;
+                jlo = 0;
+                jhi = m.Q;
+                pbase = (upper_row_base(m.N, idx[0]) + idx[1]) * m.Q;
+                return jhi > 0;
+            }
+            if (idx[0] >= m.M) return false;
             jlo = idx[0] * m.Q;
             jhi = m.N * m.Q;
             pbase = upper_row_base(m.N, idx[0]) * m.Q;

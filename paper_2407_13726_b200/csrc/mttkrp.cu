@@ -197,12 +197,51 @@ __global__ void zero_rows_kernel(float* __restrict__ M, int64_t ldm, int64_t row
         M[(t / R) * ldm + (t % R)] = 0.f;
 }
 
+// The same rule over any rank-3 structure whose fibres (i, j, :) are stored contiguously (dense box,
+// upper half cube, planes with a free trailing index: the other MTTKRP structures of Table 1 are of
+// this kind).  A warp owns a fibre: the stored interval of k comes from the hoisted row base, lane r
+// accumulates U(r) = sum_k T(i,j,k) C(k,r) with T read coalesced and broadcast by shuffles, and
+// B(j,r) U(r) is added to M(i,r) atomically.  One multiply-add per lane and element: bound by the
+// loads of C from cache, far from the tetrahedral kernel's rate; it exists for coverage.
+__global__ void __launch_bounds__(256)
+mttkrp_fibre_kernel(IndexMap m, const float* __restrict__ T, const float* __restrict__ B, int64_t ldb,
+                    const float* __restrict__ C, int64_t ldc, float* __restrict__ M, int64_t ldm, int64_t R) {
+    const int lane = threadIdx.x & 31;
+    const int64_t fibres = m.dims[0] * m.dims[1];
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t f = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); f < fibres; f += warps) {
+        const int64_t i = f / m.dims[1], j = f - i * m.dims[1];
+        int32_t idx[3] = {(int32_t)i, (int32_t)j, 0};
+        int64_t klo = 0, khi = 0, pbase = 0;
+        if (!row_span(m, idx, klo, khi, pbase)) continue;
+        const float* row = T + pbase;  // row[k] = T(i, j, k)
+        for (int64_t r0 = 0; r0 < R; r0 += 32) {
+            const int64_t r = r0 + lane;
+            float acc = 0.f;
+            for (int64_t k0 = klo; k0 < khi; k0 += 32) {
+                const float t = (k0 + lane < khi) ? __ldg(row + k0 + lane) : 0.f;
+                const int nk = (int)(khi - k0 < 32 ? khi - k0 : 32);
+                for (int kk = 0; kk < nk; ++kk) {
+                    const float tk = __shfl_sync(0xffffffffu, t, kk);
+                    if (r < R) acc = fmaf(tk, __ldg(C + (k0 + kk) * ldc + r), acc);
+                }
+            }
+            if (r < R) atomicAdd(&M[i * ldm + r], __ldg(B + j * ldb + r) * acc);
+        }
+    }
+}
+
 }  // namespace
+
+bool mttkrp_supports(const IndexMap& m) {
+    if (m.rank != 3) return false;
+    return m.kind == kTetrahedron || m.kind == kDense || m.kind == kUpper || (m.kind == kPlane && m.w != 2);
+}
 
 dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, int64_t ldb,
                             const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
                             int accumulate, cudaStream_t st) {
-    const int64_t n = m.N;
+    const int64_t n = m.dims[0];  // rows of the result
     if (n == 0 || R == 0) return DASTAC_OK;
     if (!accumulate) {
         int64_t blocks = (n * R + 255) / 256;
@@ -210,6 +249,15 @@ dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, i
         zero_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, ldm, n, R);
         dastac_status s = launch_status();
         if (s != DASTAC_OK) return s;
+    }
+    if (m.kind != kTetrahedron) {
+        const int64_t fibres = m.dims[0] * m.dims[1];
+        if (fibres == 0 || m.dims[2] == 0) return DASTAC_OK;
+        int64_t blocks = (fibres + 7) / 8;
+        const int64_t capf = (int64_t)sm_count() * 8;
+        if (blocks > capf) blocks = capf;
+        mttkrp_fibre_kernel<<<(unsigned)blocks, 256, 0, st>>>(m, T, B, ldb, C, ldc, M, ldm, R);
+        return launch_status();
     }
     // units = sum over j0 of (floor(j0/32) + 1)
     const int64_t g_full = n / kTile;

@@ -805,3 +805,33 @@ def test_matvec_single_stored_row():
     y = torch.full((N,), float("nan"), device="cuda")
     dastac.contract("ij,j->i", s, packed_dev(s, oracle.pack(desc, A)), [dev(x)], y)
     assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32 and (y[1:] == 0).all()
+
+
+MTTKRP_FIBRE_CASES = [(st.upper_half_cube(9, 14, 20), 5), (st.upper_half_cube(30, 30, 33), 32), (st.dense_box([6, 7, 40]), 40),
+                      (st.fixed_index([10, 12, 33], 1, 5), 16), (st.fixed_index([10, 12, 33], 0, 9), 32),
+                      (st.equal_indices([12, 12, 40], 0, 1), 7), (st.dense_box([1, 1, 1]), 1)]
+
+
+@pytest.mark.parametrize("desc,R", MTTKRP_FIBRE_CASES, ids=lambda v: f"{v.name}{v.dims}" if hasattr(v, "name") else str(v))
+def test_mttkrp_other_structures(desc, R):
+    """M(i,r) = sum_{j,k} T(i,j,k) B(j,r) C(k,r) over the other rank-3 structures with contiguous fibres
+    (half cube, dense box, planes with a free trailing index: the MTTKRP structures of Table 1)."""
+    s = dastac.Structure(desc)
+    ni, nj, nk = desc.dims
+    T = synth.dense(13, 0, (ni, nj, nk))
+    B = synth.dense(13, 1, (nj, R))
+    C = synth.dense(13, 2, (nk, R))
+    ref, ref_abs = oracle.mttkrp(desc, T, B, C)
+    packed = dastac.pack(s, dev(T))
+    out = torch.full((ni, R), float("nan"), device="cuda")
+    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out)
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    M0 = synth.dense(13, 3, (ni, R))
+    out2 = dev(M0)
+    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out2, accumulate=True)
+    assert rel_err(out2.cpu().numpy(), ref + M0, ref_abs + np.abs(M0)) <= TOL_F32
+    # a plane whose determined index is the trailing one has no contiguous fibres: refused
+    with pytest.raises(dastac.DastacError):
+        bad = dastac.Structure(st.fixed_index([ni + 1, nj + 1, nk + 1], 2, 0))
+        dastac.contract("ijk,jr,kr->ir", bad, bad.empty_packed(), [torch.zeros((nj + 1, R), device="cuda"), torch.zeros((nk + 1, R), device="cuda")],
+                        torch.zeros((ni + 1, R), device="cuda"))
