@@ -184,6 +184,8 @@ typedef struct {
  *   "ij,j->i"       sub-triangle j - i >= c             f32        y = A x         (batched); rows N-c .. N-1 of
  *                   y have no stored element and are set to 0 (left unchanged when accumulating)
  *   "ij,jc->ic"     band, padded diagonals or exact     f32        C = A B
+ *   "ij,jc->ic"     dense box, trapezoid, lower         f32        C = A B for the other row-contiguous classes
+ *                   triangle, offset band, single row                 (row-wise kernel, slower than the band's)
  *   "ij,jc->ic"     upper triangle (square)             bf16 -> f32 output, fp32 accumulation
  *   "ijk,jr,kr->ir" tetrahedron                         f32        M = T x_2 B x_3 C (MTTKRP)
  *   "ijk,jr,kr->ir" dense box, upper half cube, plane   f32        the same rule over the other rank-3 structures

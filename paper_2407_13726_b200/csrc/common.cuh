@@ -41,6 +41,8 @@ bool rowspan_mv_supports(const IndexMap& m);
 dastac_status launch_rowspan_mv(const IndexMap& m, const float* A, const float* x, float* y, int batch,
                                 int64_t a_stride, int64_t x_stride, int64_t y_stride, int accumulate,
                                 cudaStream_t st);
+dastac_status launch_rowspan_mm(const IndexMap& m, const float* A, const float* B, int64_t ldb, float* C,
+                                int64_t ldc, int64_t ncols, int accumulate, cudaStream_t st);
 size_t symv_workspace_bytes(const IndexMap& m);
 dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, float* y,
                           int accumulate, void* workspace, cudaStream_t st);

@@ -181,7 +181,9 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
         const bool tri_bf16 = m.kind == kUpper && m.rank == 2 && m.dims[0] == m.dims[1] &&
                               !m.symmetric && in[0].dtype == DASTAC_BF16 &&
                               in[1].dtype == DASTAC_BF16 && out->dtype == DASTAC_F32;
-        if (!band && !tri_bf16 && m.kind != kEmpty) return DASTAC_ERR_UNSUPPORTED_EXPR;
+        const bool rowwise = rowspan_mv_supports(m) && in[0].dtype == DASTAC_F32 && in[1].dtype == DASTAC_F32 &&
+                             out->dtype == DASTAC_F32;
+        if (!band && !tri_bf16 && !rowwise && m.kind != kEmpty) return DASTAC_ERR_UNSUPPORTED_EXPR;
         p.N = m.dims[1];
         p.ncols = in[1].dims[1];
         if (in[1].dims[0] != p.N || out->dims[0] != m.dims[0] || out->dims[1] != p.ncols)
@@ -330,6 +332,9 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     } else if (p.cls == kMatMat && (m.kind == kBandDiagonals || m.kind == kBandExact)) {
         st = launch_bandmm(m, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0],
                            (float*)dev_out, out->strides[0], p.ncols, accumulate, err_word, cs);
+    } else if (p.cls == kMatMat && in[0].dtype == DASTAC_F32) {
+        st = launch_rowspan_mm(m, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0], (float*)dev_out,
+                               out->strides[0], p.ncols, accumulate, cs);
     } else if (p.cls == kMatMat) {
         st = launch_trimm_bf16(m, dev_in[0], dev_in[1], in[1].strides[0], (float*)dev_out,
                                out->strides[0], p.ncols, accumulate, scratch, err_word, cs);

@@ -51,6 +51,37 @@ rowspan_mv_kernel(const IndexMap m, const float* __restrict__ A, const float* __
     if (row < rows && sub == 0) y[row] = accumulate ? y[row] + acc : acc;
 }
 
+// C = A B with a dense row-major B for the same classes: a warp owns a row of A and 32 columns of C at
+// a time; the row's elements are read coalesced and broadcast by shuffles, the rows of B coalesced.
+// One multiply-add per lane and stored element: bound by the reads of B from cache, well below the
+// symmetric band's tiled kernel; it covers the classes that kernel does not take.
+__global__ void __launch_bounds__(256)
+rowspan_mm_kernel(const IndexMap m, const float* __restrict__ A, const float* __restrict__ B, const int64_t ldb,
+                  float* __restrict__ C, const int64_t ldc, const int64_t ncols, const int64_t rows, const int accumulate) {
+    const int lane = threadIdx.x & 31;
+    const int64_t col_blocks = (ncols + 31) / 32;
+    const int64_t items = rows * col_blocks;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t it = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); it < items; it += warps) {
+        const int64_t row = it / col_blocks, c = (it - row * col_blocks) * 32 + lane;
+        int32_t idx[3] = {(int32_t)row, 0, 0};
+        int64_t jlo = 0, jhi = 0, pbase = 0;
+        float acc = 0.f;
+        if (row_span(m, idx, jlo, jhi, pbase)) {
+            const float* a = A + pbase;
+            for (int64_t j0 = jlo; j0 < jhi; j0 += 32) {
+                const float t = (j0 + lane < jhi) ? __ldg(a + j0 + lane) : 0.f;
+                const int nj = (int)(jhi - j0 < 32 ? jhi - j0 : 32);
+                for (int jj = 0; jj < nj; ++jj) {
+                    const float tj = __shfl_sync(0xffffffffu, t, jj);
+                    if (c < ncols) acc = fmaf(tj, __ldg(B + (j0 + jj) * ldb + c), acc);
+                }
+            }
+        }
+        if (c < ncols) C[row * ldc + c] = accumulate ? C[row * ldc + c] + acc : acc;
+    }
+}
+
 }  // namespace
 
 // Longest stored row of a structure whose rows are contiguous, or -1 when the class has none.
@@ -98,6 +129,18 @@ dastac_status launch_rowspan_mv(const IndexMap& m, const float* A, const float* 
         if (last != DASTAC_OK) return last;
     }
     return last;
+}
+
+dastac_status launch_rowspan_mm(const IndexMap& m, const float* A, const float* B, int64_t ldb, float* C,
+                                int64_t ldc, int64_t ncols, int accumulate, cudaStream_t st) {
+    const int64_t rows = m.dims[0];
+    if (rows == 0 || ncols == 0) return DASTAC_OK;
+    const int64_t items = rows * ((ncols + 31) / 32);
+    int64_t blocks = (items + 7) / 8;
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    rowspan_mm_kernel<<<(unsigned)blocks, 256, 0, st>>>(m, A, B, ldb, C, ldc, ncols, rows, accumulate);
+    return launch_status();
 }
 
 }  // namespace dastac

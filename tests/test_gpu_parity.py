@@ -835,3 +835,25 @@ def test_mttkrp_other_structures(desc, R):
         bad = dastac.Structure(st.fixed_index([ni + 1, nj + 1, nk + 1], 2, 0))
         dastac.contract("ijk,jr,kr->ir", bad, bad.empty_packed(), [torch.zeros((nj + 1, R), device="cuda"), torch.zeros((nk + 1, R), device="cuda")],
                         torch.zeros((ni + 1, R), device="cuda"))
+
+
+@pytest.mark.parametrize("desc,C", [(st.dense_box([7, 13]), 5), (st.lower_triangle(100), 33), (st.offset_band(200, -30, 5), 64),
+                                    (st.offset_band(64, 9, 9), 70), (_trapezoid(20, 70), 32), (st.fixed_index([30, 40], 0, 3), 17),
+                                    (st.band_exact(90, 60), 40), (st.offset_band(300, -299, -1), 8)],
+                         ids=lambda v: f"{v.name}{v.dims}" if hasattr(v, "name") else str(v))
+def test_matmat_row_contiguous_classes(desc, C):
+    """C = A B for the row-contiguous classes that the tiled band kernel does not take."""
+    s = dastac.Structure(desc)
+    M, N = desc.dims
+    A = synth.dense(14, 0, (M, N))
+    B = synth.dense(14, 1, (N, C))
+    ref, ref_abs = oracle.matmat(desc, A, B)
+    packed = packed_dev(s, oracle.pack(desc, A))
+    out = torch.full((M, C), float("nan"), device="cuda")
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out)
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    C0 = synth.dense(14, 2, (M, C))
+    out2 = torch.zeros((M, C + 3), device="cuda")[:, :C]          # padded row pitch of the result
+    out2.copy_(dev(C0))
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], out2, accumulate=True)
+    assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_F32
