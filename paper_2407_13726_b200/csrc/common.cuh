@@ -45,7 +45,7 @@ dastac_status launch_rowspan_mm(const IndexMap& m, const float* A, const float* 
                                 int64_t ldc, int64_t ncols, int accumulate, cudaStream_t st);
 size_t symv_workspace_bytes(const IndexMap& m);
 dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, float* y,
-                          int accumulate, void* workspace, cudaStream_t st);
+                          int accumulate, void* workspace, cudaStream_t st, int symmetric = 1);
 dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, int64_t ldb, float* C,
                             int64_t ldc, int64_t ncols, int accumulate, int32_t* err_word, cudaStream_t st);
 bool mttkrp_supports(const IndexMap& m);

@@ -35,7 +35,9 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // One row's contribution for alignment class R: element e of slot k is column c0 + 4 kThreads k - R + e,
 // register 3 - R + e of the slot's seven.
-template <int R, bool kMasked>
+// kSym = false gives the plain upper-triangular product (no mirrored contribution): the same
+// streaming pattern serves large triangular matrix-vector products.
+template <int R, bool kMasked, bool kSym>
 __device__ __forceinline__ void row_fma(const float4 (&a)[kQ], const float (&xw)[kQ][7], float (&cacc)[kQ][7],
                                         const float xi, float& part, const int i, const int N, const int c0) {
 #pragma unroll
@@ -51,7 +53,7 @@ __device__ __forceinline__ void row_fma(const float4 (&a)[kQ], const float (&xw)
                 vc = (in && j != i) ? v[e] : 0.f;  // the diagonal element is used once
             }
             part = fmaf(vr, xw[k][3 - R + e], part);
-            cacc[k][3 - R + e] = fmaf(vc, xi, cacc[k][3 - R + e]);
+            if (kSym) cacc[k][3 - R + e] = fmaf(vc, xi, cacc[k][3 - R + e]);
         }
     }
 }
@@ -74,22 +76,22 @@ __device__ __forceinline__ void load_row(float4 (&a)[kQ], const float4* __restri
     }
 }
 
-template <bool kMasked>
+template <bool kMasked, bool kSym>
 __device__ __forceinline__ void row_step(const float4 (&a)[kQ], const float (&xw)[kQ][7], float (&cacc)[kQ][7],
                                          const int r, const float xi, const int i, const int N, const int c0,
                                          float* row_sum_slot, const int lane) {
     float part = 0.f;
     switch (r) {
-        case 0: row_fma<0, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
-        case 1: row_fma<1, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
-        case 2: row_fma<2, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
-        default: row_fma<3, kMasked>(a, xw, cacc, xi, part, i, N, c0); break;
+        case 0: row_fma<0, kMasked, kSym>(a, xw, cacc, xi, part, i, N, c0); break;
+        case 1: row_fma<1, kMasked, kSym>(a, xw, cacc, xi, part, i, N, c0); break;
+        case 2: row_fma<2, kMasked, kSym>(a, xw, cacc, xi, part, i, N, c0); break;
+        default: row_fma<3, kMasked, kSym>(a, xw, cacc, xi, part, i, N, c0); break;
     }
     part = warp_sum(part);
     if (lane == 0) atomicAdd(row_sum_slot, part);
 }
 
-template <bool kMasked>
+template <bool kMasked, bool kSym>
 __device__ __forceinline__ void tile_rows(const int N, const int64_t cap_quads, const int i0, const int i_end,
                                           const int64_t q0, const int c0, const float4* __restrict__ A4,
                                           const float (&xw)[kQ][7], float (&cacc)[kQ][7], const float* xs,
@@ -101,18 +103,18 @@ __device__ __forceinline__ void tile_rows(const int N, const int64_t cap_quads, 
         float4 a0[kQ], a1[kQ];
         load_row<kMasked>(a0, A4, base, q0, cap_quads, i, N, c0);
         load_row<kMasked>(a1, A4, base1, q0, cap_quads, i + 1, N, c0);
-        row_step<kMasked>(a0, xw, cacc, (int)(base & 3), xs[i - i0], i, N, c0, row_sum + (i - i0), lane);
-        row_step<kMasked>(a1, xw, cacc, (int)(base1 & 3), xs[i + 1 - i0], i + 1, N, c0, row_sum + (i + 1 - i0), lane);
+        row_step<kMasked, kSym>(a0, xw, cacc, (int)(base & 3), xs[i - i0], i, N, c0, row_sum + (i - i0), lane);
+        row_step<kMasked, kSym>(a1, xw, cacc, (int)(base1 & 3), xs[i + 1 - i0], i + 1, N, c0, row_sum + (i + 1 - i0), lane);
         base = base1 + (N - i - 2);
     }
     if (i < i_end) {
         float4 a0[kQ];
         load_row<kMasked>(a0, A4, base, q0, cap_quads, i, N, c0);
-        row_step<kMasked>(a0, xw, cacc, (int)(base & 3), xs[i - i0], i, N, c0, row_sum + (i - i0), lane);
+        row_step<kMasked, kSym>(a0, xw, cacc, (int)(base & 3), xs[i - i0], i, N, c0, row_sum + (i - i0), lane);
     }
 }
 
-template <int kTileRows>
+template <int kTileRows, bool kSym>
 __global__ void __launch_bounds__(kThreads, 4)
 symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, const float* __restrict__ A,
                  const float* __restrict__ x, float* __restrict__ y) {
@@ -125,7 +127,8 @@ symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, cons
     if (col_lo + kTileCols - 1 < i0) return;          // every column of the tile lies left of the diagonal
     const int i_end = (i0 + kTileRows < N) ? i0 + kTileRows : N;
     const int tid = threadIdx.x, lane = tid & 31;
-    for (int t = tid; t < kTileCols + 8; t += kThreads) col_sum[t] = 0.f;
+    if (kSym)
+        for (int t = tid; t < kTileCols + 8; t += kThreads) col_sum[t] = 0.f;
     if (tid < kTileRows) {
         row_sum[tid] = 0.f;
         xs[tid] = (i0 + tid < N) ? x[i0 + tid] : 0.f;
@@ -147,19 +150,23 @@ symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, cons
     // strictly above the diagonal for every row and alignment, and inside the matrix
     const bool interior = (col_lo - 3 > (int64_t)i_end - 1) && (col_lo + kTileCols - 1 < N);
     if (interior)
-        tile_rows<false>(N, cap_quads, i0, i_end, q0, c0, A4, xw, cacc, xs, row_sum, lane);
+        tile_rows<false, kSym>(N, cap_quads, i0, i_end, q0, c0, A4, xw, cacc, xs, row_sum, lane);
     else
-        tile_rows<true>(N, cap_quads, i0, i_end, q0, c0, A4, xw, cacc, xs, row_sum, lane);
+        tile_rows<true, kSym>(N, cap_quads, i0, i_end, q0, c0, A4, xw, cacc, xs, row_sum, lane);
 
+    if (kSym) {
 #pragma unroll
-    for (int k = 0; k < kQ; ++k)
+        for (int k = 0; k < kQ; ++k)
 #pragma unroll
-        for (int d = 0; d < 7; ++d) atomicAdd(&col_sum[4 * (k * kThreads + tid) + 1 + d], cacc[k][d]);
+            for (int d = 0; d < 7; ++d) atomicAdd(&col_sum[4 * (k * kThreads + tid) + 1 + d], cacc[k][d]);
+    }
     __syncthreads();
     if (tid < kTileRows && i0 + tid < N) atomicAdd(&y[i0 + tid], row_sum[tid]);
-    for (int t = tid; t < kTileCols + 8; t += kThreads) {
-        const int64_t j = col_lo - 4 + t;
-        if (j > i0 && j < N) atomicAdd(&y[j], col_sum[t]);  // column j only receives from rows i < j
+    if (kSym) {
+        for (int t = tid; t < kTileCols + 8; t += kThreads) {
+            const int64_t j = col_lo - 4 + t;
+            if (j > i0 && j < N) atomicAdd(&y[j], col_sum[t]);  // column j only receives from rows i < j
+        }
     }
 }
 
@@ -167,8 +174,10 @@ symv_quad_kernel(const int N, const int64_t cap_quads, const int col_tiles, cons
 
 size_t symv_workspace_bytes(const IndexMap&) { return 0; }
 
+// symmetric = 0: the plain upper-triangular product y = A x on the same streaming kernel (used for
+// matrices too large for the shared-memory copies of x that the small-N kernel keeps).
 dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, float* y,
-                          int accumulate, void*, cudaStream_t st) {
+                          int accumulate, void*, cudaStream_t st, int symmetric) {
     const int64_t N = m.N;
     if (N == 0) return DASTAC_OK;
     if (!accumulate && cudaMemsetAsync(y, 0, (size_t)N * sizeof(float), st) != cudaSuccess)
@@ -183,12 +192,18 @@ dastac_status launch_symv(const IndexMap& m, const float* A, const float* x, flo
     if (row_tiles * col_tiles > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
     const int64_t cap_quads = (m.count + 3) / 4;
     const unsigned grid = (unsigned)(row_tiles * col_tiles);
-    if (rows == 128)
-        symv_quad_kernel<128><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
-    else if (rows == 64)
-        symv_quad_kernel<64><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
-    else
-        symv_quad_kernel<32><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y);
+#define DASTAC_SYMV_LAUNCH(ROWS, SYM) \
+    symv_quad_kernel<ROWS, SYM><<<grid, kThreads, 0, st>>>((int)N, cap_quads, (int)col_tiles, A, x, y)
+    if (symmetric) {
+        if (rows == 128) DASTAC_SYMV_LAUNCH(128, true);
+        else if (rows == 64) DASTAC_SYMV_LAUNCH(64, true);
+        else DASTAC_SYMV_LAUNCH(32, true);
+    } else {
+        if (rows == 128) DASTAC_SYMV_LAUNCH(128, false);
+        else if (rows == 64) DASTAC_SYMV_LAUNCH(64, false);
+        else DASTAC_SYMV_LAUNCH(32, false);
+    }
+#undef DASTAC_SYMV_LAUNCH
     return launch_status();
 }
 

@@ -247,3 +247,21 @@ def test_widened_row_moment3(M, n):
         exp_abs = np.concatenate([ref_abs[s, j, j:] for j in range(i, n)])
         assert exp.size == m * (m + 1) // 2
         assert rel_err(got[start: start + exp.size], exp, exp_abs) <= 4e-3 <= TOL_BF16
+
+
+def test_large_triangular_matvec_n65536():
+    """The plain upper-triangular product at the size where it runs on the streaming kernel of the
+    symmetric product (without the mirrored half): sampled rows."""
+    N = 65536
+    desc = st.upper_triangle(N)
+    s = dastac.Structure(desc)
+    x = synth.dense(2, 1, (N,), dist=synth.NORMAL)
+    packed = _packed(s, lambda h: synth.upper_triangle_stream(2, 0, N, dist=synth.NORMAL, out=h))
+    y = torch.full((N,), float("nan"), device="cuda")
+    dastac.contract("ij,j->i", s, packed, [dev(x)], y)
+    got = y.cpu().numpy()
+    assert np.isfinite(got).all()
+    sel = _rows(N, 64, extra=(1, 127, 128, 32767, 32768, N - 2))
+    Ar = np.stack([synth.linear_slice(2, 0, int(i) * N, N, dist=synth.NORMAL) for i in sel])
+    ref, ref_abs = oracle.matvec(desc, Ar, x, sel=sel)
+    assert rel_err(got[sel], ref, ref_abs) <= TOL_F32

@@ -174,7 +174,7 @@ def test_band_pack_unpack(N, w):
 
 # ---- contractions -----------------------------------------------------------------------------
 
-@pytest.mark.parametrize("N", [1, 2, 3, 31, 32, 33, 127, 128, 129, 1000, 1024, 2500])
+@pytest.mark.parametrize("N", [1, 2, 3, 31, 32, 33, 127, 128, 129, 1000, 1024, 2500, 8191, 8192, 9001])
 def test_trmv(N):
     desc = st.upper_triangle(N)
     s = dastac.Structure(desc)
