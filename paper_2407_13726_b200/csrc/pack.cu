@@ -281,6 +281,7 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
 constexpr int kBulkWin = 256;                          // chunks (16 bytes each) per window
 constexpr int kBulkBufBytes = kBulkWin * 16 + 16;      // + the granule after the last chunk
 constexpr int kBulkSmemBytes = kWarpsPerBlock * 2 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;
+constexpr int kBulkSmemBytesMul = kWarpsPerBlock * 4 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;  // Hadamard form
 constexpr long long kBulkWaitBudget = 2000000000LL;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -292,8 +293,10 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
     constexpr int E = 16 / sizeof(T);
     extern __shared__ __align__(128) uint8_t bulk_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint8_t* buf0 = bulk_smem + warp * 2 * kBulkBufBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * 2 * kBulkBufBytes) + warp * 2;
+    // MUL: two more buffers per warp hold the matching windows of the packed factor
+    constexpr int kBufs = MUL ? 4 : 2;
+    uint8_t* buf0 = bulk_smem + warp * kBufs * kBulkBufBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * kBufs * kBulkBufBytes) + warp * 2;
     if (lane == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
@@ -353,7 +356,13 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
         const uint32_t bar = smem_addr(&bars[b]);
         // the warp's earlier generic-proxy reads of this buffer come before the async-proxy overwrite
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(w.bytes) : "memory");
+        const uint32_t fbytes = MUL ? (uint32_t)(w.c_hi - w.c_lo) * 16u : 0u;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(w.bytes + fbytes) : "memory");
+        if (MUL)  // the packed factor's chunks of the window: aligned and contiguous
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                             smem_addr(buf0 + (2 + b) * kBulkBufBytes)),
+                         "l"(factor + w.c_lo * E), "r"(fbytes), "r"(bar)
+                         : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                          smem_addr(buf0 + b * kBulkBufBytes)),
                      "l"(w.g0), "r"(w.bytes), "r"(bar)
@@ -395,7 +404,7 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
                     const uint4 hi = cur.sh ? g[1] : zero4;
                     uint4 v = realign16(lo, hi, cur.sh);
                     if (MUL) {  // fp32: four elements per chunk
-                        const uint4 f = *reinterpret_cast<const uint4*>(factor + c * E);
+                        const uint4 f = *reinterpret_cast<const uint4*>(buf0 + (2 + b) * kBulkBufBytes + (c - cur.c_lo) * 16);
                         uint4 old = zero4;
                         if (accumulate) old = *reinterpret_cast<const uint4*>(packed + c * E);
                         v.x = mul_acc((T)v.x, (T)f.x, (T)old.x, accumulate != 0);
@@ -623,7 +632,7 @@ dastac_status launch_hadamard(const IndexMap& m, const float* Bp, const float* C
         cudaGetDevice(&dev);
         if (dev >= 0 && dev < 64 && !attr_set[dev]) {
             if (cudaFuncSetAttribute(pack_bulk_kernel<uint32_t, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kBulkSmemBytes) != cudaSuccess)
+                                     kBulkSmemBytesMul) != cudaSuccess)
                 return DASTAC_ERR_CUDA;
             attr_set[dev] = true;
         }
@@ -631,8 +640,8 @@ dastac_status launch_hadamard(const IndexMap& m, const float* Bp, const float* C
         if (bwpr > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
         const int64_t items = rows * bwpr;
         int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
-        if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
-        pack_bulk_kernel<uint32_t, true><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, stream>>>(
+        if (blocks > (int64_t)sm_count()) blocks = (int64_t)sm_count();  // four buffers per warp: one CTA per SM
+        pack_bulk_kernel<uint32_t, true><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytesMul, stream>>>(
             m, Cq, st, Oq, rows, (int)bwpr, Bq, accumulate);
         return launch_status();
     }
