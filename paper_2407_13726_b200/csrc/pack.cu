@@ -280,8 +280,13 @@ pack_stream_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __res
 // memory.  The source may be read up to the end of the 16-byte granule that holds a needed element.
 constexpr int kBulkWin = 256;                          // chunks (16 bytes each) per window
 constexpr int kBulkBufBytes = kBulkWin * 16 + 16;      // + the granule after the last chunk
-constexpr int kBulkSmemBytes = kWarpsPerBlock * 2 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;
-constexpr int kBulkSmemBytesMul = kWarpsPerBlock * 4 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;  // Hadamard form
+// Window buffers per warp (depth - 1 windows in flight) and the CTAs per SM their shared memory allows.
+// Measured on the bf16 triangle N = 8192: pack 29 us at depth 2 against 33 us at depth 3 and 48 us at
+// depth 4; unpack 38 us at depth 3 against 41 us at depth 2 and 63 us at depth 4.
+constexpr int kPackDepth = 2, kUnpackDepth = 3;
+constexpr int bulk_smem_bytes(int depth) { return kWarpsPerBlock * depth * kBulkBufBytes + kWarpsPerBlock * depth * 8; }
+constexpr int bulk_ctas_per_sm(int depth) { return depth <= 2 ? 3 : depth == 3 ? 2 : 1; }
+constexpr int kBulkSmemBytesMul = kWarpsPerBlock * 4 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;  // Hadamard form: depth 2, two operands
 constexpr long long kBulkWaitBudget = 2000000000LL;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -294,12 +299,12 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
     extern __shared__ __align__(128) uint8_t bulk_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // MUL: two more buffers per warp hold the matching windows of the packed factor
-    constexpr int kBufs = MUL ? 4 : 2;
+    constexpr int D = MUL ? 2 : kPackDepth;
+    constexpr int kBufs = MUL ? 2 * D : D;
     uint8_t* buf0 = bulk_smem + warp * kBufs * kBulkBufBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * kBufs * kBulkBufBytes) + warp * 2;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * kBufs * kBulkBufBytes) + warp * D;
     if (lane == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
+        for (int d = 0; d < D; ++d) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[d])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
@@ -360,7 +365,7 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(w.bytes + fbytes) : "memory");
         if (MUL)  // the packed factor's chunks of the window: aligned and contiguous
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                             smem_addr(buf0 + (2 + b) * kBulkBufBytes)),
+                             smem_addr(buf0 + (D + b) * kBulkBufBytes)),
                          "l"(factor + w.c_lo * E), "r"(fbytes), "r"(bar)
                          : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -371,14 +376,19 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
 
     Win cur, nxt;
     int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + warp;
-    describe(item, cur);
-    issue(cur, 0);
+#pragma unroll
+    for (int d = 0; d < D - 1; ++d) {  // the first D - 1 windows
+        describe(item + d * warps, nxt);
+        issue(nxt, d);
+    }
     uint32_t phases = 0;  // bit b: parity of the next completion of buffer b
     int b = 0;
-    for (; item < items; item += warps, b ^= 1) {
-        describe(item + warps, nxt);
-        // the other buffer was consumed one iteration ago (all lanes passed the __syncwarp below)
-        issue(nxt, b ^ 1);
+    for (; item < items; item += warps, b = (b + 1 == D ? 0 : b + 1)) {
+        // the window D - 1 items ahead goes into the buffer that was consumed one iteration ago (all
+        // lanes passed the __syncwarp below)
+        describe(item + (D - 1) * warps, nxt);
+        issue(nxt, b == 0 ? D - 1 : b - 1);
+        describe(item, cur);
         if (cur.live) {
             if (cur.bytes) {
                 const uint32_t bar = smem_addr(&bars[b]);
@@ -404,7 +414,7 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
                     const uint4 hi = cur.sh ? g[1] : zero4;
                     uint4 v = realign16(lo, hi, cur.sh);
                     if (MUL) {  // fp32: four elements per chunk
-                        const uint4 f = *reinterpret_cast<const uint4*>(buf0 + (2 + b) * kBulkBufBytes + (c - cur.c_lo) * 16);
+                        const uint4 f = *reinterpret_cast<const uint4*>(buf0 + (D + b) * kBulkBufBytes + (c - cur.c_lo) * 16);
                         uint4 old = zero4;
                         if (accumulate) old = *reinterpret_cast<const uint4*>(packed + c * E);
                         v.x = mul_acc((T)v.x, (T)f.x, (T)old.x, accumulate != 0);
@@ -430,7 +440,6 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
             }
         }
         __syncwarp();
-        cur = nxt;
     }
 }
 
@@ -445,11 +454,11 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
     constexpr int E = 16 / sizeof(T);
     extern __shared__ __align__(128) uint8_t bulk_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint8_t* buf0 = bulk_smem + warp * 2 * kBulkBufBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * 2 * kBulkBufBytes) + warp * 2;
+    constexpr int D = kUnpackDepth;
+    uint8_t* buf0 = bulk_smem + warp * D * kBulkBufBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem + kWarpsPerBlock * D * kBulkBufBytes) + warp * D;
     if (lane == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
+        for (int d = 0; d < D; ++d) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[d])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
@@ -525,13 +534,17 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
 
     Win cur, nxt;
     int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + warp;
-    describe(item, cur);
-    issue(cur, 0);
+#pragma unroll
+    for (int d = 0; d < D - 1; ++d) {
+        describe(item + d * warps, nxt);
+        issue(nxt, d);
+    }
     uint32_t phases = 0;
     int b = 0;
-    for (; item < items; item += warps, b ^= 1) {
-        describe(item + warps, nxt);
-        issue(nxt, b ^ 1);
+    for (; item < items; item += warps, b = (b + 1 == D ? 0 : b + 1)) {
+        describe(item + (D - 1) * warps, nxt);
+        issue(nxt, b == 0 ? D - 1 : b - 1);
+        describe(item, cur);
         if (cur.live) {
             if (cur.bytes) {
                 const uint32_t bar = smem_addr(&bars[b]);
@@ -569,7 +582,6 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
             }
         }
         __syncwarp();
-        cur = nxt;
     }
 }
 
@@ -702,22 +714,22 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
             cudaGetDevice(&dev);
             if (dev >= 0 && dev < 64 && !attr_set[dev]) {
                 if (cudaFuncSetAttribute(pack_bulk_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kBulkSmemBytes) != cudaSuccess ||
+                                         bulk_smem_bytes(kPackDepth)) != cudaSuccess ||
                     cudaFuncSetAttribute(pack_bulk_kernel<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kBulkSmemBytes) != cudaSuccess)
+                                         bulk_smem_bytes(kPackDepth)) != cudaSuccess)
                     return DASTAC_ERR_CUDA;
                 attr_set[dev] = true;
             }
             const int64_t bwpr = ((m.dims[m.rank - 1] + E - 1) / E + 2 + kBulkWin - 1) / kBulkWin;
             const int64_t items = rows * bwpr;
             int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
-            if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
+            if (blocks > (int64_t)sm_count() * bulk_ctas_per_sm(kPackDepth)) blocks = (int64_t)sm_count() * bulk_ctas_per_sm(kPackDepth);
             if (bwpr > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
             if (dtype == DASTAC_F32)
-                pack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                pack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kPackDepth), (cudaStream_t)stream>>>(
                     m, (const uint32_t*)dense, st, (uint32_t*)packed, rows, (int)bwpr);
             else
-                pack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                pack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kPackDepth), (cudaStream_t)stream>>>(
                     m, (const uint16_t*)dense, st, (uint16_t*)packed, rows, (int)bwpr);
             return launch_status();
         }
@@ -770,22 +782,22 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
             cudaGetDevice(&dev);
             if (dev >= 0 && dev < 64 && !attr_set[dev]) {
                 if (cudaFuncSetAttribute(unpack_bulk_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kBulkSmemBytes) != cudaSuccess ||
+                                         bulk_smem_bytes(kUnpackDepth)) != cudaSuccess ||
                     cudaFuncSetAttribute(unpack_bulk_kernel<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kBulkSmemBytes) != cudaSuccess)
+                                         bulk_smem_bytes(kUnpackDepth)) != cudaSuccess)
                     return DASTAC_ERR_CUDA;
                 attr_set[dev] = true;
             }
             const int64_t bwpr = (chunks_per_row + kBulkWin - 1) / kBulkWin;
             const int64_t items = rows * bwpr;
             int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
-            if (blocks > (int64_t)sm_count() * 3) blocks = (int64_t)sm_count() * 3;
+            if (blocks > (int64_t)sm_count() * bulk_ctas_per_sm(kUnpackDepth)) blocks = (int64_t)sm_count() * bulk_ctas_per_sm(kUnpackDepth);
             if (bwpr > 0x7fffffffLL || m.dims[m.rank - 1] > (int64_t(1) << 30)) return DASTAC_ERR_OVERFLOW;
             if (dtype == DASTAC_F32)
-                unpack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                unpack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kUnpackDepth), (cudaStream_t)stream>>>(
                     m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)bwpr);
             else
-                unpack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytes, (cudaStream_t)stream>>>(
+                unpack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kUnpackDepth), (cudaStream_t)stream>>>(
                     m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)bwpr);
             return launch_status();
         }
