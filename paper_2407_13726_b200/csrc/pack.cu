@@ -292,7 +292,7 @@ constexpr long long kBulkWaitBudget = 2000000000LL;
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 template <typename T, bool MUL = false>
-__global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
+__global__ void __launch_bounds__(32 * kWarpsPerBlock, MUL ? 1 : 3)
 pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed, int64_t rows,
                  int windows_per_row, const T* __restrict__ factor = nullptr, int accumulate = 0) {
     constexpr int E = 16 / sizeof(T);
@@ -374,21 +374,23 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
                      : "memory");
     };
 
-    Win cur, nxt;
+    Win ahead[D - 1];  // windows already requested, oldest first (static indices only: stays in registers)
     int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + warp;
 #pragma unroll
-    for (int d = 0; d < D - 1; ++d) {  // the first D - 1 windows
-        describe(item + d * warps, nxt);
-        issue(nxt, d);
+    for (int d = 0; d < D - 1; ++d) {
+        describe(item + d * warps, ahead[d]);
+        issue(ahead[d], d);
     }
     uint32_t phases = 0;  // bit b: parity of the next completion of buffer b
     int b = 0;
     for (; item < items; item += warps, b = (b + 1 == D ? 0 : b + 1)) {
+        const Win cur = ahead[0];
+#pragma unroll
+        for (int d = 0; d + 1 < D - 1; ++d) ahead[d] = ahead[d + 1];
         // the window D - 1 items ahead goes into the buffer that was consumed one iteration ago (all
         // lanes passed the __syncwarp below)
-        describe(item + (D - 1) * warps, nxt);
-        issue(nxt, b == 0 ? D - 1 : b - 1);
-        describe(item, cur);
+        describe(item + (D - 1) * warps, ahead[D - 2]);
+        issue(ahead[D - 2], b == 0 ? D - 1 : b - 1);
         if (cur.live) {
             if (cur.bytes) {
                 const uint32_t bar = smem_addr(&bars[b]);
@@ -532,19 +534,21 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
     };
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
 
-    Win cur, nxt;
+    Win ahead[D - 1];  // windows already requested, oldest first
     int64_t item = blockIdx.x * (int64_t)kWarpsPerBlock + warp;
 #pragma unroll
     for (int d = 0; d < D - 1; ++d) {
-        describe(item + d * warps, nxt);
-        issue(nxt, d);
+        describe(item + d * warps, ahead[d]);
+        issue(ahead[d], d);
     }
     uint32_t phases = 0;
     int b = 0;
     for (; item < items; item += warps, b = (b + 1 == D ? 0 : b + 1)) {
-        describe(item + (D - 1) * warps, nxt);
-        issue(nxt, b == 0 ? D - 1 : b - 1);
-        describe(item, cur);
+        const Win cur = ahead[0];
+#pragma unroll
+        for (int d = 0; d + 1 < D - 1; ++d) ahead[d] = ahead[d + 1];
+        describe(item + (D - 1) * warps, ahead[D - 2]);
+        issue(ahead[D - 2], b == 0 ? D - 1 : b - 1);
         if (cur.live) {
             if (cur.bytes) {
                 const uint32_t bar = smem_addr(&bars[b]);
