@@ -545,10 +545,10 @@ TRAFFIC = {
     "bandmm": int(42.104320e6 + 3.751424e6),   # outputs of this size stay in L2 past the end of the launch
     "ttm_ut": int(67.207424e6 + 18.528000e6),
     "bandmm_exact": int(42.108160e6 + 2.613248e6),
-    "thp_ut": int(134.426624e6 + 38.478080e6),
+    "thp_ut": int(134.386688e6 + 39.105536e6),
     "moment2_bf16": int(1.410541e9 + 22.173440e6),   # full size, DRAM counters only (one pass)
-    "pack_bf16": int(67.666432e6 + 18.678784e6),
-    "unpack_bf16": int(67.146496e6 + 76.666112e6),
+    "pack_bf16": int(67.670528e6 + 18.990336e6),
+    "unpack_bf16": int(67.159552e6 + 74.384896e6),
 }
 
 
