@@ -535,10 +535,10 @@ def isolated_times(order, devs, structs, run_kernel_on, z, acct, launches):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per bench launch from the ncu captures
 # summarised under profiles/, by bench kernel; a kernel changed since its capture has no entry.
-# symv and trmv_batched were captured on smaller cases (N=16384; 128 instances) and scaled by the
-# number of stored elements, which their traffic is proportional to.
+# trmv_batched was captured on a smaller case (128 instances) and scaled by the number of stored
+# elements, which its traffic is proportional to; symv, moment2 are full-size one-pass captures.
 TRAFFIC = {
-    "symv": int((537.292800e6 + 4.572672e6) * (65536 * 65537 // 2) / (16384 * 16385 // 2)),
+    "symv": int(8.598255e9 + 6.118144e6),   # full size, DRAM counters only (one pass)
     "trmv_batched": int((269.286144e6 + 4.292096e6) * 4),
     "mttkrp": int(91.026944e6 + 6.966272e6),
     "trimm_bf16": int(855.178240e6 + 215.225600e6 + 67.129856e6 + 28.432640e6),  # main kernel + tile staging
