@@ -541,10 +541,10 @@ TRAFFIC = {
     "symv": int(8.598255e9 + 6.118144e6),   # full size, DRAM counters only (one pass)
     "trmv_batched": int((269.286144e6 + 4.292096e6) * 4),
     "mttkrp": int(91.026944e6 + 6.966272e6),
-    "trimm_bf16": int(855.178240e6 + 215.225600e6 + 67.129856e6 + 28.432640e6),  # main kernel + tile staging
-    "bandmm": int(42.104320e6 + 3.751424e6),   # outputs of this size stay in L2 past the end of the launch
+    "trimm_bf16": int(852.000768e6 + 211.080704e6 + 67.132160e6 + 28.187648e6),  # main kernel + tile staging
+    "bandmm": int(42.102784e6 + 1.659136e6),   # outputs of this size stay in L2 past the end of the launch
     "ttm_ut": int(67.207424e6 + 18.528000e6),
-    "bandmm_exact": int(42.108160e6 + 2.613248e6),
+    "bandmm_exact": int(42.106880e6 + 1.919488e6),
     "thp_ut": int(134.386688e6 + 39.105536e6),
     "moment2_bf16": int(1.410541e9 + 22.173440e6),   # full size, DRAM counters only (one pass)
     "pack_bf16": int(67.670528e6 + 18.990336e6),
