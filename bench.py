@@ -510,6 +510,11 @@ def isolated_times(order, devs, structs, run_kernel_on, z, acct, launches):
 
         sets = [d] + [clone_set(d) for _ in range(nsets - 1)]
         reps = max(1, -(-launches // nsets))
+        # "alone" includes the power state: a quarter of a second of idle lets the clocks recover from the
+        # previous kernel's burst (the tensor-core kernels run into the power cap), otherwise the short
+        # kernels measured right after them inherit lowered SM clocks
+        torch.cuda.synchronize()
+        time.sleep(0.25)
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
             for sd in sets:            # warm-up outside the capture (first-call set-up happens here)
