@@ -172,12 +172,13 @@ typedef struct {
 
 /*
  * Evaluate a sum-of-products rule (Section 3, "Input"; Table 1) whose first operand is packed
- * (one rule, the last of the table, packs its output instead).
+ * (the last two rules of the table have dense inputs and pack their output instead).
  * Supported (expression, structure of in[0], dtypes):
  *   "ij,j->i"       upper triangle (square)             f32        y = A x         (batched)
  *   "ij,j->i"       upper triangle + swap (symmetric)   f32        y = S x
- *   "ij,j->i"       dense box, lower triangle, exact    f32        y = A x         (batched); rows without a
- *                   band, offset band                                 stored element give 0.  A rule with
+ *   "ij,j->i"       dense box, trapezoid, lower         f32        y = A x         (batched); rows without a
+ *                   triangle, exact band, offset band,                stored element give 0.  A rule with
+ *                   single stored row
  *                   several summands (strided band: three diagonals; Leslie matrix: first row +
  *                   sub-diagonal) is evaluated summand by summand, each with its own packed buffer
  *                   (Section 4, one buffer per summand), the later calls with accumulate = 1
