@@ -413,3 +413,61 @@ def test_hadamard_plan_is_validated_on_the_host():
     ins[1].space = 1                                    # host dense operand: staged through the workspace
     assert ws(b"ijk,ijk->ijk", *args) == 0 and nbytes.value == 768
     assert dastac.launch_count() == before
+
+
+def _check_against_enumeration(desc):
+    """Host maps of a recognised structure against the oracle's enumeration (count, rank, unrank)."""
+    try:
+        s = dastac.Structure(desc)
+    except dastac.DastacError as e:
+        assert e.status == 2          # valid descriptor, not a recognised class: nothing to compare
+        return None
+    table = oracle.rank_table(desc)
+    assert s.nnz == oracle.count(desc)
+    if s.kind == binding.KIND_BAND_DIAGONALS:
+        return s.kind
+    assert s.slots == s.nnz
+    for p, pt in enumerate(oracle.unrank_table(desc)):
+        pt = tuple(int(v) for v in pt)
+        assert dastac.unrank(s, p) == pt and dastac.rank(s, pt) == p and table[pt] == p
+    return s.kind
+
+
+def test_random_two_index_difference_bounds():
+    """Random pairs of bounds lo <= j - i <= hi in square boxes: whichever class the closure picks (dense, upper,
+    lower, exact band, sub-triangle, offset band, empty), its maps equal the enumeration."""
+    hypothesis = pytest.importorskip("hypothesis")
+    from hypothesis import given, settings, strategies as hs
+
+    seen = set()
+
+    @settings(max_examples=150, deadline=None, derandomize=True)
+    @given(hs.integers(1, 14), hs.integers(-16, 16), hs.integers(-16, 16))
+    def run(N, a, b):
+        lo, hi = min(a, b), max(a, b)
+        seen.add(_check_against_enumeration(st.offset_band(N, lo, hi)))
+
+    run()
+    assert {binding.KIND_EMPTY, binding.KIND_DENSE, binding.KIND_UPPER, binding.KIND_LOWER, binding.KIND_BAND_EXACT,
+            binding.KIND_UPPER_SHIFTED, binding.KIND_BAND_OFFSETS} <= seen
+
+
+def test_random_planes_and_boxes():
+    """Random rank-3 boxes with one index fixed or two indices equal."""
+    hypothesis = pytest.importorskip("hypothesis")
+    from hypothesis import given, settings, strategies as hs
+
+    @settings(max_examples=80, deadline=None, derandomize=True)
+    @given(hs.tuples(hs.integers(1, 6), hs.integers(1, 6), hs.integers(1, 6)), hs.integers(0, 2), hs.integers(0, 6),
+           hs.booleans(), hs.integers(0, 2))
+    def run(dims, axis, value, equal, other):
+        if equal:
+            a, b = sorted((axis, other))
+            if a == b:
+                return
+            desc = st.equal_indices(list(dims), a, b)
+        else:
+            desc = st.fixed_index(list(dims), axis, value)
+        _check_against_enumeration(desc)
+
+    run()
