@@ -857,3 +857,52 @@ def test_matmat_row_contiguous_classes(desc, C):
     out2.copy_(dev(C0))
     dastac.contract("ij,jc->ic", s, packed, [dev(B)], out2, accumulate=True)
     assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_F32
+
+
+def _random_descriptors(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        kind = rng.integers(0, 6)
+        if kind == 0:
+            N = int(rng.integers(1, 700))
+            a, b = sorted(int(v) for v in rng.integers(-N - 3, N + 4, 2))
+            out.append(st.offset_band(N, a, b))
+        elif kind == 1:
+            out.append(st.upper_half_cube(int(rng.integers(1, 40)), int(rng.integers(1, 40)), int(rng.integers(1, 70))))
+        elif kind == 2:
+            out.append(st.tetrahedron(int(rng.integers(1, 60))))
+        elif kind == 3:
+            dims = [int(v) for v in rng.integers(1, 30, 3)]
+            axis = int(rng.integers(0, 3))
+            out.append(st.fixed_index(dims, axis, int(rng.integers(0, dims[axis]))))
+        elif kind == 4:
+            dims = [int(v) for v in rng.integers(1, 30, 3)]
+            a, b = sorted(int(v) for v in rng.choice(3, 2, replace=False))
+            out.append(st.equal_indices(dims, a, b))
+        else:
+            out.append(st.dense_box([int(v) for v in rng.integers(1, 50, int(rng.integers(1, 4)))]))
+    return out
+
+
+@pytest.mark.parametrize("sixteen", [False, True], ids=["f32", "bf16"])
+def test_pack_unpack_random_structures(sixteen):
+    """Forty random descriptors of the recognised families: pack and unpack bit for bit against the oracle."""
+    tdt = torch.bfloat16 if sixteen else torch.float32
+    idt = torch.int16 if sixteen else torch.int32
+    for k, desc in enumerate(_random_descriptors(40, 123)):
+        try:
+            s = dastac.Structure(desc)
+        except dastac.DastacError as e:
+            assert e.status == 2
+            continue
+        bits = _bits(tuple(desc.dims), 50 + k, sixteen)
+        d_dense = torch.from_numpy(bits.view(np.int16 if sixteen else np.int32)).cuda().view(tdt)
+        packed = dastac.pack(s, d_dense)
+        exp = oracle.pack(desc, bits)
+        got = packed.view(idt).cpu().numpy().view(bits.dtype)
+        assert np.array_equal(got[: s.nnz], exp), (desc.name, desc.dims, desc.meta)
+        out = torch.full(desc.dims, float("nan"), dtype=tdt, device="cuda")
+        dastac.unpack(s, packed, out)
+        back = out.view(idt).cpu().numpy().view(bits.dtype)
+        assert np.array_equal(back, oracle.unpack(desc, exp)), (desc.name, desc.dims, desc.meta)
