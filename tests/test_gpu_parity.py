@@ -906,3 +906,49 @@ def test_pack_unpack_random_structures(sixteen):
         dastac.unpack(s, packed, out)
         back = out.view(idt).cpu().numpy().view(bits.dtype)
         assert np.array_equal(back, oracle.unpack(desc, exp)), (desc.name, desc.dims, desc.meta)
+
+
+def test_contractions_random_structures():
+    """Random descriptors: matrix-vector, matrix x dense and Hadamard product wherever the structure's class has them."""
+    done = {"mv": 0, "mm": 0, "had": 0}
+    for k, desc in enumerate(_random_descriptors(60, 321)):
+        try:
+            s = dastac.Structure(desc)
+        except dastac.DastacError:
+            continue
+        shape = tuple(desc.dims)
+        if s.nnz == 0 or desc.name == "dense" and len(shape) == 1:
+            continue
+        A = synth.dense(60 + k, 0, shape)
+        packed = packed_dev(s, oracle.pack(desc, A))
+        # Hadamard product: every class and rank
+        Cf = synth.dense(60 + k, 1, shape)
+        ref, _ = oracle.hadamard(desc, A, Cf)
+        out = s.empty_packed()
+        dastac.contract({1: "i,i->i", 2: "ij,ij->ij", 3: "ijk,ijk->ijk"}[len(shape)], s, packed, [dev(Cf)], out, out_structure=s)
+        assert np.array_equal(out.cpu().numpy()[: s.nnz], oracle.pack(desc, ref).astype(np.float32)), (desc.name, shape, desc.meta)
+        done["had"] += 1
+        if len(shape) != 2:
+            continue
+        M, N = shape
+        x = synth.dense(60 + k, 2, (N,))
+        r, ra = oracle.matvec(desc, A, x)
+        y = torch.full((M,), float("nan"), device="cuda")
+        try:
+            dastac.contract("ij,j->i", s, packed, [dev(x)], y)
+        except dastac.DastacError as e:
+            assert e.status == 3
+        else:
+            assert rel_err(y.cpu().numpy(), r, ra) <= TOL_F32, (desc.name, shape, desc.meta)
+            done["mv"] += 1
+        B = synth.dense(60 + k, 3, (N, 19))
+        r, ra = oracle.matmat(desc, A, B)
+        Cm = torch.full((M, 19), float("nan"), device="cuda")
+        try:
+            dastac.contract("ij,jc->ic", s, packed, [dev(B)], Cm)
+        except dastac.DastacError as e:
+            assert e.status == 3
+        else:
+            assert rel_err(Cm.cpu().numpy(), r, ra) <= TOL_F32, (desc.name, shape, desc.meta)
+            done["mm"] += 1
+    assert done["mv"] >= 5 and done["mm"] >= 5 and done["had"] >= 30
