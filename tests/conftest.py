@@ -14,9 +14,13 @@ def pytest_configure(config):
 
 @pytest.fixture(scope="session", autouse=True)
 def _built_cpu_libs():
-    """The generator and the oracle are small gcc builds; make sure they exist."""
+    """The generator and the oracle are small gcc builds, the library an nvcc build; make sure they exist."""
     import oracle
     import synth
 
     synth.build()
     oracle.build()
+    # the CUDA library: a no-op when it is up to date, an nvcc build (no GPU needed) when it is missing or stale
+    from paper_2407_13726_b200 import build as cuda_build
+
+    cuda_build.build()
