@@ -10,17 +10,18 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # The CUDA library is loaded when the test modules are imported, i.e. during collection: build it
+    # before that (a no-op when it is up to date; an nvcc build, which needs no GPU, otherwise).
+    from paper_2407_13726_b200 import build as cuda_build
+
+    cuda_build.build()
 
 
 @pytest.fixture(scope="session", autouse=True)
 def _built_cpu_libs():
-    """The generator and the oracle are small gcc builds, the library an nvcc build; make sure they exist."""
+    """The generator and the oracle are small gcc builds; make sure they exist."""
     import oracle
     import synth
 
     synth.build()
     oracle.build()
-    # the CUDA library: a no-op when it is up to date, an nvcc build (no GPU needed) when it is missing or stale
-    from paper_2407_13726_b200 import build as cuda_build
-
-    cuda_build.build()
