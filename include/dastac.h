@@ -16,6 +16,12 @@
  *     library allocates no device memory; scratch space is passed in as `workspace`.
  *   - Indices are int32 per dimension (extents up to 2^30); packed positions are int64.
  *   - Dense operands are described by element strides; packed operands are contiguous.
+ *   - State kept by the library in the calling process, none of it visible in results: a launch
+ *     counter (dastac_launch_count), per-device caches of attribute set-up and of work partitions,
+ *     and, on every GPU that loads it, one device error word (dastac_device_error) and the
+ *     scratch array of dastac_trimm_bf16_noalloc.
+ *   - fp32 arithmetic flushes subnormal inputs and results to zero (the kernels are compiled
+ *     that way); pack and unpack copy bits and are not affected.
  *   - Packed buffers must be 16-byte aligned and have a capacity of `slots` elements as reported
  *     by dastac_structure_count (the point count rounded up to a multiple of 16 bytes); the
  *     library never reads element values beyond `count` into a result, but it may load the
@@ -41,7 +47,7 @@ typedef enum {
     DASTAC_ERR_OVERFLOW = 6,              /* an extent exceeds 2^30 or a count exceeds 2^62        */
     DASTAC_ERR_WORKSPACE = 7,             /* workspace missing, misaligned or too small            */
     DASTAC_ERR_CUDA = 8,                  /* a CUDA runtime/driver call failed                     */
-    DASTAC_ERR_TIMEOUT = 9                /* a bounded device-side wait expired (see err_word)     */
+    DASTAC_ERR_TIMEOUT = 9                /* a bounded device-side wait expired (dastac_device_error) */
 } dastac_status;
 
 typedef enum { DASTAC_F32 = 0, DASTAC_BF16 = 1 } dastac_dtype;
@@ -140,6 +146,9 @@ dastac_status dastac_unrank_batch(const dastac_structure* s, const int64_t* off,
  *   unpack  dense = 0 everywhere in the box, then dense[idx] = packed[P(idx)]; with a redundancy
  *           swap the mirrored element receives the same bits.  Padding slots are ignored.
  * dense_strides: host array of `rank` element strides of the dense tensor.
+ * The row-wise kernels fetch windows of a row by bulk copies and wait for them with a budget; a
+ * wait that runs out (never expected) leaves the rest of the launch's output unwritten and sets
+ * the device error word, which dastac_device_error reports as DASTAC_ERR_TIMEOUT.
  */
 dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dtype, const void* dense,
                           const int64_t* dense_strides, void* packed, void* stream);
@@ -258,6 +267,23 @@ const char* dastac_status_string(dastac_status st);
 dastac_status dastac_trimm_bf16_noalloc(const dastac_structure* s, const void* A, const void* B,
                                         int64_t ldb, int64_t ncols, float* C, int64_t ldc,
                                         int32_t accumulate, int32_t* err_word, void* stream);
+
+/*
+ * Device error word (no counterpart in the paper: it belongs to the execution model, not to the
+ * method).  Kernels whose entry points take no `err_word` (pack, unpack) record an expired bounded
+ * wait in a device int32 owned by the library, one per GPU.  dastac_device_error copies the current
+ * device's word to *word (host, may be NULL), clears it on the device when `clear` != 0, and
+ * returns DASTAC_OK when it was 0 and DASTAC_ERR_TIMEOUT otherwise.  Unlike the other device
+ * calls it SYNCHRONISES `stream`, so it reports everything enqueued on that stream before it.
+ */
+dastac_status dastac_device_error(int32_t* word, int32_t clear, void* stream);
+/*
+ * Self-test of the expiry path: enqueues one warp that waits `budget_cycles` SM clock cycles
+ * (0 .. 2e9) on a shared-memory barrier that nothing arrives on, then records a code in the
+ * device error word and returns normally.  Afterwards dastac_device_error reports
+ * DASTAC_ERR_TIMEOUT and the device is as usable as before: no trap, no fault, no unbounded loop.
+ */
+dastac_status dastac_selftest_wait_expiry(int64_t budget_cycles, void* stream);
 
 /* Number of kernels this library has launched in the calling process (for launch accounting). */
 int64_t dastac_launch_count(void);

@@ -69,6 +69,15 @@ def _load():
         lib.orc_moment3.argtypes = [P, ctypes.c_int, i64, vp, vp, i64, vp, vp]
         lib.orc_hadamard.argtypes = [P, vp, vp, vp, vp]
         lib.orc_num_threads.restype = ctypes.c_int
+        ci = ctypes.c_int
+        lib.orc_clip_matvec_upper.argtypes = [i64, vp, vp, vp, ci]
+        lib.orc_clip_symv.argtypes = [i64, vp, vp, vp, ci]
+        lib.orc_clip_band_matmat.argtypes = [i64, i64, vp, vp, i64, vp, ci]
+        lib.orc_clip_mttkrp_tetra.argtypes = [i64, vp, vp, vp, i64, vp, ci]
+        lib.orc_clip_matmat_upper_bf16.argtypes = [i64, i64, vp, vp, vp, i64, vp, ci]
+        for name in ("orc_clip_matvec_upper", "orc_clip_symv", "orc_clip_band_matmat", "orc_clip_mttkrp_tetra",
+                     "orc_clip_matmat_upper_bf16"):
+            getattr(lib, name).restype = None
         for name in ("orc_rank_table", "orc_unrank_table", "orc_pack", "orc_unpack", "orc_band_pack",
                      "orc_band_unpack", "orc_band_slot_table", "orc_matvec", "orc_symv",
                      "orc_matmat", "orc_mttkrp", "orc_ttm", "orc_moment2", "orc_moment3", "orc_hadamard"):
@@ -302,3 +311,55 @@ def hadamard(desc, B, C):
     out, out_abs = np.empty(shape), np.empty(shape)
     _load().orc_hadamard(h.ref, B.ctypes.data, C.ctypes.data, out.ctypes.data, out_abs.ctypes.data)
     return out, out_abs
+
+
+# ---- timed variants: loops clipped to the domain, packed operand (the CPU baseline) --------------
+# Same products as the masked forms; see the header of ``oracle.c``.  ``threads`` = OpenMP threads.
+
+def _threads(threads):
+    return int(threads) if threads else num_threads()
+
+
+def clip_matvec_upper(N, packed, x, threads=None):
+    packed, x = _f32(packed), _f32(x)
+    assert packed.size >= N * (N + 1) // 2 and x.shape == (N,)
+    y = np.empty(N)
+    _load().orc_clip_matvec_upper(N, packed.ctypes.data, x.ctypes.data, y.ctypes.data, _threads(threads))
+    return y
+
+
+def clip_symv(N, packed, x, threads=None):
+    packed, x = _f32(packed), _f32(x)
+    assert packed.size >= N * (N + 1) // 2 and x.shape == (N,)
+    y = np.empty(N)
+    _load().orc_clip_symv(N, packed.ctypes.data, x.ctypes.data, y.ctypes.data, _threads(threads))
+    return y
+
+
+def clip_band_matmat(N, w, diags, B, threads=None):
+    diags, B = _f32(diags), _f32(B)
+    assert diags.size == (2 * w + 1) * N and B.shape[0] == N
+    out = np.empty((N, B.shape[1]))
+    _load().orc_clip_band_matmat(N, w, diags.ctypes.data, B.ctypes.data, B.shape[1], out.ctypes.data,
+                                 _threads(threads))
+    return out
+
+
+def clip_mttkrp_tetra(n, packed, B, C, threads=None):
+    packed, B, C = _f32(packed), _f32(B), _f32(C)
+    R = B.shape[1]
+    assert packed.size >= n * (n + 1) * (n + 2) // 6 and B.shape == (n, R) and C.shape == (n, R)
+    out = np.empty((n, R))
+    _load().orc_clip_mttkrp_tetra(n, packed.ctypes.data, B.ctypes.data, C.ctypes.data, R, out.ctypes.data,
+                                  _threads(threads))
+    return out
+
+
+def clip_matmat_upper_bf16(N, packed, B, sel=None, threads=None):
+    sel = _sel(sel, N)
+    packed, B = np.ascontiguousarray(packed), np.ascontiguousarray(B)
+    assert packed.dtype == np.uint16 and B.dtype == np.uint16 and B.shape[0] == N
+    out = np.empty((len(sel), B.shape[1]))
+    _load().orc_clip_matmat_upper_bf16(N, len(sel), sel.ctypes.data, packed.ctypes.data, B.ctypes.data,
+                                       B.shape[1], out.ctypes.data, _threads(threads))
+    return out

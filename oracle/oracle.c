@@ -23,6 +23,9 @@
  * parallelisation the paper itself applies (Section 5.2, "Parallelization").
  */
 #include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -397,9 +400,144 @@ void orc_hadamard(const orc_desc* d, const float* B, const float* C, double* out
     } while (box_next(d, idx));
 }
 
+/* ---- timed variants: loops clipped to the domain ---------------------------------------------
+ * The same products as the masked forms above, but the loops run over the stored elements only
+ * (Section 5.3, "Compressed Compute Code Generation": the generated loops visit the accessed
+ * indices, and the operand is read from its compressed buffer).  The operand is the packed vector
+ * in the enumeration order of the masked oracle; the position of a row's first element is a
+ * counter advanced by the trip count of the clipped inner loop, never a ranking polynomial.
+ * These exist to be timed as the CPU baseline (1 thread, or `threads` OpenMP threads with a static
+ * schedule over the outermost output index, the paper's own parallelisation); a test checks them
+ * against the masked forms on small sizes.  Results are double. */
+
+/* y[i] = sum_{j >= i} A[i][j] x[j], A packed row after row (upper triangle). */
+void orc_clip_matvec_upper(int64_t N, const float* packed, const float* x, double* y, int threads) {
+    int64_t* start = (int64_t*)malloc(sizeof(int64_t) * (size_t)(N + 1));
+    int64_t counter = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        start[i] = counter;
+        for (int64_t j = i; j < N; ++j) ++counter;
+    }
+#pragma omp parallel for schedule(static) num_threads(threads)
+    for (int64_t i = 0; i < N; ++i) {
+        const float* row = packed + start[i];
+        double acc = 0.0;
+        for (int64_t j = i; j < N; ++j) acc += (double)row[j - i] * (double)x[j];
+        y[i] = acc;
+    }
+    free(start);
+}
+
+/* y = Sfull x from the packed upper triangle: every stored off-diagonal element is used for the two
+ * outputs it contributes to.  Threads own blocks of rows of the stored triangle and private copies
+ * of y, summed at the end. */
+void orc_clip_symv(int64_t N, const float* packed, const float* x, double* y, int threads) {
+    int64_t* start = (int64_t*)malloc(sizeof(int64_t) * (size_t)(N + 1));
+    int64_t counter = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        start[i] = counter;
+        counter += N - i; /* trip count of j = i .. N-1 */
+    }
+    if (threads < 1) threads = 1;
+    double* priv = (double*)calloc((size_t)threads * (size_t)N, sizeof(double));
+#pragma omp parallel num_threads(threads)
+    {
+        int t = 0, nt = 1;
+#ifdef _OPENMP
+        t = omp_get_thread_num();
+        nt = omp_get_num_threads();
+#endif
+        double* mine = priv + (size_t)t * (size_t)N;
+        /* rows dealt round-robin so that every thread gets long and short rows */
+        for (int64_t i = t; i < N; i += nt) {
+            const float* row = packed + start[i];
+            double acc = (double)row[0] * (double)x[i];
+            const double xi = (double)x[i];
+            for (int64_t j = i + 1; j < N; ++j) {
+                const double v = (double)row[j - i];
+                acc += v * (double)x[j];
+                mine[j] += v * xi;
+            }
+            mine[i] += acc;
+        }
+    }
+    for (int64_t i = 0; i < N; ++i) {
+        double acc = 0.0;
+        for (int t = 0; t < threads; ++t) acc += priv[(size_t)t * (size_t)N + i];
+        y[i] = acc;
+    }
+    free(priv);
+    free(start);
+}
+
+/* C[i][c] = sum_{|i-j| <= w} A[i][j] B[j][c], A as 2w+1 padded diagonals of N slots (slot (d, i)). */
+void orc_clip_band_matmat(int64_t N, int64_t w, const float* diags, const float* B, int64_t ncols,
+                          double* out, int threads) {
+#pragma omp parallel for schedule(static) num_threads(threads)
+    for (int64_t i = 0; i < N; ++i) {
+        double* o = out + i * ncols;
+        for (int64_t c = 0; c < ncols; ++c) o[c] = 0.0;
+        const int64_t jlo = i - w < 0 ? 0 : i - w, jhi = i + w > N - 1 ? N - 1 : i + w;
+        for (int64_t j = jlo; j <= jhi; ++j) {
+            const double a = (double)diags[(j - i + w) * N + i];
+            const float* b = B + j * ncols;
+            for (int64_t c = 0; c < ncols; ++c) o[c] += a * (double)b[c];
+        }
+    }
+}
+
+/* M[i][r] = sum_{i <= j <= k} T[i][j][k] B[j][r] C[k][r], T packed in lexicographic order. */
+void orc_clip_mttkrp_tetra(int64_t n, const float* packed, const float* B, const float* C, int64_t R,
+                           double* M, int threads) {
+    int64_t* start = (int64_t*)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    int64_t counter = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        start[i] = counter;
+        for (int64_t j = i; j < n; ++j) counter += n - j; /* trip count of k = j .. n-1 */
+    }
+#pragma omp parallel for schedule(dynamic, 1) num_threads(threads)
+    for (int64_t i = 0; i < n; ++i) {
+        double* m = M + i * R;
+        for (int64_t r = 0; r < R; ++r) m[r] = 0.0;
+        const float* t = packed + start[i];
+        for (int64_t j = i; j < n; ++j) {
+            const float* b = B + j * R;
+            for (int64_t k = j; k < n; ++k) {
+                const double v = (double)*t++;
+                const float* c = C + k * R;
+                for (int64_t r = 0; r < R; ++r) m[r] += v * (double)b[r] * (double)c[r];
+            }
+        }
+    }
+    free(start);
+}
+
+/* C[i][c] = sum_{j >= i} A[i][j] B[j][c] for the rows i in sel, bf16 bit patterns, A packed. */
+void orc_clip_matmat_upper_bf16(int64_t N, int64_t nsel, const int64_t* sel, const uint16_t* packed,
+                                const uint16_t* B, int64_t ncols, double* out, int threads) {
+    int64_t* start = (int64_t*)malloc(sizeof(int64_t) * (size_t)(N + 1));
+    int64_t counter = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        start[i] = counter;
+        counter += N - i;
+    }
+#pragma omp parallel for schedule(dynamic, 1) num_threads(threads)
+    for (int64_t s = 0; s < nsel; ++s) {
+        const int64_t i = sel[s];
+        double* o = out + s * ncols;
+        for (int64_t c = 0; c < ncols; ++c) o[c] = 0.0;
+        const uint16_t* row = packed + start[i];
+        for (int64_t j = i; j < N; ++j) {
+            const double a = widen(row, j - i, 1);
+            const uint16_t* b = B + j * ncols;
+            for (int64_t c = 0; c < ncols; ++c) o[c] += a * widen(b, c, 1);
+        }
+    }
+    free(start);
+}
+
 /* Thread count the contractions above will use. */
 #ifdef _OPENMP
-#include <omp.h>
 int orc_num_threads(void) { return omp_get_max_threads(); }
 #else
 int orc_num_threads(void) { return 1; }

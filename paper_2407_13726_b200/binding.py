@@ -27,6 +27,7 @@ EXPORTS = [
     "dastac_structure_kind", "dastac_rank", "dastac_unrank", "dastac_rank_batch",
     "dastac_unrank_batch", "dastac_pack", "dastac_unpack", "dastac_contract_workspace",
     "dastac_contract", "dastac_status_string", "dastac_launch_count", "dastac_trimm_bf16_noalloc",
+    "dastac_device_error", "dastac_selftest_wait_expiry",
 ]
 NOALLOC_MAX_N = 2048
 
@@ -77,6 +78,8 @@ _lib.dastac_status_string.restype = ctypes.c_char_p
 _lib.dastac_trimm_bf16_noalloc.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _i32, _vp, _vp]
 _lib.dastac_launch_count.argtypes = []
 _lib.dastac_launch_count.restype = _i64
+_lib.dastac_device_error.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
+_lib.dastac_selftest_wait_expiry.argtypes = [_i64, _vp]
 
 
 def status_string(status: int) -> str:
@@ -85,6 +88,18 @@ def status_string(status: int) -> str:
 
 def launch_count() -> int:
     return int(_lib.dastac_launch_count())
+
+
+def device_error(clear: bool = True):
+    """``(status, word)`` of the current device's error word after everything enqueued on the current
+    stream (synchronises it): status 0, or 9 (TIMEOUT) with the recorded code."""
+    word = _i32(0)
+    st = _lib.dastac_device_error(ctypes.byref(word), int(bool(clear)), _stream())
+    return int(st), int(word.value)
+
+
+def selftest_wait_expiry(budget_cycles: int) -> None:
+    _check(_lib.dastac_selftest_wait_expiry(int(budget_cycles), _stream()), "dastac_selftest_wait_expiry")
 
 
 def _check(status: int, where: str):

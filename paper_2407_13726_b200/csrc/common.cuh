@@ -51,7 +51,7 @@ dastac_status launch_bandmm(const IndexMap& m, const float* A, const float* B, i
 bool mttkrp_supports(const IndexMap& m);
 dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, int64_t ldb,
                             const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
-                            int accumulate, cudaStream_t st);
+                            int accumulate, int32_t* err_word, cudaStream_t st);
 dastac_status launch_ttm(int64_t P, int64_t Q, int64_t K, const float* X, const float* C, int64_t ldc, float* Y,
                          int accumulate, cudaStream_t st);
 size_t trimm_workspace_bytes(const IndexMap& m, int64_t ncols, int64_t ldb);

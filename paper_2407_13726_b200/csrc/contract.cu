@@ -341,7 +341,7 @@ extern "C" dastac_status dastac_contract(const char* expr, const dastac_operand*
     } else {
         st = launch_mttkrp(m, (const float*)dev_in[0], (const float*)dev_in[1], in[1].strides[0],
                            (const float*)dev_in[2], in[2].strides[0], (float*)dev_out,
-                           out->strides[0], p.R, accumulate, cs);
+                           out->strides[0], p.R, accumulate, err_word, cs);
     }
     if (st != DASTAC_OK) return st;
     if (out->space == DASTAC_MEM_HOST && out_bytes > 0 &&

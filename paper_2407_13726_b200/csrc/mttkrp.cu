@@ -240,7 +240,8 @@ bool mttkrp_supports(const IndexMap& m) {
 
 dastac_status launch_mttkrp(const IndexMap& m, const float* T, const float* B, int64_t ldb,
                             const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
-                            int accumulate, cudaStream_t st) {
+                            int accumulate, int32_t* err_word, cudaStream_t st) {
+    (void)err_word;  // no kernel of this rule has a bounded wait
     const int64_t n = m.dims[0];  // rows of the result
     if (n == 0 || R == 0) return DASTAC_OK;
     if (!accumulate) {

@@ -17,6 +17,7 @@
 // packed stream, a thread unranks the first of its positions and steps with index increments;
 // unpack walks the dense box and ranks every point.
 #include "common.cuh"
+#include "waits.cuh"
 
 namespace dastac {
 namespace {
@@ -287,14 +288,14 @@ constexpr int kPackDepth = 2, kUnpackDepth = 3;
 constexpr int bulk_smem_bytes(int depth) { return kWarpsPerBlock * depth * kBulkBufBytes + kWarpsPerBlock * depth * 8; }
 constexpr int bulk_ctas_per_sm(int depth) { return depth <= 2 ? 3 : depth == 3 ? 2 : 1; }
 constexpr int kBulkSmemBytesMul = kWarpsPerBlock * 4 * kBulkBufBytes + kWarpsPerBlock * 2 * 8;  // Hadamard form: depth 2, two operands
-constexpr long long kBulkWaitBudget = 2000000000LL;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 template <typename T, bool MUL = false>
 __global__ void __launch_bounds__(32 * kWarpsPerBlock, MUL ? 1 : 3)
 pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restrict__ packed, int64_t rows,
-                 int windows_per_row, const T* __restrict__ factor = nullptr, int accumulate = 0) {
+                 int windows_per_row, long long wait_budget, int32_t* __restrict__ err_word,
+                 const T* __restrict__ factor = nullptr, int accumulate = 0) {
     constexpr int E = 16 / sizeof(T);
     extern __shared__ __align__(128) uint8_t bulk_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -356,8 +357,11 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
             w.bytes = (uint32_t)(w.c_hi - w.c_lo) * 16 + (w.sh ? 16u : 0u);
         }
     };
+    uint32_t pending = 0;  // bit b: a copy into buffer b has been requested and not yet waited for
     auto issue = [&](const Win& w, int b) {
-        if (w.bytes == 0 || lane != 0) return;
+        if (w.bytes == 0) return;
+        pending |= 1u << b;
+        if (lane != 0) return;
         const uint32_t bar = smem_addr(&bars[b]);
         // the warp's earlier generic-proxy reads of this buffer come before the async-proxy overwrite
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -382,6 +386,7 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
         issue(ahead[d], d);
     }
     uint32_t phases = 0;  // bit b: parity of the next completion of buffer b
+    bool dead = false;    // a wait ran out: stop, report, let the copies in flight land
     int b = 0;
     for (; item < items; item += warps, b = (b + 1 == D ? 0 : b + 1)) {
         const Win cur = ahead[0];
@@ -393,19 +398,12 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
         issue(ahead[D - 2], b == 0 ? D - 1 : b - 1);
         if (cur.live) {
             if (cur.bytes) {
-                const uint32_t bar = smem_addr(&bars[b]);
-                const long long t0 = clock64();
-                uint32_t done = 0;
-                while (!done) {
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\t"
-                        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                        "selp.u32 %0, 1, 0, p;\n\t}"
-                        : "=r"(done)
-                        : "r"(bar), "r"((phases >> b) & 1u)
-                        : "memory");
-                    if (!done && clock64() - t0 > kBulkWaitBudget) break;  // never expected; gives up instead of spinning
+                // never expected to run out; if it does, nothing of this window is stored
+                if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&bars[b]), (phases >> b) & 1u, wait_budget))) {
+                    dead = true;
+                    break;
                 }
+                pending &= ~(1u << b);
                 phases ^= 1u << b;
                 const uint8_t* src = buf0 + b * kBulkBufBytes;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
@@ -443,6 +441,11 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
         }
         __syncwarp();
     }
+    if (dead) {
+        if (lane == 0 && err_word) atomicExch(err_word, kErrWordPack);
+        for (int d = 0; d < D; ++d)  // the copies still in flight get one more budget to land
+            if (pending & (1u << d)) mbar_wait_bounded(smem_addr(&bars[d]), (phases >> d) & 1u, wait_budget);
+    }
 }
 
 // unpack through shared memory, the mirror image: a window is 256 aligned chunks of a dense row; the
@@ -452,7 +455,7 @@ pack_bulk_kernel(IndexMap m, const T* __restrict__ dense, Strides st, T* __restr
 template <typename T>
 __global__ void __launch_bounds__(32 * kWarpsPerBlock, 3)
 unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ dense, Strides st, int64_t rows,
-                   int windows_per_row) {
+                   int windows_per_row, long long wait_budget, int32_t* __restrict__ err_word) {
     constexpr int E = 16 / sizeof(T);
     extern __shared__ __align__(128) uint8_t bulk_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -518,8 +521,11 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
             w.bytes = (uint32_t)((hi - lo) / E) * 16 + (w.sh ? 16u : 0u);
         }
     };
+    uint32_t pending = 0;  // bit b: a copy into buffer b has been requested and not yet waited for
     auto issue = [&](const Win& w, int b) {
-        if (w.bytes == 0 || lane != 0) return;
+        if (w.bytes == 0) return;
+        pending |= 1u << b;
+        if (lane != 0) return;
         const uint32_t bar = smem_addr(&bars[b]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(w.bytes) : "memory");
@@ -542,6 +548,7 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
         issue(ahead[d], d);
     }
     uint32_t phases = 0;
+    bool dead = false;
     int b = 0;
     for (; item < items; item += warps, b = (b + 1 == D ? 0 : b + 1)) {
         const Win cur = ahead[0];
@@ -551,19 +558,12 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
         issue(ahead[D - 2], b == 0 ? D - 1 : b - 1);
         if (cur.live) {
             if (cur.bytes) {
-                const uint32_t bar = smem_addr(&bars[b]);
-                const long long t0 = clock64();
-                uint32_t done = 0;
-                while (!done) {
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\t"
-                        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                        "selp.u32 %0, 1, 0, p;\n\t}"
-                        : "=r"(done)
-                        : "r"(bar), "r"((phases >> b) & 1u)
-                        : "memory");
-                    if (!done && clock64() - t0 > kBulkWaitBudget) break;
+                // never expected to run out; if it does, nothing of this window is stored
+                if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&bars[b]), (phases >> b) & 1u, wait_budget))) {
+                    dead = true;
+                    break;
                 }
+                pending &= ~(1u << b);
                 phases ^= 1u << b;
             }
             const uint8_t* src = buf0 + b * kBulkBufBytes;
@@ -586,6 +586,11 @@ unpack_bulk_kernel(IndexMap m, const T* __restrict__ packed, T* __restrict__ den
             }
         }
         __syncwarp();
+    }
+    if (dead) {
+        if (lane == 0 && err_word) atomicExch(err_word, kErrWordUnpack);
+        for (int d = 0; d < D; ++d)  // the copies still in flight get one more budget to land
+            if (pending & (1u << d)) mbar_wait_bounded(smem_addr(&bars[d]), (phases >> d) & 1u, wait_budget);
     }
 }
 
@@ -658,7 +663,7 @@ dastac_status launch_hadamard(const IndexMap& m, const float* Bp, const float* C
         int64_t blocks = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (blocks > (int64_t)sm_count()) blocks = (int64_t)sm_count();  // four buffers per warp: one CTA per SM
         pack_bulk_kernel<uint32_t, true><<<(unsigned)blocks, 32 * kWarpsPerBlock, kBulkSmemBytesMul, stream>>>(
-            m, Cq, st, Oq, rows, (int)bwpr, Bq, accumulate);
+            m, Cq, st, Oq, rows, (int)bwpr, kDefaultWaitBudget, device_error_word(), Bq, accumulate);
         return launch_status();
     }
     const int grid = grid_for((m.slots + E - 1) / E, 256);
@@ -731,10 +736,10 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
             if (bwpr > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
             if (dtype == DASTAC_F32)
                 pack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kPackDepth), (cudaStream_t)stream>>>(
-                    m, (const uint32_t*)dense, st, (uint32_t*)packed, rows, (int)bwpr);
+                    m, (const uint32_t*)dense, st, (uint32_t*)packed, rows, (int)bwpr, kDefaultWaitBudget, device_error_word());
             else
                 pack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kPackDepth), (cudaStream_t)stream>>>(
-                    m, (const uint16_t*)dense, st, (uint16_t*)packed, rows, (int)bwpr);
+                    m, (const uint16_t*)dense, st, (uint16_t*)packed, rows, (int)bwpr, kDefaultWaitBudget, device_error_word());
             return launch_status();
         }
         const int grid = grid_for(rows * gpr * 32, 32 * kWarpsPerBlock);
@@ -764,7 +769,8 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
     IndexMap m = s->map;
     if (!strides_ok(m, dense_strides)) return DASTAC_ERR_INVALID_ARG;
     int64_t box = 1;
-    for (int k = 0; k < m.rank; ++k) box *= m.dims[k];
+    for (int k = 0; k < m.rank; ++k)
+        if (__builtin_mul_overflow(box, m.dims[k], &box)) return DASTAC_ERR_OVERFLOW;  // no such tensor fits in memory
     if (box == 0) return DASTAC_OK;
     if (!dense || (m.slots > 0 && !packed)) return DASTAC_ERR_INVALID_ARG;
     if (m.slots > 0 && !aligned16(packed)) return DASTAC_ERR_ALIGNMENT;
@@ -799,10 +805,10 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
             if (bwpr > 0x7fffffffLL || m.dims[m.rank - 1] > (int64_t(1) << 30)) return DASTAC_ERR_OVERFLOW;
             if (dtype == DASTAC_F32)
                 unpack_bulk_kernel<uint32_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kUnpackDepth), (cudaStream_t)stream>>>(
-                    m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)bwpr);
+                    m, (const uint32_t*)packed, (uint32_t*)dense, st, rows, (int)bwpr, kDefaultWaitBudget, device_error_word());
             else
                 unpack_bulk_kernel<uint16_t><<<(unsigned)blocks, 32 * kWarpsPerBlock, bulk_smem_bytes(kUnpackDepth), (cudaStream_t)stream>>>(
-                    m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)bwpr);
+                    m, (const uint16_t*)packed, (uint16_t*)dense, st, rows, (int)bwpr, kDefaultWaitBudget, device_error_word());
             return launch_status();
         }
     }

@@ -336,11 +336,13 @@ extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* de
             m.N = m.dims[1];
             m.M = hi[0] + 1;
             m.Q = m.dims[2];
-            m.count = upper_row_start(m.N, m.M) * m.Q;
+            // rows <= 2^59 points, Q <= 2^30: the product may not fit
+            if (__builtin_mul_overflow(upper_row_start(m.N, m.M), m.Q, &m.count)) return DASTAC_ERR_OVERFLOW;
             matched = true;
         } else if (full && free_pair(0, 1) && free_pair(0, 2) && free_pair(1, 2)) {
             m.kind = kDense;
-            m.count = m.dims[0] * m.dims[1] * m.dims[2];
+            // three extents of up to 2^30 each: checked product
+            if (__builtin_mul_overflow(m.dims[0] * m.dims[1], m.dims[2], &m.count)) return DASTAC_ERR_OVERFLOW;
             matched = true;
         }
     }

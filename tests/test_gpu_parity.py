@@ -403,7 +403,8 @@ def test_band_matmat(N, w, C):
     assert rel_err(outp.cpu().numpy(), ref, ref_abs) <= TOL_F32
 
 
-@pytest.mark.parametrize("n,R", [(1, 1), (2, 5), (7, 32), (33, 32), (70, 40), (130, 32), (96, 7)])
+@pytest.mark.parametrize("n,R", [(1, 1), (2, 5), (7, 32), (8, 3), (9, 32), (33, 32), (63, 16), (64, 32), (65, 8),
+                                 (70, 40), (130, 32), (96, 7), (200, 32), (257, 33), (300, 64)])
 def test_mttkrp(n, R):
     desc = st.tetrahedron(n)
     s = dastac.Structure(desc)
@@ -413,13 +414,25 @@ def test_mttkrp(n, R):
     ref, ref_abs = oracle.mttkrp(desc, T, B, C)
     packed = packed_dev(s, synth.tetrahedron_stream(3, 0, n))
     out = torch.full((n, R), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
     ws = _workspace("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out)
-    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out, workspace=ws)
+    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
     assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
     M0 = synth.dense(3, 3, (n, R))
     out2 = dev(M0)
-    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out2, accumulate=True, workspace=ws)
+    dastac.contract("ijk,jr,kr->ir", s, packed, [dev(B), dev(C)], out2, accumulate=True, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
     assert rel_err(out2.cpu().numpy(), ref + M0, ref_abs + np.abs(M0)) <= TOL_F32
+    # factor matrices and result with padded leading dimensions (rows not 16-byte aligned)
+    Bp = torch.zeros((n, R + 3), device="cuda")[:, :R]
+    Bp.copy_(dev(B))
+    Cp = torch.zeros((n, R + 1), device="cuda")[:, :R]
+    Cp.copy_(dev(C))
+    outp = torch.full((n, R + 5), float("nan"), device="cuda")[:, :R]
+    dastac.contract("ijk,jr,kr->ir", s, packed, [Bp, Cp], outp, workspace=ws, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(outp.cpu().numpy(), ref, ref_abs) <= TOL_F32
 
 
 @pytest.mark.parametrize("N,C", [(1, 1), (17, 9), (128, 256), (129, 64), (300, 200), (1000, 264), (512, 512)])
@@ -952,3 +965,48 @@ def test_contractions_random_structures():
             assert rel_err(Cm.cpu().numpy(), r, ra) <= TOL_F32, (desc.name, shape, desc.meta)
             done["mm"] += 1
     assert done["mv"] >= 5 and done["mm"] >= 5 and done["had"] >= 30
+
+
+@pytest.mark.parametrize("desc", [st.upper_triangle(1024), st.tetrahedron(512), st.upper_triangle(8192)],
+                         ids=["triangle1024", "tetrahedron512", "triangle8192"])
+def test_index_maps_exhaustive_against_the_oracle_at_kernel_sizes(desc):
+    """Every point of the sets the kernels run on (all but the 2^31-point triangle): the device maps
+    against the oracle's enumeration, bit for bit, in both directions."""
+    s = dastac.Structure(desc)
+    table = oracle.unrank_table(desc)                       # [count, rank]: the point at every position
+    assert table.shape[0] == s.nnz
+    idx = torch.from_numpy(table).cuda()
+    positions = torch.arange(s.nnz, dtype=torch.int64, device="cuda")
+    assert torch.equal(dastac.rank_batch(s, idx), positions)
+    assert torch.equal(dastac.unrank_batch(s, positions), idx)
+    if desc.rank == 2 and desc.dims[0] <= 1024:             # the whole box: points outside rank to -1
+        full = oracle.rank_table(desc)
+        N = desc.dims[0]
+        ij = np.stack(np.meshgrid(np.arange(N), np.arange(N), indexing="ij"), -1).reshape(-1, 2).astype(np.int32)
+        got = dastac.rank_batch(s, torch.from_numpy(ij).cuda()).cpu().numpy()
+        assert np.array_equal(got, full.reshape(-1))
+
+
+def test_expired_wait_is_reported_and_the_device_stays_usable():
+    """The expiry path of the bounded waits, run on purpose: one warp waits about a millisecond on a
+    barrier nothing arrives on, records its code and returns.  The host sees DASTAC_ERR_TIMEOUT with
+    that code, the word clears, and the next kernels (a pack/unpack round trip through the bulk-copy
+    kernels, which wait on barriers of the same kind) run as usual."""
+    st0, _ = dastac.device_error(clear=True)          # whatever earlier tests left: cleared
+    st1, word1 = dastac.device_error(clear=True)
+    assert (st1, word1) == (0, 0)
+    dastac.selftest_wait_expiry(2_000_000)
+    st2, word2 = dastac.device_error(clear=False)
+    assert st2 == 9 and word2 == 0x5354
+    assert "wait" in dastac.status_string(st2)
+    st3, word3 = dastac.device_error(clear=True)       # still set until cleared
+    assert (st3, word3) == (9, 0x5354)
+    assert dastac.device_error(clear=True) == (0, 0)
+    N = 1500
+    d = st.upper_triangle(N)
+    s = dastac.Structure(d)
+    A = synth.dense(7, 0, (N, N))
+    pk = dastac.pack(s, dev(A))
+    assert np.array_equal(pk.cpu().numpy()[: s.nnz], oracle.pack(d, A))
+    assert np.array_equal(dastac.unpack(s, pk).cpu().numpy(), oracle.unpack(d, oracle.pack(d, A)))
+    assert dastac.device_error(clear=True) == (0, 0)

@@ -143,6 +143,13 @@ def test_config_cardinalities_and_overflow():
     with pytest.raises(dastac.DastacError) as e:
         dastac.Structure(st.tetrahedron(2 ** 20 + 1))
     assert e.value.status == 6
+    # products of three accepted extents that leave 63 bits: the dense box and the half cube
+    for desc in (st.dense_box([2 ** 22, 2 ** 22, 2 ** 22]), st.upper_half_cube(2 ** 30, 2 ** 30, 2 ** 30)):
+        with pytest.raises(dastac.DastacError) as e:
+            dastac.Structure(desc)
+        assert e.value.status == 6
+    # the largest products that still fit are accepted, with the exact count
+    assert dastac.Structure(st.dense_box([2 ** 20, 2 ** 20, 2 ** 20])).nnz == 2 ** 60
 
 
 def test_large_offsets_round_trip_on_host():

@@ -501,3 +501,37 @@ def test_hadamard_structured_times_dense():
         assert ones.sum() == oracle.count(desc)
         # the packed result is the element-wise product of the two packed operands
         assert np.array_equal(oracle.pack(desc, out), oracle.pack(desc, B).astype(np.float64) * oracle.pack(desc, C))
+
+
+@pytest.mark.parametrize("threads", [1, 3])
+def test_clipped_timed_variants_equal_the_masked_forms(threads):
+    """The loops that are timed as the CPU baseline visit only the stored elements of the packed
+    operand; they must give the masked definition's sums (same products, fp64; only the order of
+    the additions may differ)."""
+    tol = dict(rtol=1e-12, atol=1e-12)
+    for N in (1, 2, 37, 130):
+        d = st.upper_triangle(N)
+        A = synth.dense(0, 0, (N, N), dist=synth.NORMAL)
+        x = synth.dense(0, 1, (N,), dist=synth.NORMAL)
+        pk = oracle.pack(d, A)
+        np.testing.assert_allclose(oracle.clip_matvec_upper(N, pk, x, threads), oracle.matvec(d, A, x)[0], **tol)
+        np.testing.assert_allclose(oracle.clip_symv(N, pk, x, threads), oracle.symv(A, x)[0], **tol)
+    for N, w, C in ((1, 0, 3), (9, 2, 5), (70, 8, 33), (40, 19, 4)):
+        A = synth.dense(1, 0, (N, N))
+        B = synth.dense(1, 1, (N, C))
+        got = oracle.clip_band_matmat(N, w, oracle.band_pack(N, w, A), B, threads)
+        np.testing.assert_allclose(got, oracle.matmat(st.band(N, w), A, B)[0], **tol)
+    for n, R in ((1, 1), (5, 3), (33, 8)):
+        d = st.tetrahedron(n)
+        T = synth.dense(3, 0, (n, n, n))
+        B = synth.dense(3, 1, (n, R))
+        C = synth.dense(3, 2, (n, R))
+        got = oracle.clip_mttkrp_tetra(n, oracle.pack(d, T), B, C, threads)
+        np.testing.assert_allclose(got, oracle.mttkrp(d, T, B, C)[0], **tol)
+    for N, C in ((1, 1), (50, 7)):
+        d = st.upper_triangle(N)
+        A = synth.dense(4, 0, (N, N), dist=synth.NORMAL, bf16=True)
+        B = synth.dense(4, 1, (N, C), dist=synth.NORMAL, bf16=True)
+        sel = np.arange(0, N, 3, dtype=np.int64)
+        got = oracle.clip_matmat_upper_bf16(N, oracle.pack(d, A), B, sel=sel, threads=threads)
+        np.testing.assert_allclose(got, oracle.matmat(d, A[sel], B, sel=sel)[0], **tol)

@@ -1,15 +1,17 @@
 """The bf16 triangular x dense contraction through the entry point that takes no workspace and
 allocates nothing (for callers that cannot obtain device memory around the call), checked against
-the regular entry point on the same operands.  Collected last on purpose: a failure here leaves
-every other test already run."""
+the regular entry point on the same operands (same kernels, same tile order, no atomics: the bits
+must agree) and against the oracle.  Collected last on purpose: a failure here leaves every other
+test already run."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import synth
 from synth import structures as st
 
-from _util import TOL_BF16, dev, packed_dev
+from _util import TOL_BF16, dev, packed_dev, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -23,6 +25,15 @@ def _operands(N, C, seed):
                         dtype=torch.bfloat16)
     B = dev(synth.dense(seed, 1, (N, C), dist=synth.NORMAL, scale=scale, bf16=True), "bf16")
     return s, packed, B
+
+
+def _oracle_err(N, C, seed, got):
+    """Forward error of `got` against the oracle on the same seeded operands (the parity tests' measure)."""
+    scale = N ** -0.5
+    A = synth.dense(seed, 0, (N, N), dist=synth.NORMAL, scale=scale, bf16=True)
+    B = synth.dense(seed, 1, (N, C), dist=synth.NORMAL, scale=scale, bf16=True)
+    ref, ref_abs = oracle.matmat(st.upper_triangle(N), A, B)
+    return rel_err(got.cpu().numpy(), ref, ref_abs)
 
 
 def _regular(s, packed, B, accumulate=False, out=None):
@@ -59,8 +70,13 @@ def test_two_calls_in_a_row_match_the_regular_entry_point():
     dastac.trimm_bf16_noalloc(s2, p2, B2, out2, err_word=err)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
-    assert _close(out1, _regular(s1, p1, B1))
-    assert _close(out2, _regular(s2, p2, B2))
+    ref1, ref2 = _regular(s1, p1, B1), _regular(s2, p2, B2)
+    assert _close(out1, ref1) and _close(out2, ref2)
+    # stronger than the tolerance: the two entry points run the same kernels in the same order
+    assert torch.equal(out1, ref1) and torch.equal(out2, ref2)
+    # and against the oracle, element by element
+    assert _oracle_err(1000, 264, 41, out1) <= TOL_BF16
+    assert _oracle_err(300, 200, 42, out2) <= TOL_BF16
     # accumulate and the largest supported size
     s3, p3, B3 = _operands(dastac.NOALLOC_MAX_N, 256, 43)
     C0 = dev(synth.dense(43, 2, (dastac.NOALLOC_MAX_N, 256)))
