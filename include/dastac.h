@@ -67,9 +67,13 @@ typedef enum {
     DASTAC_KIND_BAND_OFFSETS = 8,   /* lo<=j-i<=hi, square, any lo<=hi: rows packed back to back.  One
                                        off-diagonal (lo=hi=s) is a per-summand buffer of the strided band
                                        of Section 6.4; chosen when no class above applies           */
-    DASTAC_KIND_PLANE = 9           /* one index fixed (idx_a = c) or equal to an earlier one (idx_b = idx_a),
+    DASTAC_KIND_PLANE = 9,          /* one index fixed (idx_a = c) or equal to an earlier one (idx_b = idx_a),
                                        everything else dense: "Fixed i", "Fixed j", "Diagonal (plane)" of
                                        Table 1; packed as the dense box over the free indices        */
+    DASTAC_KIND_GENERIC = 10        /* any other conjunction of affine comparisons (rank 2 or 3, unit
+                                       coefficients on the inner indices) whose counting function the
+                                       library could fit when the structure was created: index maps, pack
+                                       and unpack only, through slower element-wise kernels           */
 } dastac_kind;
 
 #define DASTAC_LAYOUT_LEXICOGRAPHIC 0 /* exact pack in lexicographic order                         */
@@ -105,11 +109,18 @@ typedef struct {
 typedef struct dastac_structure dastac_structure;
 
 /*
- * Analyse a descriptor (Algorithm 1, "Symbolic Indexing", restricted to classes whose counting
- * polynomial is known in closed form).  The comparisons are normalised to difference bounds,
- * closed under implication, and matched against the recognised classes, so redundant or
- * re-ordered rows do not matter.  Errors: INVALID_ARG, OVERFLOW, UNSUPPORTED_STRUCTURE (a row that
- * is not a bound or a difference of two indices, or a set that is none of the classes).
+ * Analyse a descriptor (Algorithm 1, "Symbolic Indexing").  The comparisons are normalised to
+ * difference bounds, closed under implication, and matched against the classes whose counting
+ * polynomial is known in closed form, so redundant or re-ordered rows do not matter.
+ * A set that is none of those classes (or has rows that are not difference bounds, such as
+ * i + j <= N - 1 or 2 i <= j) gets DASTAC_KIND_GENERIC when it can: the library counts every slab
+ * of the set by brute force, fits the piecewise polynomial "points before slab i" to those counts
+ * (the stand-in for the symbolic counting step of Algorithm 1), fuses pieces that agree
+ * (Algorithm 2) and verifies the map.  Conditions: lexicographic layout, no redundancy map, rank 2
+ * or 3, coefficients -1, 0 or 1 on the last index (rank 3: on the last two), extents up to 2^20
+ * and at most 2^24 slabs (rank 2) or fibres (rank 3), at most 12 polynomial pieces; creation
+ * costs time proportional to the number of fibres.
+ * Errors: INVALID_ARG, OVERFLOW, UNSUPPORTED_STRUCTURE (none of the above applies).
  */
 dastac_status dastac_structure_create(const dastac_structure_desc* desc, dastac_structure** out);
 void dastac_structure_destroy(dastac_structure* s);
@@ -267,6 +278,76 @@ const char* dastac_status_string(dastac_status st);
 dastac_status dastac_trimm_bf16_noalloc(const dastac_structure* s, const void* A, const void* B,
                                         int64_t ldb, int64_t ncols, float* C, int64_t ldc,
                                         int32_t accumulate, int32_t* err_word, void* stream);
+
+/*
+ * A structured operand given as several summands (Section 4: the method works on the individual
+ * summands of a rule; every summand's region has its own compressed buffer, and a summand whose
+ * region equals an earlier one reuses that buffer instead of getting a second copy).  Examples:
+ * the strided band of Section 6.4 (three diagonals), the Leslie matrix of Table 1 (first row and
+ * sub-diagonal).
+ *   dastac_rule_create   one structure per summand descriptor (each as for
+ *                        dastac_structure_create, all over the same box) and the buffer index of
+ *                        each; summands with equal regions get the same index.  n = 1..64.
+ *   dastac_rule_size     number of summands and of distinct buffers.
+ *   dastac_rule_summand  structure (owned by the rule) and buffer index of summand k.
+ *   dastac_rule_pack     fills every distinct buffer from the dense tensor: `packed` is a host
+ *                        array of n_buffers device pointers, buffer b sized and aligned for the
+ *                        structure of the first summand that uses it.
+ *   dastac_rule_contract the rule `expr` with the summed operand in first place:
+ *                        out = sum_k contract(expr, summand k, rest...), enqueued in one call; the
+ *                        first summand overwrites `out` (adds to it when accumulate != 0), the
+ *                        others add.  `rest` holds the remaining inputs (in[1..] of
+ *                        dastac_contract), `packed` the device buffers as for dastac_rule_pack,
+ *                        `packed_batch_strides` (host, may be NULL) their batch strides.  Every
+ *                        summand must be a supported (expression, structure) pair; all are
+ *                        checked before anything is enqueued.  Workspace: the largest need of any
+ *                        summand (dastac_rule_contract_workspace).
+ * Regions of different summands that overlap without being equal are stored twice and counted
+ * twice, as the summed rule says.
+ */
+typedef struct dastac_rule dastac_rule;
+dastac_status dastac_rule_create(const dastac_structure_desc* summands, int32_t n, dastac_rule** out);
+void dastac_rule_destroy(dastac_rule* r);
+dastac_status dastac_rule_size(const dastac_rule* r, int32_t* n_summands, int32_t* n_buffers);
+dastac_status dastac_rule_summand(const dastac_rule* r, int32_t k, const dastac_structure** s, int32_t* buffer);
+dastac_status dastac_rule_pack(const dastac_rule* r, dastac_dtype dtype, const void* dense,
+                               const int64_t* dense_strides, void* const* packed, void* stream);
+dastac_status dastac_rule_contract_workspace(const char* expr, const dastac_rule* r, dastac_dtype dtype,
+                                             const dastac_operand* rest, int32_t n_rest,
+                                             const dastac_operand* out, size_t* bytes);
+dastac_status dastac_rule_contract(const char* expr, const dastac_rule* r, dastac_dtype dtype,
+                                   void* const* packed, const int64_t* packed_batch_strides,
+                                   const dastac_operand* rest, int32_t n_rest, const dastac_operand* out,
+                                   int32_t accumulate, void* workspace, size_t workspace_bytes,
+                                   int32_t* err_word, void* stream);
+
+/*
+ * Algorithm 2, "Piecewise QuasiPolynomial Fusion" (Section 4, "Piecewise Polynomial
+ * Simplification"), as a host procedure.  The counting step returns one polynomial per piece of
+ * the counted set; a piece (D', P') is dropped when another piece's polynomial P equals P' on D',
+ * and that piece's domain grows by D'.
+ *   poly     sum_t num[t] / den * prod_v x_v ^ exps[t * nvars + v]   (host arrays; den > 0;
+ *            exponents 0..6; nvars = the domain's rank)
+ *   domain   a descriptor as for dastac_structure_create (rows may be equalities; mirror and
+ *            layout are ignored); the box 0 <= x_v < dims[v] is implied
+ *   owner    host, n entries out: owner[k] = index of the piece whose polynomial holds on piece k
+ *            after fusion (owner[k] == k for the pieces that remain)
+ * "(P - P') restricted to D' is zero" is decided exactly: symbolically when the equalities of D'
+ * make the difference vanish, else at every integer point of D' when its box has at most 2^22
+ * points; a larger domain that is not decided symbolically is left alone.
+ */
+typedef struct {
+    int32_t nvars;
+    int32_t nterms;
+    const int32_t* exps;
+    const int64_t* num;
+    int64_t den;
+} dastac_poly;
+typedef struct {
+    dastac_structure_desc domain;
+    dastac_poly poly;
+} dastac_piece;
+dastac_status dastac_piecewise_fuse(const dastac_piece* pieces, int32_t n, int32_t* owner);
 
 /*
  * Device error word (no counterpart in the paper: it belongs to the execution model, not to the

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libdastac.so")
 F32, BF16 = 0, 1
 MEM_DEVICE, MEM_HOST = 0, 1
 (KIND_EMPTY, KIND_DENSE, KIND_UPPER, KIND_LOWER, KIND_BAND_DIAGONALS, KIND_TETRAHEDRON, KIND_BAND_EXACT,
- KIND_UPPER_SHIFTED, KIND_BAND_OFFSETS, KIND_PLANE) = range(10)
+ KIND_UPPER_SHIFTED, KIND_BAND_OFFSETS, KIND_PLANE, KIND_GENERIC) = range(11)
 LAYOUT_LEXICOGRAPHIC, LAYOUT_PADDED_DIAGONALS = 0, 1
 
 EXPORTS = [
@@ -27,7 +27,9 @@ EXPORTS = [
     "dastac_structure_kind", "dastac_rank", "dastac_unrank", "dastac_rank_batch",
     "dastac_unrank_batch", "dastac_pack", "dastac_unpack", "dastac_contract_workspace",
     "dastac_contract", "dastac_status_string", "dastac_launch_count", "dastac_trimm_bf16_noalloc",
-    "dastac_device_error", "dastac_selftest_wait_expiry",
+    "dastac_device_error", "dastac_selftest_wait_expiry", "dastac_piecewise_fuse",
+    "dastac_rule_create", "dastac_rule_destroy", "dastac_rule_size", "dastac_rule_summand", "dastac_rule_pack",
+    "dastac_rule_contract_workspace", "dastac_rule_contract",
 ]
 NOALLOC_MAX_N = 2048
 
@@ -80,6 +82,15 @@ _lib.dastac_launch_count.argtypes = []
 _lib.dastac_launch_count.restype = _i64
 _lib.dastac_device_error.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
 _lib.dastac_selftest_wait_expiry.argtypes = [_i64, _vp]
+_lib.dastac_piecewise_fuse.argtypes = [_vp, _i32, _vp]
+_lib.dastac_rule_create.argtypes = [_vp, _i32, ctypes.POINTER(_vp)]
+_lib.dastac_rule_destroy.argtypes = [_vp]
+_lib.dastac_rule_destroy.restype = None
+_lib.dastac_rule_size.argtypes = [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]
+_lib.dastac_rule_summand.argtypes = [_vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_i32)]
+_lib.dastac_rule_pack.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
+_lib.dastac_rule_contract_workspace.argtypes = [_vp, _vp, _i32, _vp, _i32, _vp, ctypes.POINTER(ctypes.c_size_t)]
+_lib.dastac_rule_contract.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, _vp, _i32, _vp, ctypes.c_size_t, _vp, _vp]
 
 
 def status_string(status: int) -> str:
@@ -119,25 +130,63 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 
+def _marshal_desc(desc):
+    """The C descriptor of ``desc`` plus the arrays its pointers refer to (keep them alive)."""
+    import numpy as np
+
+    dims = np.ascontiguousarray(desc.dims, dtype=np.int64)
+    params = np.ascontiguousarray(desc.params, dtype=np.int64)
+    rows = np.ascontiguousarray(desc.rows, dtype=np.int64)
+    is_eq = np.ascontiguousarray(desc.is_eq, dtype=np.uint8)
+    mirror = getattr(desc, "mirror", None)
+    mirror_arr = None if mirror is None else np.ascontiguousarray(mirror, dtype=np.int32)
+    layout = LAYOUT_PADDED_DIAGONALS if getattr(desc, "padded_diagonals", False) else LAYOUT_LEXICOGRAPHIC
+    nrows = rows.shape[0] if rows.ndim == 2 else 0
+    c = _StructureDesc(len(dims), len(params), nrows, dims.ctypes.data,
+                       rows.ctypes.data if nrows else None, is_eq.ctypes.data if nrows else None,
+                       params.ctypes.data if len(params) else None,
+                       None if mirror_arr is None else mirror_arr.ctypes.data, layout)
+    return c, (dims, params, rows, is_eq, mirror_arr)
+
+
+class _Poly(ctypes.Structure):
+    _fields_ = [("nvars", ctypes.c_int32), ("nterms", ctypes.c_int32), ("exps", ctypes.c_void_p),
+                ("num", ctypes.c_void_p), ("den", ctypes.c_int64)]
+
+
+class _Piece(ctypes.Structure):
+    _fields_ = [("domain", _StructureDesc), ("poly", _Poly)]
+
+
+def piecewise_fuse(pieces):
+    """Algorithm 2 on ``[(descriptor, terms, den), ...]`` where ``terms`` is a list of
+    ``(numerator, exponents)``: returns ``owner`` (see ``dastac_piecewise_fuse``)."""
+    import numpy as np
+
+    n = len(pieces)
+    arr = (_Piece * max(n, 1))()
+    keep = []
+    for k, (desc, terms, den) in enumerate(pieces):
+        c, held = _marshal_desc(desc)
+        nv = len(desc.dims)
+        exps = np.ascontiguousarray([list(e) for _, e in terms], dtype=np.int32).reshape(len(terms), nv)
+        num = np.ascontiguousarray([v for v, _ in terms], dtype=np.int64)
+        keep.append((held, exps, num))
+        arr[k].domain = c
+        arr[k].poly = _Poly(nv, len(terms), exps.ctypes.data if len(terms) else None,
+                            num.ctypes.data if len(terms) else None, int(den))
+    owner = (ctypes.c_int32 * max(n, 1))()
+    _check(_lib.dastac_piecewise_fuse(arr, n, owner), "dastac_piecewise_fuse")
+    return [int(owner[k]) for k in range(n)]
+
+
 class Structure:
     """Owns a ``dastac_structure`` created from a descriptor (any object with ``dims``,
     ``params``, ``rows``, ``is_eq``, ``mirror`` and ``padded_diagonals`` attributes)."""
 
     def __init__(self, desc):
-        import numpy as np
-
-        dims = np.ascontiguousarray(desc.dims, dtype=np.int64)
-        params = np.ascontiguousarray(desc.params, dtype=np.int64)
-        rows = np.ascontiguousarray(desc.rows, dtype=np.int64)
-        is_eq = np.ascontiguousarray(desc.is_eq, dtype=np.uint8)
-        mirror = getattr(desc, "mirror", None)
-        mirror_arr = None if mirror is None else np.ascontiguousarray(mirror, dtype=np.int32)
-        layout = LAYOUT_PADDED_DIAGONALS if getattr(desc, "padded_diagonals", False) else LAYOUT_LEXICOGRAPHIC
-        nrows = rows.shape[0] if rows.ndim == 2 else 0
-        c = _StructureDesc(len(dims), len(params), nrows, dims.ctypes.data,
-                           rows.ctypes.data if nrows else None, is_eq.ctypes.data if nrows else None,
-                           params.ctypes.data if len(params) else None,
-                           None if mirror_arr is None else mirror_arr.ctypes.data, layout)
+        c, keep = _marshal_desc(desc)
+        dims = keep[0]
         handle = _vp()
         _check(_lib.dastac_structure_create(ctypes.byref(c), ctypes.byref(handle)),
                "dastac_structure_create")
@@ -290,6 +339,91 @@ def contract(expr: str, s: Structure, packed: torch.Tensor, dense_inputs: Sequen
                                 None if err_word is None else err_word.data_ptr(), _stream()),
            "dastac_contract")
     return out
+
+
+class _SummandView:
+    """Counts and kind of a summand's structure (the structure itself belongs to the rule)."""
+
+    def __init__(self, handle, dims):
+        self._h = handle
+        self.rank, self.dims = len(dims), list(dims)
+        slots, nnz, kind, sym = _i64(), _i64(), _i32(), _i32()
+        _check(_lib.dastac_structure_count(handle, ctypes.byref(slots), ctypes.byref(nnz)), "dastac_structure_count")
+        _check(_lib.dastac_structure_kind(handle, ctypes.byref(kind), ctypes.byref(sym)), "dastac_structure_kind")
+        self.slots, self.nnz, self.kind = int(slots.value), int(nnz.value), int(kind.value)
+
+    capacity = Structure.capacity
+    empty_packed = Structure.empty_packed
+
+
+class Rule:
+    """Owns a ``dastac_rule``: a structured operand given as a list of summand descriptors."""
+
+    def __init__(self, descs):
+        arr = (_StructureDesc * len(descs))()
+        keep = []
+        for k, d in enumerate(descs):
+            arr[k], held = _marshal_desc(d)
+            keep.append(held)
+        handle = _vp()
+        _check(_lib.dastac_rule_create(arr, len(descs), ctypes.byref(handle)), "dastac_rule_create")
+        self._h = handle
+        ns, nb = _i32(), _i32()
+        _check(_lib.dastac_rule_size(handle, ctypes.byref(ns), ctypes.byref(nb)), "dastac_rule_size")
+        self.n_summands, self.n_buffers = int(ns.value), int(nb.value)
+        self.summands, self.buffer = [], []
+        for k in range(self.n_summands):
+            sh, b = _vp(), _i32()
+            _check(_lib.dastac_rule_summand(handle, k, ctypes.byref(sh), ctypes.byref(b)), "dastac_rule_summand")
+            self.summands.append(_SummandView(sh, descs[k].dims))
+            self.buffer.append(int(b.value))
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h and _lib is not None:
+            _lib.dastac_rule_destroy(h)
+
+    def empty_buffers(self, dtype=torch.float32, device="cuda"):
+        """One packed buffer per distinct region, sized for the first summand that uses it."""
+        bufs = [None] * self.n_buffers
+        for s, b in zip(self.summands, self.buffer):
+            if bufs[b] is None:
+                bufs[b] = s.empty_packed(dtype, device)
+        return bufs
+
+    def pack(self, dense: torch.Tensor, buffers=None):
+        buffers = buffers if buffers is not None else self.empty_buffers(dense.dtype, dense.device)
+        ptrs = (_vp * self.n_buffers)(*[t.data_ptr() for t in buffers])
+        strides = (_i64 * dense.dim())(*dense.stride())
+        _check(_lib.dastac_rule_pack(self._h, _dtype_code(dense), dense.data_ptr(), strides, ptrs, _stream()),
+               "dastac_rule_pack")
+        return buffers
+
+    def _rest(self, dense_inputs, out, batch):
+        rest = (_Operand * len(dense_inputs))()
+        for k, t in enumerate(dense_inputs):
+            rest[k] = _operand(t, None, batch)
+        return rest, _operand(out, None, batch)
+
+    def contract_workspace(self, expr, buffers, dense_inputs, out, batch: int = 1) -> int:
+        rest, o = self._rest(dense_inputs, out, batch)
+        nbytes = ctypes.c_size_t()
+        _check(_lib.dastac_rule_contract_workspace(expr.encode(), self._h, _dtype_code(buffers[0]), rest, len(dense_inputs),
+                                                   ctypes.byref(o), ctypes.byref(nbytes)), "dastac_rule_contract_workspace")
+        return int(nbytes.value)
+
+    def contract(self, expr, buffers, dense_inputs, out, accumulate=False, workspace=None, err_word=None, batch: int = 1):
+        """``out = sum over the summands of contract(expr, summand, dense_inputs...)`` in one call."""
+        rest, o = self._rest(dense_inputs, out, batch)
+        ptrs = (_vp * self.n_buffers)(*[t.data_ptr() for t in buffers])
+        ws_ptr, ws_bytes = None, 0
+        if workspace is not None:
+            ws_ptr, ws_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+        _check(_lib.dastac_rule_contract(expr.encode(), self._h, _dtype_code(buffers[0]), ptrs, None, rest, len(dense_inputs),
+                                         ctypes.byref(o), int(accumulate), ws_ptr, ws_bytes,
+                                         None if err_word is None else err_word.data_ptr(), _stream()),
+               "dastac_rule_contract")
+        return out
 
 
 def trimm_bf16_noalloc(s: Structure, packed: torch.Tensor, B: torch.Tensor, out: torch.Tensor,

@@ -6,10 +6,13 @@
 #include <cstdint>
 
 #include "../../include/dastac.h"
+#include "generic.cuh"
 #include "indexmap.cuh"
 
 struct dastac_structure {
     dastac::IndexMap map;
+    dastac::GenericMap* generic = nullptr;  // map.kind == kGeneric: the fitted map (owned)
+    ~dastac_structure() { delete generic; }
 };
 
 namespace dastac {

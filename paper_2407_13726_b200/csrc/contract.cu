@@ -69,6 +69,10 @@ dastac_status make_plan(const char* expr, const dastac_operand* in, int32_t n_in
     if (p.cls == kNoExpr) return DASTAC_ERR_UNSUPPORTED_EXPR;
     const int want_in = (p.cls == kMttkrp || p.cls == kMoment3) ? 3 : 2;  // the tensor-times-matrix rule has two inputs as well
     if (n_in != want_in) return DASTAC_ERR_INVALID_ARG;
+    // fitted maps have element-wise kernels only (index maps, pack, unpack)
+    for (int k = 0; k < n_in; ++k)
+        if (in[k].structure && in[k].structure->map.kind == kGeneric) return DASTAC_ERR_UNSUPPORTED_EXPR;
+    if (out->structure && out->structure->map.kind == kGeneric) return DASTAC_ERR_UNSUPPORTED_EXPR;
     if (p.cls == kMoment2 || p.cls == kMoment3) {
         // dense B (samples x features) as every factor, packed unique part of the symmetric result out
         for (int k = 0; k < n_in; ++k)

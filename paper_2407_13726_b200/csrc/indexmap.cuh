@@ -43,7 +43,10 @@ enum Kind : int32_t {
     // "Fixed i", "Fixed j" of Table 1.  The packed layout is the dense box over the free indices
     // in their own order.  dep is kept in `w`, src (or -1) in `lo_off`, c in `hi_off`; M and Q hold
     // the extents of the first and second free index.
-    kPlane = 9
+    kPlane = 9,
+    // Any other conjunction of affine comparisons whose counting function could be fitted when the
+    // structure was created; the map itself is a GenericMap (generic.cuh), not this struct.
+    kGeneric = 10
 };
 
 // Plain data, passed to kernels by value.

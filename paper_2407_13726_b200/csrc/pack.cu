@@ -51,6 +51,56 @@ __global__ void unrank_batch_kernel(IndexMap m, const int64_t* __restrict__ off,
     }
 }
 
+// ---- structures with a fitted map (generic.cuh): element-wise kernels ---------------------------
+__global__ void g_rank_batch_kernel(GenericMap g, const int32_t* __restrict__ idx, int64_t n, int64_t* __restrict__ off) {
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < n; t += (int64_t)gridDim.x * blockDim.x) {
+        int64_t p[3] = {0, 0, 0};
+        for (int k = 0; k < g.rank; ++k) p[k] = idx[t * g.rank + k];
+        off[t] = g_in_domain(g, p) ? g_rank(g, p) : -1;
+    }
+}
+
+__global__ void g_unrank_batch_kernel(GenericMap g, const int64_t* __restrict__ off, int64_t n, int32_t* __restrict__ idx) {
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < n; t += (int64_t)gridDim.x * blockDim.x) {
+        int64_t p[3] = {-1, -1, -1};
+        const int64_t o = off[t];
+        if (o >= 0 && o < g.count) g_unrank(g, o, p);
+        for (int k = 0; k < g.rank; ++k) idx[t * g.rank + k] = (int32_t)p[k];
+    }
+}
+
+// A warp per fibre of the last index: the position of the fibre's first stored element is evaluated
+// once, the lanes then move along the fibre (contiguous in the packed vector, and in the dense tensor
+// when its last stride is 1).  UNPACK writes the whole fibre of the box, zeros outside the set.
+template <typename T, bool UNPACK>
+__global__ void g_fibre_copy_kernel(GenericMap g, T* __restrict__ dense, Strides st, T* __restrict__ packed) {
+    const int lane = threadIdx.x & 31;
+    const int64_t fibres = g.rank == 2 ? g.dims[0] : g.dims[0] * g.dims[1];
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t last = g.dims[g.rank - 1];
+    for (int64_t f = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); f < fibres; f += warps) {
+        int64_t outer[3] = {f, 0, 0};
+        if (g.rank == 3) {
+            outer[0] = f / g.dims[1];
+            outer[1] = f - outer[0] * g.dims[1];
+        }
+        int64_t lo, hi;
+        const bool live = g_last_bounds(g, outer, lo, hi) && hi >= lo;
+        int64_t base = 0;
+        if (live) {
+            base = g_s1(g, outer[0]);
+            if (g.rank == 3) base += g_s2(g, outer[0], outer[1]);
+        }
+        T* drow = dense + outer[0] * st.s[0] + (g.rank == 3 ? outer[1] * st.s[1] : 0);
+        const int64_t ls = st.s[g.rank - 1];
+        if (UNPACK) {
+            for (int64_t x = lane; x < last; x += 32) drow[x * ls] = (live && x >= lo && x <= hi) ? packed[base + (x - lo)] : T(0);
+        } else if (live) {
+            for (int64_t x = lo + lane; x <= hi; x += 32) packed[base + (x - lo)] = drow[x * ls];
+        }
+    }
+}
+
 template <typename T>
 struct Vec16 {
     static constexpr int kElems = 16 / sizeof(T);
@@ -679,6 +729,10 @@ extern "C" dastac_status dastac_rank_batch(const dastac_structure* s, const int3
                                            int64_t* off, void* stream) {
     if (!s || n < 0 || (n > 0 && (!idx || !off))) return DASTAC_ERR_INVALID_ARG;
     if (n == 0) return DASTAC_OK;
+    if (s->map.kind == kGeneric) {
+        g_rank_batch_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(*s->generic, idx, n, off);
+        return launch_status();
+    }
     rank_batch_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(s->map, idx, n, off);
     return launch_status();
 }
@@ -687,6 +741,10 @@ extern "C" dastac_status dastac_unrank_batch(const dastac_structure* s, const in
                                              int64_t n, int32_t* idx, void* stream) {
     if (!s || n < 0 || (n > 0 && (!idx || !off))) return DASTAC_ERR_INVALID_ARG;
     if (n == 0) return DASTAC_OK;
+    if (s->map.kind == kGeneric) {
+        g_unrank_batch_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(*s->generic, off, n, idx);
+        return launch_status();
+    }
     unrank_batch_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(s->map, off, n, idx);
     return launch_status();
 }
@@ -703,6 +761,16 @@ extern "C" dastac_status dastac_pack(const dastac_structure* s, dastac_dtype dty
     if (!aligned16(packed)) return DASTAC_ERR_ALIGNMENT;
     Strides st{{0, 0, 0}};
     for (int k = 0; k < m.rank; ++k) st.s[k] = dense_strides[k];
+    if (m.kind == kGeneric) {
+        const GenericMap& g = *s->generic;
+        const int64_t fibres = g.rank == 2 ? g.dims[0] : g.dims[0] * g.dims[1];
+        const int grid = grid_for(fibres * 32, 256);
+        if (dtype == DASTAC_F32)
+            g_fibre_copy_kernel<uint32_t, false><<<grid, 256, 0, (cudaStream_t)stream>>>(g, (uint32_t*)const_cast<void*>(dense), st, (uint32_t*)packed);
+        else
+            g_fibre_copy_kernel<uint16_t, false><<<grid, 256, 0, (cudaStream_t)stream>>>(g, (uint16_t*)const_cast<void*>(dense), st, (uint16_t*)packed);
+        return launch_status();
+    }
     const int E = 16 / elt_size(dtype);
     // (the row kernels below only use the row intervals, which the collapsed view provides)
     if ((reinterpret_cast<uintptr_t>(dense) % elt_size(dtype)) == 0) collapse_half_cube(m, st);
@@ -776,6 +844,16 @@ extern "C" dastac_status dastac_unpack(const dastac_structure* s, dastac_dtype d
     if (m.slots > 0 && !aligned16(packed)) return DASTAC_ERR_ALIGNMENT;
     Strides st{{0, 0, 0}};
     for (int k = 0; k < m.rank; ++k) st.s[k] = dense_strides[k];
+    if (m.kind == kGeneric) {
+        const GenericMap& g = *s->generic;
+        const int64_t fibres = g.rank == 2 ? g.dims[0] : g.dims[0] * g.dims[1];
+        const int grid = grid_for(fibres * 32, 256);
+        if (dtype == DASTAC_F32)
+            g_fibre_copy_kernel<uint32_t, true><<<grid, 256, 0, (cudaStream_t)stream>>>(g, (uint32_t*)dense, st, (uint32_t*)const_cast<void*>(packed));
+        else
+            g_fibre_copy_kernel<uint16_t, true><<<grid, 256, 0, (cudaStream_t)stream>>>(g, (uint16_t*)dense, st, (uint16_t*)const_cast<void*>(packed));
+        return launch_status();
+    }
     const int esz = elt_size(dtype);
     const int E = 16 / esz;
     // 128-bit stores need a unit inner stride, a 16-byte aligned base and outer strides that keep

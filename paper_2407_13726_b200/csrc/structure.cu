@@ -8,11 +8,16 @@
 // The closed matrix is matched against the classes whose counting polynomial is known.
 #include <climits>
 #include <cstring>
+#include <array>
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
 namespace dastac {
+
+dastac_status build_generic_map(int rank, const int64_t* dims, const std::vector<std::array<int64_t, 4>>& user_rows,
+                                GenericMap** out);
 
 std::atomic<int64_t> g_launches{0};
 
@@ -95,8 +100,52 @@ bool add_row(Bounds& b, int rank, const int64_t* a, int64_t c) {
 
 using namespace dastac;
 
-extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* desc,
-                                                 dastac_structure** out) {
+static dastac_status create_recognised(const dastac_structure_desc* desc, dastac_structure** out);
+
+// A descriptor that is none of the recognised classes gets a fitted map when it can (generic.cuh):
+// exact lexicographic layout, no redundancy map, rank 2 or 3.
+extern "C" dastac_status dastac_structure_create(const dastac_structure_desc* desc, dastac_structure** out) {
+    const dastac_status st = create_recognised(desc, out);
+    if (st != DASTAC_ERR_UNSUPPORTED_STRUCTURE) return st;
+    if (desc->layout != DASTAC_LAYOUT_LEXICOGRAPHIC || desc->rank < 2) return st;
+    if (desc->mirror)
+        for (int k = 0; k < desc->rank; ++k)
+            if (desc->mirror[k] != k) return st;
+    const int rank = desc->rank, np = desc->nparams, width = rank + np + 1;
+    std::vector<std::array<int64_t, 4>> rows;
+    for (int r = 0; r < desc->nrows; ++r) {
+        const int64_t* row = desc->rows + (size_t)r * width;
+        std::array<int64_t, 4> a{0, 0, 0, row[width - 1]};
+        for (int k = 0; k < rank; ++k) a[(size_t)k] = row[k];
+        for (int p = 0; p < np; ++p) {
+            if (desc->params[p] > (int64_t(1) << 40) || desc->params[p] < -(int64_t(1) << 40) || row[rank + p] > 1024 ||
+                row[rank + p] < -1024)
+                return st;
+            a[3] += row[rank + p] * desc->params[p];
+        }
+        rows.push_back(a);
+        if (desc->is_eq[r]) rows.push_back({-a[0], -a[1], -a[2], -a[3]});
+    }
+    GenericMap* g = nullptr;
+    const dastac_status gs = build_generic_map(rank, desc->dims, rows, &g);
+    if (gs != DASTAC_OK) return gs == DASTAC_ERR_OVERFLOW ? gs : st;
+    dastac_structure* s = new (std::nothrow) dastac_structure;
+    if (!s) {
+        delete g;
+        return DASTAC_ERR_INVALID_ARG;
+    }
+    std::memset(&s->map, 0, sizeof(s->map));
+    s->map.kind = kGeneric;
+    s->map.rank = rank;
+    s->map.Q = 1;
+    for (int k = 0; k < rank; ++k) s->map.dims[k] = desc->dims[k];
+    s->map.count = s->map.slots = g->count;
+    s->generic = g;
+    *out = s;
+    return DASTAC_OK;
+}
+
+static dastac_status create_recognised(const dastac_structure_desc* desc, dastac_structure** out) {
     if (!desc || !out) return DASTAC_ERR_INVALID_ARG;
     *out = nullptr;
     const int rank = desc->rank, np = desc->nparams, nr = desc->nrows;
@@ -384,6 +433,12 @@ extern "C" dastac_status dastac_structure_kind(const dastac_structure* s, int32_
 
 extern "C" dastac_status dastac_rank(const dastac_structure* s, const int32_t* idx, int64_t* off) {
     if (!s || !idx || !off) return DASTAC_ERR_INVALID_ARG;
+    if (s->map.kind == kGeneric) {
+        const int64_t x[3] = {idx[0], s->map.rank > 1 ? idx[1] : 0, s->map.rank > 2 ? idx[2] : 0};
+        if (!g_in_domain(*s->generic, x)) return DASTAC_ERR_INVALID_ARG;
+        *off = g_rank(*s->generic, x);
+        return DASTAC_OK;
+    }
     if (!in_set(s->map, idx)) return DASTAC_ERR_INVALID_ARG;
     *off = rank_of(s->map, idx);
     return DASTAC_OK;
@@ -392,6 +447,12 @@ extern "C" dastac_status dastac_rank(const dastac_structure* s, const int32_t* i
 extern "C" dastac_status dastac_unrank(const dastac_structure* s, int64_t off, int32_t* idx) {
     if (!s || !idx) return DASTAC_ERR_INVALID_ARG;
     if (off < 0 || off >= s->map.slots) return DASTAC_ERR_INVALID_ARG;
+    if (s->map.kind == kGeneric) {
+        int64_t x[3] = {0, 0, 0};
+        g_unrank(*s->generic, off, x);
+        for (int k = 0; k < s->map.rank; ++k) idx[k] = (int32_t)x[k];
+        return DASTAC_OK;
+    }
     unrank_of(s->map, off, idx);
     return DASTAC_OK;
 }

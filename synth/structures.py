@@ -152,3 +152,19 @@ def equal_indices(dims: Sequence[int], a: int, b: int) -> Descriptor:
     eq[-1] = 1
     return Descriptor(list(dims), list(dims), _rows(rank, rank, items), eq, name="equal_indices",
                       meta={"a": a, "b": b})
+
+
+def affine_set(dims: Sequence[int], comparisons: Sequence[Sequence[int]], name: str = "affine_set") -> Descriptor:
+    """Any conjunction of affine comparisons inside the box ``dims``: every item of ``comparisons``
+    is ``(a_0, ..., a_{rank-1}, c)`` and states ``sum a_k idx_k + c >= 0``.  params = dims."""
+    rank = len(dims)
+    items = _box_rows(rank, rank, list(range(rank)))
+    for cmp_ in comparisons:
+        assert len(cmp_) == rank + 1
+        items.append(list(cmp_[:rank]) + [0] * rank + [cmp_[rank]])
+    return Descriptor(list(dims), list(dims), _rows(rank, rank, items), np.zeros(len(items), np.uint8), name=name)
+
+
+def anti_triangle(N: int) -> Descriptor:
+    """{(i, j) : i + j <= N - 1}: the triangle above the anti-diagonal."""
+    return affine_set([N, N], [[-1, -1, N - 1]], name="anti_triangle")

@@ -1010,3 +1010,105 @@ def test_expired_wait_is_reported_and_the_device_stays_usable():
     assert np.array_equal(pk.cpu().numpy()[: s.nnz], oracle.pack(d, A))
     assert np.array_equal(dastac.unpack(s, pk).cpu().numpy(), oracle.unpack(d, oracle.pack(d, A)))
     assert dastac.device_error(clear=True) == (0, 0)
+
+
+FITTED = [
+    st.anti_triangle(301),
+    st.affine_set([150, 400], [[-2, 1, 0]], name="2i<=j"),
+    st.affine_set([97, 97], [[-1, -1, 130], [1, 1, -40], [3, -1, 30]], name="polygon"),
+    st.affine_set([40, 41, 45], [[-1, 1, 0, 0], [1, -1, 1, 0]], name="i<=j<=i+k"),
+    st.affine_set([33, 47, 29], [[-1, -1, -1, 60]], name="i+j+k<=60"),
+    st.affine_set([50, 50, 50], [[-1, 1, 0, 0], [0, -1, 1, 0], [1, 0, -1, 9]], name="i<=j<=k<=i+9"),
+]
+
+
+@pytest.mark.parametrize("desc", FITTED, ids=lambda d: f"{d.name}{d.dims}")
+def test_fitted_maps_and_copies_on_the_device(desc):
+    """Descriptors outside the recognised classes: device rank/unrank against the oracle's enumeration at
+    every point of the box, pack and unpack bit for bit (fp32 with NaN payloads and -0, and bf16)."""
+    s = dastac.Structure(desc)
+    assert s.kind == dastac.KIND_GENERIC
+    table = oracle.rank_table(desc)
+    points = oracle.unrank_table(desc)
+    assert s.nnz == len(points)
+    box = np.stack(np.meshgrid(*[np.arange(n) for n in desc.dims], indexing="ij"), -1).reshape(-1, desc.rank).astype(np.int32)
+    assert np.array_equal(dastac.rank_batch(s, torch.from_numpy(box).cuda()).cpu().numpy(), table.reshape(-1))
+    pos = torch.arange(s.nnz, dtype=torch.int64, device="cuda")
+    assert np.array_equal(dastac.unrank_batch(s, pos).cpu().numpy(), points)
+    A = synth.dense(12, 0, tuple(desc.dims))
+    bits = A.view(np.uint32).reshape(-1)
+    bits[::7] = 0x7FC00123            # NaN with a payload
+    bits[3::11] = 0x80000000          # -0.0
+    pk = dastac.pack(s, dev(A))
+    assert np.array_equal(pk.cpu().numpy().view(np.uint32)[: s.nnz], oracle.pack(desc, A).view(np.uint32))
+    back = dastac.unpack(s, pk, torch.full(tuple(desc.dims), float("nan"), device="cuda"))
+    assert np.array_equal(back.cpu().numpy().view(np.uint32), oracle.unpack(desc, oracle.pack(desc, A)).view(np.uint32))
+    # bf16, and a dense tensor with padded strides
+    H = synth.dense(12, 1, tuple(desc.dims), dist=synth.NORMAL, bf16=True)
+    wide = torch.zeros(tuple(desc.dims[:-1]) + (desc.dims[-1] + 3,), dtype=torch.bfloat16, device="cuda")[..., : desc.dims[-1]]
+    wide.copy_(dev(H, "bf16"))
+    pkh = dastac.pack(s, wide)
+    assert np.array_equal(pkh.view(torch.int16).cpu().numpy().view(np.uint16)[: s.nnz], oracle.pack(desc, H))
+    backh = dastac.unpack(s, pkh)
+    assert np.array_equal(backh.view(torch.int16).cpu().numpy().view(np.uint16), oracle.unpack(desc, oracle.pack(desc, H)))
+    # a fitted map has no contraction kernels
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.contract("ij,j->i" if desc.rank == 2 else "ijk,jr,kr->ir", s, pk,
+                        [torch.zeros(desc.dims[1], device="cuda")] if desc.rank == 2 else
+                        [torch.zeros((desc.dims[1], 4), device="cuda"), torch.zeros((desc.dims[2], 4), device="cuda")],
+                        torch.zeros(desc.dims[0], device="cuda") if desc.rank == 2 else torch.zeros((desc.dims[0], 4), device="cuda"))
+    assert e.value.status == 3
+
+
+def _rule_reference(descs, A, x):
+    """Sum over the summands of the masked definition (the regions of these rules are disjoint)."""
+    ref, ref_abs = np.zeros(A.shape[0]), np.zeros(A.shape[0])
+    for d in descs:
+        r, ra = oracle.matvec(d, A, x)
+        ref, ref_abs = ref + r, ref_abs + ra
+    return ref, ref_abs
+
+
+@pytest.mark.parametrize("name", ["strided_band", "leslie"])
+def test_rule_with_several_summands_in_one_call(name):
+    """A structured operand that is a sum of summands, each with its own compressed buffer (Section 4):
+    the strided band j = i, j - i = +-s of Section 6.4 and the Leslie matrix of Table 1 (first row and
+    sub-diagonal), packed and multiplied with a vector through one call each."""
+    N = 1000
+    if name == "strided_band":
+        descs = [st.offset_band(N, 0, 0), st.offset_band(N, 37, 37), st.offset_band(N, -37, -37)]
+    else:
+        descs = [st.fixed_index([N, N], 0, 0), st.offset_band(N, -1, -1)]
+    rule = dastac.Rule(descs)
+    assert rule.n_buffers == len(descs)
+    A = synth.dense(13, 0, (N, N))
+    x = synth.dense(13, 1, (N,))
+    bufs = rule.pack(dev(A))
+    for d, b, v in zip(descs, bufs, rule.summands):
+        assert np.array_equal(b.cpu().numpy()[: v.nnz], oracle.pack(d, A))
+    ref, ref_abs = _rule_reference(descs, A, x)
+    # the rule's value is the masked dense product as well
+    mask = np.zeros((N, N), bool)
+    for d in descs:
+        mask |= oracle.rank_table(d) >= 0
+    assert np.allclose((np.where(mask, A, 0).astype(np.float64) @ x.astype(np.float64)), ref, rtol=1e-12, atol=1e-12)
+    y = torch.full((N,), float("nan"), device="cuda")
+    n = rule.contract_workspace("ij,j->i", bufs, [dev(x)], y)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda") if n else None
+    rule.contract("ij,j->i", bufs, [dev(x)], y, workspace=ws)
+    assert rel_err(y.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    y0 = synth.dense(13, 2, (N,))
+    y2 = dev(y0)
+    rule.contract("ij,j->i", bufs, [dev(x)], y2, accumulate=True, workspace=ws)
+    assert rel_err(y2.cpu().numpy(), ref + y0, ref_abs + np.abs(y0)) <= TOL_F32
+    # matrix times dense matrix through the same rule object
+    B = synth.dense(13, 3, (N, 24))
+    C = torch.full((N, 24), float("nan"), device="cuda")
+    n = rule.contract_workspace("ij,jc->ic", bufs, [dev(B)], C)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda") if n else None
+    rule.contract("ij,jc->ic", bufs, [dev(B)], C, workspace=ws)
+    refC, refC_abs = np.zeros((N, 24)), np.zeros((N, 24))
+    for d in descs:
+        r, ra = oracle.matmat(d, A, B)
+        refC, refC_abs = refC + r, refC_abs + ra
+    assert rel_err(C.cpu().numpy(), refC, refC_abs) <= TOL_F32

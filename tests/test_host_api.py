@@ -93,18 +93,33 @@ def test_recognition_is_independent_of_how_rows_are_written():
     strict = st.Descriptor([N, N], [N], np.array([[-1, 1, 0, -1]], dtype=np.int64), np.zeros(1, np.uint8))
     ss = dastac.Structure(strict)
     assert (ss.kind, ss.nnz) == (dastac.KIND_UPPER_SHIFTED, N * (N - 1) // 2) and oracle.count(strict) == ss.nnz
-    # a lower bound on i alone (i >= 2) is not a recognised class
+    # a lower bound on i alone (i >= 2) is none of the recognised classes: it gets a fitted map
+    rows_from_2 = st.Descriptor([N, N], [N], np.array([[1, 0, 0, -2]], dtype=np.int64), np.zeros(1, np.uint8))
+    g = dastac.Structure(rows_from_2)
+    assert (g.kind, g.nnz) == (dastac.KIND_GENERIC, (N - 2) * N) and oracle.count(rows_from_2) == g.nnz
+    # ... unless the innermost index carries a coefficient other than -1, 0, 1 (i <= 2j: a quasi-polynomial count)
     with pytest.raises(dastac.DastacError) as e:
-        dastac.Structure(st.Descriptor([N, N], [N], np.array([[1, 0, 0, -2]], dtype=np.int64), np.zeros(1, np.uint8)))
+        dastac.Structure(st.Descriptor([N, N], [N], np.array([[-1, 2, 0, 0]], dtype=np.int64), np.zeros(1, np.uint8)))
     assert e.value.status == 2
     # an equality row (diagonal) closes to the band of half width 0, packed exactly: N points, rank(i, i) = i
     diag = dastac.Structure(st.diagonal(5))
     assert (diag.kind, diag.nnz) == (dastac.KIND_BAND_EXACT, 5) and dastac.rank(diag, (3, 3)) == 3
     assert oracle.count(st.diagonal(5)) == 5
-    # a row coupling three indices is not a difference bound
+    # a row coupling three indices is not a difference bound: fitted map as well
     three = st.Descriptor([4, 4, 4], [4], np.array([[1, 1, -1, 0, 0]], dtype=np.int64), np.zeros(1, np.uint8))
-    with pytest.raises(dastac.DastacError):
-        dastac.Structure(three)
+    g3 = dastac.Structure(three)
+    assert (g3.kind, g3.nnz) == (dastac.KIND_GENERIC, oracle.count(three))
+    # the padded-diagonal layout and a redundancy map are for recognised classes only
+    odd = st.anti_triangle(6)
+    odd.padded_diagonals = True
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(odd)
+    assert e.value.status == 2
+    odd = st.anti_triangle(6)
+    odd.mirror = [1, 0]
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Structure(odd)
+    assert e.value.status == 2
     # contradictory rows give the empty set
     empty = st.Descriptor([5, 5], [5], np.array([[1, -1, 0, -1], [-1, 1, 0, -1]], dtype=np.int64),
                           np.zeros(2, np.uint8))
@@ -277,17 +292,17 @@ def test_plane_structures_kind_and_refusals():
     assert f.kind == dastac.KIND_PLANE and f.nnz == 800 and dastac.unrank(f, 17) == (2, 49, 1)
     assert dastac.Structure(st.fixed_index([100, 50, 8], 1, 50)).nnz == 0        # outside the box: empty
     assert dastac.Structure(st.equal_indices([9, 9], 0, 1)).kind == dastac.KIND_BAND_EXACT   # square matrix: the w = 0 band
-    # two determined indices (a line) and an equality combined with an order are not classes
+    # two determined indices (a line) and an equality combined with an order are not planes: they get fitted maps
     two = st.fixed_index([5, 6, 7], 0, 1)
     two.rows = np.vstack([two.rows, [0, 1, 0, 0, 0, 0, -2]])
     two.is_eq = np.append(two.is_eq, 1).astype(np.uint8)
-    with pytest.raises(dastac.DastacError):
-        dastac.Structure(two)
+    line = dastac.Structure(two)
+    assert (line.kind, line.nnz) == (dastac.KIND_GENERIC, 7) and dastac.unrank(line, 4) == (1, 2, 4)
     mixed = st.equal_indices([6, 6, 6], 0, 1)
     mixed.rows = np.vstack([mixed.rows, [0, -1, 1, 0, 0, 0, 0]])                  # j <= k as well
     mixed.is_eq = np.append(mixed.is_eq, 0).astype(np.uint8)
-    with pytest.raises(dastac.DastacError):
-        dastac.Structure(mixed)
+    wedge = dastac.Structure(mixed)
+    assert (wedge.kind, wedge.nnz) == (dastac.KIND_GENERIC, oracle.count(mixed))
 
 
 def test_exact_band_limits_and_kind():
@@ -478,3 +493,121 @@ def test_random_planes_and_boxes():
         _check_against_enumeration(desc)
 
     run()
+
+
+# ---- descriptors outside the recognised classes: fitted maps ----------------------------------------
+
+GENERIC_CASES = [
+    st.anti_triangle(1), st.anti_triangle(2), st.anti_triangle(23),
+    st.affine_set([17, 40], [[-2, 1, 0]], name="2i<=j"),
+    st.affine_set([14, 40], [[3, -1, 2]], name="j<=3i+2"),
+    st.affine_set([30, 30], [[-1, -1, 40], [1, 1, -12], [3, -1, 9]], name="polygon"),
+    st.affine_set([25, 25], [[1, 0, -4], [-1, 0, 19], [-1, 1, 3]], name="rows4to19_band"),
+    st.affine_set([12, 12, 12], [[-1, 1, 0, 0], [1, -1, 1, 0]], name="i<=j<=i+k"),
+    st.affine_set([9, 11, 13], [[-1, -1, -1, 15]], name="i+j+k<=15"),
+    st.affine_set([14, 14, 14], [[-1, 1, 0, 0], [0, -1, 1, 0], [1, 0, -1, 4]], name="i<=j<=k<=i+4"),
+    st.affine_set([10, 12, 9], [[1, 1, -1, 0], [-1, 0, 1, 3], [0, -1, 0, 8]], name="k<=i+j,k>=i-3,j<=8"),
+    st.affine_set([8, 8, 8], [[2, -1, 0, 0], [0, 1, -1, 2], [-3, 0, 1, 6]], name="j<=2i,k<=j+2,k>=3i-6"),
+    st.affine_set([6, 6, 6], [[1, -1, 0, -10]], name="empty_by_rows_3d"),
+]
+
+
+@pytest.mark.parametrize("desc", GENERIC_CASES, ids=lambda d: f"{d.name}{d.dims}")
+def test_fitted_maps_match_enumeration(desc):
+    """Sets that are none of the recognised classes: the map fitted to the library's own slab counts
+    equals the oracle's enumeration at every point, in both directions."""
+    s = dastac.Structure(desc)
+    table = oracle.rank_table(desc)
+    points = oracle.unrank_table(desc)
+    assert s.nnz == oracle.count(desc) == s.slots
+    if s.nnz:
+        assert s.kind == dastac.KIND_GENERIC
+    for idx in np.ndindex(*desc.dims):
+        if table[idx] >= 0:
+            assert dastac.rank(s, idx) == table[idx]
+        else:
+            with pytest.raises(dastac.DastacError):
+                dastac.rank(s, idx)
+    for p, pt in enumerate(points):
+        assert dastac.unrank(s, p) == tuple(int(v) for v in pt)
+
+
+def test_fitted_maps_on_random_affine_sets():
+    rng = np.random.default_rng(11)
+    made = 0
+    for trial in range(60):
+        rank = int(rng.integers(2, 4))
+        dims = [int(v) for v in rng.integers(3, 11, rank)]
+        cmps = []
+        for _ in range(int(rng.integers(1, 4))):
+            a = [int(v) for v in rng.integers(-2, 3, rank)]
+            a[-1] = int(rng.integers(-1, 2))
+            if rank == 3:
+                a[1] = int(rng.integers(-1, 2))
+            cmps.append(a + [int(rng.integers(-4, 12))])
+        desc = st.affine_set(dims, cmps, name=f"random{trial}")
+        try:
+            s = dastac.Structure(desc)
+        except dastac.DastacError as e:
+            assert e.status == 2
+            continue
+        made += 1
+        points = oracle.unrank_table(desc)
+        assert s.nnz == len(points)
+        for p, pt in enumerate(points):
+            assert dastac.rank(s, [int(v) for v in pt]) == p
+            assert dastac.unrank(s, p) == tuple(int(v) for v in pt)
+    assert made >= 40
+
+
+def test_piecewise_fusion_on_the_printed_triangle_example():
+    """Section 4, "Piecewise Polynomial Simplification": counting the lower triangle gives the piece
+    j > 0 with i/2 + i^2/2 + j and the piece j = 0 with i/2 + i^2/2; the second agrees with the first on
+    its own domain and is fused away.  The polynomials are the golden file's entries."""
+    golden = {}
+    for line in open(os.path.join(ROOT, "tests", "golden", "printed_polynomials.txt")):
+        if line.strip() and not line.startswith("#"):
+            name, _, _, _, expr = [f.strip() for f in line.split("|")]
+            golden[name] = expr
+    assert golden["lower_triangle"] == "H * i + H * i**2 + j" and golden["lower_triangle_piece_j0"] == "H * i + H * i**2"
+    P = [(1, (1, 0)), (1, (2, 0)), (2, (0, 1))]     # (i + i^2 + 2 j) / 2
+    Pj0 = [(1, (1, 0)), (1, (2, 0))]                # (i + i^2) / 2
+    N = 37
+    base = st.lower_triangle(N)
+
+    def piece(extra_row, is_eq):
+        rows = np.vstack([base.rows, np.array([extra_row], dtype=np.int64)])
+        return st.Descriptor([N, N], [N], rows, np.append(base.is_eq, np.uint8(is_eq)))
+
+    D, Dj0 = piece([0, 1, 0, -1], 0), piece([0, 1, 0, 0], 1)      # j >= 1 ; j == 0
+    assert dastac.piecewise_fuse([(D, P, 2), (Dj0, Pj0, 2)]) == [0, 0]
+    assert dastac.piecewise_fuse([(Dj0, Pj0, 2), (D, P, 2)]) == [1, 1]   # whichever comes first, P survives
+    # the fused polynomial is the oracle's position on the whole triangle
+    table = oracle.rank_table(base)
+    for i in range(N):
+        for j in range(i + 1):
+            assert (i + i * i + 2 * j) // 2 == table[i, j]
+    # a piece that does not agree stays: i/2 + i^2/2 + 1 on j = 0
+    assert dastac.piecewise_fuse([(D, P, 2), (Dj0, Pj0 + [(2, (0, 0))], 2)]) == [0, 1]
+    # equality between two variables: on the diagonal j = i the polynomial j^2 equals i*j
+    diag = piece([1, -1, 0, 0], 1)
+    assert dastac.piecewise_fuse([(D, [(1, (1, 1))], 1), (diag, [(1, (0, 2))], 1)]) == [0, 0]
+    # no symbolic argument, decided on the integer points: i (i - 1) (i - 2) vanishes on 0 <= i <= 2
+    small = st.Descriptor([3], [3], np.zeros((0, 3), np.int64), np.zeros(0, np.uint8))
+    cubic = [(1, (3,)), (-3, (2,)), (2, (1,))]
+    assert dastac.piecewise_fuse([(small, cubic, 1), (small, [], 1)]) == [0, 0]
+    big = st.Descriptor([4], [4], np.zeros((0, 3), np.int64), np.zeros(0, np.uint8))
+    assert dastac.piecewise_fuse([(big, cubic, 1), (big, [], 1)]) == [0, 1]
+
+
+def test_rule_summands_share_buffers_of_equal_regions():
+    N, s = 50, 7
+    rule = dastac.Rule([st.offset_band(N, 0, 0), st.offset_band(N, s, s), st.offset_band(N, -s, -s), st.offset_band(N, s, s)])
+    assert (rule.n_summands, rule.n_buffers, rule.buffer) == (4, 3, [0, 1, 2, 1])
+    assert [v.nnz for v in rule.summands] == [N, N - s, N - s, N - s]
+    # summands must live in the same box
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.Rule([st.offset_band(N, 0, 0), st.offset_band(N + 1, 1, 1)])
+    assert e.value.status == 4
+    with pytest.raises(dastac.DastacError):
+        dastac.Rule([])
