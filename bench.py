@@ -82,6 +82,8 @@ def accounting(z):
         # useful flops by the paper's convention (two multiplies and an add per element and rank column);
         # the factored evaluation issues one multiply-add per element and rank column
         "mttkrp": dict(flops=3 * tet(n4) * R, exec_flops=2 * tet(n4) * R, bytes=4 * (tet(n4) + 3 * n4 * R), bound="alu"),
+        # widened row: the same rule through the opt-in split-precision (TF32 hi/lo) tensor-core entry point: HBM-bound
+        "mttkrp_tc": dict(flops=3 * tet(n4) * R, bytes=4 * (tet(n4) + 3 * n4 * R), bound="hbm"),
         "trimm_bf16": dict(flops=2 * tri(N5) * N5, bytes=2 * tri(N5) + 2 * N5 * N5 + 4 * N5 * N5, bound="tensor"),
         "pack_bf16": dict(flops=0, bytes=2 * (2 * tri(N5)), bound="hbm"),          # read the set, write it
         "unpack_bf16": dict(flops=0, bytes=2 * (tri(N5) + N5 * N5), bound="hbm"),  # read packed, write box
@@ -97,7 +99,7 @@ def accounting(z):
     return acc
 
 
-ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
+ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "mttkrp_tc", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
          "moment2_bf16", "moment3_bf16", "thp_ut", "symv"]
 # the kernels of the five configurations; the others are widened rows and never the roofline's kernel
 CONFIG_KERNELS = ("trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv")
@@ -156,6 +158,12 @@ def generate_host(z, pin, only=None):
         synth.tetrahedron_stream(3, 0, n4, out=a4)
         h["mttkrp"] = dict(desc=st.tetrahedron(n4), A=host(a4),
                            ins=[host(synth.dense(3, 1, (n4, R))), host(synth.dense(3, 2, (n4, R)))], out=(n4, R))
+    if want("mttkrp_tc"):
+        n4, R = z["n4"], z["R"]
+        a4 = np.zeros(cap(tet(n4), 4), np.float32)
+        synth.tetrahedron_stream(3, 0, n4, out=a4)
+        h["mttkrp_tc"] = dict(desc=st.tetrahedron(n4), A=host(a4),
+                              ins=[host(synth.dense(3, 1, (n4, R))), host(synth.dense(3, 2, (n4, R)))], out=(n4, R))
     if want("trimm_bf16"):
         N5 = z["N5"]
         sc = N5 ** -0.5
@@ -191,7 +199,7 @@ def generate_host(z, pin, only=None):
     return h
 
 
-EXPR = {"trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
+EXPR = {"mttkrp_tc": "ijk,jr,kr->ir", "trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
         "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
         "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij", "moment3_bf16": "xi,xj,xk->ijk", "thp_ut": "ijk,ijk->ijk"}
 
@@ -322,6 +330,8 @@ def run_gpu(args):
             dastac.pack(structs["trimm_bf16"], d["A"], d["out"])
         elif name == "unpack_bf16":
             dastac.unpack(structs["trimm_bf16"], d["A"], d["out"])
+        elif name == "mttkrp_tc":
+            dastac.mttkrp_split_tf32(structs[name], d["A"], d["ins"][0], d["ins"][1], d["out"], err_word=err_word)
         else:
             dastac.contract(EXPR[name], structs[name], d["A"], d["ins"], d["out"], workspace=d["ws"],
                             err_word=err_word, batch=d["batch"], out_structure=d.get("out_s"))
@@ -440,7 +450,7 @@ def run_gpu(args):
         hd = {}
         h2d = d2h = 0
         for name, hw in host.items():
-            if name not in order:
+            if name not in order or name == "mttkrp_tc":   # a device-only entry point
                 continue
             out_h = torch.empty(hw["out"], dtype=torch.float32).pin_memory()
             n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1),

@@ -280,6 +280,26 @@ dastac_status dastac_trimm_bf16_noalloc(const dastac_structure* s, const void* A
                                         int32_t accumulate, int32_t* err_word, void* stream);
 
 /*
+ * Split-precision tensor-core form of the tetrahedral MTTKRP (opt-in; dastac_contract keeps the
+ * plain fp32 multiply-add kernel).  The same rule M(i,r) = sum_{i<=j<=k} T(i,j,k) B(j,r) C(k,r)
+ * (Table 1 "MTTKRP" over the hyper-triangular domain of Section 1) with the product T_i C of
+ * every slab evaluated on the tensor cores in TF32: each fp32 value is split into a high and a
+ * low part and the three products hi*hi, hi*lo, lo*hi are accumulated in fp32, which keeps the
+ * error per product near 2^-21 (a single TF32 pass would be 2^-11); the multiplication by B and
+ * the sum over j are fp32.  Results agree with dastac_contract's within the same 1e-5 bound.
+ *   s         tetrahedron, n <= 512 (the factor C is kept in shared memory as hi / lo tiles);
+ *             anything else returns DASTAC_ERR_UNSUPPORTED_EXPR
+ *   T         device, packed fp32 tensor of s, 16-byte aligned
+ *   B, C      device, n x R fp32, row pitches ldb, ldc elements; R <= 32
+ *   M         device, n x R fp32, row pitch ldm; accumulate as for dastac_contract
+ *   err_word  optional device int32, set when a bounded wait inside the kernel expires
+ * Needs no workspace.
+ */
+dastac_status dastac_mttkrp_split_tf32(const dastac_structure* s, const float* T, const float* B, int64_t ldb,
+                                       const float* C, int64_t ldc, float* M, int64_t ldm, int64_t R,
+                                       int32_t accumulate, int32_t* err_word, void* stream);
+
+/*
  * A structured operand given as several summands (Section 4: the method works on the individual
  * summands of a rule; every summand's region has its own compressed buffer, and a summand whose
  * region equals an earlier one reuses that buffer instead of getting a second copy).  Examples:

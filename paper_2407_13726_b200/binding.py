@@ -29,7 +29,7 @@ EXPORTS = [
     "dastac_contract", "dastac_status_string", "dastac_launch_count", "dastac_trimm_bf16_noalloc",
     "dastac_device_error", "dastac_selftest_wait_expiry", "dastac_piecewise_fuse",
     "dastac_rule_create", "dastac_rule_destroy", "dastac_rule_size", "dastac_rule_summand", "dastac_rule_pack",
-    "dastac_rule_contract_workspace", "dastac_rule_contract",
+    "dastac_rule_contract_workspace", "dastac_rule_contract", "dastac_mttkrp_split_tf32",
 ]
 NOALLOC_MAX_N = 2048
 
@@ -83,6 +83,7 @@ _lib.dastac_launch_count.restype = _i64
 _lib.dastac_device_error.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
 _lib.dastac_selftest_wait_expiry.argtypes = [_i64, _vp]
 _lib.dastac_piecewise_fuse.argtypes = [_vp, _i32, _vp]
+_lib.dastac_mttkrp_split_tf32.argtypes = [_vp, _vp, _vp, _i64, _vp, _i64, _vp, _i64, _i64, _i32, _vp, _vp]
 _lib.dastac_rule_create.argtypes = [_vp, _i32, ctypes.POINTER(_vp)]
 _lib.dastac_rule_destroy.argtypes = [_vp]
 _lib.dastac_rule_destroy.restype = None
@@ -424,6 +425,20 @@ class Rule:
                                          None if err_word is None else err_word.data_ptr(), _stream()),
                "dastac_rule_contract")
         return out
+
+
+def mttkrp_split_tf32(s: Structure, packed: torch.Tensor, B: torch.Tensor, C: torch.Tensor, out: torch.Tensor,
+                      accumulate: bool = False, err_word: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The tetrahedral MTTKRP through the split-precision tensor-core entry point (see ``dastac.h``)."""
+    assert packed.is_cuda and B.is_cuda and C.is_cuda and out.is_cuda
+    assert packed.dtype == B.dtype == C.dtype == out.dtype == torch.float32
+    assert B.dim() == 2 and C.dim() == 2 and out.dim() == 2 and B.shape[1] == C.shape[1] == out.shape[1]
+    assert (B.shape[1] <= 1 or (B.stride(1) == 1 and C.stride(1) == 1 and out.stride(1) == 1))
+    _check(_lib.dastac_mttkrp_split_tf32(s._h, packed.data_ptr(), B.data_ptr(), B.stride(0), C.data_ptr(), C.stride(0),
+                                         out.data_ptr(), out.stride(0), B.shape[1], int(accumulate),
+                                         None if err_word is None else err_word.data_ptr(), _stream()),
+           "dastac_mttkrp_split_tf32")
+    return out
 
 
 def trimm_bf16_noalloc(s: Structure, packed: torch.Tensor, B: torch.Tensor, out: torch.Tensor,

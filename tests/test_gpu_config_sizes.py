@@ -122,6 +122,26 @@ def test_config4_mttkrp_n512_r32():
     assert rel_err(got[sel], ref, ref_abs) <= TOL_F32
 
 
+def test_config4_mttkrp_split_precision_tensor_core_form():
+    """The opt-in TF32 hi/lo form at the configuration's size, same sampled slabs, same bound."""
+    n, R = 512, 32
+    desc = st.tetrahedron(n)
+    s = dastac.Structure(desc)
+    B = synth.dense(3, 1, (n, R))
+    C = synth.dense(3, 2, (n, R))
+    packed = _packed(s, lambda h: synth.tetrahedron_stream(3, 0, n, out=h))
+    out = torch.full((n, R), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dastac.mttkrp_split_tf32(s, packed, dev(B), dev(C), out, err_word=err)
+    assert int(err.item()) == 0
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    sel = _rows(n, 20, extra=(1, 31, 32, 33, 127, 128, 129, 383, 384, 479, 480, 510))
+    Ts = np.stack([synth.linear_slice(3, 0, int(i) * n * n, n * n).reshape(n, n) for i in sel])
+    ref, ref_abs = oracle.mttkrp(desc, Ts, B, C, sel=sel)
+    assert rel_err(got[sel], ref, ref_abs) <= TOL_F32
+
+
 @pytest.mark.parametrize("n,R", [(700, 32), (1100, 24), (1500, 32)])
 def test_mttkrp_beyond_config4(n, R):
     """Sizes at which the factor matrix leaves room for fewer warps per block (n = 1100) or no longer

@@ -1112,3 +1112,47 @@ def test_rule_with_several_summands_in_one_call(name):
         r, ra = oracle.matmat(d, A, B)
         refC, refC_abs = refC + r, refC_abs + ra
     assert rel_err(C.cpu().numpy(), refC, refC_abs) <= TOL_F32
+
+
+@pytest.mark.parametrize("n,R", [(1, 1), (2, 5), (7, 32), (31, 32), (32, 16), (33, 32), (64, 32), (65, 8), (127, 32),
+                                 (128, 32), (129, 32), (130, 7), (200, 32), (257, 24), (300, 32)])
+def test_mttkrp_split_precision_tensor_core_form(n, R):
+    """The opt-in TF32 hi/lo form of the tetrahedral MTTKRP against the oracle, at the fp32 kernels' bound."""
+    desc = st.tetrahedron(n)
+    s = dastac.Structure(desc)
+    T = synth.dense(3, 0, (n, n, n))
+    B = synth.dense(3, 1, (n, R))
+    C = synth.dense(3, 2, (n, R))
+    ref, ref_abs = oracle.mttkrp(desc, T, B, C)
+    packed = packed_dev(s, synth.tetrahedron_stream(3, 0, n))
+    out = torch.full((n, R), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dastac.mttkrp_split_tf32(s, packed, dev(B), dev(C), out, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    M0 = synth.dense(3, 3, (n, R))
+    out2 = dev(M0)
+    dastac.mttkrp_split_tf32(s, packed, dev(B), dev(C), out2, accumulate=True, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out2.cpu().numpy(), ref + M0, ref_abs + np.abs(M0)) <= TOL_F32
+    # padded leading dimensions
+    Bp = torch.zeros((n, R + 3), device="cuda")[:, :R]
+    Bp.copy_(dev(B))
+    Cp = torch.zeros((n, R + 1), device="cuda")[:, :R]
+    Cp.copy_(dev(C))
+    outp = torch.full((n, R + 5), float("nan"), device="cuda")[:, :R]
+    dastac.mttkrp_split_tf32(s, packed, Bp, Cp, outp, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(outp.cpu().numpy(), ref, ref_abs) <= TOL_F32
+
+
+def test_mttkrp_split_precision_refusals():
+    big = dastac.Structure(st.tetrahedron(513))
+    z = torch.zeros((513, 4), device="cuda")
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.mttkrp_split_tf32(big, big.empty_packed(), z, z, torch.zeros((513, 4), device="cuda"))
+    assert e.value.status == 3
+    tri = dastac.Structure(st.upper_triangle(16))
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.mttkrp_split_tf32(tri, tri.empty_packed(), z[:16], z[:16], torch.zeros((16, 4), device="cuda"))
+    assert e.value.status == 3
