@@ -4,7 +4,7 @@
 // Section 1), factored as in mttkrp.cu: for a slab i, U = T_i C is a triangular matrix times the
 // tall matrix C, and M(i,:) = sum_j B(j,:) o U(j,:).  Here U is computed on the tensor cores in
 // TF32 with every fp32 operand split into a high and a low part (hi = the value with its low 13
-// mantissa bits cleared, lo = value - hi, exact in fp32, cleared the same way):
+// mantissa bits cleared, lo = value - hi, exact in fp32, of which the tensor core reads the upper 19 bits):
 //     T C  ~  Thi Chi + Thi Clo + Tlo Chi        (the dropped Tlo Clo is 2^-22 relative)
 // accumulated in fp32 in tensor memory; the error per product is about 2^-21, far inside the 1e-5
 // bound of the fp32 kernels, which a single TF32 pass (2^-11) would break.
@@ -35,9 +35,11 @@ constexpr int kTcBlockK = 32;            // k per K block: one 128-byte swizzle 
 constexpr int kTcTileBytes = kTcRows * 128;          // 16 KiB: a 128 x 32 fp32 tile
 constexpr int kTcStageBytes = 2 * kTcTileBytes;      // hi + lo
 constexpr int kTcMaxN = 512;
-constexpr int kTcProducerWarps = 8;
+constexpr int kTcProducerWarps = 8;                  // warps that fill one stage
+constexpr int kTcProducerGroups = 2;                 // groups of such warps, taking the items in turn
 constexpr int kTcWarpMma = 4;                        // warps 0-3 epilogue, 4 MMA, 5.. producers
-constexpr int kTcThreads = (5 + kTcProducerWarps) * 32;
+constexpr int kTcThreads = (5 + kTcProducerWarps * kTcProducerGroups) * 32;
+constexpr int kTcAhead = 2;                         // items whose loads are in flight per producer thread
 constexpr int kTcTmemCols = 128;                     // two accumulators of 64 columns
 constexpr long long kTcWaitBudget = 2000000000LL;
 constexpr int32_t kErrWordMttkrpTc = 0x4d43;         // "MC"
@@ -90,7 +92,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // hi / lo parts of an fp32 value as TF32 operands
 __device__ __forceinline__ void tc_split(float v, float& hi, float& lo) {
     hi = __uint_as_float(__float_as_uint(v) & 0xffffe000u);
-    lo = __uint_as_float(__float_as_uint(v - hi) & 0xffffe000u);
+    lo = v - hi;  // exact; the tensor core reads its upper 19 bits
 }
 
 struct TcParams {
@@ -147,6 +149,30 @@ __device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile 
     }
 }
 
+// Writes a thread's 16 values of k (element k0 + x is v[x + SH]) as hi / lo parts into its row of the
+// two swizzled tiles; outside j <= k < n (or for a fibre beyond n) zeros are written.
+template <int SH>
+__device__ __forceinline__ void tc_store_item(const float (&v)[20], uint8_t* row_hi, int h, int m, int k0, int j, int n,
+                                              bool live, bool interior) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        float hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int x = 4 * c + e;
+            float val = v[x + SH];
+            if (!interior) {
+                const int k = k0 + x;
+                if (!(live && k >= j && k < n)) val = 0.f;
+            }
+            tc_split(val, hi[e], lo[e]);
+        }
+        const uint32_t off = (uint32_t)(((h * 4 + c) ^ (m & 7)) << 4);
+        *reinterpret_cast<float4*>(row_hi + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<float4*>(row_hi + kTcTileBytes + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+    }
+}
+
 __global__ void __launch_bounds__(kTcThreads, 1) mttkrp_tc_kernel(const TcParams p) {
     extern __shared__ uint8_t tc_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_raw) + 1023) & ~(uintptr_t)1023);
@@ -181,17 +207,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) mttkrp_tc_kernel(const TcParams
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // C(:, 0..31) as hi / lo K-major tiles: element (k, r) -> block k / 32, rows r (hi) and 32 + r (lo)
-    for (int idx = threadIdx.x; idx < p.n_kb * 32 * 32; idx += blockDim.x) {
-        const int k = idx >> 5, r = idx & 31;
-        float c = 0.f;
-        if (k < p.n && r < p.R) c = __ldg(p.C + (int64_t)k * p.ldc + r);
-        float hi, lo;
-        tc_split(c, hi, lo);
-        const int kk = k & 31;
-        uint8_t* blk = Cb + (size_t)(k >> 5) * 8192;
-        const uint32_t in_row = (uint32_t)((((kk >> 2) ^ (r & 7)) << 4) + (kk & 3) * 4);
-        *reinterpret_cast<float*>(blk + (r >> 3) * 1024 + (r & 7) * 128 + in_row) = hi;
-        *reinterpret_cast<float*>(blk + 4096 + (r >> 3) * 1024 + (r & 7) * 128 + in_row) = lo;
+    for (int base = threadIdx.x; base < p.n_kb * 32 * 32; base += 8 * blockDim.x) {
+        float cv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {  // eight independent loads in flight per thread
+            const int idx = base + u * blockDim.x, k = idx >> 5, r = idx & 31;
+            cv[u] = (idx < p.n_kb * 32 * 32 && k < p.n && r < p.R) ? __ldg(p.C + (int64_t)k * p.ldc + r) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * blockDim.x, k = idx >> 5, r = idx & 31;
+            if (idx >= p.n_kb * 32 * 32) break;
+            float hi, lo;
+            tc_split(cv[u], hi, lo);
+            const int kk = k & 31;
+            uint8_t* blk = Cb + (size_t)(k >> 5) * 8192;
+            const uint32_t in_row = (uint32_t)((((kk >> 2) ^ (r & 7)) << 4) + (kk & 3) * 4);
+            *reinterpret_cast<float*>(blk + (r >> 3) * 1024 + (r & 7) * 128 + in_row) = hi;
+            *reinterpret_cast<float*>(blk + 4096 + (r >> 3) * 1024 + (r & 7) * 128 + in_row) = lo;
+        }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -206,63 +240,122 @@ __global__ void __launch_bounds__(kTcThreads, 1) mttkrp_tc_kernel(const TcParams
 
     if (warp > kTcWarpMma) {
         // ---- producers: thread = (row m, half h) of the 128 x 32 tile ----
-        const int pt = threadIdx.x - (kTcWarpMma + 1) * 32;
-        const int m = pt >> 1, h = pt & 1;
-        uint32_t it = 0;
+        // The loads of an item (tile, K block) are issued kTcAhead items before its tile is written,
+        // so that several K blocks of packed data are in flight per thread.
+        // Warp w owns the rows m = w + 8 r (r = 0..15): fibres eight apart share their misalignment
+        // (the row base advances by n-j-1 per fibre, eight steps sum to a multiple of 4), so the
+        // realignment shift is uniform in the warp and is resolved by one switch, not per element.
+        // Two groups of eight warps take the items in turn, so that the dependent chain of one item
+        // (wait, realign, split, store, fence, arrive) overlaps with the other group's.
+        const int pw = (warp - (kTcWarpMma + 1)) % kTcProducerWarps, grp = (warp - (kTcWarpMma + 1)) / kTcProducerWarps;
+        const int m = pw + 8 * (lane >> 1), h = lane & 1;
+        const float4* Tq = reinterpret_cast<const float4*>(p.T);
+        struct Item {
+            int j, k0, s;       // fibre of this thread, first of its 16 values of k, misalignment
+            bool valid, live;   // an item exists; the fibre exists
+            bool interior;      // every (row, k) of the tile's K block lies inside the set
+        };
+        // iterator over this CTA's items
+        int round = -1, kb = 0, kb_end = 0, cur_j = 0, cur_s = 0, cur_j0 = 0;
+        bool cur_live = false;
+        int64_t cur_rb = 0;
+        auto next_item = [&](Item& itx, int64_t& q0) {
+            while (kb >= kb_end) {  // next tile
+                ++round;
+                if (round >= rounds) {
+                    itx.valid = false;
+                    return;
+                }
+                const int q = tile_of(round);
+                if (q >= p.tiles) continue;
+                int i, j0;
+                tc_decode(q, i, j0);
+                cur_j = j0 + m;
+                cur_j0 = j0;
+                cur_live = cur_j < n;
+                cur_rb = cur_live ? p.tetn - tet((int64_t)(n - i)) + tri((int64_t)(n - i)) - tri((int64_t)(n - cur_j)) - cur_j : 0;
+                cur_s = (int)(cur_rb & 3);
+                kb = j0 >> 5;
+                kb_end = p.n_kb;
+            }
+            itx.valid = true;
+            itx.live = cur_live;
+            itx.j = cur_j;
+            itx.s = cur_s;
+            itx.k0 = kb * 32 + h * 16;
+            itx.interior = kb * 32 >= cur_j0 + kTcRows - 1 && kb * 32 + 31 < n && cur_j0 + kTcRows - 1 < n;
+            q0 = (cur_rb + itx.k0) >> 2;  // memory quad that holds element k0
+            ++kb;
+        };
+        auto load_item = [&](const Item& itx, int64_t q0, float (&v)[20]) {
+#pragma unroll
+            for (int e = 0; e < 20; ++e) v[e] = 0.f;
+            if (itx.valid && itx.live && itx.k0 + 15 >= itx.j && itx.k0 < n) {
+#pragma unroll
+                for (int c = 0; c < 5; ++c) {
+                    // quad c holds k = k0 - s + 4c .. +3: loaded when it holds an element of the row
+                    const int klo = itx.k0 - itx.s + 4 * c;
+                    if (klo + 3 >= itx.j && klo < n && q0 + c < p.cap_quads) {
+                        const float4 t4 = __ldg(Tq + q0 + c);
+                        v[4 * c] = t4.x, v[4 * c + 1] = t4.y, v[4 * c + 2] = t4.z, v[4 * c + 3] = t4.w;
+                    }
+                }
+            }
+        };
+        auto next_own_item = [&](Item& itx, int64_t& q0) {  // this group's next item: every kTcProducerGroups-th
+            next_item(itx, q0);
+#pragma unroll
+            for (int g = 1; g < kTcProducerGroups; ++g) {
+                Item skip;
+                int64_t qs = 0;
+                next_item(skip, qs);
+            }
+        };
+        Item items[kTcAhead];
+        float vals[kTcAhead][20];
+        for (int g = 0; g < grp; ++g) {  // items 0 .. grp-1 belong to the groups before this one
+            Item skip;
+            int64_t qs = 0;
+            next_item(skip, qs);
+        }
+#pragma unroll
+        for (int d = 0; d < kTcAhead; ++d) {
+            int64_t q0 = 0;
+            next_own_item(items[d], q0);
+            load_item(items[d], q0, vals[d]);
+        }
+        uint32_t it = (uint32_t)grp;
         bool ok = true;
-        for (int round = 0; round < rounds && ok; ++round) {
-            const int q = tile_of(round);
-            if (q >= p.tiles) continue;
-            int i, j0;
-            tc_decode(q, i, j0);
-            const int j = j0 + m;
-            const bool row_live = j < n;
-            // T(i, j, k) sits at rb + k; s = misalignment of the row against the 16-byte grid
-            const int64_t rb = row_live ? p.tetn - tet((int64_t)(n - i)) + tri((int64_t)(n - i)) - tri((int64_t)(n - j)) - j : 0;
-            const int s = (int)(rb & 3);
-            const float4* Tq = reinterpret_cast<const float4*>(p.T);
-            for (int kb = j0 >> 5; kb < p.n_kb && ok; ++kb, ++it) {
+        while (ok) {
+#pragma unroll
+            for (int d = 0; d < kTcAhead; ++d) {
+                if (!ok) break;
+                const Item itx = items[d];
+                if (!itx.valid) {
+                    ok = false;
+                    break;
+                }
                 const int st = it % S;
                 if (it >= (uint32_t)S && !tc_wait(empty(st), ((it / S) & 1) ^ 1, abort_flag, p.err_word)) {
                     ok = false;
                     break;
                 }
-                const int k0 = kb * 32 + h * 16;  // this thread's 16 values of k
-                float v[20];
-#pragma unroll
-                for (int e = 0; e < 20; ++e) v[e] = 0.f;
-                if (row_live && k0 + 15 >= j && k0 < n) {
-                    const int64_t q0 = (rb + k0) >> 2;  // memory quad that holds element k0
-#pragma unroll
-                    for (int c = 0; c < 5; ++c) {
-                        // quad c holds k = k0 - s + 4c .. +3: loaded when it holds an element of the row
-                        const int klo = k0 - s + 4 * c;
-                        if (klo + 3 >= j && klo < n && q0 + c < p.cap_quads) {
-                            const float4 t4 = __ldg(Tq + q0 + c);
-                            v[4 * c] = t4.x, v[4 * c + 1] = t4.y, v[4 * c + 2] = t4.z, v[4 * c + 3] = t4.w;
-                        }
-                    }
-                }
-                uint8_t* hi_tile = stage0 + (size_t)st * kTcStageBytes;
-                uint8_t* row_hi = hi_tile + (m >> 3) * 1024 + (m & 7) * 128;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    float hi[4], lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int x = 4 * c + e;  // element k0 + x is v[x + s]
-                        float val = s == 0 ? v[x] : s == 1 ? v[x + 1] : s == 2 ? v[x + 2] : v[x + 3];
-                        const int k = k0 + x;
-                        if (!(row_live && k >= j && k < n)) val = 0.f;
-                        tc_split(val, hi[e], lo[e]);
-                    }
-                    const uint32_t off = (uint32_t)(((h * 4 + c) ^ (m & 7)) << 4);
-                    *reinterpret_cast<float4*>(row_hi + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<float4*>(row_hi + kTcTileBytes + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                uint8_t* row_hi = stage0 + (size_t)st * kTcStageBytes + (m >> 3) * 1024 + (m & 7) * 128;
+                // lane 0 holds the warp's first row: if that fibre does not exist none of the warp's does
+                const int s_warp = __shfl_sync(0xffffffffu, itx.s, 0);
+                switch (s_warp) {
+                    case 0: tc_store_item<0>(vals[d], row_hi, h, m, itx.k0, itx.j, n, itx.live, itx.interior); break;
+                    case 1: tc_store_item<1>(vals[d], row_hi, h, m, itx.k0, itx.j, n, itx.live, itx.interior); break;
+                    case 2: tc_store_item<2>(vals[d], row_hi, h, m, itx.k0, itx.j, n, itx.live, itx.interior); break;
+                    default: tc_store_item<3>(vals[d], row_hi, h, m, itx.k0, itx.j, n, itx.live, itx.interior); break;
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) tc_mbar_arrive(full(st));
+                it += kTcProducerGroups;
+                int64_t q0 = 0;
+                next_own_item(items[d], q0);
+                load_item(items[d], q0, vals[d]);
             }
         }
     }
