@@ -569,8 +569,9 @@ TRAFFIC = {
     "bandmm_exact": int(42.106880e6 + 1.919488e6),
     "thp_ut": int(134.386688e6 + 39.105536e6),
     "moment2_bf16": int(1.410541e9 + 22.173440e6),   # full size, DRAM counters only (one pass)
-    "pack_bf16": int(67.670528e6 + 18.990336e6),
-    "unpack_bf16": int(67.159552e6 + 74.384896e6),
+    "pack_bf16": int(67.685888e6 + 18.702336e6),
+    "unpack_bf16": int(67.160576e6 + 74.180864e6),
+    "mttkrp_tc": int(90.289408e6 + 3.652608e6),
 }
 
 
