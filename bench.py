@@ -78,6 +78,9 @@ def accounting(z):
         "bandmm": dict(flops=2 * nnz2 * C2, exec_flops=2 * nnz2 * C2, bytes=4 * ((2 * w + 1) * N2 + 2 * N2 * C2), bound="alu"),
         # widened row: the same band product over the exact (un-padded) layout
         "bandmm_exact": dict(flops=2 * nnz2 * C2, exec_flops=2 * nnz2 * C2, bytes=4 * (nnz2 + 2 * N2 * C2), bound="alu"),
+        # widened row: the padded-diagonal band product through the opt-in split-precision (TF32 hi/lo) tensor-core
+        # entry point: HBM-bound
+        "bandmm_tc": dict(flops=2 * nnz2 * C2, bytes=4 * ((2 * w + 1) * N2 + 2 * N2 * C2), bound="hbm"),
         "symv": dict(flops=2 * N3 * N3, bytes=4 * (tri(N3) + 2 * N3), bound="hbm"),
         # useful flops by the paper's convention (two multiplies and an add per element and rank column);
         # the factored evaluation issues one multiply-add per element and rank column
@@ -99,7 +102,7 @@ def accounting(z):
     return acc
 
 
-ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "mttkrp", "mttkrp_tc", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
+ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "bandmm_tc", "mttkrp", "mttkrp_tc", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
          "moment2_bf16", "moment3_bf16", "thp_ut", "symv"]
 # the kernels of the five configurations; the others are widened rows and never the roofline's kernel
 CONFIG_KERNELS = ("trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv")
@@ -139,6 +142,10 @@ def generate_host(z, pin, only=None):
         N2, w, C2 = z["N2"], z["w"], z["C2"]
         h["bandmm"] = dict(desc=st.band(N2, w), A=host(synth.band_diagonals_stream(1, 0, N2, w).reshape(-1)),
                            ins=[host(synth.dense(1, 1, (N2, C2)))], out=(N2, C2))
+    if want("bandmm_tc"):
+        N2, w, C2 = z["N2"], z["w"], z["C2"]
+        h["bandmm_tc"] = dict(desc=st.band(N2, w), A=host(synth.band_diagonals_stream(1, 0, N2, w).reshape(-1)),
+                              ins=[host(synth.dense(1, 1, (N2, C2)))], out=(N2, C2))
     if want("bandmm_exact"):
         N2, w, C2 = z["N2"], z["w"], z["C2"]
         nnz2 = (2 * w + 1) * N2 - w * (w + 1)
@@ -199,7 +206,7 @@ def generate_host(z, pin, only=None):
     return h
 
 
-EXPR = {"mttkrp_tc": "ijk,jr,kr->ir", "trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
+EXPR = {"mttkrp_tc": "ijk,jr,kr->ir", "bandmm_tc": "ij,jc->ic", "trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
         "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
         "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij", "moment3_bf16": "xi,xj,xk->ijk", "thp_ut": "ijk,ijk->ijk"}
 
@@ -330,6 +337,8 @@ def run_gpu(args):
             dastac.pack(structs["trimm_bf16"], d["A"], d["out"])
         elif name == "unpack_bf16":
             dastac.unpack(structs["trimm_bf16"], d["A"], d["out"])
+        elif name == "bandmm_tc":
+            dastac.bandmm_split_tf32(structs[name], d["A"], d["ins"][0], d["out"], err_word=err_word)
         elif name == "mttkrp_tc":
             dastac.mttkrp_split_tf32(structs[name], d["A"], d["ins"][0], d["ins"][1], d["out"], err_word=err_word)
         else:
@@ -450,7 +459,7 @@ def run_gpu(args):
         hd = {}
         h2d = d2h = 0
         for name, hw in host.items():
-            if name not in order or name == "mttkrp_tc":   # a device-only entry point
+            if name not in order or name in ("mttkrp_tc", "bandmm_tc"):   # device-only entry points
                 continue
             out_h = torch.empty(hw["out"], dtype=torch.float32).pin_memory()
             n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1),

@@ -300,6 +300,28 @@ dastac_status dastac_mttkrp_split_tf32(const dastac_structure* s, const float* T
                                        int32_t accumulate, int32_t* err_word, void* stream);
 
 /*
+ * Split-precision tensor-core form of band x dense (opt-in; dastac_contract keeps the plain fp32
+ * multiply-add kernel).  C = A B (or C += A B) for a band |i - j| <= w (Section 1, the banded
+ * motivation; Section 6.4): a tile of 128 rows of C is the dense product of the 128 x (128 + 2w)
+ * slice of A that holds its band with the B rows i0-w .. i0+127+w, taken on the tensor cores in
+ * TF32 with both operands split into a high and a low part and the three products hi*hi, hi*lo,
+ * lo*hi accumulated in fp32 (about 2^-21 per product).  Results agree with dastac_contract's
+ * within the same 1e-5 bound.  Padding slots of the diagonal layout are never read.
+ *   s         band as padded diagonals or packed exactly; anything else returns
+ *             DASTAC_ERR_UNSUPPORTED_EXPR
+ *   A         device, packed fp32 values of s (no alignment requirement)
+ *   B         device, N x ncols fp32, row pitch ldb elements (no alignment requirement)
+ *   C         device, N x ncols fp32, row pitch ldc elements; 128-bit stores when C is 16-byte
+ *             aligned and ldc is a multiple of 4, scalar stores otherwise
+ *   accumulate, stream   as for dastac_contract
+ *   err_word  optional device int32, set when a bounded wait inside the kernel expires
+ * Needs no workspace.
+ */
+dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, const float* A, const float* B, int64_t ldb,
+                                       float* C, int64_t ldc, int64_t ncols, int32_t accumulate,
+                                       int32_t* err_word, void* stream);
+
+/*
  * A structured operand given as several summands (Section 4: the method works on the individual
  * summands of a rule; every summand's region has its own compressed buffer, and a summand whose
  * region equals an earlier one reuses that buffer instead of getting a second copy).  Examples:

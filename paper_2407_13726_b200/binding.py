@@ -30,6 +30,7 @@ EXPORTS = [
     "dastac_device_error", "dastac_selftest_wait_expiry", "dastac_piecewise_fuse",
     "dastac_rule_create", "dastac_rule_destroy", "dastac_rule_size", "dastac_rule_summand", "dastac_rule_pack",
     "dastac_rule_contract_workspace", "dastac_rule_contract", "dastac_mttkrp_split_tf32",
+    "dastac_bandmm_split_tf32",
 ]
 NOALLOC_MAX_N = 2048
 
@@ -84,6 +85,7 @@ _lib.dastac_device_error.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
 _lib.dastac_selftest_wait_expiry.argtypes = [_i64, _vp]
 _lib.dastac_piecewise_fuse.argtypes = [_vp, _i32, _vp]
 _lib.dastac_mttkrp_split_tf32.argtypes = [_vp, _vp, _vp, _i64, _vp, _i64, _vp, _i64, _i64, _i32, _vp, _vp]
+_lib.dastac_bandmm_split_tf32.argtypes = [_vp, _vp, _vp, _i64, _vp, _i64, _i64, _i32, _vp, _vp]
 _lib.dastac_rule_create.argtypes = [_vp, _i32, ctypes.POINTER(_vp)]
 _lib.dastac_rule_destroy.argtypes = [_vp]
 _lib.dastac_rule_destroy.restype = None
@@ -438,6 +440,20 @@ def mttkrp_split_tf32(s: Structure, packed: torch.Tensor, B: torch.Tensor, C: to
                                          out.data_ptr(), out.stride(0), B.shape[1], int(accumulate),
                                          None if err_word is None else err_word.data_ptr(), _stream()),
            "dastac_mttkrp_split_tf32")
+    return out
+
+
+def bandmm_split_tf32(s: Structure, packed: torch.Tensor, B: torch.Tensor, out: torch.Tensor,
+                      accumulate: bool = False, err_word: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``out = A B`` (or ``+=``) for a packed band through the split-precision tensor-core entry point
+    (see ``dastac.h``)."""
+    assert packed.is_cuda and B.is_cuda and out.is_cuda and B.dim() == 2 and out.dim() == 2
+    assert packed.dtype == B.dtype == out.dtype == torch.float32
+    assert (B.shape[1] <= 1 or (B.stride(1) == 1 and out.stride(1) == 1)) and out.shape == (s.dims[0], B.shape[1])
+    _check(_lib.dastac_bandmm_split_tf32(s._h, packed.data_ptr(), B.data_ptr(), B.stride(0), out.data_ptr(),
+                                         out.stride(0), B.shape[1], int(accumulate),
+                                         None if err_word is None else err_word.data_ptr(), _stream()),
+           "dastac_bandmm_split_tf32")
     return out
 
 

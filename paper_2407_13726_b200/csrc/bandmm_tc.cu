@@ -1,0 +1,401 @@
+// Split-precision tensor-core form of band x dense (opt-in, its own entry point).
+//
+// C = A B with A banded, |i - j| <= w (Section 1, the banded motivation; Section 6.4), stored as
+// padded diagonals or packed exactly row after row; B and C dense row-major fp32.  A tile of 128
+// rows i0 .. i0+127 touches the B rows i0-w .. i0+127+w only, so the product of the tile is the
+// dense product of a 128 x (128 + 2w) slice of A (the band inside it, zeros elsewhere) with that
+// window of B.  It runs on the tensor cores in TF32 with both operands split into a high and a low
+// part (tf32_mma.cuh): A B ~ Ahi Bhi + Ahi Blo + Alo Bhi, accumulated in fp32 in tensor memory,
+// about 2^-21 per product, inside the 1e-5 bound of the fp32 kernels.
+//
+// Tile = (128 rows, 256 columns); K blocks of 32 rows of the B window.
+//   producer warps   (two groups of eight, taking the K blocks in turn, one stage each) thread n of 256 reads column n of the K block of B (32 coalesced 4-byte loads
+//                    per thread, no alignment requirement on B), splits and writes row n of the two
+//                    K-major, 128-byte-swizzled 256 x 32 tiles Bhi, Blo with 128-bit stores.  The
+//                    slice of A is zeroed and the band written into it diagonal by diagonal: for
+//                    diagonal d the 32 rows whose entry falls into this K block are consecutive in
+//                    memory in the padded layout (one coalesced load) and land on 32 different
+//                    banks of the swizzled tile.
+//   MMA thread       per K block and k-step of 8: three tcgen05.mma kind::tf32 M128 N256 K8
+//                    (Ahi Bhi, Ahi Blo, Alo Bhi) into one accumulator
+//   epilogue warps   one per lane quarter of tensor memory: tcgen05.ld, 128-bit stores to C
+//                    (read-add-write when accumulating)
+// Two stages of operands (96 KiB each), two accumulators of 256 columns (all of tensor memory).
+// K blocks that lie outside the matrix (first and last tiles) are skipped.  Every wait is bounded.
+#include "common.cuh"
+#include "tf32_mma.cuh"
+#include "waits.cuh"
+
+namespace dastac {
+namespace {
+
+constexpr int kBtRows = 128;                 // rows of C per tile
+constexpr int kBtCols = 256;                 // columns of C per tile
+constexpr int kBtATile = kBtRows * 128;      // 16 KiB: 128 x 32 fp32
+constexpr int kBtBTile = kBtCols * 128;      // 32 KiB: 256 x 32 fp32
+constexpr int kBtStageBytes = 2 * kBtATile + 2 * kBtBTile;  // Ahi, Alo, Bhi, Blo
+constexpr int kBtStages = 2;
+constexpr int kBtEpiWarps = 4, kBtWarpMma = 4, kBtProducerWarps = 8;  // warps 0-3 epilogue, 4 MMA, 5.. producers
+constexpr int kBtEpiCols = kBtCols / (kBtEpiWarps / 4);  // columns of the tile per epilogue warp
+constexpr int kBtProducerGroups = 2;         // = kBtStages: group g fills stage g
+constexpr int kBtThreads = (kBtEpiWarps + 1 + kBtProducerWarps * kBtProducerGroups) * 32;
+// diagonals of one K block per producer warp: at most ceil(min(2w + 1, 159) / 8), a template parameter
+// of the kernel (10 for 2w + 1 <= 80, else 20) so that narrow bands hold fewer values in registers
+constexpr int kBtTmemCols = 512;
+constexpr long long kBtWaitBudget = 2000000000LL;
+constexpr int32_t kErrWordBandTc = 0x4254;   // "BT"
+constexpr size_t kBtSmemBytes = (size_t)kBtStages * kBtStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+
+struct BtParams {
+    const float* A;
+    const float* B;
+    float* C;
+    int64_t N, w, ldb, ldc, ncols;
+    int32_t row_tiles, col_tiles, tiles;
+    int32_t exact;       // A packed row after row instead of padded diagonals
+    int32_t accumulate;
+    int32_t vec_c;       // C allows 128-bit accesses
+    int32_t* err_word;
+};
+
+// K blocks of a tile that intersect the matrix: window row kk of the tile is B row i0 - w + kk
+__device__ __forceinline__ void bt_k_range(const BtParams& p, int64_t i0, int& kb_lo, int& kb_hi) {
+    const int64_t row0 = i0 - p.w;
+    const int64_t rows_live = p.N - i0 < kBtRows ? p.N - i0 : kBtRows;
+    int64_t kk_end = rows_live + 2 * p.w;          // one past the last window row any live row reads
+    if (p.N - row0 < kk_end) kk_end = p.N - row0;  // ... that exists
+    kb_lo = row0 < 0 ? (int)((-row0) >> 5) : 0;
+    kb_hi = (int)((kk_end + 31) >> 5);
+}
+
+__device__ __forceinline__ bool bt_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* err_word) {
+    return tc_wait_coded(bar, parity, abort_flag, err_word, kErrWordBandTc, kBtWaitBudget);
+}
+// Barrier of the eight warps of a producer group (barrier 1 + group) that also tells every one of them whether any thread raised
+// `flag`: the warps leave their loop together, so none is left waiting at this barrier.
+template <int ID>
+__device__ __forceinline__ bool bt_bar_or(bool flag) {
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, %2, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(any)
+        : "r"((uint32_t)flag), "n"(ID), "n"(kBtProducerWarps * 32)
+        : "memory");
+    return any != 0;
+}
+__device__ __forceinline__ bool bt_producer_sync_any(bool flag, int group) {
+    return group == 0 ? bt_bar_or<1>(flag) : bt_bar_or<2>(flag);
+}
+
+template <int kBtSegs>
+__global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams p) {
+    extern __shared__ uint8_t bt_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(bt_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint64_t* const bars = reinterpret_cast<uint64_t*>(smem + (size_t)kBtStages * kBtStageBytes);
+    constexpr int S = kBtStages;
+    auto full = [&](int s) { return tc_smem(&bars[s]); };
+    auto empty = [&](int s) { return tc_smem(&bars[S + s]); };
+    auto tmem_full = [&](int a) { return tc_smem(&bars[2 * S + a]); };
+    auto tmem_empty = [&](int a) { return tc_smem(&bars[2 * S + 2 + a]); };
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(&bars[2 * S + 4]);
+    volatile int* const abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            tc_mbar_init(full(s), kBtProducerWarps);
+            tc_mbar_init(empty(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            tc_mbar_init(tmem_full(a), 1);
+            tc_mbar_init(tmem_empty(a), kBtEpiWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem(tmem_slot)),
+                     "r"((uint32_t)kBtTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int G = gridDim.x;
+    const int rounds = (p.tiles + G - 1) / G;
+    auto tile_of = [&](int round) { return round * G + (int)blockIdx.x; };
+    const int64_t N = p.N, w = p.w;
+
+    if (warp > kBtWarpMma) {
+        // ---- producers: two groups of eight warps take the items (tile, K block) in turn, group g
+        // fills stage g.  A group issues the loads of its next item right after it has published the
+        // current one, so they are in flight while the tensor core works on the other group's stage.
+        const int pw = (warp - (kBtWarpMma + 1)) % kBtProducerWarps, grp = (warp - (kBtWarpMma + 1)) / kBtProducerWarps;
+        const int t = pw * 32 + lane;  // column of the tile whose B values this thread splits
+        int round = -1, kb = -1, kb_end = 0;
+        int64_t i0 = 0, cb = 0;
+        bool valid = true;
+        auto next_item = [&]() {  // advances to the next (tile, K block) of this CTA
+            if (!valid) return;
+            ++kb;
+            while (kb >= kb_end) {
+                ++round;
+                if (round >= rounds || tile_of(round) >= p.tiles) {
+                    valid = false;
+                    return;
+                }
+                const int q = tile_of(round);
+                i0 = (int64_t)(q / p.col_tiles) * kBtRows;
+                cb = (int64_t)(q % p.col_tiles) * kBtCols;
+                bt_k_range(p, i0, kb, kb_end);
+            }
+        };
+        float bv[32], av[kBtSegs];
+        auto load_item = [&]() {
+            const int64_t j0 = i0 - w + 32 * (int64_t)kb;  // B row of the block's first window row
+            const int64_t col = cb + t;
+            const bool col_ok = col < p.ncols;
+            const float* bsrc = p.B + j0 * p.ldb + col;  // dereferenced only where the row and column exist
+            if (j0 >= 0 && j0 + 31 < N) {  // block-uniform: every row of the K block exists
+#pragma unroll
+                for (int e = 0; e < 32; ++e) bv[e] = col_ok ? __ldg(bsrc + e * p.ldb) : 0.f;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int64_t j = j0 + e;
+                    bv[e] = (col_ok && j >= 0 && j < N) ? __ldg(bsrc + e * p.ldb) : 0.f;
+                }
+            }
+            // diagonals d whose entries fall into this K block for some row of the tile:
+            // row r holds diagonal d at window row kk = r + d, so d in [32 kb - 127, 32 kb + 31]
+            const int d_lo = 32 * kb - (kBtRows - 1) > 0 ? 32 * kb - (kBtRows - 1) : 0;
+            const int d_hi = (int)(32 * (int64_t)kb + 31 < 2 * w ? 32 * (int64_t)kb + 31 : 2 * w);
+            const int64_t j = j0 + lane;  // the column of A this lane reads, whatever the diagonal
+            const bool j_ok = j >= 0 && j < N;
+#pragma unroll
+            for (int u = 0; u < kBtSegs; ++u) {
+                const int d = d_lo + pw + 8 * u;
+                if (d > d_hi) break;  // warp-uniform
+                const int r = 32 * kb - d + lane;
+                const int64_t i = i0 + r;
+                float v = 0.f;
+                if (j_ok && r >= 0 && r < kBtRows && i < N) {
+                    const int64_t off = p.exact ? band_row_start(N, w, i) - band_jlo(w, i) + j : (int64_t)d * N + i;
+                    v = __ldg(p.A + off);
+                }
+                av[u] = v;
+            }
+        };
+        for (int g = 0; g <= grp; ++g) next_item();  // group g starts at item g
+        if (valid) load_item();
+        const int st = grp;
+        uint8_t* const a_hi = smem + (size_t)st * kBtStageBytes;
+        uint8_t* const b_hi = a_hi + 2 * kBtATile;
+        uint32_t use = 0;  // items this group has written into its stage
+        while (valid) {
+            // one lane per warp waits for the stage; the group's barrier below spreads the outcome
+            bool ok = true;
+            if (use >= 1 && lane == 0) ok = bt_wait(empty(st), (use - 1) & 1, abort_flag, p.err_word);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (ok) {
+                // row t of Bhi / Blo
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    float hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) tc_split(bv[4 * c + e], hi[e], lo[e]);
+                    const uint32_t off = tc_tile_offset(t, c);
+                    *reinterpret_cast<float4*>(b_hi + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<float4*>(b_hi + kBtBTile + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                }
+                // the slice of A: zeros, then the band
+#pragma unroll
+                for (int u = 0; u < 2 * kBtATile / (16 * kBtProducerWarps * 32); ++u)
+                    *reinterpret_cast<float4*>(a_hi + (size_t)(u * kBtProducerWarps * 32 + t) * 16) =
+                        make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (bt_producer_sync_any(!ok, grp)) break;  // a wait ran out somewhere: all eight warps stop here
+            {
+                const int d_lo = 32 * kb - (kBtRows - 1) > 0 ? 32 * kb - (kBtRows - 1) : 0;
+                const int d_hi = (int)(32 * (int64_t)kb + 31 < 2 * w ? 32 * (int64_t)kb + 31 : 2 * w);
+#pragma unroll
+                for (int u = 0; u < kBtSegs; ++u) {
+                    const int d = d_lo + pw + 8 * u;
+                    if (d > d_hi) break;
+                    const int r = 32 * kb - d + lane;
+                    if (r >= 0 && r < kBtRows) {
+                        float hi, lo;
+                        tc_split(av[u], hi, lo);
+                        const uint32_t off = tc_tile_offset(r, lane >> 2) + (uint32_t)(lane & 3) * 4u;
+                        *reinterpret_cast<float*>(a_hi + off) = hi;
+                        *reinterpret_cast<float*>(a_hi + kBtATile + off) = lo;
+                    }
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) tc_mbar_arrive(full(st));
+            ++use;
+            next_item();
+            next_item();
+            if (valid) load_item();
+        }
+    }
+    else if (warp == kBtWarpMma) {
+        // ---- MMA issuer: one thread ----
+        if (lane == 0) {
+            constexpr uint32_t kIdesc = tc_idesc_mn(kBtRows, kBtCols);
+            uint32_t it = 0, tile_n = 0;
+            bool ok = true;
+            for (int round = 0; round < rounds && ok; ++round) {
+                const int q = tile_of(round);
+                if (q >= p.tiles) break;
+                const int64_t i0 = (int64_t)(q / p.col_tiles) * kBtRows;
+                int kb_lo, kb_hi;
+                bt_k_range(p, i0, kb_lo, kb_hi);
+                const int acc = tile_n & 1;
+                const uint32_t use = tile_n >> 1;  // earlier uses of this accumulator
+                if (use >= 1 && !bt_wait(tmem_empty(acc), (use - 1) & 1, abort_flag, p.err_word)) {
+                    ok = false;
+                    break;
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + acc * kBtCols;
+                for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+                    const int st = it % S;
+                    if (!bt_wait(full(st), (it / S) & 1, abort_flag, p.err_word)) {
+                        ok = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_hi = tc_smem(smem + (size_t)st * kBtStageBytes);
+                    const uint32_t a_lo = a_hi + kBtATile;
+                    const uint32_t b_hi = a_hi + 2 * kBtATile;
+                    const uint32_t b_lo = b_hi + kBtBTile;
+#pragma unroll
+                    for (int k8 = 0; k8 < 4; ++k8) {
+                        tc_mma_tf32(d_tmem, tc_desc(a_hi + k8 * 32), tc_desc(b_hi + k8 * 32), kIdesc,
+                                    (kb > kb_lo || k8 > 0) ? 1u : 0u);
+                        tc_mma_tf32(d_tmem, tc_desc(a_hi + k8 * 32), tc_desc(b_lo + k8 * 32), kIdesc, 1u);
+                        tc_mma_tf32(d_tmem, tc_desc(a_lo + k8 * 32), tc_desc(b_hi + k8 * 32), kIdesc, 1u);
+                    }
+                    tc_commit(empty(st));
+                }
+                if (ok) tc_commit(tmem_full(acc));
+                ++tile_n;
+            }
+        }
+    } else {
+        // ---- epilogue: warp = (lane quarter of tensor memory, column half); thread = row ----
+        const int quarter = warp & 3, half = warp >> 2;
+        uint32_t tile_n = 0;
+        for (int round = 0; round < rounds; ++round) {
+            const int q = tile_of(round);
+            if (q >= p.tiles) break;
+            const int64_t i0 = (int64_t)(q / p.col_tiles) * kBtRows;
+            const int64_t cb = (int64_t)(q % p.col_tiles) * kBtCols + half * kBtEpiCols;
+            const int acc = tile_n & 1;
+            const uint32_t use = tile_n >> 1;
+            int got = 1;
+            if (lane == 0) got = bt_wait(tmem_full(acc), use & 1, abort_flag, p.err_word) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (!got) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int64_t i = i0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBtCols + half * kBtEpiCols;
+            float* crow = p.C + i * p.ldc + cb;
+#pragma unroll 1
+            for (int cc = 0; cc < kBtEpiCols / 32; ++cc) {
+                uint32_t r[32];
+                tc_ld32(taddr + cc * 32, r);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const int64_t col0 = cb + cc * 32;
+                if (i < N) {
+                    if (p.vec_c && col0 + 32 <= p.ncols) {
+                        float4* dst = reinterpret_cast<float4*>(crow + cc * 32);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                   __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                            if (p.accumulate) {
+                                const float4 old = dst[v];
+                                o.x += old.x, o.y += old.y, o.z += old.z, o.w += old.w;
+                            }
+                            dst[v] = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 32; ++v)
+                            if (col0 + v < p.ncols) {
+                                float o = __uint_as_float(r[v]);
+                                if (p.accumulate) o += crow[cc * 32 + v];
+                                crow[cc * 32 + v] = o;
+                            }
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) tc_mbar_arrive(tmem_empty(acc));  // the accumulator may be overwritten
+            ++tile_n;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kBtTmemCols) : "memory");
+    }
+}
+
+}  // namespace
+}  // namespace dastac
+
+using namespace dastac;
+
+extern "C" dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, const float* A, const float* B, int64_t ldb,
+                                                  float* C, int64_t ldc, int64_t ncols, int32_t accumulate,
+                                                  int32_t* err_word, void* stream) {
+    if (!s) return DASTAC_ERR_INVALID_ARG;
+    const IndexMap& m = s->map;
+    if (m.kind == kEmpty) return DASTAC_OK;
+    if (m.kind != kBandDiagonals && m.kind != kBandExact) return DASTAC_ERR_UNSUPPORTED_EXPR;
+    const int64_t N = m.N;
+    if (ncols < 0) return DASTAC_ERR_INVALID_ARG;
+    if (N == 0 || ncols == 0) return DASTAC_OK;
+    if (!A || !B || !C || ldb < ncols || ldc < ncols) return DASTAC_ERR_INVALID_ARG;
+    // window rows and diagonals are counted in 32-bit integers inside the kernel
+    if (m.w > (int64_t)1 << 24 || N > (int64_t)1 << 40) return DASTAC_ERR_OVERFLOW;
+    BtParams p;
+    p.A = A, p.B = B, p.C = C;
+    p.N = N, p.w = m.w, p.ldb = ldb, p.ldc = ldc, p.ncols = ncols;
+    const int64_t row_tiles = (N + kBtRows - 1) / kBtRows, col_tiles = (ncols + kBtCols - 1) / kBtCols;
+    if (row_tiles * col_tiles > 0x7fffffffLL) return DASTAC_ERR_OVERFLOW;
+    p.row_tiles = (int32_t)row_tiles, p.col_tiles = (int32_t)col_tiles, p.tiles = (int32_t)(row_tiles * col_tiles);
+    p.exact = m.kind == kBandExact;
+    p.accumulate = accumulate;
+    p.vec_c = ((ldc & 3) == 0) && aligned16(C);
+    p.err_word = err_word;
+    static bool attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(bandmm_tc_kernel<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBtSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(bandmm_tc_kernel<20>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBtSmemBytes) != cudaSuccess)
+            return DASTAC_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    int grid = sm_count();
+    if (grid > p.tiles) grid = p.tiles;
+    if (2 * m.w + 1 <= 80)
+        bandmm_tc_kernel<10><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(p);
+    else
+        bandmm_tc_kernel<20><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(p);
+    return launch_status();
+}

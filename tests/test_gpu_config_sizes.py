@@ -82,6 +82,26 @@ def test_config2_band_n32768_w32_c256():
     assert rel_err(got[sel], ref, ref_abs) <= TOL_F32
 
 
+def test_config2_band_split_precision_tensor_core_form():
+    """Configuration 2 through the opt-in TF32 hi/lo entry point, same sampled rows and bound."""
+    N, w, C = 32768, 32, 256
+    desc = st.band(N, w)
+    s = dastac.Structure(desc)
+    B = synth.dense(1, 1, (N, C))
+    packed = _packed(s, lambda h: synth.band_diagonals_stream(1, 0, N, w, pad_bits=0x7FC00000, out=h))
+    out = torch.full((N, C), float("nan"), device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dastac.bandmm_split_tf32(s, packed, dev(B), out, err_word=err)
+    assert int(err.item()) == 0
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    sel = _rows(N, 300, extra=range(0, 40))
+    sel = np.union1d(sel, np.arange(N - 40, N))
+    Ar = np.stack([synth.linear_slice(1, 0, int(i) * N, N) for i in sel])
+    ref, ref_abs = oracle.matmat(desc, Ar, B, sel=sel)
+    assert rel_err(got[sel], ref, ref_abs) <= TOL_F32
+
+
 def test_config3_symv_n65536():
     N = 65536
     desc = st.upper_triangle(N, symmetric=True)

@@ -1146,6 +1146,50 @@ def test_mttkrp_split_precision_tensor_core_form(n, R):
     assert rel_err(outp.cpu().numpy(), ref, ref_abs) <= TOL_F32
 
 
+@pytest.mark.parametrize("exact", [False, True], ids=["diagonals", "exact"])
+@pytest.mark.parametrize("N,w,C", [(2, 0, 1), (7, 0, 3), (40, 3, 5), (128, 32, 256), (129, 16, 257), (300, 32, 256),
+                                   (1000, 7, 130), (2048, 32, 64), (200, 40, 33), (513, 90, 64), (190, 94, 12),
+                                   (700, 200, 300)])
+def test_band_matmat_split_precision_tensor_core_form(N, w, C, exact):
+    """The opt-in TF32 hi/lo form of band x dense against the oracle, at the fp32 kernels' bound."""
+    desc = st.band_exact(N, w) if exact else st.band(N, w)
+    s = dastac.Structure(desc)
+    A = synth.dense(1, 0, (N, N))
+    B = synth.dense(1, 1, (N, C))
+    ref, ref_abs = oracle.matmat(desc, A, B)
+    # padding slots of the diagonal layout are poisoned: the product must not depend on them
+    packed = packed_dev(s, oracle.pack(desc, A) if exact else synth.band_diagonals_stream(1, 0, N, w, pad_bits=0x7FC00000))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full((N, C), float("nan"), device="cuda")
+    dastac.bandmm_split_tf32(s, packed, dev(B), out, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    C0 = synth.dense(1, 2, (N, C))
+    out2 = dev(C0)
+    dastac.bandmm_split_tf32(s, packed, dev(B), out2, accumulate=True, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out2.cpu().numpy(), ref + C0, ref_abs + np.abs(C0)) <= TOL_F32
+    # padded leading dimensions (rows of B and C not 16-byte aligned)
+    Bp = torch.zeros((N, C + 3), device="cuda")[:, :C]
+    Bp.copy_(dev(B))
+    outp = torch.full((N, C + 5), float("nan"), device="cuda")[:, :C]
+    dastac.bandmm_split_tf32(s, packed, Bp, outp, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(outp.cpu().numpy(), ref, ref_abs) <= TOL_F32
+    # the fp32 kernel and this form agree far inside the bound
+    plain = torch.empty((N, C), device="cuda")
+    dastac.contract("ij,jc->ic", s, packed, [dev(B)], plain)
+    assert rel_err(out.cpu().numpy(), plain.cpu().numpy().astype(np.float64), ref_abs) <= TOL_F32
+
+
+def test_band_matmat_split_precision_refusals():
+    tri = dastac.Structure(st.upper_triangle(16))
+    z = torch.zeros((16, 4), device="cuda")
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.bandmm_split_tf32(tri, tri.empty_packed(), z, torch.zeros((16, 4), device="cuda"))
+    assert e.value.status == 3
+
+
 def test_mttkrp_split_precision_refusals():
     big = dastac.Structure(st.tetrahedron(513))
     z = torch.zeros((513, 4), device="cuda")
