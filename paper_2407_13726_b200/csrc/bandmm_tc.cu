@@ -22,6 +22,10 @@
 //                    (read-add-write when accumulating)
 // Two stages of operands (96 KiB each), two accumulators of 256 columns (all of tensor memory).
 // K blocks that lie outside the matrix (first and last tiles) are skipped.  Every wait is bounded.
+#include <cuda.h>
+
+#include <cstring>
+
 #include "common.cuh"
 #include "tf32_mma.cuh"
 #include "waits.cuh"
@@ -44,7 +48,9 @@ constexpr int kBtThreads = (kBtEpiWarps + 1 + kBtProducerWarps * kBtProducerGrou
 constexpr int kBtTmemCols = 512;
 constexpr long long kBtWaitBudget = 2000000000LL;
 constexpr int32_t kErrWordBandTc = 0x4254;   // "BT"
-constexpr size_t kBtSmemBytes = (size_t)kBtStages * kBtStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr int kBtEpiBufBytes = 32 * 128;     // a 32 x 32 fp32 chunk of C on its way out
+constexpr int kBtEpiBytes = kBtEpiWarps * 2 * kBtEpiBufBytes;  // two buffers per epilogue warp
+constexpr size_t kBtSmemBytes = (size_t)kBtStages * kBtStageBytes + kBtEpiBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 
 struct BtParams {
     const float* A;
@@ -55,6 +61,7 @@ struct BtParams {
     int32_t exact;       // A packed row after row instead of padded diagonals
     int32_t accumulate;
     int32_t vec_c;       // C allows 128-bit accesses
+    int32_t tma_c;       // C is described by the tensor map: chunks leave through shared memory by bulk stores
     int32_t* err_word;
 };
 
@@ -91,11 +98,12 @@ __device__ __forceinline__ bool bt_producer_sync_any(bool flag, int group) {
 }
 
 template <int kBtSegs>
-__global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams p) {
+__global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_constant__ CUtensorMap tmap_c, const BtParams p) {
     extern __shared__ uint8_t bt_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(bt_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint64_t* const bars = reinterpret_cast<uint64_t*>(smem + (size_t)kBtStages * kBtStageBytes);
+    uint8_t* const epi0 = smem + (size_t)kBtStages * kBtStageBytes;
+    uint64_t* const bars = reinterpret_cast<uint64_t*>(epi0 + kBtEpiBytes);
     constexpr int S = kBtStages;
     auto full = [&](int s) { return tc_smem(&bars[s]); };
     auto empty = [&](int s) { return tc_smem(&bars[S + s]); };
@@ -161,35 +169,43 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams
             const int64_t j0 = i0 - w + 32 * (int64_t)kb;  // B row of the block's first window row
             const int64_t col = cb + t;
             const bool col_ok = col < p.ncols;
-            const float* bsrc = p.B + j0 * p.ldb + col;  // dereferenced only where the row and column exist
+            int64_t boff = j0 * p.ldb + col;  // used only where the row and column exist
             if (j0 >= 0 && j0 + 31 < N) {  // block-uniform: every row of the K block exists
 #pragma unroll
-                for (int e = 0; e < 32; ++e) bv[e] = col_ok ? __ldg(bsrc + e * p.ldb) : 0.f;
+                for (int e = 0; e < 32; ++e, boff += p.ldb) bv[e] = col_ok ? __ldg(p.B + boff) : 0.f;
             } else {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
+                for (int e = 0; e < 32; ++e, boff += p.ldb) {
                     const int64_t j = j0 + e;
-                    bv[e] = (col_ok && j >= 0 && j < N) ? __ldg(bsrc + e * p.ldb) : 0.f;
+                    bv[e] = (col_ok && j >= 0 && j < N) ? __ldg(p.B + boff) : 0.f;
                 }
             }
-            // diagonals d whose entries fall into this K block for some row of the tile:
-            // row r holds diagonal d at window row kk = r + d, so d in [32 kb - 127, 32 kb + 31]
-            const int d_lo = 32 * kb - (kBtRows - 1) > 0 ? 32 * kb - (kBtRows - 1) : 0;
+            // Diagonals d whose entries fall into this K block for some row of the tile: row r holds
+            // diagonal d at window row kk = r + d, so d in [32 kb - 127, 32 kb + 31].  This warp takes
+            // d = d_lo + pw + 8u; its lane reads row r0 - 8u, always column j of A.
+            const int d0 = (32 * kb - (kBtRows - 1) > 0 ? 32 * kb - (kBtRows - 1) : 0) + pw;
             const int d_hi = (int)(32 * (int64_t)kb + 31 < 2 * w ? 32 * (int64_t)kb + 31 : 2 * w);
-            const int64_t j = j0 + lane;  // the column of A this lane reads, whatever the diagonal
+            const int r0 = 32 * kb - d0 + lane;
+            const int r_lim = (int)(N - i0 < kBtRows ? N - i0 : kBtRows);  // rows of the tile that exist
+            const int64_t j = j0 + lane;
             const bool j_ok = j >= 0 && j < N;
+            if (!p.exact) {
+                int64_t aoff = (int64_t)d0 * N + i0 + r0;  // slot (d, i) = d N + i; next segment: + 8 (N - 1)
+                const int64_t astep = 8 * (N - 1);
 #pragma unroll
-            for (int u = 0; u < kBtSegs; ++u) {
-                const int d = d_lo + pw + 8 * u;
-                if (d > d_hi) break;  // warp-uniform
-                const int r = 32 * kb - d + lane;
-                const int64_t i = i0 + r;
-                float v = 0.f;
-                if (j_ok && r >= 0 && r < kBtRows && i < N) {
-                    const int64_t off = p.exact ? band_row_start(N, w, i) - band_jlo(w, i) + j : (int64_t)d * N + i;
-                    v = __ldg(p.A + off);
+                for (int u = 0; u < kBtSegs; ++u, aoff += astep) {
+                    if (d0 + 8 * u > d_hi) break;  // warp-uniform
+                    const int r = r0 - 8 * u;
+                    av[u] = (j_ok && r >= 0 && r < r_lim) ? __ldg(p.A + aoff) : 0.f;
                 }
-                av[u] = v;
+            } else {
+#pragma unroll
+                for (int u = 0; u < kBtSegs; ++u) {
+                    if (d0 + 8 * u > d_hi) break;
+                    const int r = r0 - 8 * u;
+                    const int64_t i = i0 + r;
+                    av[u] = (j_ok && r >= 0 && r < r_lim) ? __ldg(p.A + (band_row_start(N, w, i) - band_jlo(w, i) + j)) : 0.f;
+                }
             }
         };
         for (int g = 0; g <= grp; ++g) next_item();  // group g starts at item g
@@ -222,19 +238,20 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams
             }
             if (bt_producer_sync_any(!ok, grp)) break;  // a wait ran out somewhere: all eight warps stop here
             {
-                const int d_lo = 32 * kb - (kBtRows - 1) > 0 ? 32 * kb - (kBtRows - 1) : 0;
+                // segment u lands in row r0 - 8u, column lane of the K block: eight rows up is 1024 bytes back
+                const int d0 = (32 * kb - (kBtRows - 1) > 0 ? 32 * kb - (kBtRows - 1) : 0) + pw;
                 const int d_hi = (int)(32 * (int64_t)kb + 31 < 2 * w ? 32 * (int64_t)kb + 31 : 2 * w);
+                const int r0 = 32 * kb - d0 + lane;
+                const int off0 = (r0 >> 3) * 1024 + (r0 & 7) * 128 + (((lane >> 2) ^ (r0 & 7)) << 4) + (lane & 3) * 4;
 #pragma unroll
                 for (int u = 0; u < kBtSegs; ++u) {
-                    const int d = d_lo + pw + 8 * u;
-                    if (d > d_hi) break;
-                    const int r = 32 * kb - d + lane;
+                    if (d0 + 8 * u > d_hi) break;
+                    const int r = r0 - 8 * u;
                     if (r >= 0 && r < kBtRows) {
                         float hi, lo;
                         tc_split(av[u], hi, lo);
-                        const uint32_t off = tc_tile_offset(r, lane >> 2) + (uint32_t)(lane & 3) * 4u;
-                        *reinterpret_cast<float*>(a_hi + off) = hi;
-                        *reinterpret_cast<float*>(a_hi + kBtATile + off) = lo;
+                        *reinterpret_cast<float*>(a_hi + off0 - 1024 * u) = hi;
+                        *reinterpret_cast<float*>(a_hi + kBtATile + off0 - 1024 * u) = lo;
                     }
                 }
             }
@@ -294,7 +311,7 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams
     } else {
         // ---- epilogue: warp = (lane quarter of tensor memory, column half); thread = row ----
         const int quarter = warp & 3, half = warp >> 2;
-        uint32_t tile_n = 0;
+        uint32_t tile_n = 0, chunk_n = 0;
         for (int round = 0; round < rounds; ++round) {
             const int q = tile_of(round);
             if (q >= p.tiles) break;
@@ -310,6 +327,41 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams
             const int64_t i = i0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBtCols + half * kBtEpiCols;
             float* crow = p.C + i * p.ldc + cb;
+            if (p.tma_c) {
+                // A 32 x 32 chunk goes to one of the warp's two buffers (rows of 128 bytes, 16-byte
+                // pieces swizzled like the tensor map's 128-byte mode, so the lanes' stores spread
+                // over the banks) and leaves by one bulk tensor store, or reduce-add when
+                // accumulating; rows and columns outside C are clipped by the copy.
+#pragma unroll 1
+                for (int cc = 0; cc < kBtEpiCols / 32; ++cc, ++chunk_n) {
+                    uint8_t* const buf = epi0 + (size_t)(warp * 2 + (chunk_n & 1)) * kBtEpiBufBytes;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");  // its last store has read it
+                    __syncwarp();
+                    uint32_t r[32];
+                    tc_ld32(taddr + cc * 32, r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        *reinterpret_cast<float4*>(buf + lane * 128 + ((v ^ (lane & 7)) << 4)) =
+                            make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                        __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    const int64_t col0 = cb + cc * 32, row0 = i0 + quarter * 32;
+                    if (lane == 0 && col0 < p.ncols && row0 < N) {
+                        if (p.accumulate)
+                            asm volatile(
+                                "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                ::"l"(&tmap_c), "r"((int)col0), "r"((int)row0), "r"(tc_smem(buf))
+                                : "memory");
+                        else
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(&tmap_c), "r"((int)col0), "r"((int)row0), "r"(tc_smem(buf))
+                                         : "memory");
+                    }
+                    if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            } else {
 #pragma unroll 1
             for (int cc = 0; cc < kBtEpiCols / 32; ++cc) {
                 uint32_t r[32];
@@ -340,11 +392,14 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams
                     }
                 }
             }
+            }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) tc_mbar_arrive(tmem_empty(acc));  // the accumulator may be overwritten
             ++tile_n;
         }
+        // shared memory stays allocated until the bulk stores have read it and written C
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -352,6 +407,22 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const BtParams
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kBtTmemCols) : "memory");
     }
+}
+
+typedef CUresult (*BtEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+BtEncodeTiledFn bt_encode_fn() {
+    static BtEncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (BtEncodeTiledFn)ptr;
+    }
+    return fn;
 }
 
 }  // namespace
@@ -382,6 +453,22 @@ extern "C" dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, con
     p.accumulate = accumulate;
     p.vec_c = ((ldc & 3) == 0) && aligned16(C);
     p.err_word = err_word;
+    // C as a 2-D tensor of 32 x 32 boxes in the 128-byte swizzle, when its rows are 16-byte aligned
+    CUtensorMap tmap_c;
+    std::memset(&tmap_c, 0, sizeof(tmap_c));
+    p.tma_c = 0;
+    if (p.vec_c && N < ((int64_t)1 << 31) && ncols < ((int64_t)1 << 31)) {
+        BtEncodeTiledFn enc = bt_encode_fn();
+        if (!enc) return DASTAC_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)ncols, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+        const cuuint32_t box[2] = {32, 32};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&tmap_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DASTAC_ERR_CUDA;
+        p.tma_c = 1;
+    }
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -394,8 +481,8 @@ extern "C" dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, con
     int grid = sm_count();
     if (grid > p.tiles) grid = p.tiles;
     if (2 * m.w + 1 <= 80)
-        bandmm_tc_kernel<10><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(p);
+        bandmm_tc_kernel<10><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(tmap_c, p);
     else
-        bandmm_tc_kernel<20><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(p);
+        bandmm_tc_kernel<20><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(tmap_c, p);
     return launch_status();
 }
