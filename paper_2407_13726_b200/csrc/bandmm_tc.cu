@@ -9,17 +9,21 @@
 // about 2^-21 per product, inside the 1e-5 bound of the fp32 kernels.
 //
 // Tile = (128 rows, 256 columns); K blocks of 32 rows of the B window.
-//   producer warps   (two groups of eight, taking the K blocks in turn, one stage each) thread n of 256 reads column n of the K block of B (32 coalesced 4-byte loads
-//                    per thread, no alignment requirement on B), splits and writes row n of the two
-//                    K-major, 128-byte-swizzled 256 x 32 tiles Bhi, Blo with 128-bit stores.  The
-//                    slice of A is zeroed and the band written into it diagonal by diagonal: for
-//                    diagonal d the 32 rows whose entry falls into this K block are consecutive in
-//                    memory in the padded layout (one coalesced load) and land on 32 different
-//                    banks of the swizzled tile.
+//   producer warps   two groups of eight, taking the K blocks in turn, one stage each.  The K block of
+//                    B arrives by bulk tensor copies (eight 32 x 32 boxes) straight into the N-major
+//                    operand layout of 4-byte types (rows of 128 bytes, 32-byte pieces swizzled with
+//                    the row); the block itself serves as Bhi, since the tensor core reads only the
+//                    upper 19 bits of a value, and the warps write Blo = B - trunc(B) beside it.  (A B
+//                    whose rows are not 16-byte aligned is read column by column with plain loads
+//                    and stored in the same layout.)  The slice of A is K-major: it is zeroed and the
+//                    band written into it diagonal by diagonal: for diagonal d the 32 rows whose
+//                    entry falls into this K block are consecutive in memory in the padded layout
+//                    (one coalesced load) and land on 32 different banks of the swizzled tile.
 //   MMA thread       per K block and k-step of 8: three tcgen05.mma kind::tf32 M128 N256 K8
 //                    (Ahi Bhi, Ahi Blo, Alo Bhi) into one accumulator
-//   epilogue warps   one per lane quarter of tensor memory: tcgen05.ld, 128-bit stores to C
-//                    (read-add-write when accumulating)
+//   epilogue warps   one per lane quarter of tensor memory: tcgen05.ld, then 32 x 32 chunks leave
+//                    through shared memory by bulk tensor stores (reduce-add when accumulating);
+//                    a C whose rows are not 16-byte aligned is written with plain stores
 // Two stages of operands (96 KiB each), two accumulators of 256 columns (all of tensor memory).
 // K blocks that lie outside the matrix (first and last tiles) are skipped.  Every wait is bounded.
 #include <cuda.h>
@@ -61,6 +65,7 @@ struct BtParams {
     int32_t exact;       // A packed row after row instead of padded diagonals
     int32_t accumulate;
     int32_t vec_c;       // C allows 128-bit accesses
+    int32_t tma_b;       // B is described by a tensor map: its K blocks arrive by bulk tensor copies
     int32_t tma_c;       // C is described by the tensor map: chunks leave through shared memory by bulk stores
     int32_t* err_word;
 };
@@ -75,6 +80,18 @@ __device__ __forceinline__ void bt_k_range(const BtParams& p, int64_t i0, int& k
     kb_hi = (int)((kk_end + 31) >> 5);
 }
 
+// N-major B operand of a 4-byte type: rows (one k, 32 consecutive n) of 128 bytes whose 32-byte
+// pieces are swizzled with the row; groups of four rows 512 bytes apart, blocks of 32 columns one
+// 32 x 32 box (4096 bytes) apart.
+__device__ __forceinline__ uint64_t bt_desc_b(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(4096 >> 4) << 16;  // leading byte offset: next block of 32 columns
+    d |= (uint64_t)(512 >> 4) << 32;   // stride byte offset: next group of four rows
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)1 << 61;            // 128-byte swizzle of 32-byte pieces
+    return d;
+}
 __device__ __forceinline__ bool bt_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* err_word) {
     return tc_wait_coded(bar, parity, abort_flag, err_word, kErrWordBandTc, kBtWaitBudget);
 }
@@ -98,7 +115,7 @@ __device__ __forceinline__ bool bt_producer_sync_any(bool flag, int group) {
 }
 
 template <int kBtSegs>
-__global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_constant__ CUtensorMap tmap_c, const BtParams p) {
+__global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_c, const BtParams p) {
     extern __shared__ uint8_t bt_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(bt_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -109,13 +126,15 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
     auto empty = [&](int s) { return tc_smem(&bars[S + s]); };
     auto tmem_full = [&](int a) { return tc_smem(&bars[2 * S + a]); };
     auto tmem_empty = [&](int a) { return tc_smem(&bars[2 * S + 2 + a]); };
-    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(&bars[2 * S + 4]);
+    auto raw = [&](int s) { return tc_smem(&bars[2 * S + 4 + s]); };  // the stage's block of B has landed
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(&bars[3 * S + 4]);
     volatile int* const abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             tc_mbar_init(full(s), kBtProducerWarps);
             tc_mbar_init(empty(s), 1);
+            tc_mbar_init(raw(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             tc_mbar_init(tmem_full(a), 1);
@@ -170,7 +189,9 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
             const int64_t col = cb + t;
             const bool col_ok = col < p.ncols;
             int64_t boff = j0 * p.ldb + col;  // used only where the row and column exist
-            if (j0 >= 0 && j0 + 31 < N) {  // block-uniform: every row of the K block exists
+            if (p.tma_b) {
+                // the block arrives by bulk copies once the stage is free
+            } else if (j0 >= 0 && j0 + 31 < N) {  // block-uniform: every row of the K block exists
 #pragma unroll
                 for (int e = 0; e < 32; ++e, boff += p.ldb) bv[e] = col_ok ? __ldg(p.B + boff) : 0.f;
             } else {
@@ -220,21 +241,44 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
             if (use >= 1 && lane == 0) ok = bt_wait(empty(st), (use - 1) & 1, abort_flag, p.err_word);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (ok) {
-                // row t of Bhi / Blo
+                if (p.tma_b) {
+                    // The K block of B, 32 rows x 256 columns, as eight 32 x 32 boxes: rows of 128 bytes
+                    // whose 32-byte pieces are swizzled with the row (the N-major operand layout of
+                    // 4-byte types).  Rows and columns outside B arrive as zeros.  The block itself is
+                    // the high part: the tensor core reads the upper 19 bits of every value.
+                    if (pw == 0 && lane == 0) {
+                        const int64_t j0 = i0 - w + 32 * (int64_t)kb;
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw(st)), "r"((uint32_t)kBtBTile)
+                                     : "memory");
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    float hi[4], lo[4];
+                        for (int a = 0; a < kBtCols / 32; ++a)
+                            asm volatile(
+                                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                                ::"r"(tc_smem(b_hi + a * 4096)), "l"(&tmap_b), "r"((int)(cb + 32 * a)), "r"((int)j0), "r"(raw(st))
+                                : "memory");
+                    }
+                } else {
+                    // column t of the block from registers: element (k, n) of the N-major layout sits at
+                    // (n / 32) * 4096 + k * 128 + (((n % 32) / 8) ^ (k % 4)) * 32 + (n % 8) * 4
+                    uint8_t* const colp = b_hi + (t >> 5) * 4096 + (t & 7) * 4;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) tc_split(bv[4 * c + e], hi[e], lo[e]);
-                    const uint32_t off = tc_tile_offset(t, c);
-                    *reinterpret_cast<float4*>(b_hi + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<float4*>(b_hi + kBtBTile + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                    for (int e = 0; e < 32; ++e) {
+                        float hi, lo;
+                        tc_split(bv[e], hi, lo);
+                        const uint32_t off = (uint32_t)(e * 128 + ((((t & 31) >> 3) ^ (e & 3)) << 5));
+                        *reinterpret_cast<float*>(colp + off) = hi;
+                        *reinterpret_cast<float*>(colp + kBtBTile + off) = lo;
+                    }
                 }
                 // the slice of A: zeros, then the band
 #pragma unroll
                 for (int u = 0; u < 2 * kBtATile / (16 * kBtProducerWarps * 32); ++u)
                     *reinterpret_cast<float4*>(a_hi + (size_t)(u * kBtProducerWarps * 32 + t) * 16) =
                         make_float4(0.f, 0.f, 0.f, 0.f);
+                if (p.tma_b) {  // the block of B has landed (every warp's lane 0 looks for itself)
+                    if (lane == 0) ok = bt_wait(raw(st), use & 1, abort_flag, p.err_word);
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                }
             }
             if (bt_producer_sync_any(!ok, grp)) break;  // a wait ran out somewhere: all eight warps stop here
             {
@@ -255,6 +299,17 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
                     }
                 }
             }
+            if (p.tma_b) {
+                // low parts of the block: same layout, element by element
+#pragma unroll
+                for (int u = 0; u < kBtBTile / (16 * kBtProducerWarps * 32); ++u) {
+                    const size_t off = (size_t)(u * kBtProducerWarps * 32 + t) * 16;
+                    const float4 v = *reinterpret_cast<const float4*>(b_hi + off);
+                    float4 h, l;
+                    tc_split(v.x, h.x, l.x), tc_split(v.y, h.y, l.y), tc_split(v.z, h.z, l.z), tc_split(v.w, h.w, l.w);
+                    *reinterpret_cast<float4*>(b_hi + kBtBTile + off) = l;
+                }
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) tc_mbar_arrive(full(st));
@@ -267,7 +322,7 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
     else if (warp == kBtWarpMma) {
         // ---- MMA issuer: one thread ----
         if (lane == 0) {
-            constexpr uint32_t kIdesc = tc_idesc_mn(kBtRows, kBtCols);
+            constexpr uint32_t kIdesc = tc_idesc_mn(kBtRows, kBtCols) | (1u << 16);  // B operand N-major
             uint32_t it = 0, tile_n = 0;
             bool ok = true;
             for (int round = 0; round < rounds && ok; ++round) {
@@ -297,10 +352,10 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
                     const uint32_t b_lo = b_hi + kBtBTile;
 #pragma unroll
                     for (int k8 = 0; k8 < 4; ++k8) {
-                        tc_mma_tf32(d_tmem, tc_desc(a_hi + k8 * 32), tc_desc(b_hi + k8 * 32), kIdesc,
+                        tc_mma_tf32(d_tmem, tc_desc(a_hi + k8 * 32), bt_desc_b(b_hi + k8 * 1024), kIdesc,
                                     (kb > kb_lo || k8 > 0) ? 1u : 0u);
-                        tc_mma_tf32(d_tmem, tc_desc(a_hi + k8 * 32), tc_desc(b_lo + k8 * 32), kIdesc, 1u);
-                        tc_mma_tf32(d_tmem, tc_desc(a_lo + k8 * 32), tc_desc(b_hi + k8 * 32), kIdesc, 1u);
+                        tc_mma_tf32(d_tmem, tc_desc(a_hi + k8 * 32), bt_desc_b(b_lo + k8 * 1024), kIdesc, 1u);
+                        tc_mma_tf32(d_tmem, tc_desc(a_lo + k8 * 32), bt_desc_b(b_hi + k8 * 1024), kIdesc, 1u);
                     }
                     tc_commit(empty(st));
                 }
@@ -469,6 +524,23 @@ extern "C" dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, con
             return DASTAC_ERR_CUDA;
         p.tma_c = 1;
     }
+    // B as a 2-D tensor of 32 x 32 boxes, 32-byte pieces swizzled within 128 bytes, under the same conditions
+    CUtensorMap tmap_b;
+    std::memset(&tmap_b, 0, sizeof(tmap_b));
+    p.tma_b = 0;
+    if ((ldb & 3) == 0 && aligned16(B) && N < ((int64_t)1 << 31) && ncols < ((int64_t)1 << 31)) {
+        BtEncodeTiledFn enc = bt_encode_fn();
+        if (!enc) return DASTAC_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)ncols, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)ldb * 4};
+        const cuuint32_t box[2] = {32, 32};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(B), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DASTAC_ERR_CUDA;
+        p.tma_b = 1;
+    }
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -481,8 +553,8 @@ extern "C" dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, con
     int grid = sm_count();
     if (grid > p.tiles) grid = p.tiles;
     if (2 * m.w + 1 <= 80)
-        bandmm_tc_kernel<10><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(tmap_c, p);
+        bandmm_tc_kernel<10><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(tmap_b, tmap_c, p);
     else
-        bandmm_tc_kernel<20><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(tmap_c, p);
+        bandmm_tc_kernel<20><<<grid, kBtThreads, kBtSmemBytes, (cudaStream_t)stream>>>(tmap_b, tmap_c, p);
     return launch_status();
 }
