@@ -315,7 +315,9 @@ dastac_status dastac_mttkrp_split_tf32(const dastac_structure* s, const float* T
  *             aligned and ldc is a multiple of 4, scalar stores otherwise
  *   accumulate, stream   as for dastac_contract
  *   err_word  optional device int32, set when a bounded wait inside the kernel expires
- * Needs no workspace.
+ * Needs no workspace.  Unlike dastac_contract, which visits the band only, a row of B meets every
+ * row of the 128-row tile whose window holds it, with a zero factor outside the band: an infinity
+ * or NaN in B therefore reaches rows of C that the band does not connect it to.
  */
 dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, const float* A, const float* B, int64_t ldb,
                                        float* C, int64_t ldc, int64_t ncols, int32_t accumulate,
