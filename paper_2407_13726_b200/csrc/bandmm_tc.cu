@@ -183,24 +183,9 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
                 bt_k_range(p, i0, kb, kb_end);
             }
         };
-        float bv[32], av[kBtSegs];
+        float av[kBtSegs];
         auto load_item = [&]() {
             const int64_t j0 = i0 - w + 32 * (int64_t)kb;  // B row of the block's first window row
-            const int64_t col = cb + t;
-            const bool col_ok = col < p.ncols;
-            int64_t boff = j0 * p.ldb + col;  // used only where the row and column exist
-            if (p.tma_b) {
-                // the block arrives by bulk copies once the stage is free
-            } else if (j0 >= 0 && j0 + 31 < N) {  // block-uniform: every row of the K block exists
-#pragma unroll
-                for (int e = 0; e < 32; ++e, boff += p.ldb) bv[e] = col_ok ? __ldg(p.B + boff) : 0.f;
-            } else {
-#pragma unroll
-                for (int e = 0; e < 32; ++e, boff += p.ldb) {
-                    const int64_t j = j0 + e;
-                    bv[e] = (col_ok && j >= 0 && j < N) ? __ldg(p.B + boff) : 0.f;
-                }
-            }
             // Diagonals d whose entries fall into this K block for some row of the tile: row r holds
             // diagonal d at window row kk = r + d, so d in [32 kb - 127, 32 kb + 31].  This warp takes
             // d = d_lo + pw + 8u; its lane reads row r0 - 8u, always column j of A.
@@ -215,17 +200,15 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
                 const int64_t astep = 8 * (N - 1);
 #pragma unroll
                 for (int u = 0; u < kBtSegs; ++u, aoff += astep) {
-                    if (d0 + 8 * u > d_hi) break;  // warp-uniform
                     const int r = r0 - 8 * u;
-                    av[u] = (j_ok && r >= 0 && r < r_lim) ? __ldg(p.A + aoff) : 0.f;
+                    av[u] = (d0 + 8 * u <= d_hi && j_ok && r >= 0 && r < r_lim) ? __ldg(p.A + aoff) : 0.f;
                 }
             } else {
 #pragma unroll
                 for (int u = 0; u < kBtSegs; ++u) {
-                    if (d0 + 8 * u > d_hi) break;
                     const int r = r0 - 8 * u;
                     const int64_t i = i0 + r;
-                    av[u] = (j_ok && r >= 0 && r < r_lim) ? __ldg(p.A + (band_row_start(N, w, i) - band_jlo(w, i) + j)) : 0.f;
+                    av[u] = (d0 + 8 * u <= d_hi && j_ok && r >= 0 && r < r_lim) ? __ldg(p.A + (band_row_start(N, w, i) - band_jlo(w, i) + j)) : 0.f;
                 }
             }
         };
@@ -258,7 +241,24 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
                                 : "memory");
                     }
                 } else {
-                    // column t of the block from registers: element (k, n) of the N-major layout sits at
+                    // column t of the block with plain loads (issued here, when the stage is free: this
+                    // path holds no values across K blocks)
+                    float bv[32];
+                    const int64_t j0 = i0 - w + 32 * (int64_t)kb;
+                    const int64_t col = cb + t;
+                    const bool col_ok = col < p.ncols;
+                    int64_t boff = j0 * p.ldb + col;  // used only where the row and column exist
+                    if (j0 >= 0 && j0 + 31 < N) {  // block-uniform: every row of the K block exists
+#pragma unroll
+                        for (int e = 0; e < 32; ++e, boff += p.ldb) bv[e] = col_ok ? __ldg(p.B + boff) : 0.f;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e, boff += p.ldb) {
+                            const int64_t j = j0 + e;
+                            bv[e] = (col_ok && j >= 0 && j < N) ? __ldg(p.B + boff) : 0.f;
+                        }
+                    }
+                    // element (k, n) of the N-major layout sits at
                     // (n / 32) * 4096 + k * 128 + (((n % 32) / 8) ^ (k % 4)) * 32 + (n % 8) * 4
                     uint8_t* const colp = b_hi + (t >> 5) * 4096 + (t & 7) * 4;
 #pragma unroll
@@ -289,9 +289,8 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
                 const int off0 = (r0 >> 3) * 1024 + (r0 & 7) * 128 + (((lane >> 2) ^ (r0 & 7)) << 4) + (lane & 3) * 4;
 #pragma unroll
                 for (int u = 0; u < kBtSegs; ++u) {
-                    if (d0 + 8 * u > d_hi) break;
                     const int r = r0 - 8 * u;
-                    if (r >= 0 && r < kBtRows) {
+                    if (d0 + 8 * u <= d_hi && r >= 0 && r < kBtRows) {
                         float hi, lo;
                         tc_split(av[u], hi, lo);
                         *reinterpret_cast<float*>(a_hi + off0 - 1024 * u) = hi;
@@ -301,13 +300,19 @@ __global__ void __launch_bounds__(kBtThreads, 1) bandmm_tc_kernel(const __grid_c
             }
             if (p.tma_b) {
                 // low parts of the block: same layout, element by element
+                constexpr int kPer = kBtBTile / (16 * kBtProducerWarps * 32);
 #pragma unroll
-                for (int u = 0; u < kBtBTile / (16 * kBtProducerWarps * 32); ++u) {
-                    const size_t off = (size_t)(u * kBtProducerWarps * 32 + t) * 16;
-                    const float4 v = *reinterpret_cast<const float4*>(b_hi + off);
-                    float4 h, l;
-                    tc_split(v.x, h.x, l.x), tc_split(v.y, h.y, l.y), tc_split(v.z, h.z, l.z), tc_split(v.w, h.w, l.w);
-                    *reinterpret_cast<float4*>(b_hi + kBtBTile + off) = l;
+                for (int half = 0; half < 2; ++half) {
+                    float4 v[kPer / 2];  // loads first: the stores below must not wait on them one by one
+#pragma unroll
+                    for (int u = 0; u < kPer / 2; ++u)
+                        v[u] = *reinterpret_cast<const float4*>(b_hi + (size_t)((half * (kPer / 2) + u) * kBtProducerWarps * 32 + t) * 16);
+#pragma unroll
+                    for (int u = 0; u < kPer / 2; ++u) {
+                        float4 h, l;
+                        tc_split(v[u].x, h.x, l.x), tc_split(v[u].y, h.y, l.y), tc_split(v[u].z, h.z, l.z), tc_split(v[u].w, h.w, l.w);
+                        *reinterpret_cast<float4*>(b_hi + kBtBTile + (size_t)((half * (kPer / 2) + u) * kBtProducerWarps * 32 + t) * 16) = l;
+                    }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
