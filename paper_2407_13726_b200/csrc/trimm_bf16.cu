@@ -406,6 +406,14 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
     };
     auto kb_first = [&](int P) { return MOMENT2 ? 0 : 4 * P; };
+    // Degree 3: in the column block that holds i1 itself the columns i3 < i1 belong to no element of
+    // the slab; the MMAs of such a tile start at column c0 = i1 rounded down to 16 within the block
+    // and are N = 256 - c0 wide (each CTA supplies half of those columns).
+    auto col_skip = [&](int P, int J, int slot) {
+        if (MODE != kModeMoment3) return 0;
+        const int i1 = p.i1_first + slot;
+        return (J == P && i1 / kTileN == J) ? ((i1 - J * kTileN) & ~15) : 0;
+    };
     constexpr uint32_t kIdesc = MOMENT2 ? (kPIdesc | (1u << 15)) : kPIdesc;  // A operand M-major
     const int64_t G = gridDim.x >> 1, cid = blockIdx.x >> 1;
     auto tile_of = [&](uint32_t n) -> int64_t { return (int64_t)n * G + ((n & 1) ? (G - 1 - cid) : cid); };
@@ -446,10 +454,11 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     } else {
                         tma_load_2d_pair(dst, &tmap_a, 0, (int)((tile_base + kb) * kTileM), bar);
                     }
+                    const int c0 = col_skip(P, J, slot);
 #pragma unroll
                     for (int q = 0; q < kTileN / 128; ++q)
                         tma_load_2d_pair(dst + kABytes + q * (kBlockK * 128), &tmap_b,
-                                         J * kTileN + (int)rank * (kTileN / 2) + q * 64, kb * kBlockK, bar);
+                                         J * kTileN + c0 + (int)rank * ((kTileN - c0) / 2) + q * 64, kb * kBlockK, bar);
                 }
             }
             if (!ok) {
@@ -566,6 +575,8 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileN;
+                // degree 3: the instruction's N is the tile's width without the skipped columns
+                const uint32_t idesc3 = (kPIdesc & ~(0x3Fu << 17)) | ((uint32_t)((kTileN - col_skip(P, J, slot)) >> 3) << 17);
                 for (int kb = kb_first(P); kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kPStages;
                     if (!mbar_wait_cluster(full(s), (it / kPStages) & 1, abort_flag, p.err_word, kErrFull)) {
@@ -581,7 +592,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                                     : smem_desc(a_addr + k16 * 32, 16, 1024);
                         const uint64_t db = smem_desc(b_addr + k16 * 2048, kBlockK * 128, 1024);
                         if (MODE == kModeMoment3)
-                            umma_bf16_pair_ts(d_tmem, tmem_base + kTmemAStage0 + s * kTmemAStageCols + k16 * 8, db, kPIdesc,
+                            umma_bf16_pair_ts(d_tmem, tmem_base + kTmemAStage0 + s * kTmemAStageCols + k16 * 8, db, idesc3,
                                               (kb > 0 || k16 > 0) ? 1u : 0u);
                         else
                             umma_bf16_pair(d_tmem, da, db, kIdesc, (kb > kb_first(P) || k16 > 0) ? 1u : 0u);
@@ -635,8 +646,10 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                  : upper_row_base(p.N, i);
                     float* prow = p.C + rb;
 #pragma unroll 1
-                    for (int cc = 0; cc < kTileN / 32; ++cc) {
-                        const int64_t col0 = (int64_t)J * kTileN + cc * 32;
+                    const int c0 = col_skip(P, J, slot);  // accumulator column 0 is column c0 of the block
+                    const int64_t col_end = (int64_t)(J + 1) * kTileN;
+                    for (int cc = 0; cc * 32 < kTileN - c0; ++cc) {
+                        const int64_t col0 = (int64_t)J * kTileN + c0 + cc * 32;
                         if (col0 + 32 <= (int64_t)I * kTileM + warp * 32 || col0 >= p.N) continue;  // warp-uniform: nothing kept
                         uint32_t r[32];
                         tmem_ld32(taddr + cc * 32, r);
@@ -645,7 +658,7 @@ trimm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                             for (int v = 0; v < 32; ++v) {
                                 const int64_t j = col0 + v;
-                                if (j >= i && j < p.N) {
+                                if (j >= i && j < p.N && j < col_end) {
                                     float o = __uint_as_float(r[v]);
                                     if (p.accumulate) o += prow[j];
                                     prow[j] = o;
