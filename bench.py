@@ -92,6 +92,8 @@ def accounting(z):
         "unpack_bf16": dict(flops=0, bytes=2 * (tri(N5) + N5 * N5), bound="hbm"),  # read packed, write box
         # widened row: tensor times matrix over the upper half cube, packed in and out (8 flop/B: HBM first)
         "ttm_ut": dict(flops=2 * tri(N6) * Q6 * K6, bytes=4 * (tri(N6) * (Q6 + K6) + K6 * Q6), bound="hbm"),
+        # widened row: the same rule through the opt-in split-precision (TF32 hi/lo) tensor-core entry point
+        "ttm_ut_tc": dict(flops=2 * tri(N6) * Q6 * K6, bytes=4 * (tri(N6) * (Q6 + K6) + K6 * Q6), bound="hbm"),
         # widened row: degree-2 moments B^T B on i1 <= i2 (M7 samples x N7 features, bf16), packed fp32 output
         "moment2_bf16": dict(flops=2 * tri(N7) * M7, bytes=2 * M7 * N7 + 4 * tri(N7), bound="tensor"),
         # widened row: degree-3 moments on i1 <= i2 <= i3 (two multiplies and an add per term), packed tetrahedron out
@@ -102,7 +104,7 @@ def accounting(z):
     return acc
 
 
-ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "bandmm_tc", "mttkrp", "mttkrp_tc", "ttm_ut", "trimm_bf16", "pack_bf16", "unpack_bf16",
+ORDER = ["trmv", "trmv_batched", "bandmm", "bandmm_exact", "bandmm_tc", "mttkrp", "mttkrp_tc", "ttm_ut", "ttm_ut_tc", "trimm_bf16", "pack_bf16", "unpack_bf16",
          "moment2_bf16", "moment3_bf16", "thp_ut", "symv"]
 # the kernels of the five configurations; the others are widened rows and never the roofline's kernel
 CONFIG_KERNELS = ("trmv", "trmv_batched", "bandmm", "mttkrp", "trimm_bf16", "pack_bf16", "unpack_bf16", "symv")
@@ -185,6 +187,12 @@ def generate_host(z, pin, only=None):
         synth.upper_half_cube_stream(5, 0, N6, N6, Q6, out=a6)
         h["ttm_ut"] = dict(desc=st.upper_half_cube(N6, N6, Q6), out_desc=st.upper_half_cube(N6, N6, K6), A=host(a6),
                            ins=[host(synth.dense(5, 1, (K6, Q6)))], out=(cap(tri(N6) * K6, 4),))
+    if want("ttm_ut_tc"):
+        N6, Q6, K6 = z["N6"], z["Q6"], z["K6"]
+        a6 = np.zeros(cap(tri(N6) * Q6, 4), np.float32)
+        synth.upper_half_cube_stream(5, 0, N6, N6, Q6, out=a6)
+        h["ttm_ut_tc"] = dict(desc=st.upper_half_cube(N6, N6, Q6), out_desc=st.upper_half_cube(N6, N6, K6), A=host(a6),
+                              ins=[host(synth.dense(5, 1, (K6, Q6)))], out=(cap(tri(N6) * K6, 4),))
     if want("thp_ut"):
         N6, Q6 = z["N6"], z["Q6"]
         a9 = np.zeros(cap(tri(N6) * Q6, 4), np.float32)
@@ -207,7 +215,7 @@ def generate_host(z, pin, only=None):
 
 
 EXPR = {"mttkrp_tc": "ijk,jr,kr->ir", "bandmm_tc": "ij,jc->ic", "trmv": "ij,j->i", "trmv_batched": "ij,j->i", "bandmm": "ij,jc->ic", "symv": "ij,j->i",
-        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk",
+        "mttkrp": "ijk,jr,kr->ir", "trimm_bf16": "ij,jc->ic", "ttm_ut": "ijl,kl->ijk", "ttm_ut_tc": "ijl,kl->ijk",
         "bandmm_exact": "ij,jc->ic", "moment2_bf16": "xi,xj->ij", "moment3_bf16": "xi,xj,xk->ijk", "thp_ut": "ijk,ijk->ijk"}
 
 
@@ -337,6 +345,8 @@ def run_gpu(args):
             dastac.pack(structs["trimm_bf16"], d["A"], d["out"])
         elif name == "unpack_bf16":
             dastac.unpack(structs["trimm_bf16"], d["A"], d["out"])
+        elif name == "ttm_ut_tc":
+            dastac.ttm_split_tf32(structs[name], d["A"], d["ins"][0], d["out"], err_word=err_word)
         elif name == "bandmm_tc":
             dastac.bandmm_split_tf32(structs[name], d["A"], d["ins"][0], d["out"], err_word=err_word)
         elif name == "mttkrp_tc":
@@ -459,7 +469,7 @@ def run_gpu(args):
         hd = {}
         h2d = d2h = 0
         for name, hw in host.items():
-            if name not in order or name in ("mttkrp_tc", "bandmm_tc"):   # device-only entry points
+            if name not in order or name in ("mttkrp_tc", "bandmm_tc", "ttm_ut_tc"):   # device-only entry points
                 continue
             out_h = torch.empty(hw["out"], dtype=torch.float32).pin_memory()
             n = dastac.contract_workspace(EXPR[name], structs[name], hw["A"], hw["ins"], out_h, batch=hw.get("batch", 1),

@@ -324,6 +324,30 @@ dastac_status dastac_bandmm_split_tf32(const dastac_structure* s, const float* A
                                        int32_t* err_word, void* stream);
 
 /*
+ * Split-precision tensor-core form of tensor times matrix with packed input and output (opt-in;
+ * dastac_contract keeps the plain fp32 multiply-add kernel).  A(i,j,k) = sum_l B(i,j,l) C(k,l) (the
+ * running example of Section 3) over a rank-3 structure whose trailing index is dense: in packed
+ * form the rule is the dense product Y[p][k] = sum_l X[p][l] C[k][l] of the packed input, viewed as
+ * a [count / Q][Q] matrix, with C.  It is taken on the tensor cores in TF32 with both operands
+ * split into a high and a low part and the three products hi*hi, hi*lo, lo*hi accumulated in fp32
+ * (about 2^-21 per product); results agree with dastac_contract's within the same 1e-5 bound.
+ *   s         rank-3 structure with a dense trailing index of extent Q (upper half cube, dense
+ *             box, planes with a free last index); anything else returns DASTAC_ERR_UNSUPPORTED_EXPR,
+ *             as does Q > 256
+ *   X         device, packed fp32 values of s, 16-byte aligned, Q a multiple of 4
+ *             (DASTAC_ERR_ALIGNMENT otherwise: a packed row must be a row of a tensor map)
+ *   C         device, K x Q fp32, row pitch ldc elements
+ *   Y         device, packed fp32 output over the same leading index set with trailing extent K
+ *             (count / Q * K values); bulk tensor stores when Y is 16-byte aligned and K is a
+ *             multiple of 4, plain stores otherwise
+ *   accumulate, stream   as for dastac_contract
+ *   err_word  optional device int32, set when a bounded wait inside the kernel expires
+ * Needs no workspace.
+ */
+dastac_status dastac_ttm_split_tf32(const dastac_structure* s, const float* X, const float* C, int64_t ldc,
+                                    int64_t K, float* Y, int32_t accumulate, int32_t* err_word, void* stream);
+
+/*
  * A structured operand given as several summands (Section 4: the method works on the individual
  * summands of a rule; every summand's region has its own compressed buffer, and a summand whose
  * region equals an earlier one reuses that buffer instead of getting a second copy).  Examples:

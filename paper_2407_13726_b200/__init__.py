@@ -9,7 +9,7 @@ import importlib
 
 _PUBLIC = ("DastacError", "Structure", "contract", "contract_workspace", "launch_count", "pack",
            "rank", "rank_batch", "status_string", "structure_count", "structure_create", "unpack",
-           "unrank", "unrank_batch", "trimm_bf16_noalloc", "device_error", "selftest_wait_expiry", "piecewise_fuse", "KIND_GENERIC", "Rule", "mttkrp_split_tf32", "bandmm_split_tf32", "NOALLOC_MAX_N", "F32", "BF16", "MEM_DEVICE", "MEM_HOST", "KIND_EMPTY",
+           "unrank", "unrank_batch", "trimm_bf16_noalloc", "device_error", "selftest_wait_expiry", "piecewise_fuse", "KIND_GENERIC", "Rule", "mttkrp_split_tf32", "bandmm_split_tf32", "ttm_split_tf32", "NOALLOC_MAX_N", "F32", "BF16", "MEM_DEVICE", "MEM_HOST", "KIND_EMPTY",
            "KIND_DENSE", "KIND_UPPER", "KIND_LOWER", "KIND_BAND_DIAGONALS", "KIND_TETRAHEDRON", "KIND_BAND_EXACT", "KIND_UPPER_SHIFTED", "KIND_BAND_OFFSETS", "KIND_PLANE",
            "LAYOUT_LEXICOGRAPHIC", "LAYOUT_PADDED_DIAGONALS", "EXPORTS", "LIB_PATH")
 

@@ -30,7 +30,7 @@ EXPORTS = [
     "dastac_device_error", "dastac_selftest_wait_expiry", "dastac_piecewise_fuse",
     "dastac_rule_create", "dastac_rule_destroy", "dastac_rule_size", "dastac_rule_summand", "dastac_rule_pack",
     "dastac_rule_contract_workspace", "dastac_rule_contract", "dastac_mttkrp_split_tf32",
-    "dastac_bandmm_split_tf32",
+    "dastac_bandmm_split_tf32", "dastac_ttm_split_tf32",
 ]
 NOALLOC_MAX_N = 2048
 
@@ -86,6 +86,7 @@ _lib.dastac_selftest_wait_expiry.argtypes = [_i64, _vp]
 _lib.dastac_piecewise_fuse.argtypes = [_vp, _i32, _vp]
 _lib.dastac_mttkrp_split_tf32.argtypes = [_vp, _vp, _vp, _i64, _vp, _i64, _vp, _i64, _i64, _i32, _vp, _vp]
 _lib.dastac_bandmm_split_tf32.argtypes = [_vp, _vp, _vp, _i64, _vp, _i64, _i64, _i32, _vp, _vp]
+_lib.dastac_ttm_split_tf32.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp]
 _lib.dastac_rule_create.argtypes = [_vp, _i32, ctypes.POINTER(_vp)]
 _lib.dastac_rule_destroy.argtypes = [_vp]
 _lib.dastac_rule_destroy.restype = None
@@ -454,6 +455,19 @@ def bandmm_split_tf32(s: Structure, packed: torch.Tensor, B: torch.Tensor, out: 
                                          out.stride(0), B.shape[1], int(accumulate),
                                          None if err_word is None else err_word.data_ptr(), _stream()),
            "dastac_bandmm_split_tf32")
+    return out
+
+
+def ttm_split_tf32(s: Structure, packed: torch.Tensor, C: torch.Tensor, out: torch.Tensor,
+                   accumulate: bool = False, err_word: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Tensor times matrix, packed in and packed out (``out`` holds ``count / Q * K`` values), through the
+    split-precision tensor-core entry point (see ``dastac.h``)."""
+    assert packed.is_cuda and C.is_cuda and out.is_cuda and C.dim() == 2
+    assert packed.dtype == C.dtype == out.dtype == torch.float32
+    assert C.shape[0] <= 1 or C.stride(1) == 1 or C.shape[1] <= 1
+    _check(_lib.dastac_ttm_split_tf32(s._h, packed.data_ptr(), C.data_ptr(), C.stride(0), C.shape[0], out.data_ptr(),
+                                      int(accumulate), None if err_word is None else err_word.data_ptr(), _stream()),
+           "dastac_ttm_split_tf32")
     return out
 
 

@@ -217,9 +217,11 @@ def test_config5_triangular_bf16_n8192():
     assert torch.equal(repacked.view(torch.int16)[: s.nnz], packed.view(torch.int16)[: s.nnz])
 
 
-def test_widened_row_ttm_n1024_q32_k32():
+@pytest.mark.parametrize("tensor_cores", [False, True], ids=["fp32", "split_tf32"])
+def test_widened_row_ttm_n1024_q32_k32(tensor_cores):
     """The tensor-times-matrix running example at the size the benchmark times: sampled slabs i of
-    the packed result (slab i is the contiguous run of positions that starts at (i, i, 0))."""
+    the packed result (slab i is the contiguous run of positions that starts at (i, i, 0)); through
+    dastac_contract and through the opt-in tensor-core entry point."""
     N, Q, K = 1024, 32, 32
     dB, dA = st.upper_half_cube(N, N, Q), st.upper_half_cube(N, N, K)
     sB, sA = dastac.Structure(dB), dastac.Structure(dA)
@@ -227,7 +229,10 @@ def test_widened_row_ttm_n1024_q32_k32():
     C = synth.dense(5, 1, (K, Q))
     packedB = _packed(sB, lambda h: synth.upper_half_cube_stream(5, 0, N, N, Q, out=h))
     out = torch.full((sA.capacity(torch.float32),), float("nan"), device="cuda")
-    dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out, out_structure=sA)
+    if tensor_cores:
+        dastac.ttm_split_tf32(sB, packedB, dev(C), out)
+    else:
+        dastac.contract("ijl,kl->ijk", sB, packedB, [dev(C)], out, out_structure=sA)
     got = out.cpu().numpy()[: sA.nnz]
     assert np.isfinite(got).all()
     sel = _rows(N, 12, extra=(1, 255, 256, 257, N - 2))

@@ -1190,6 +1190,50 @@ def test_band_matmat_split_precision_refusals():
     assert e.value.status == 3
 
 
+@pytest.mark.parametrize("M,N,Q,K", [(1, 1, 4, 1), (5, 7, 4, 6), (7, 5, 8, 5), (33, 40, 32, 32), (64, 64, 20, 12),
+                                     (130, 130, 32, 64), (97, 97, 36, 33), (300, 300, 8, 40), (40, 50, 100, 32),
+                                     (20, 30, 256, 7)])
+def test_ttm_split_precision_tensor_core_form(M, N, Q, K):
+    """The opt-in TF32 hi/lo form of the running example, packed in and out, at the fp32 kernels' bound."""
+    dB, dA = st.upper_half_cube(M, N, Q), st.upper_half_cube(M, N, K)
+    sB, sA = dastac.Structure(dB), dastac.Structure(dA)
+    B = synth.dense(5, 0, (M, N, Q))
+    C = synth.dense(5, 1, (K, Q))
+    ref, ref_abs = oracle.ttm(dB, B, C)
+    exp, exp_abs = oracle.pack(dA, ref), oracle.pack(dA, ref_abs)
+    packedB = packed_dev(sB, synth.upper_half_cube_stream(5, 0, M, N, Q))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = sA.empty_packed()
+    out.fill_(float("nan"))
+    dastac.ttm_split_tf32(sB, packedB, dev(C), out, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out.cpu().numpy()[: sA.nnz], exp, exp_abs) <= TOL_F32
+    A0 = synth.dense(5, 2, (sA.nnz,))
+    out2 = sA.empty_packed()
+    out2[: sA.nnz] = dev(A0)
+    dastac.ttm_split_tf32(sB, packedB, dev(C), out2, accumulate=True, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out2.cpu().numpy()[: sA.nnz], exp + A0, exp_abs + np.abs(A0)) <= TOL_F32
+    # a padded leading dimension of C
+    Cp = torch.zeros((K, Q + 3), device="cuda")[:, :Q]
+    Cp.copy_(dev(C))
+    out3 = sA.empty_packed()
+    dastac.ttm_split_tf32(sB, packedB, Cp, out3, err_word=err)
+    assert int(err.item()) == 0
+    assert rel_err(out3.cpu().numpy()[: sA.nnz], exp, exp_abs) <= TOL_F32
+
+
+def test_ttm_split_precision_refusals():
+    tri = dastac.Structure(st.upper_triangle(16))
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.ttm_split_tf32(tri, tri.empty_packed(), torch.zeros((4, 16), device="cuda"), torch.zeros(64, device="cuda"))
+    assert e.value.status == 3
+    odd = dastac.Structure(st.upper_half_cube(8, 8, 3))   # a packed row of 12 bytes is no tensor-map row
+    with pytest.raises(dastac.DastacError) as e:
+        dastac.ttm_split_tf32(odd, odd.empty_packed(), torch.zeros((4, 3), device="cuda"), torch.zeros(36 * 4, device="cuda"))
+    assert e.value.status == 5
+
+
 def test_mttkrp_split_precision_refusals():
     big = dastac.Structure(st.tetrahedron(513))
     z = torch.zeros((513, 4), device="cuda")
