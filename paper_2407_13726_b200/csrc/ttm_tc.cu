@@ -13,11 +13,12 @@
 //
 // Tile = 128 packed rows x 32 output columns, l in blocks of 32.
 //   loader thread    waits for a free stage and starts the copy of the next block of X
-//   producer warps   two groups of eight, taking the blocks in turn: wait for the copy, write Xlo
+//   producer warps   three groups of four, taking the blocks in turn: wait for the copy, write Xlo
 //   MMA thread       per block and k-step of 8: tcgen05.mma kind::tf32 M128 N64 K8 with A = X,
 //                    B = [Chi ; Clo] (columns 0..31 get Xhi Chi, 32..63 get Xhi Clo), and M128 N32 K8
 //                    with A = Xlo, B = Chi into columns 0..31
-//   epilogue warps   tcgen05.ld of both halves, their sum leaves as a 32 x 32 chunk through shared
+//   epilogue warps   two sets of four, one per accumulator (the proxy fence before a bulk store
+//                    costs about a thousand cycles): tcgen05.ld of both halves, their sum leaves as a 32 x 32 chunk through shared
 //                    memory by a bulk tensor store (reduce-add when accumulating; plain stores when
 //                    the rows of Y are not 16-byte aligned)
 // C is staged once per CTA as hi / lo K-major tiles (8 KiB per block of l, Q <= 256).  Accumulators
@@ -40,12 +41,15 @@ constexpr int kTtStageBytes = 2 * kTtTile;   // X (= Xhi), Xlo
 constexpr int kTtCBlock = 2 * kTtCols * 128; // 8 KiB: [Chi ; Clo] of one block of l
 constexpr int kTtMaxQBlocks = 8;
 constexpr int kTtMaxStages = 6;
-constexpr int kTtEpiWarps = 4, kTtWarpMma = 4, kTtWarpLoad = 5, kTtWarpLo0 = 6;
-constexpr int kTtLoWarps = 8, kTtLoGroups = 2;
+// warps 0-7 epilogue (two sets of four: set e drains accumulator e, i.e. every second tile), 8-9 MMA
+// (issuer e fills accumulator e: the eight small MMAs of a tile cost one thread more than a thousand
+// cycles to issue), 10 loader, 11.. low parts (three groups of four, taking the blocks in turn)
+constexpr int kTtEpiSets = 2, kTtEpiWarps = 4 * kTtEpiSets, kTtWarpMma = 8, kTtMmaWarps = 2, kTtWarpLoad = 10, kTtWarpLo0 = 11;
+constexpr int kTtLoWarps = 4, kTtLoGroups = 3;
 constexpr int kTtThreads = (kTtWarpLo0 + kTtLoWarps * kTtLoGroups) * 32;
 constexpr int kTtTmemCols = 128;             // two accumulators of 64 columns
 constexpr int kTtEpiBufBytes = 32 * 128;
-constexpr int kTtEpiBytes = kTtEpiWarps * 2 * kTtEpiBufBytes;
+constexpr int kTtEpiBytes = kTtEpiWarps * kTtEpiBufBytes;  // one buffer per epilogue warp
 constexpr long long kTtWaitBudget = 2000000000LL;
 constexpr int32_t kErrWordTtmTc = 0x5454;    // "TT"
 
@@ -89,7 +93,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             tc_mbar_init(tmem_full(a), 1);
-            tc_mbar_init(tmem_empty(a), kTtEpiWarps);
+            tc_mbar_init(tmem_empty(a), 4);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -164,14 +168,15 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             if (lane == 0) tc_mbar_arrive(full(s));
         }
     }
-    else if (warp == kTtWarpMma) {
-        // ---- MMA issuer: one thread ----
+    else if (warp >= kTtWarpMma && warp < kTtWarpMma + kTtMmaWarps) {
+        // ---- MMA issuers: one thread per accumulator, taking the tiles in turn ----
         if (lane == 0) {
             constexpr uint32_t kIdesc64 = tc_idesc_mn(kTtRows, 64), kIdesc32 = tc_idesc_mn(kTtRows, 32);
-            int64_t it = 0;
+            const int me = warp - kTtWarpMma;
             bool ok = true;
-            for (int64_t tile_n = 0; tile_n < my_tiles && ok; ++tile_n) {
-                const int acc = (int)(tile_n & 1);
+            for (int64_t tile_n = me; tile_n < my_tiles && ok; tile_n += kTtMmaWarps) {
+                int64_t it = tile_n * p.q_blocks;
+                const int acc = me;
                 const int64_t use = tile_n >> 1;  // earlier uses of this accumulator
                 if (use >= 1 && !tt_wait(tmem_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.err_word)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -198,17 +203,17 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         }
     } else if (warp < kTtEpiWarps) {
         // ---- epilogue: warp = lane quarter of tensor memory, thread = packed row ----
-        uint32_t chunk_n = 0;
-        for (int64_t tile_n = 0; tile_n < my_tiles; ++tile_n) {
-            const int64_t p0 = (blockIdx.x + tile_n * G) * kTtRows + warp * 32;
-            const int acc = (int)(tile_n & 1);
+        const int set = warp >> 2, quarter = warp & 3;
+        for (int64_t tile_n = set; tile_n < my_tiles; tile_n += kTtEpiSets) {
+            const int64_t p0 = (blockIdx.x + tile_n * G) * kTtRows + quarter * 32;
+            const int acc = set;
             const int64_t use = tile_n >> 1;
             int got = 1;
             if (lane == 0) got = tt_wait(tmem_full(acc), (uint32_t)(use & 1), abort_flag, p.err_word) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + acc * 64;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 64;
             uint32_t d0[32], d1[32];
             tc_ld32(taddr, d0);
             tc_ld32(taddr + 32, d1);
@@ -220,8 +225,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 #pragma unroll
             for (int v = 0; v < 32; ++v) o[v] = __uint_as_float(d0[v]) + __uint_as_float(d1[v]);
             if (p.tma_y) {
-                uint8_t* const buf = epi0 + (size_t)(warp * 2 + (chunk_n & 1)) * kTtEpiBufBytes;
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");  // its last store has read it
+                uint8_t* const buf = epi0 + (size_t)warp * kTtEpiBufBytes;
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // its last store has read it
                 __syncwarp();
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
@@ -241,7 +246,6 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                                      : "memory");
                 }
                 if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                ++chunk_n;
             } else {
                 const int64_t row = p0 + lane;
                 if (row < p.P) {
