@@ -14,15 +14,16 @@
 // Tile = 128 packed rows x 32 output columns, l in blocks of 32.
 //   loader thread    waits for a free stage and starts the copy of the next block of X
 //   producer warps   three groups of four, taking the blocks in turn: wait for the copy, write Xlo
-//   MMA thread       per block and k-step of 8: tcgen05.mma kind::tf32 M128 N64 K8 with A = X,
+//   MMA threads      four, taking the tiles in turn (one accumulator each: issuing the eight small MMAs
+//                    of a tile costs a thread more than a thousand cycles); per block and k-step of 8: tcgen05.mma kind::tf32 M128 N64 K8 with A = X,
 //                    B = [Chi ; Clo] (columns 0..31 get Xhi Chi, 32..63 get Xhi Clo), and M128 N32 K8
 //                    with A = Xlo, B = Chi into columns 0..31
 //   epilogue warps   two sets of four, one per accumulator (the proxy fence before a bulk store
 //                    costs about a thousand cycles): tcgen05.ld of both halves, their sum leaves as a 32 x 32 chunk through shared
 //                    memory by a bulk tensor store (reduce-add when accumulating; plain stores when
 //                    the rows of Y are not 16-byte aligned)
-// C is staged once per CTA as hi / lo K-major tiles (8 KiB per block of l, Q <= 256).  Accumulators
-// are double buffered in tensor memory (2 x 64 columns).  Every wait is bounded.
+// C is staged once per CTA as hi / lo K-major tiles (8 KiB per block of l, Q <= 256).  Four
+// accumulators of 64 columns in tensor memory, one per MMA issuer.  Every wait is bounded.
 #include <cuda.h>
 
 #include <cstring>
@@ -44,10 +45,11 @@ constexpr int kTtMaxStages = 6;
 // warps 0-7 epilogue (two sets of four: set e drains accumulator e, i.e. every second tile), 8-9 MMA
 // (issuer e fills accumulator e: the eight small MMAs of a tile cost one thread more than a thousand
 // cycles to issue), 10 loader, 11.. low parts (three groups of four, taking the blocks in turn)
-constexpr int kTtEpiSets = 2, kTtEpiWarps = 4 * kTtEpiSets, kTtWarpMma = 8, kTtMmaWarps = 2, kTtWarpLoad = 10, kTtWarpLo0 = 11;
+constexpr int kTtEpiSets = 2, kTtEpiWarps = 4 * kTtEpiSets, kTtWarpMma = 8, kTtMmaWarps = 4, kTtWarpLoad = 12, kTtWarpLo0 = 13;
 constexpr int kTtLoWarps = 4, kTtLoGroups = 3;
 constexpr int kTtThreads = (kTtWarpLo0 + kTtLoWarps * kTtLoGroups) * 32;
-constexpr int kTtTmemCols = 128;             // two accumulators of 64 columns
+constexpr int kTtAccs = kTtMmaWarps;         // accumulators of 64 columns, one per issuer
+constexpr int kTtTmemCols = 64 * kTtAccs;
 constexpr int kTtEpiBufBytes = 32 * 128;
 constexpr int kTtEpiBytes = kTtEpiWarps * kTtEpiBufBytes;  // one buffer per epilogue warp
 constexpr long long kTtWaitBudget = 2000000000LL;
@@ -81,8 +83,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     auto full = [&](int s) { return tc_smem(&bars[kTtMaxStages + s]); };
     auto empty = [&](int s) { return tc_smem(&bars[2 * kTtMaxStages + s]); };
     auto tmem_full = [&](int a) { return tc_smem(&bars[3 * kTtMaxStages + a]); };
-    auto tmem_empty = [&](int a) { return tc_smem(&bars[3 * kTtMaxStages + 2 + a]); };
-    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(&bars[3 * kTtMaxStages + 4]);
+    auto tmem_empty = [&](int a) { return tc_smem(&bars[3 * kTtMaxStages + kTtAccs + a]); };
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(&bars[3 * kTtMaxStages + 2 * kTtAccs]);
     volatile int* const abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     if (threadIdx.x == 0) {
@@ -91,7 +93,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             tc_mbar_init(full(s), kTtLoWarps);
             tc_mbar_init(empty(s), 1);
         }
-        for (int a = 0; a < 2; ++a) {
+        for (int a = 0; a < kTtAccs; ++a) {
             tc_mbar_init(tmem_full(a), 1);
             tc_mbar_init(tmem_empty(a), 4);
         }
@@ -177,7 +179,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             for (int64_t tile_n = me; tile_n < my_tiles && ok; tile_n += kTtMmaWarps) {
                 int64_t it = tile_n * p.q_blocks;
                 const int acc = me;
-                const int64_t use = tile_n >> 1;  // earlier uses of this accumulator
+                const int64_t use = tile_n / kTtMmaWarps;  // earlier uses of this accumulator
                 if (use >= 1 && !tt_wait(tmem_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.err_word)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + acc * 64;
@@ -206,8 +208,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int set = warp >> 2, quarter = warp & 3;
         for (int64_t tile_n = set; tile_n < my_tiles; tile_n += kTtEpiSets) {
             const int64_t p0 = (blockIdx.x + tile_n * G) * kTtRows + quarter * 32;
-            const int acc = set;
-            const int64_t use = tile_n >> 1;
+            const int acc = (int)(tile_n % kTtAccs);
+            const int64_t use = tile_n / kTtAccs;
             int got = 1;
             if (lane == 0) got = tt_wait(tmem_full(acc), (uint32_t)(use & 1), abort_flag, p.err_word) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
