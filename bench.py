@@ -398,7 +398,7 @@ def run_gpu(args):
     launches = dastac.launch_count() - launches0
     total_ms = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
-    assert int(err_word.item()) == 0, "a device-side bounded wait expired"
+    assert int(err_word.item()) == 0, "a device-side bounded wait expired, code %#x" % int(err_word.item())
     total_ms = max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
     step_flops = sum(acct[n]["flops"] for n in order)

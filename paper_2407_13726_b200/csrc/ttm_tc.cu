@@ -65,8 +65,9 @@ struct TtParams {
     int32_t* err_word;
 };
 
-__device__ __forceinline__ bool tt_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* err_word) {
-    return tc_wait_coded(bar, parity, abort_flag, err_word, kErrWordTtmTc, kTtWaitBudget);
+// `site` (1..5) is added to the code so that the word tells which wait ran out
+__device__ __forceinline__ bool tt_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* err_word, int site = 0) {
+    return tc_wait_coded(bar, parity, abort_flag, err_word, kErrWordTtmTc + (site << 16), kTtWaitBudget);
 }
 
 __global__ void __launch_bounds__(kTtThreads, 1)
@@ -134,7 +135,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (lane == 0) {
             for (int64_t it = 0; it < items; ++it) {
                 const int s = (int)(it % S);
-                if (it >= S && !tt_wait(empty(s), (uint32_t)(((it / S) - 1) & 1), abort_flag, p.err_word)) break;
+                if (it >= S && !tt_wait(empty(s), (uint32_t)(((it / S) - 1) & 1), abort_flag, p.err_word, 1)) break;
                 const int64_t tile = blockIdx.x + (it / p.q_blocks) * G;
                 const int qb = (int)(it % p.q_blocks);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw(s)), "r"((uint32_t)kTtTile) : "memory");
@@ -151,7 +152,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         for (int64_t it = grp; it < items; it += kTtLoGroups) {
             const int s = (int)(it % S);
             bool ok = true;
-            if (lane == 0) ok = tt_wait(raw(s), (uint32_t)((it / S) & 1), abort_flag, p.err_word);
+            if (lane == 0) ok = tt_wait(raw(s), (uint32_t)((it / S) & 1), abort_flag, p.err_word, 2);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
             uint8_t* const x = stage0 + (size_t)s * kTtStageBytes;
@@ -180,12 +181,12 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 int64_t it = tile_n * p.q_blocks;
                 const int acc = me;
                 const int64_t use = tile_n / kTtMmaWarps;  // earlier uses of this accumulator
-                if (use >= 1 && !tt_wait(tmem_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.err_word)) break;
+                if (use >= 1 && !tt_wait(tmem_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.err_word, 3)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + acc * 64;
                 for (int qb = 0; qb < p.q_blocks; ++qb, ++it) {
                     const int s = (int)(it % S);
-                    if (!tt_wait(full(s), (uint32_t)((it / S) & 1), abort_flag, p.err_word)) {
+                    if (!tt_wait(full(s), (uint32_t)((it / S) & 1), abort_flag, p.err_word, 4)) {
                         ok = false;
                         break;
                     }
@@ -211,7 +212,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const int acc = (int)(tile_n % kTtAccs);
             const int64_t use = tile_n / kTtAccs;
             int got = 1;
-            if (lane == 0) got = tt_wait(tmem_full(acc), (uint32_t)(use & 1), abort_flag, p.err_word) ? 1 : 0;
+            if (lane == 0) got = tt_wait(tmem_full(acc), (uint32_t)(use & 1), abort_flag, p.err_word, 5) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
